@@ -1,0 +1,180 @@
+/*
+ * gc.h -- C ABI of libgc: sparse gradient compression with error feedback on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * Per training iteration and per worker the library
+ *   1. folds the error-feedback residual into the fresh gradient      a = g + r   (fp32)
+ *   2. selects, per tensor, the k entries of largest magnitude (exact top-k, ties to the
+ *      lower index) or, in threshold mode, every entry at or above a sampled threshold
+ *   3. emits them as index-sorted (uint32 flat index, fp32 value) pairs
+ *   4. writes the residual back: +0 where sent, a elsewhere
+ * and, across W workers,
+ *   5. decodes and sums the W sparse sets into one dense fp32 buffer in worker order.
+ *
+ * Where the definitions come from.  The source paper of this project (erasure-coded fault
+ * tolerance for recommendation-model training) defines none of these steps; its only words
+ * on gradient compression are a remark in its Section 3.3.2 that its own deltas are dense.
+ * Every operation below therefore follows the problem statement of the benchmark workload,
+ * and each comment says which clause.
+ *
+ * Conventions
+ *   - All tensors of a plan live back to back in one flat fp32 buffer ("flat layout");
+ *     indices in the output are offsets into that flat buffer.
+ *   - "device" pointers are CUDA device memory on the plan's device; "host" pointers are
+ *     ordinary process memory.  The caller owns every buffer it passes in, including the
+ *     workspace; the plan owns only its own small host and device tables.
+ *   - gc_compress and gc_decompress_accumulate enqueue work on the given stream and return
+ *     without synchronising.  No call allocates device memory except gc_plan.
+ *   - Return value: 0 = GC_OK, negative = error, positive = warning.  Conditions detected on
+ *     the device (truncation in threshold mode, an internal wait that ran out) are written
+ *     to a status word at the head of the workspace; read it with gc_last_status.
+ *   - Nothing here aborts, throws or traps.
+ *
+ * Limits: total elements per plan <= 2^31 - 1; at most GC_MAX_WORKERS sparse sets per
+ * gc_decompress_accumulate call (chain calls with zero_first = 0 for more).
+ */
+#ifndef GC_H_
+#define GC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gc_plan_s gc_plan_t;
+
+/* status codes */
+#define GC_OK             0
+#define GC_E_INVALID     (-1)   /* bad argument (null pointer, misaligned buffer, density out of (0,1]) */
+#define GC_E_UNSUPPORTED (-2)   /* not available in this build / on this device                        */
+#define GC_E_CUDA        (-3)   /* a CUDA runtime call failed; see gc_last_cuda_error                   */
+#define GC_E_TOO_LARGE   (-4)   /* size beyond a stated limit                                           */
+#define GC_E_TIMEOUT     (-5)   /* a bounded device-side wait gave up (device status only)              */
+#define GC_W_TRUNCATED     1    /* threshold mode: more hits than capacity; the rest stayed in r       */
+
+/* selection modes */
+#define GC_TOPK       0
+#define GC_THRESHOLD  1
+
+#define GC_MAX_WORKERS 64
+
+/* gc_plan_query keys.  "tensor" is ignored for plan-wide keys. */
+#define GC_Q_N_TENSORS          0   /* number of tensors                                            */
+#define GC_Q_TOTAL_N            1   /* elements in the flat buffer                                  */
+#define GC_Q_TOTAL_CAP          2   /* length of out_idx / out_val (sum of per-tensor capacities)   */
+#define GC_Q_WORKSPACE_BYTES    3   /* bytes of device workspace gc_compress / decode need          */
+#define GC_Q_TENSOR_N           4   /* elements of tensor t                                         */
+#define GC_Q_TENSOR_K           5   /* k of tensor t = min(n, max(1, ceil(density*n)))              */
+#define GC_Q_TENSOR_CAP         6   /* output capacity of tensor t (= k in top-k mode)              */
+#define GC_Q_TENSOR_OFFSET      7   /* first flat index of tensor t                                 */
+#define GC_Q_TENSOR_OUT_OFFSET  8   /* first output slot of tensor t                                */
+#define GC_Q_TENSOR_STRIDE      9   /* threshold mode: sampling stride used for tensor t            */
+#define GC_Q_MODE              10
+#define GC_Q_KERNEL_LAUNCHES   11   /* kernels + memsets enqueued by the library so far (host count) */
+
+/*
+ * gc_plan -- describe the flat gradient once; computes k per tensor, output offsets and the
+ * workspace size.  (Problem statement: "top-k at density d applied per tensor" for layer-wise
+ * workloads, "global top-k" when the model is given as one tensor.  k = min(n, max(1,
+ * ceil(density * n))) with density in double precision -- the statement prints k = 10,486
+ * for 1 % of 1,048,576 elements, which excludes a floor.)
+ *
+ *   out            host; receives the new plan
+ *   device         CUDA device ordinal the plan is bound to; -1 = host-only plan that answers
+ *                  gc_plan_query but makes every compute call return GC_E_UNSUPPORTED
+ *   n_tensors      number of tensors (may be 0)
+ *   sizes          host; n_tensors element counts (zeros allowed); the tensors are laid back
+ *                  to back in that order in every flat buffer
+ *   density        in (0, 1]
+ *   mode           GC_TOPK or GC_THRESHOLD
+ *   sample_stride  threshold mode: sample one 4-element group out of this many (0 = 64);
+ *                  tensors of <= 65,536 elements are always sampled in full
+ *   cap_factor     threshold mode: per-tensor output capacity = min(n, ceil(cap_factor*k))
+ *                  (0 = 2.0; must be >= 1)
+ * Allocates a few KB of device memory for the tensor table (freed by gc_destroy).
+ * Errors: GC_E_INVALID, GC_E_TOO_LARGE (total > 2^31-1), GC_E_CUDA.
+ */
+int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *sizes,
+            double density, int mode, uint32_t sample_stride, double cap_factor);
+
+/* gc_plan_query -- host-side lookup of plan facts; never touches the device.
+ * Errors: GC_E_INVALID for an unknown key, a null pointer or tensor >= n_tensors. */
+int gc_plan_query(const gc_plan_t *plan, int what, uint32_t tensor, uint64_t *value);
+
+/*
+ * gc_compress -- one worker, one iteration (problem statement: "fold the error-feedback
+ * residual into the fresh gradient, select the top-k entries by magnitude, compact them
+ * into (index, value) pairs, write back the residual").
+ *
+ *   grad       device, const, fp32[total_n], 16-byte aligned
+ *   residual   device, in/out, fp32[total_n], 16-byte aligned; on return (after the stream
+ *              drains) holds +0 where an entry was sent and g + r elsewhere
+ *   out_idx    device, uint32[total_cap]; pairs of tensor t start at its out offset and are in
+ *              ascending flat index; magnitude = bit pattern with the sign cleared, ties go to
+ *              the lower index, so the selected set is unique
+ *   out_val    device, fp32[total_cap]; bit copy of a = g + r at each sent index
+ *   out_count  device, uint32[2 * n_tensors] or NULL: [t] = pairs written for tensor t,
+ *              [n_tensors + t] = hits (threshold mode: entries at or above the threshold,
+ *              which may exceed the capacity; top-k mode: both equal k)
+ *   workspace  device, GC_Q_WORKSPACE_BYTES bytes, 256-byte aligned; scratch -- contents
+ *              need not survive between calls, but two calls in flight at once must not
+ *              share one workspace
+ *   stream     cudaStream_t (0 = legacy default stream)
+ * Threshold mode (own reading; nothing external defines it): sample = elements whose
+ * 4-element group number within the tensor is a multiple of the stride; tau = the
+ * max(1, ceil(density*|sample|))-th largest sampled magnitude; every element with magnitude
+ * >= tau is a hit; hits are sent in index order up to the capacity.
+ * Errors: GC_E_INVALID (null / misaligned pointer), GC_E_CUDA.  Asynchronous.
+ */
+int gc_compress(gc_plan_t *plan, const float *grad, float *residual,
+                uint32_t *out_idx, float *out_val, uint32_t *out_count,
+                void *workspace, void *stream);
+
+/*
+ * gc_decompress_accumulate -- decode W sparse sets and sum them into a dense buffer
+ * (problem statement: "decode and sum the sparse contributions of W simulated workers into
+ * one dense buffer"; a sum, not a mean).  For every flat index the additions happen in
+ * worker order 0..W-1 in fp32, so the result is reproducible bit for bit.
+ *
+ *   W          number of sparse sets, 1..GC_MAX_WORKERS (0 with zero_first just clears)
+ *   idx, val   host arrays of W device pointers, each laid out as gc_compress wrote them
+ *   count      host array of W device pointers to the out_count arrays gc_compress wrote, or
+ *              NULL = every tensor carries exactly its capacity (top-k mode)
+ *   dense_out  device, fp32[total_n]
+ *   zero_first non-zero: dense_out is set to +0 first; zero: sums are added to its content
+ *   workspace  device, GC_Q_WORKSPACE_BYTES bytes, 256-byte aligned; either one that
+ *              gc_compress has used (ordered before this call on the stream) or zero-filled
+ *              by the caller -- this call does not reset the status word
+ * An index >= total_n is skipped and GC_E_INVALID is recorded in the device status.
+ * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_CUDA.  Asynchronous.
+ */
+int gc_decompress_accumulate(gc_plan_t *plan, uint32_t W,
+                             const uint32_t *const *idx, const float *const *val,
+                             const uint32_t *const *count,
+                             float *dense_out, int zero_first,
+                             void *workspace, void *stream);
+
+/*
+ * gc_last_status -- copy the device status word of a workspace to the host.  This call
+ * SYNCHRONISES the stream.  *status receives GC_OK, GC_W_TRUNCATED, GC_E_TIMEOUT or
+ * GC_E_INVALID as recorded by the kernels since the last gc_compress on that workspace;
+ * *detail (may be NULL) receives a code-specific value (e.g. the tensor that overflowed).
+ */
+int gc_last_status(gc_plan_t *plan, const void *workspace, void *stream,
+                   int32_t *status, uint64_t *detail);
+
+/* gc_last_cuda_error -- host; the cudaError_t value of the most recent failed runtime call
+ * made on behalf of this plan (0 if none). */
+int gc_last_cuda_error(const gc_plan_t *plan);
+
+/* gc_destroy -- free the plan and its device table.  NULL is accepted. */
+int gc_destroy(gc_plan_t *plan);
+
+/* gc_version -- ABI version of the loaded library (host, constant). */
+uint32_t gc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GC_H_ */

@@ -1,0 +1,264 @@
+// libgc: host side of the C ABI declared in include/gc.h.
+#include "gc.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "gc_kernels.cuh"
+
+using namespace gc;
+
+struct gc_plan_s {
+    int device = 0;
+    int mode = GC_TOPK;
+    double density = 0.0;
+    double cap_factor = 2.0;
+    uint32_t stride = 64;
+    uint32_t T = 0;
+    uint64_t total_n = 0, total_cap = 0;
+    uint32_t ntiles = 0;
+    std::vector<TensorDesc> desc;
+    TensorDesc* d_desc = nullptr;
+    // workspace layout (byte offsets)
+    size_t off_sel = 0, off_hist = 0, off_state = 0, control_bytes = 0, ws_bytes = 0;
+    int sm_count = 0;
+    int grid_hist = 0, grid_compact = 0;
+    unsigned long long launches = 0;
+    int last_cuda_error = 0;
+};
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline uint64_t k_rule(uint64_t n, double density) {
+    if (n == 0) return 0;
+    double x = std::ceil(density * (double)n);
+    uint64_t k = x < 1.0 ? 1ull : (uint64_t)x;
+    return k < n ? k : n;
+}
+
+#define GC_CUDA(plan, expr)                                           \
+    do {                                                              \
+        cudaError_t e__ = (expr);                                     \
+        if (e__ != cudaSuccess) {                                     \
+            (plan)->last_cuda_error = (int)e__;                       \
+            (void)cudaGetLastError();                                 \
+            return GC_E_CUDA;                                         \
+        }                                                             \
+    } while (0)
+
+WsView view(const gc_plan_s* p, void* ws) {
+    char* b = static_cast<char*>(ws);
+    WsView v;
+    v.hdr = reinterpret_cast<WsHeader*>(b);
+    v.sel = reinterpret_cast<TensorSel*>(b + p->off_sel);
+    v.hist = reinterpret_cast<uint32_t*>(b + p->off_hist);
+    v.tile_state = reinterpret_cast<unsigned long long*>(b + p->off_state);
+    return v;
+}
+
+template <typename K>
+int blocks_per_sm(K kernel, int threads) {
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, threads, 0) != cudaSuccess || nb < 1) {
+        (void)cudaGetLastError();
+        nb = 1;
+    }
+    return nb;
+}
+
+}  // namespace
+
+extern "C" {
+
+uint32_t gc_version(void) { return 1u; }
+
+int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* sizes,
+            double density, int mode, uint32_t sample_stride, double cap_factor) {
+    if (out == nullptr) return GC_E_INVALID;
+    *out = nullptr;
+    if (n_tensors > 0 && sizes == nullptr) return GC_E_INVALID;
+    if (!(density > 0.0) || !(density <= 1.0)) return GC_E_INVALID;
+    if (mode != GC_TOPK && mode != GC_THRESHOLD) return GC_E_INVALID;
+    if (cap_factor == 0.0) cap_factor = 2.0;
+    if (!(cap_factor >= 1.0)) return GC_E_INVALID;
+    if (sample_stride == 0) sample_stride = 64;
+    uint64_t total = 0;
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        total += sizes[t];
+        if (total > 0x7FFFFFFFull) return GC_E_TOO_LARGE;
+    }
+    gc_plan_s* p = new (std::nothrow) gc_plan_s();
+    if (p == nullptr) return GC_E_INVALID;
+    p->device = device; p->mode = mode; p->density = density;
+    p->cap_factor = cap_factor; p->stride = sample_stride; p->T = n_tensors;
+    p->total_n = total;
+    p->desc.resize(n_tensors);
+    uint64_t off = 0, out_off = 0, tile0 = 0;
+    for (uint32_t t = 0; t < n_tensors; ++t) {
+        TensorDesc& d = p->desc[t];
+        uint64_t n = sizes[t];
+        uint64_t k = k_rule(n, density);
+        uint64_t cap = k;
+        if (mode == GC_THRESHOLD) {
+            double c = std::ceil(cap_factor * (double)k);
+            cap = c >= (double)n ? n : (uint64_t)c;
+        }
+        uint64_t lead = off & 3ull;                       // elements before the tensor in its first group
+        uint64_t nt = n == 0 ? 0 : (lead + n + kTile - 1) / kTile;
+        d.off = (uint32_t)off; d.n = (uint32_t)n; d.k = (uint32_t)k; d.cap = (uint32_t)cap;
+        d.out_off = (uint32_t)out_off; d.tile0 = (uint32_t)tile0; d.ntiles = (uint32_t)nt;
+        d.stride = n <= 65536 ? 1u : sample_stride;
+        off += n; out_off += cap; tile0 += nt;
+    }
+    p->total_cap = out_off;
+    p->ntiles = (uint32_t)tile0;
+    p->off_sel = sizeof(WsHeader);
+    p->off_hist = align_up(p->off_sel + sizeof(TensorSel) * (size_t)n_tensors, 256);
+    p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * n_tensors, 256);
+    p->control_bytes = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
+    p->ws_bytes = p->control_bytes;
+
+    if (device < 0) {            // host-only plan: answers queries, refuses compute calls
+        *out = p;
+        return GC_OK;
+    }
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess && n_tensors > 0) {
+        e = cudaMalloc(reinterpret_cast<void**>(&p->d_desc), sizeof(TensorDesc) * (size_t)n_tensors);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(p->d_desc, p->desc.data(), sizeof(TensorDesc) * (size_t)n_tensors,
+                           cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (p->d_desc) cudaFree(p->d_desc);
+        delete p;
+        return GC_E_CUDA;
+    }
+    p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, true>, kBlock);
+    p->grid_compact = p->sm_count * blocks_per_sm(k_compact, kBlock);
+    *out = p;
+    return GC_OK;
+}
+
+int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value) {
+    if (p == nullptr || value == nullptr) return GC_E_INVALID;
+    switch (what) {
+        case GC_Q_N_TENSORS: *value = p->T; return GC_OK;
+        case GC_Q_TOTAL_N: *value = p->total_n; return GC_OK;
+        case GC_Q_TOTAL_CAP: *value = p->total_cap; return GC_OK;
+        case GC_Q_WORKSPACE_BYTES: *value = p->ws_bytes; return GC_OK;
+        case GC_Q_MODE: *value = (uint64_t)p->mode; return GC_OK;
+        case GC_Q_KERNEL_LAUNCHES: *value = p->launches; return GC_OK;
+        default: break;
+    }
+    if (tensor >= p->T) return GC_E_INVALID;
+    const TensorDesc& d = p->desc[tensor];
+    switch (what) {
+        case GC_Q_TENSOR_N: *value = d.n; return GC_OK;
+        case GC_Q_TENSOR_K: *value = d.k; return GC_OK;
+        case GC_Q_TENSOR_CAP: *value = d.cap; return GC_OK;
+        case GC_Q_TENSOR_OFFSET: *value = d.off; return GC_OK;
+        case GC_Q_TENSOR_OUT_OFFSET: *value = d.out_off; return GC_OK;
+        case GC_Q_TENSOR_STRIDE: *value = d.stride; return GC_OK;
+        default: return GC_E_INVALID;
+    }
+}
+
+int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_idx, float* out_val,
+                uint32_t* out_count, void* workspace, void* stream) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (p->total_n == 0) return GC_OK;
+    if (grad == nullptr || residual == nullptr || out_idx == nullptr || out_val == nullptr ||
+        workspace == nullptr)
+        return GC_E_INVALID;
+    if ((reinterpret_cast<uintptr_t>(grad) & 15u) || (reinterpret_cast<uintptr_t>(residual) & 15u) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(out_idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out_val) & 3u))
+        return GC_E_INVALID;
+    if (p->mode != GC_TOPK) return GC_E_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    WsView ws = view(p, workspace);
+    GC_CUDA(p, cudaMemsetAsync(workspace, 0, p->control_bytes, s));
+    ++p->launches;
+    if (out_count != nullptr) {
+        GC_CUDA(p, cudaMemsetAsync(out_count, 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
+        ++p->launches;
+    }
+    const uint32_t nt = p->ntiles;
+    const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
+    const int gc_ = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
+    k_hist<0, true><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws);
+    k_hist<1, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
+    k_hist<2, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
+    k_compact<<<gc_, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, ws, 0);
+    p->launches += 4;
+    GC_CUDA(p, cudaGetLastError());
+    return GC_OK;
+}
+
+int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* idx,
+                             const float* const* val, const uint32_t* const* count,
+                             float* dense_out, int zero_first, void* workspace, void* stream) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (W > GC_MAX_WORKERS) return GC_E_TOO_LARGE;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (p->total_n == 0) return GC_OK;
+    if (dense_out == nullptr || workspace == nullptr) return GC_E_INVALID;
+    if (W > 0 && (idx == nullptr || val == nullptr)) return GC_E_INVALID;
+    for (uint32_t w = 0; w < W; ++w) {
+        if (idx[w] == nullptr || val[w] == nullptr) return GC_E_INVALID;
+        if (count != nullptr && count[w] == nullptr) return GC_E_INVALID;
+    }
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return GC_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    WsView ws = view(p, workspace);
+    if (zero_first) {
+        GC_CUDA(p, cudaMemsetAsync(dense_out, 0, sizeof(float) * (size_t)p->total_n, s));
+        ++p->launches;
+    }
+    if (p->total_cap == 0) return GC_OK;
+    const uint32_t cap = (uint32_t)p->total_cap;
+    const int grid = (int)((cap + 255u) / 256u);
+    for (uint32_t w = 0; w < W; ++w) {
+        k_scatter_add<<<grid, 256, 0, s>>>(p->d_desc, p->T, cap, (uint32_t)p->total_n, idx[w], val[w],
+                                           count ? count[w] : nullptr, dense_out, ws.hdr);
+        ++p->launches;
+    }
+    GC_CUDA(p, cudaGetLastError());
+    return GC_OK;
+}
+
+int gc_last_status(gc_plan_t* p, const void* workspace, void* stream, int32_t* status, uint64_t* detail) {
+    if (p == nullptr || workspace == nullptr || status == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    WsHeader h;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
+    GC_CUDA(p, cudaStreamSynchronize(s));
+    *status = h.status;
+    if (detail) *detail = h.detail;
+    return GC_OK;
+}
+
+int gc_last_cuda_error(const gc_plan_t* p) { return p ? p->last_cuda_error : 0; }
+
+int gc_destroy(gc_plan_t* p) {
+    if (p == nullptr) return GC_OK;
+    int rc = GC_OK;
+    if (p->d_desc) {
+        (void)cudaSetDevice(p->device);
+        if (cudaFree(p->d_desc) != cudaSuccess) { (void)cudaGetLastError(); rc = GC_E_CUDA; }
+    }
+    delete p;
+    return rc;
+}
+
+}  // extern "C"

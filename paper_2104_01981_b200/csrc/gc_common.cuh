@@ -1,0 +1,208 @@
+// Shared device-side definitions of libgc: tensor table, workspace layout, tile geometry,
+// warp/block scan helpers and the ordered-tile prefix exchange ("look-back").
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gc {
+
+// ----------------------------------------------------------------------------- geometry
+constexpr int kBlock = 512;                 // threads per CTA for the streaming kernels
+constexpr int kWarps = kBlock / 32;
+constexpr int kVpt = 4;                     // 128-bit vectors per thread per tile
+constexpr int kTile = kBlock * kVpt * 4;    // 8192 elements per tile
+constexpr int kWarpChunk = 32 * kVpt * 4;   // contiguous elements owned by one warp
+constexpr uint32_t kKeyMask = 0x7FFFFFFFu;
+
+// radix-select levels over the 31-bit magnitude key: 11 + 10 + 10 bits
+constexpr int kLevels = 3;
+__host__ __device__ constexpr int level_bits(int l) { return l == 0 ? 11 : 10; }
+__host__ __device__ constexpr int level_shift(int l) { return l == 0 ? 20 : (l == 1 ? 10 : 0); }
+constexpr int kHistBins = 2048;             // bins reserved per tensor (largest level)
+
+// Bounded waits: a predecessor tile is always already running (tiles are handed out by an
+// atomic ticket), so these limits are a safety net, not a schedule.
+constexpr uint32_t kSpinLimit = 1u << 21;
+
+// ----------------------------------------------------------------------------- tables
+struct TensorDesc {          // one per tensor, immutable, plan-owned device memory
+    uint32_t off;            // first flat index
+    uint32_t n;              // elements
+    uint32_t k;              // entries to keep (top-k) / reference k (threshold)
+    uint32_t cap;            // output capacity
+    uint32_t out_off;        // first output slot
+    uint32_t tile0;          // first tile id
+    uint32_t ntiles;         // tiles of this tensor
+    uint32_t stride;         // threshold mode: sampling stride in 4-element groups
+};
+
+struct TensorSel {           // one per tensor, in the workspace, rewritten every call
+    uint32_t prefix;         // key bits fixed so far by the radix select
+    uint32_t krem;           // entries still to take inside the current prefix bucket
+    uint32_t T;              // k-th largest key (valid after the last level)
+    uint32_t m_eq;           // how many of the entries with key == T are taken
+    uint32_t done[kLevels];  // tiles histogrammed per level
+    uint32_t pad;
+};
+
+struct WsHeader {            // head of the workspace, 256 bytes
+    int32_t status;          // GC_OK / warning / error recorded by kernels
+    uint32_t abort;          // non-zero: a bounded wait gave up, everyone leaves
+    unsigned long long detail;
+    uint32_t ticket[8];      // tile tickets, one per ordered kernel
+    uint32_t reserved[52];
+};
+static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
+
+struct WsView {              // host-computed pointers into the workspace
+    WsHeader* hdr;
+    TensorSel* sel;          // [n_tensors]
+    uint32_t* hist;          // [n_tensors][kHistBins]
+    unsigned long long* tile_state;   // [ntiles]
+};
+
+// ----------------------------------------------------------------------------- small helpers
+__device__ __forceinline__ uint32_t key_of(float a) { return __float_as_uint(a) & kKeyMask; }
+
+__device__ __forceinline__ void record_status(WsHeader* h, int32_t code, unsigned long long detail) {
+    // errors (negative) win over warnings; first writer of a kind keeps its detail
+    int32_t old = atomicCAS(&h->status, 0, code);
+    if (old == 0) { h->detail = detail; return; }
+    if (old > 0 && code < 0) { atomicExch(&h->status, code); h->detail = detail; }
+}
+
+// tensor that owns `tile`: last t with tile0[t] <= tile and ntiles[t] > 0 covering it
+__device__ __forceinline__ uint32_t find_tensor(const TensorDesc* __restrict__ d, uint32_t T, uint32_t tile) {
+    uint32_t lo = 0, hi = T;                 // invariant: answer in [lo, hi)
+    while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(&d[mid].tile0) <= tile) lo = mid; else hi = mid;
+    }
+    // tensors with zero tiles share tile0 with their successor; step back is never needed
+    // because the search keeps the LAST t with tile0 <= tile, which is the one with tiles.
+    return lo;
+}
+
+struct TileGeom { uint32_t base, lo, hi; };  // aligned start, first and one-past-last valid flat index
+__device__ __forceinline__ TileGeom tile_geom(const TensorDesc& d, uint32_t tile_in_tensor) {
+    TileGeom g;
+    g.base = (d.off & ~3u) + tile_in_tensor * (uint32_t)kTile;
+    g.lo = max(d.off, g.base);
+    uint32_t end = d.off + d.n;
+    g.hi = min(end, g.base + (uint32_t)kTile);
+    return g;
+}
+
+// flat index of element 0 of this thread's j-th vector inside a tile
+__device__ __forceinline__ uint32_t vec_index(uint32_t base, int warp, int lane, int j) {
+    return base + warp * kWarpChunk + (j * 32 + lane) * 4;
+}
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_incl_scan64(unsigned long long v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
+}
+
+// Per-thread counts c[j] (0..4) for its kVpt vectors -> exclusive rank of each vector within
+// the warp's chunk in element order (vector j, then lane), plus the warp total.
+// Counts are packed as 8-bit fields (a field never exceeds 32*4 = 128).
+__device__ __forceinline__ void warp_rank(const uint32_t (&c)[kVpt], int lane,
+                                          uint32_t (&rank)[kVpt], uint32_t& total) {
+    uint32_t packed = 0;
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) packed |= c[j] << (8 * j);
+    uint32_t incl = warp_incl_scan(packed, lane);
+    uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    uint32_t excl = incl - packed;
+    uint32_t run = 0;
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) {
+        rank[j] = run + ((excl >> (8 * j)) & 0xFFu);
+        run += (tot >> (8 * j)) & 0xFFu;
+    }
+    total = run;
+}
+
+// ----------------------------------------------------------------------------- ordered tiles
+// Tile descriptors: bits 63..62 = flag (0 none, 1 aggregate of this tile, 2 inclusive prefix
+// up to and including this tile), bits 61..0 = value.  Flag and value travel in one 64-bit
+// word, so a relaxed load sees a consistent pair.
+constexpr unsigned long long kFlagAgg = 1ull << 62;
+constexpr unsigned long long kFlagPre = 2ull << 62;
+constexpr unsigned long long kValMask = (1ull << 62) - 1;
+
+__device__ __forceinline__ unsigned long long ld_state(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_state(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
+}
+
+// Called by all 32 lanes of one warp.  Publishes this tile's aggregate, walks back over the
+// predecessor tiles of the same tensor until an inclusive prefix is met, publishes this
+// tile's inclusive prefix and returns the exclusive one.  `ok` is cleared if a wait ran out
+// (status GC_E_TIMEOUT recorded, abort raised).
+__device__ __forceinline__ unsigned long long lookback(unsigned long long* state, uint32_t tile,
+                                                       uint32_t first_tile, unsigned long long agg,
+                                                       int lane, WsHeader* hdr, bool& ok) {
+    ok = true;
+    if (tile == first_tile) {
+        if (lane == 0) st_state(state + tile, kFlagPre | agg);
+        return 0ull;
+    }
+    if (lane == 0) st_state(state + tile, kFlagAgg | agg);
+    unsigned long long excl = 0;
+    long long base = (long long)tile - 1;
+    while (true) {
+        long long p = base - lane;
+        unsigned long long v = kFlagPre;                 // before the tensor's first tile: prefix 0
+        bool timed_out = false;
+        if (p >= (long long)first_tile) {
+            uint32_t spins = 0;
+            v = ld_state(state + p);
+            while ((v >> 62) == 0) {
+                if (++spins > kSpinLimit) { timed_out = true; break; }
+                if (spins > 16) __nanosleep(spins > 1024 ? 200 : 40);
+                if ((spins & 1023u) == 0 && *(volatile uint32_t*)&hdr->abort) { timed_out = true; break; }
+                v = ld_state(state + p);
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, timed_out)) {
+            if (lane == 0) {
+                record_status(hdr, -5 /*GC_E_TIMEOUT*/, tile);
+                atomicExch(&hdr->abort, 1u);
+            }
+            ok = false;
+            return 0ull;
+        }
+        unsigned pmask = __ballot_sync(0xFFFFFFFFu, (v >> 62) == 2);
+        int first_p = pmask ? (__ffs(pmask) - 1) : 32;
+        unsigned long long contrib = (lane <= first_p) ? (v & kValMask) : 0ull;
+        excl += warp_sum64(contrib);
+        if (pmask) break;
+        base -= 32;
+    }
+    if (lane == 0) st_state(state + tile, kFlagPre | ((excl + agg) & kValMask));
+    return excl;
+}
+
+}  // namespace gc

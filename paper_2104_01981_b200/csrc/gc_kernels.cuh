@@ -1,0 +1,328 @@
+// Kernels of the exact multi-pass path: fold + radix-select histograms over the magnitude
+// key, ordered compaction with residual zeroing, and the sparse decode.
+#pragma once
+#include "gc_common.cuh"
+
+namespace gc {
+
+// ----------------------------------------------------------------------------- tile I/O
+struct Tile {
+    float a[kVpt][4];
+    uint32_t valid;          // bit j*4+e set: element e of vector j belongs to this tile
+};
+
+// Loads the thread's vectors of one tile.  FOLD: a = g + r (one rounded fp32 add) and a is
+// stored to r; otherwise a is read from r.  Interior vectors use 128-bit accesses; vectors
+// that straddle the tensor's first or last element fall back to guarded scalar accesses.
+template <bool FOLD>
+__device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __restrict__ r,
+                                          const TileGeom& tg, int warp, int lane, Tile& t) {
+    t.valid = 0;
+    float4 gv[kVpt], rv[kVpt];
+    bool full[kVpt];
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) {
+        uint32_t f0 = vec_index(tg.base, warp, lane, j);
+        full[j] = (f0 >= tg.lo) && (f0 + 4 <= tg.hi);
+        if (full[j]) {
+            rv[j] = *reinterpret_cast<const float4*>(r + f0);
+            if (FOLD) gv[j] = __ldg(reinterpret_cast<const float4*>(g + f0));
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) {
+        uint32_t f0 = vec_index(tg.base, warp, lane, j);
+        if (full[j]) {
+            if (FOLD) {
+                float4 s;
+                s.x = __fadd_rn(gv[j].x, rv[j].x); s.y = __fadd_rn(gv[j].y, rv[j].y);
+                s.z = __fadd_rn(gv[j].z, rv[j].z); s.w = __fadd_rn(gv[j].w, rv[j].w);
+                *reinterpret_cast<float4*>(r + f0) = s;
+                rv[j] = s;
+            }
+            t.a[j][0] = rv[j].x; t.a[j][1] = rv[j].y; t.a[j][2] = rv[j].z; t.a[j][3] = rv[j].w;
+            t.valid |= 0xFu << (4 * j);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                uint32_t f = f0 + e;
+                float v = 0.0f;
+                if (f >= tg.lo && f < tg.hi) {
+                    v = r[f];
+                    if (FOLD) { v = __fadd_rn(__ldg(g + f), v); r[f] = v; }
+                    t.valid |= 1u << (4 * j + e);
+                }
+                t.a[j][e] = v;
+            }
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------- block scans
+// Exclusive scan of one value per warp (kWarps values) by warp 0; result in smem.
+__device__ __forceinline__ void scan_warp_totals(uint32_t* s_tot, uint32_t* s_excl, uint32_t* s_sum,
+                                                 int warp, int lane) {
+    if (warp == 0) {
+        uint32_t v = lane < kWarps ? s_tot[lane] : 0u;
+        uint32_t inc = warp_incl_scan(v, lane);
+        if (lane < kWarps) s_excl[lane] = inc - v;
+        if (lane == 31) *s_sum = inc;
+    }
+}
+
+// ----------------------------------------------------------------------------- select step
+// Run by the CTA that completes the last tile of a tensor at one level: scans that tensor's
+// histogram from the top bin down, finds the bin that holds the krem-th largest key, and
+// clears the histogram for the next level.  NB = bins at this level.
+template <int LEVEL>
+__device__ void select_step(const TensorDesc* __restrict__ desc, const WsView& ws, uint32_t t,
+                            uint32_t* s_scratch /* >= kWarps + 4 words */) {
+    constexpr int NB = 1 << level_bits(LEVEL);
+    constexpr int BPT = (NB + kBlock - 1) / kBlock;          // bins per thread
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t* hist = ws.hist + (size_t)t * kHistBins;
+    TensorSel* sel = ws.sel + t;
+    const uint32_t krem = (LEVEL == 0) ? desc[t].k : sel->krem;
+    const uint32_t prefix = (LEVEL == 0) ? 0u : sel->prefix;
+    // thread `tid` owns the bins [top - BPT*tid - BPT + 1 .. top - BPT*tid], i.e. it walks
+    // the histogram from the largest key downwards
+    uint32_t c[BPT];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        int b = NB - 1 - (tid * BPT + i);
+        c[i] = (b >= 0) ? __ldcg(hist + b) : 0u;
+        if (b >= 0) hist[b] = 0u;
+        sum += c[i];
+    }
+    uint32_t inc = warp_incl_scan(sum, lane);
+    if (lane == 31) s_scratch[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t v = lane < kWarps ? s_scratch[lane] : 0u;
+        uint32_t wi = warp_incl_scan(v, lane);
+        if (lane < kWarps) s_scratch[lane] = wi - v;
+    }
+    __syncthreads();
+    uint32_t above = s_scratch[warp] + inc - sum;            // keys in bins above this thread's
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        int b = NB - 1 - (tid * BPT + i);
+        if (b >= 0 && above < krem && krem <= above + c[i]) {
+            uint32_t np = (prefix << level_bits(LEVEL)) | (uint32_t)b;
+            sel->prefix = np;
+            sel->krem = krem - above;
+            if (LEVEL == kLevels - 1) { sel->T = np; sel->m_eq = krem - above; }
+        }
+        above += c[i];
+    }
+    __syncthreads();
+}
+
+// ----------------------------------------------------------------------------- histogram pass
+// One radix-select level over all tensors.  CTAs take contiguous runs of tiles, keep a
+// shared-memory histogram while the tensor stays the same, flush it with global atomics when
+// it changes, and the CTA that completes a tensor's last tile runs the select step.
+//   LEVEL 0, FOLD: reads g and r, writes a = g + r into r (12 bytes per element)
+//   otherwise:     reads a from r (4 bytes per element); only keys under the prefix count
+template <int LEVEL, bool FOLD>
+__global__ void __launch_bounds__(kBlock)
+k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+       const float* __restrict__ g, float* __restrict__ r, WsView ws) {
+    constexpr int NB = 1 << level_bits(LEVEL);
+    constexpr int SH = level_shift(LEVEL);
+    __shared__ uint32_t s_hist[NB];
+    __shared__ uint32_t s_scratch[kWarps + 4];
+    __shared__ uint32_t s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t first = blockIdx.x * per;
+    const uint32_t last = min(ntiles, first + per);
+    if (first >= last) return;
+    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    __syncthreads();
+
+    uint32_t t = find_tensor(desc, T, first);
+    TensorDesc d = desc[t];
+    uint32_t prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
+    uint32_t tiles_here = 0;
+
+    auto flush = [&]() {
+        __syncthreads();
+        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
+        for (int b = tid; b < NB; b += kBlock) {
+            uint32_t c = s_hist[b];
+            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
+            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            select_step<LEVEL>(desc, ws, t, s_scratch);
+        }
+        tiles_here = 0;
+    };
+
+    for (uint32_t tile = first; tile < last; ++tile) {
+        if (tile >= d.tile0 + d.ntiles) {
+            flush();
+            t = find_tensor(desc, T, tile);
+            d = desc[t];
+            prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
+        }
+        TileGeom tg = tile_geom(d, tile - d.tile0);
+        Tile tl;
+        load_tile<FOLD>(g, r, tg, warp, lane, tl);
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                uint32_t key = key_of(tl.a[j][e]);
+                bool in = (tl.valid >> (4 * j + e)) & 1u;
+                if (LEVEL > 0) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
+                if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+            }
+        }
+        ++tiles_here;
+    }
+    flush();
+}
+
+// ----------------------------------------------------------------------------- compaction
+// Ordered emission of the selected entries.  Tiles are handed out by an atomic ticket so
+// that every predecessor of a running tile is itself running or finished; the exclusive
+// counts (keys above T, keys equal to T) of a tile within its tensor come from the look-back
+// exchange.  An element is sent iff key > T, or key == T and fewer than m_eq equal keys
+// precede it in the tensor.  Sent elements are written as (flat index, value) at their rank
+// and zeroed in the residual.
+__global__ void __launch_bounds__(kBlock)
+k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+          float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+          uint32_t* __restrict__ out_count, WsView ws, int ticket_slot) {
+    __shared__ uint32_t s_tile;
+    __shared__ uint32_t s_gt_tot[kWarps], s_eq_tot[kWarps], s_gt_ex[kWarps], s_eq_ex[kWarps];
+    __shared__ uint32_t s_gt_sum, s_eq_sum;
+    __shared__ unsigned long long s_excl;
+    __shared__ int s_ok;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    while (true) {
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t tk = atomicAdd(&ws.hdr->ticket[ticket_slot], 1u);
+            if (*(volatile uint32_t*)&ws.hdr->abort) tk = 0xFFFFFFFFu;
+            s_tile = tk;
+        }
+        __syncthreads();
+        const uint32_t tile = s_tile;
+        if (tile >= ntiles) break;
+        const uint32_t t = find_tensor(desc, T, tile);
+        const TensorDesc d = desc[t];
+        const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
+        const TileGeom tg = tile_geom(d, tile - d.tile0);
+        Tile tl;
+        load_tile<false>(nullptr, r, tg, warp, lane, tl);
+
+        uint32_t cg[kVpt], ce[kVpt], gtm = 0, eqm = 0;
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            cg[j] = 0; ce[j] = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                uint32_t key = key_of(tl.a[j][e]);
+                bool v = (tl.valid >> (4 * j + e)) & 1u;
+                bool gt = v && key > Tkey, eq = v && key == Tkey;
+                cg[j] += gt; ce[j] += eq;
+                gtm |= (uint32_t)gt << (4 * j + e);
+                eqm |= (uint32_t)eq << (4 * j + e);
+            }
+        }
+        uint32_t rg[kVpt], re[kVpt], wg, we;
+        warp_rank(cg, lane, rg, wg);
+        warp_rank(ce, lane, re, we);
+        if (lane == 0) { s_gt_tot[warp] = wg; s_eq_tot[warp] = we; }
+        __syncthreads();
+        scan_warp_totals(s_gt_tot, s_gt_ex, &s_gt_sum, warp, lane);
+        if (warp == 1) {
+            uint32_t v = lane < kWarps ? s_eq_tot[lane] : 0u;
+            uint32_t inc = warp_incl_scan(v, lane);
+            if (lane < kWarps) s_eq_ex[lane] = inc - v;
+            if (lane == 31) s_eq_sum = inc;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long agg = ((unsigned long long)s_gt_sum << 31) | (unsigned long long)s_eq_sum;
+            bool ok;
+            unsigned long long ex = lookback(ws.tile_state, tile, d.tile0, agg, lane, ws.hdr, ok);
+            if (lane == 0) { s_excl = ex; s_ok = ok ? 1 : 0; }
+        }
+        __syncthreads();
+        if (!s_ok) break;
+        const uint32_t gt_before = (uint32_t)(s_excl >> 31) + s_gt_ex[warp];
+        const uint32_t eq_before = (uint32_t)(s_excl & 0x7FFFFFFFull) + s_eq_ex[warp];
+        if ((gtm | eqm) != 0u) {
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                uint32_t gpos = gt_before + rg[j], epos = eq_before + re[j];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    bool gt = (gtm >> (4 * j + e)) & 1u, eq = (eqm >> (4 * j + e)) & 1u;
+                    if (gt || (eq && epos < m_eq)) {
+                        uint32_t slot = gpos + min(epos, m_eq);
+                        uint32_t f = vec_index(tg.base, warp, lane, j) + e;
+                        if (slot >= d.cap) {          // cannot happen with a correct select; never write outside
+                            record_status(ws.hdr, -1 /*GC_E_INVALID*/, f);
+                            continue;
+                        }
+                        uint32_t pos = d.out_off + slot;
+                        out_idx[pos] = f;
+                        out_val[pos] = tl.a[j][e];
+                        r[f] = 0.0f;
+                    }
+                    gpos += gt; epos += eq;
+                }
+            }
+        }
+        if (out_count != nullptr && tile == d.tile0 && tid == 0) {
+            out_count[t] = d.k;
+            out_count[T + t] = d.k;
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------- decode
+struct DecodeArgs {
+    const uint32_t* idx[64];
+    const float* val[64];
+    const uint32_t* count[64];
+};
+
+// One sparse set added into the dense buffer.  Indices of one set are distinct, so plain
+// read-modify-write is race free; sets are applied by consecutive launches in worker order,
+// which fixes the order of the fp32 additions per element.
+__global__ void __launch_bounds__(256)
+k_scatter_add(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t total_cap, uint32_t total_n,
+              const uint32_t* __restrict__ idx, const float* __restrict__ val,
+              const uint32_t* __restrict__ count, float* __restrict__ out, WsHeader* hdr) {
+    uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= total_cap) return;
+    if (count != nullptr) {
+        // slot j belongs to the last tensor whose out_off <= j; it is live iff below the count
+        uint32_t lo = 0, hi = T;
+        while (hi - lo > 1) {
+            uint32_t mid = (lo + hi) >> 1;
+            if (__ldg(&desc[mid].out_off) <= j) lo = mid; else hi = mid;
+        }
+        if (j - __ldg(&desc[lo].out_off) >= __ldg(count + lo)) return;
+    }
+    uint32_t i = __ldg(idx + j);
+    if (i >= total_n) { record_status(hdr, -1 /*GC_E_INVALID*/, j); return; }
+    out[i] = __fadd_rn(out[i], __ldg(val + j));
+}
+
+}  // namespace gc

@@ -1,0 +1,89 @@
+"""The C-ABI library loads, exports every symbol the header declares, and its host-side
+logic (k rule, offsets, capacities, argument checks) is right.  No GPU needed."""
+import ctypes
+import math
+import os
+import re
+
+import pytest
+
+import oracle
+from paper_2104_01981_b200 import api, build, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return api.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "gc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gc_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    syms = declared_symbols()
+    assert {"gc_plan", "gc_compress", "gc_decompress_accumulate", "gc_destroy"} <= set(syms)
+    for s in syms:
+        assert hasattr(lib, s), s
+    assert lib.gc_version() >= 1
+
+
+def test_host_plan_k_offsets_match_the_oracle_rule(lib):
+    for cfg in (0, 1, 2, 4):
+        w = synth.workload(cfg)
+        p = api.Plan(w.sizes, w.density, device=-1)
+        ks = p.tensor_k()
+        assert ks == [oracle.k_from_density(n, w.density) for n in w.sizes]
+        offs = p.tensor_out_offset()
+        assert offs == [sum(ks[:t]) for t in range(len(ks))]
+        assert p.total_n == w.total_n and p.total_cap == sum(ks)
+        assert p.workspace_bytes % 256 == 0
+        p.destroy()
+    p = api.Plan([1 << 20], 0.01, device=-1)
+    assert p.tensor_k() == [10486]
+
+
+def test_threshold_plan_capacity_and_stride(lib):
+    sizes = [64, 65536, 65537, 1_000_000]
+    p = api.Plan(sizes, 0.001, mode=api.GC_THRESHOLD, device=-1)
+    ks = [oracle.k_from_density(n, 0.001) for n in sizes]
+    assert p.tensor_cap() == [min(n, math.ceil(2.0 * k)) for n, k in zip(sizes, ks)]
+    assert [p.query(api.GC_Q_TENSOR_STRIDE, t) for t in range(4)] == \
+        [oracle.effective_stride(n, 64) for n in sizes]
+    p2 = api.Plan(sizes, 0.001, mode=api.GC_THRESHOLD, device=-1, sample_stride=16, cap_factor=1.5)
+    assert p2.tensor_cap() == [min(n, math.ceil(1.5 * k)) for n, k in zip(sizes, ks)]
+    assert p2.query(api.GC_Q_TENSOR_STRIDE, 3) == 16
+
+
+def test_plan_rejects_bad_arguments(lib):
+    for density in (0.0, -0.1, 1.5, float("nan")):
+        with pytest.raises(api.GcError) as e:
+            api.Plan([10], density, device=-1)
+        assert e.value.code == api.GC_E_INVALID
+    with pytest.raises(api.GcError) as e:
+        api.Plan([1 << 30, 1 << 30], 0.01, device=-1)
+    assert e.value.code == api.GC_E_TOO_LARGE
+    with pytest.raises(api.GcError):
+        api.Plan([10], 0.5, mode=7, device=-1)
+    with pytest.raises(api.GcError):
+        api.Plan([10], 0.5, mode=api.GC_THRESHOLD, device=-1, cap_factor=0.5)
+
+
+def test_empty_and_zero_sized_tensors(lib):
+    p = api.Plan([], 0.5, device=-1)
+    assert p.total_n == 0 and p.total_cap == 0
+    p = api.Plan([0, 5, 0], 0.5, device=-1)
+    assert p.tensor_k() == [0, 3, 0] and p.tensor_out_offset() == [0, 0, 3]
+    with pytest.raises(api.GcError):
+        p.query(api.GC_Q_TENSOR_K, 3)
+
+
+def test_host_only_plan_refuses_compute(lib):
+    p = api.Plan([16], 0.5, device=-1)
+    assert p.compress_ptr(16, 16, 16, 16, None, 256, 0) == api.GC_E_UNSUPPORTED
+    assert lib.gc_destroy(None) == api.GC_OK

@@ -1,0 +1,125 @@
+"""GPU parity of gc_decompress_accumulate against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_01981_b200 import api, build, synth
+from helpers import GpuWorker, bits, to_np_u32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    api.lib()
+
+
+def run_workers(sizes, density, W, seed, steps=1, dist_scale=None):
+    """W workers compress `steps` times on GPU; returns plan, workers, last gradients (cpu)."""
+    plan = api.Plan(sizes, density, device=0)
+    workers = [GpuWorker(plan) for _ in range(W)]
+    n = plan.total_n
+    grads = []
+    for w, wk in enumerate(workers):
+        for s in range(steps):
+            gen = torch.Generator().manual_seed(seed + 1000 * w + s)
+            g = torch.randn(n, generator=gen) * (dist_scale[w] if dist_scale else 1.0)
+            wk.step(g.cuda())
+        grads.append(g)
+    return plan, workers, grads
+
+
+def oracle_pairs(workers, plan):
+    tot = plan.total_cap
+    return [(to_np_u32(w.idx[:tot]).copy(), w.val[:tot].cpu().numpy().copy()) for w in workers]
+
+
+@pytest.mark.parametrize("W", [1, 2, 8])
+@pytest.mark.parametrize("sizes,density", [([100_000], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02),
+                                           ([40_000], 0.5)])
+def test_decode_matches_oracle_bitwise(W, sizes, density):
+    plan, workers, _ = run_workers(sizes, density, W, seed=3, steps=2,
+                                   dist_scale=[10.0 ** (w % 4 - 2) for w in range(W)])
+    n = plan.total_n
+    out = torch.full((n,), 7.0, device="cuda")
+    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out, True,
+                               workers[0].ws)
+    want = oracle.decode_accumulate(oracle_pairs(workers, plan), np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
+    # with explicit count arrays the result is the same
+    out2 = torch.full((n,), 7.0, device="cuda")
+    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers],
+                               [w.count for w in workers], out2, True, workers[0].ws)
+    assert torch.equal(out, out2)
+    # accumulate mode adds on top of the existing content
+    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out2, False,
+                               workers[0].ws)
+    want2 = oracle.decode_accumulate(oracle_pairs(workers, plan), want.copy(), False)
+    assert np.array_equal(to_np_u32(out2), bits(want2))
+    st, _ = plan.last_status(workers[0].ws)
+    assert st == api.GC_OK
+
+
+def test_density_one_reproduces_the_dense_sum():
+    sizes, W = [9, 30_000, 4097], 5
+    plan, workers, grads = run_workers(sizes, 1.0, W, seed=11, dist_scale=[1.0, 1e3, 1e-3, 50.0, 0.1])
+    n = plan.total_n
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out, True,
+                               workers[0].ws)
+    dense = np.zeros(n, np.float32)
+    for g in grads:
+        dense = (dense + g.numpy()).astype(np.float32)
+    assert np.array_equal(to_np_u32(out), bits(dense))
+    for w in workers:
+        assert not w.residual.any()
+
+
+def test_worker_order_is_observable_and_fixed():
+    plan = api.Plan([8], 1.0, device=0)
+    ws = plan.alloc_workspace()
+    idx = torch.arange(8, dtype=torch.int32, device="cuda")
+    a = torch.full((8,), 1e8, device="cuda")
+    b = torch.ones(8, device="cuda")
+    out = torch.empty(8, device="cuda")
+    plan.decompress_accumulate([idx, idx, idx], [a, b, -a], None, out, True, ws)
+    assert out.tolist() == [0.0] * 8
+    plan.decompress_accumulate([idx, idx, idx], [a, -a, b], None, out, True, ws)
+    assert out.tolist() == [1.0] * 8
+
+
+def test_out_of_range_index_is_skipped_and_reported():
+    plan = api.Plan([100], 0.04, device=0)          # k = 4
+    ws = plan.alloc_workspace()
+    idx = torch.tensor([1, 50, 100, 99], dtype=torch.int32, device="cuda")
+    val = torch.ones(4, device="cuda")
+    out = torch.empty(100, device="cuda")
+    plan.decompress_accumulate([idx], [val], None, out, True, ws)
+    st, det = plan.last_status(ws)
+    assert st == api.GC_E_INVALID and det == 2
+    assert out.sum().item() == 3.0
+
+
+def test_config4_eight_resnet_workers_decode():
+    w = synth.workload(3)
+    plan = api.Plan(w.sizes, w.density, device=0)
+    ks = plan.tensor_k()
+    n = plan.total_n
+    workers = [GpuWorker(plan) for _ in range(w.workers)]
+    pairs = []
+    for i, wk in enumerate(workers):
+        g = synth.gradient(w, i, 0, device="cuda")
+        wk.step(g)
+        r = np.zeros(n, np.float32)
+        oi, ov = oracle.topk_compress_tensors(w.sizes, ks, g.cpu().numpy(), r)
+        assert np.array_equal(to_np_u32(wk.idx[:plan.total_cap]), oi)
+        assert np.array_equal(to_np_u32(wk.val[:plan.total_cap]), bits(ov))
+        assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r))
+        pairs.append((oi, ov))
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([x.idx for x in workers], [x.val for x in workers], None, out, True,
+                               workers[0].ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))

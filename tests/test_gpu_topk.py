@@ -1,0 +1,99 @@
+"""GPU parity of gc_compress (top-k mode) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_01981_b200 import api, build, synth
+from helpers import GpuWorker, bits, check_topk_against_oracle, to_np_u32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    api.lib()
+
+
+def randn(n, seed, scale=1.0):
+    gen = torch.Generator().manual_seed(seed)
+    return torch.randn(n, generator=gen) * scale
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 31, 32, 33, 1023, 1024, 1025, 8191, 8192, 8193, 8196,
+                               16384, 16385, 100_003, (1 << 20) - 1, (1 << 20) + 1])
+@pytest.mark.parametrize("density", [1e-9, 0.01, 1.0])
+def test_single_tensor_sizes_and_extreme_k(n, density):
+    grads = [randn(n, 17 * n + s) for s in range(2)]
+    check_topk_against_oracle([n], density, grads, r0=randn(n, 5 * n + 1, 0.3))
+
+
+def test_many_ragged_tensors_misaligned_offsets():
+    sizes = [5, 3, 1000, 7, 8193, 64, 1, 0, 2, 16384, 9, 70001, 0, 6]
+    n = sum(sizes)
+    grads = [randn(n, 100 + s) for s in range(3)]
+    for density in (0.001, 0.05, 0.5):
+        check_topk_against_oracle(sizes, density, grads)
+
+
+def test_tie_stress_quantised_values():
+    n = 300_000
+    grads = [synth.quantised_gradient(n, 40 + s) for s in range(3)]
+    for density in (0.01, 0.2):
+        check_topk_against_oracle([n], density, grads)
+        check_topk_against_oracle([100_000, 100_000, 100_000], density, grads)
+
+
+def test_degenerate_values():
+    n = 20_000
+    for g in (torch.zeros(n), torch.full((n,), -2.5), torch.cat([torch.ones(n // 2), -torch.ones(n // 2)])):
+        check_topk_against_oracle([n], 0.01, [g, g])
+    g = randn(n, 9)
+    g[::7] = float("inf")
+    g[3::11] = float("nan")
+    g[5::13] = -0.0
+    g[1::17] = 1e-42                  # denormal
+    check_topk_against_oracle([n], 0.05, [g])
+
+
+def test_config1_three_steps_error_feedback():
+    w = synth.workload(0)
+    grads = [synth.gradient(w, 0, s, device="cuda") for s in range(w.steps)]
+    check_topk_against_oracle(w.sizes, w.density, grads)
+
+
+def test_config2_resnet50_layerwise():
+    w = synth.workload(1)
+    grads = [synth.gradient(w, 0, s, device="cuda") for s in range(4)]
+    check_topk_against_oracle(w.sizes, w.density, grads)
+
+
+def test_config3_bert_full_size():
+    w = synth.workload(2)
+    grads = [synth.gradient(w, 0, s, device="cuda") for s in range(2)]
+    check_topk_against_oracle(w.sizes, w.density, grads)
+
+
+def test_config5_gpt2_medium_full_size_two_workers():
+    w = synth.workload(4)
+    for worker in (0, 15):
+        grads = [synth.gradient(w, worker, 0, device="cuda")]
+        check_topk_against_oracle(w.sizes, w.density, grads)
+        torch.cuda.empty_cache()
+
+
+def test_rejects_misaligned_and_null_buffers():
+    plan = api.Plan([1024], 0.1, device=0)
+    wk = GpuWorker(plan)
+    g = torch.zeros(1028, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    base = dict(grad=g.data_ptr(), residual=wk.residual.data_ptr(), out_idx=wk.idx.data_ptr(),
+                out_val=wk.val.data_ptr(), out_count=None, workspace=wk.ws.data_ptr(), stream=s)
+    assert plan.compress_ptr(**base) == api.GC_OK
+    for key, bad in (("grad", g.data_ptr() + 4), ("residual", 0), ("workspace", wk.ws.data_ptr() + 16),
+                     ("out_idx", 0)):
+        args = dict(base)
+        args[key] = bad
+        assert plan.compress_ptr(**args) == api.GC_E_INVALID
+    torch.cuda.synchronize()
