@@ -164,6 +164,44 @@ int gc_decompress_accumulate(gc_plan_t *plan, uint32_t W,
 int gc_last_status(gc_plan_t *plan, const void *workspace, void *stream,
                    int32_t *status, uint64_t *detail);
 
+/*
+ * gc_compress_host -- gc_compress for a gradient that lives in HOST memory, with the
+ * compressed pairs returned to HOST memory (what a worker would hand to its network stack).
+ * Enqueues, on the stream: copy host_grad -> grad_staging, gc_compress, copy the pairs
+ * device -> host.  No counterpart in the source paper; it exists so that end-to-end
+ * throughput including both PCIe copies can be measured through this ABI.
+ *
+ *   host_grad     host (pinned for a truly asynchronous copy), fp32[total_n]
+ *   grad_staging  device, fp32[total_n], 16-byte aligned; overwritten
+ *   host_idx/val  host (pinned recommended), uint32/fp32[total_cap]; valid after the stream drains
+ *   the other arguments are those of gc_compress
+ * Bytes moved per call: 4*total_n host->device, 8*total_cap device->host.
+ */
+int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_staging, float *residual,
+                     uint32_t *out_idx, float *out_val, uint32_t *out_count,
+                     uint32_t *host_idx, float *host_val, void *workspace, void *stream);
+
+/*
+ * Per-kernel timing with CUDA events (a measuring aid; not part of the hot path).
+ * gc_profile_enable(plan, max_records): from now on every kernel or memset the library
+ * enqueues for this plan is bracketed by a pair of CUDA events recorded on the same stream,
+ * up to max_records launches (later ones run untimed).  max_records = 0 switches timing off
+ * and frees the events.  gc_profile_read synchronises the device, sums the elapsed time and
+ * the launches per kernel id (GC_K_*; arrays of GC_K_COUNT entries) and clears the records.
+ */
+#define GC_K_CLEAR_CTRL     0   /* memset of the workspace control block                  */
+#define GC_K_FOLD_HIST      1   /* fold + level-0 histogram (reads g, r; writes r)        */
+#define GC_K_HIST_REFINE    2   /* level-1 / level-2 histogram over r                      */
+#define GC_K_COMPACT        3   /* ordered compaction + residual zeroing                   */
+#define GC_K_DECODE_CLEAR   4   /* memset of the dense output                              */
+#define GC_K_DECODE_ADD     5   /* sparse set added into the dense output                  */
+#define GC_K_COPY           6   /* host<->device copies of gc_compress_host                */
+#define GC_K_OTHER          7
+#define GC_K_COUNT         16
+int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
+int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);
+const char *gc_kernel_name(int kernel_id);
+
 /* gc_last_cuda_error -- host; the cudaError_t value of the most recent failed runtime call
  * made on behalf of this plan (0 if none). */
 int gc_last_cuda_error(const gc_plan_t *plan);

@@ -20,6 +20,7 @@ GC_OK, GC_E_INVALID, GC_E_UNSUPPORTED, GC_E_CUDA, GC_E_TOO_LARGE, GC_E_TIMEOUT =
 GC_W_TRUNCATED = 1
 GC_TOPK, GC_THRESHOLD = 0, 1
 GC_MAX_WORKERS = 64
+GC_K_COUNT = 16
 (GC_Q_N_TENSORS, GC_Q_TOTAL_N, GC_Q_TOTAL_CAP, GC_Q_WORKSPACE_BYTES, GC_Q_TENSOR_N, GC_Q_TENSOR_K,
  GC_Q_TENSOR_CAP, GC_Q_TENSOR_OFFSET, GC_Q_TENSOR_OUT_OFFSET, GC_Q_TENSOR_STRIDE, GC_Q_MODE,
  GC_Q_KERNEL_LAUNCHES) = range(12)
@@ -58,6 +59,14 @@ def lib() -> ctypes.CDLL:
         L.gc_decompress_accumulate.argtypes = [vp, u32, vp, vp, vp, vp, i32, vp, vp]
         L.gc_last_status.restype = i32
         L.gc_last_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(u64)]
+        L.gc_compress_host.restype = i32
+        L.gc_compress_host.argtypes = [vp] * 11
+        L.gc_profile_enable.restype = i32
+        L.gc_profile_enable.argtypes = [vp, u32]
+        L.gc_profile_read.restype = i32
+        L.gc_profile_read.argtypes = [vp, vp, vp]
+        L.gc_kernel_name.restype = ctypes.c_char_p
+        L.gc_kernel_name.argtypes = [i32]
         L.gc_last_cuda_error.restype = i32
         L.gc_last_cuda_error.argtypes = [vp]
         L.gc_destroy.restype = i32
@@ -138,6 +147,38 @@ class Plan:
                      workspace: int, stream: int) -> int:
         """Raw-address form of ``compress`` (host or device addresses are passed through as is)."""
         return lib().gc_compress(self._h, grad, residual, out_idx, out_val, out_count, workspace, stream)
+
+    # --- gc_compress_host
+    def compress_host(self, host_grad: torch.Tensor, grad_staging: torch.Tensor, residual: torch.Tensor,
+                      out_idx: torch.Tensor, out_val: torch.Tensor, out_count: Optional[torch.Tensor],
+                      host_idx: torch.Tensor, host_val: torch.Tensor, workspace: torch.Tensor,
+                      stream=None) -> int:
+        assert not host_grad.is_cuda and not host_idx.is_cuda and not host_val.is_cuda
+        rc = lib().gc_compress_host(self._h, _ptr(host_grad), _ptr(grad_staging), _ptr(residual),
+                                    _ptr(out_idx), _ptr(out_val), _ptr(out_count), _ptr(host_idx),
+                                    _ptr(host_val), _ptr(workspace), _stream_handle(stream))
+        if rc < 0:
+            raise GcError("gc_compress_host", rc)
+        return rc
+
+    # --- gc_profile_enable / gc_profile_read
+    def profile_enable(self, max_records: int) -> None:
+        rc = lib().gc_profile_enable(self._h, max_records)
+        if rc < 0:
+            raise GcError("gc_profile_enable", rc)
+
+    def profile_read(self):
+        """{kernel name: (total ms, launches)} since the last read; synchronises the device."""
+        ms = (ctypes.c_float * GC_K_COUNT)()
+        cnt = (ctypes.c_uint32 * GC_K_COUNT)()
+        rc = lib().gc_profile_read(self._h, ms, cnt)
+        if rc < 0:
+            raise GcError("gc_profile_read", rc)
+        out = {}
+        for i in range(GC_K_COUNT):
+            if cnt[i]:
+                out[lib().gc_kernel_name(i).decode()] = (float(ms[i]), int(cnt[i]))
+        return out
 
     # --- gc_decompress_accumulate
     def decompress_accumulate(self, idx: Sequence[torch.Tensor], val: Sequence[torch.Tensor],

@@ -28,6 +28,10 @@ struct gc_plan_s {
     int grid_hist = 0, grid_compact = 0;
     unsigned long long launches = 0;
     int last_cuda_error = 0;
+    // optional per-kernel event timing
+    struct Rec { cudaEvent_t a, b; int id; };
+    std::vector<Rec> recs;
+    size_t recs_used = 0;
 };
 
 namespace {
@@ -50,6 +54,20 @@ inline uint64_t k_rule(uint64_t n, double density) {
             return GC_E_CUDA;                                         \
         }                                                             \
     } while (0)
+
+// Brackets one enqueued operation with events when timing is on; always counts the launch.
+struct Timed {
+    gc_plan_s* p; cudaStream_t s; gc_plan_s::Rec* r = nullptr;
+    Timed(gc_plan_s* p_, cudaStream_t s_, int id) : p(p_), s(s_) {
+        ++p->launches;
+        if (p->recs_used < p->recs.size()) {
+            r = &p->recs[p->recs_used++];
+            r->id = id;
+            cudaEventRecord(r->a, s);
+        }
+    }
+    ~Timed() { if (r) cudaEventRecord(r->b, s); }
+};
 
 WsView view(const gc_plan_s* p, void* ws) {
     char* b = static_cast<char*>(ws);
@@ -186,20 +204,33 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     if (p->mode != GC_TOPK) return GC_E_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
-    GC_CUDA(p, cudaMemsetAsync(workspace, 0, p->control_bytes, s));
-    ++p->launches;
+    {
+        Timed tm(p, s, GC_K_CLEAR_CTRL);
+        GC_CUDA(p, cudaMemsetAsync(workspace, 0, p->control_bytes, s));
+    }
     if (out_count != nullptr) {
+        Timed tm(p, s, GC_K_CLEAR_CTRL);
         GC_CUDA(p, cudaMemsetAsync(out_count, 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
-        ++p->launches;
     }
     const uint32_t nt = p->ntiles;
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
     const int gc_ = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
-    k_hist<0, true><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws);
-    k_hist<1, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
-    k_hist<2, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
-    k_compact<<<gc_, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, ws, 0);
-    p->launches += 4;
+    {
+        Timed tm(p, s, GC_K_FOLD_HIST);
+        k_hist<0, true><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws);
+    }
+    {
+        Timed tm(p, s, GC_K_HIST_REFINE);
+        k_hist<1, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
+    }
+    {
+        Timed tm(p, s, GC_K_HIST_REFINE);
+        k_hist<2, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
+    }
+    {
+        Timed tm(p, s, GC_K_COMPACT);
+        k_compact<<<gc_, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, ws, 0);
+    }
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
 }
@@ -221,16 +252,16 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
     if (zero_first) {
+        Timed tm(p, s, GC_K_DECODE_CLEAR);
         GC_CUDA(p, cudaMemsetAsync(dense_out, 0, sizeof(float) * (size_t)p->total_n, s));
-        ++p->launches;
     }
     if (p->total_cap == 0) return GC_OK;
     const uint32_t cap = (uint32_t)p->total_cap;
     const int grid = (int)((cap + 255u) / 256u);
     for (uint32_t w = 0; w < W; ++w) {
+        Timed tm(p, s, GC_K_DECODE_ADD);
         k_scatter_add<<<grid, 256, 0, s>>>(p->d_desc, p->T, cap, (uint32_t)p->total_n, idx[w], val[w],
                                            count ? count[w] : nullptr, dense_out, ws.hdr);
-        ++p->launches;
     }
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
@@ -248,11 +279,88 @@ int gc_last_status(gc_plan_t* p, const void* workspace, void* stream, int32_t* s
     return GC_OK;
 }
 
+int gc_compress_host(gc_plan_t* p, const float* host_grad, float* grad_staging, float* residual,
+                     uint32_t* out_idx, float* out_val, uint32_t* out_count, uint32_t* host_idx,
+                     float* host_val, void* workspace, void* stream) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (p->total_n == 0) return GC_OK;
+    if (host_grad == nullptr || grad_staging == nullptr || host_idx == nullptr || host_val == nullptr)
+        return GC_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    {
+        Timed tm(p, s, GC_K_COPY);
+        GC_CUDA(p, cudaMemcpyAsync(grad_staging, host_grad, sizeof(float) * (size_t)p->total_n,
+                                   cudaMemcpyHostToDevice, s));
+    }
+    int rc = gc_compress(p, grad_staging, residual, out_idx, out_val, out_count, workspace, stream);
+    if (rc < 0) return rc;
+    {
+        Timed tm(p, s, GC_K_COPY);
+        GC_CUDA(p, cudaMemcpyAsync(host_idx, out_idx, sizeof(uint32_t) * (size_t)p->total_cap,
+                                   cudaMemcpyDeviceToHost, s));
+    }
+    {
+        Timed tm(p, s, GC_K_COPY);
+        GC_CUDA(p, cudaMemcpyAsync(host_val, out_val, sizeof(float) * (size_t)p->total_cap,
+                                   cudaMemcpyDeviceToHost, s));
+    }
+    return rc;
+}
+
+int gc_profile_enable(gc_plan_t* p, uint32_t max_records) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    for (auto& r : p->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    p->recs.clear();
+    p->recs_used = 0;
+    p->recs.reserve(max_records);
+    for (uint32_t i = 0; i < max_records; ++i) {
+        gc_plan_s::Rec r{};
+        cudaError_t e = cudaEventCreate(&r.a);
+        if (e == cudaSuccess) e = cudaEventCreate(&r.b);
+        if (e != cudaSuccess) { p->last_cuda_error = (int)e; (void)cudaGetLastError(); return GC_E_CUDA; }
+        p->recs.push_back(r);
+    }
+    return GC_OK;
+}
+
+int gc_profile_read(gc_plan_t* p, float* total_ms, uint32_t* launches) {
+    if (p == nullptr || total_ms == nullptr || launches == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    for (int i = 0; i < GC_K_COUNT; ++i) { total_ms[i] = 0.f; launches[i] = 0; }
+    GC_CUDA(p, cudaDeviceSynchronize());
+    for (size_t i = 0; i < p->recs_used; ++i) {
+        float ms = 0.f;
+        GC_CUDA(p, cudaEventElapsedTime(&ms, p->recs[i].a, p->recs[i].b));
+        int id = p->recs[i].id;
+        if (id < 0 || id >= GC_K_COUNT) id = GC_K_OTHER;
+        total_ms[id] += ms;
+        launches[id] += 1;
+    }
+    p->recs_used = 0;
+    return GC_OK;
+}
+
+const char* gc_kernel_name(int id) {
+    switch (id) {
+        case GC_K_CLEAR_CTRL: return "clear_ctrl";
+        case GC_K_FOLD_HIST: return "fold_hist";
+        case GC_K_HIST_REFINE: return "hist_refine";
+        case GC_K_COMPACT: return "compact";
+        case GC_K_DECODE_CLEAR: return "decode_clear";
+        case GC_K_DECODE_ADD: return "decode_add";
+        case GC_K_COPY: return "copy";
+        default: return "other";
+    }
+}
+
 int gc_last_cuda_error(const gc_plan_t* p) { return p ? p->last_cuda_error : 0; }
 
 int gc_destroy(gc_plan_t* p) {
     if (p == nullptr) return GC_OK;
     int rc = GC_OK;
+    for (auto& r : p->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     if (p->d_desc) {
         (void)cudaSetDevice(p->device);
         if (cudaFree(p->d_desc) != cudaSuccess) { (void)cudaGetLastError(); rc = GC_E_CUDA; }
