@@ -202,6 +202,36 @@ int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
 int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);
 const char *gc_kernel_name(int kernel_id);
 
+/*
+ * gc_compress_noalloc -- exact top-k compression of ONE tensor without any device allocation
+ * (nothing in the source paper corresponds to this call; it is an addition of this library).
+ *
+ * Who needs it: code that runs where allocating is off the table -- a gradient hook called by
+ * a training framework whose caching allocator already owns nearly all device memory (so a
+ * cudaMalloc can fail, and would in any case stall every stream of the device while it
+ * runs), or a latency-bound loop that may not touch the allocator.  Such callers cannot use
+ * gc_plan, which allocates its tensor table.  Here the scratch the kernels need (histograms,
+ * tile words, selection record; about 26 KB) is a fixed array inside the library image, so
+ * every GPU that loads libgc carries it until the process exits.
+ *
+ *   grad, residual  device, fp32[n], 16-byte aligned; residual is in/out exactly as in gc_compress
+ *   n               elements, at most GC_NOALLOC_MAX_N; larger -> GC_E_TOO_LARGE (use gc_plan)
+ *   k               entries to keep, k <= n (k > n -> GC_E_INVALID); same selection rule,
+ *                   same output order and same residual rule as gc_compress in top-k mode
+ *   out_idx/out_val device, uint32/fp32[k]
+ *   device_status   device int32 or NULL: receives GC_OK or GC_E_TIMEOUT when the work is done
+ *   stream          cudaStream_t; the call is asynchronous
+ * The current device is used.  The first call on each device resolves the device address of
+ * the array (cudaGetSymbolAddress) and sizes its grids; make that first call outside any
+ * stream capture.  All calls on a device share the one array: each call clears what it
+ * needs, so back-to-back calls on one stream are fine, but two calls whose kernels can
+ * overlap on the GPU (different streams, different threads) race on it -- serialise them.
+ * Calls no cudaMalloc/cudaFree and no allocating library routine.
+ */
+#define GC_NOALLOC_MAX_N (1u << 24)
+int gc_compress_noalloc(const float *grad, float *residual, uint32_t n, uint32_t k,
+                        uint32_t *out_idx, float *out_val, int32_t *device_status, void *stream);
+
 /* gc_last_cuda_error -- host; the cudaError_t value of the most recent failed runtime call
  * made on behalf of this plan (0 if none). */
 int gc_last_cuda_error(const gc_plan_t *plan);

@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.gc_profile_read.argtypes = [vp, vp, vp]
         L.gc_kernel_name.restype = ctypes.c_char_p
         L.gc_kernel_name.argtypes = [i32]
+        L.gc_compress_noalloc.restype = i32
+        L.gc_compress_noalloc.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
         L.gc_last_cuda_error.restype = i32
         L.gc_last_cuda_error.argtypes = [vp]
         L.gc_destroy.restype = i32
@@ -85,6 +87,17 @@ def _stream_handle(stream) -> int:
     if isinstance(stream, int):
         return stream
     return stream.cuda_stream
+
+
+GC_NOALLOC_MAX_N = 1 << 24
+
+
+def compress_noalloc(grad: torch.Tensor, residual: torch.Tensor, n: int, k: int, out_idx: torch.Tensor,
+                     out_val: torch.Tensor, device_status: Optional[torch.Tensor] = None, stream=None) -> int:
+    """gc_compress_noalloc: one tensor, scratch inside the library, no plan and no allocation.
+    Returns the status code (negative codes are returned, not raised, so callers can test them)."""
+    return lib().gc_compress_noalloc(_ptr(grad), _ptr(residual), n, k, _ptr(out_idx), _ptr(out_val),
+                                     _ptr(device_status), _stream_handle(stream))
 
 
 class Plan:

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 SO = os.path.join(_HERE, "libgc.so")
-SOURCES = ["gc.cu"]
+SOURCES = ["gc.cu", "gc_noalloc.cu"]
 
 
 def _nvcc() -> str:

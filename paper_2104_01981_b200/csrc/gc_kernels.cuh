@@ -200,7 +200,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
 // exchange.  An element is sent iff key > T, or key == T and fewer than m_eq equal keys
 // precede it in the tensor.  Sent elements are written as (flat index, value) at their rank
 // and zeroed in the residual.
-__global__ void __launch_bounds__(kBlock)
+static __global__ void __launch_bounds__(kBlock)
 k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
           float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
           uint32_t* __restrict__ out_count, WsView ws, int ticket_slot) {
@@ -305,7 +305,7 @@ struct DecodeArgs {
 // One sparse set added into the dense buffer.  Indices of one set are distinct, so plain
 // read-modify-write is race free; sets are applied by consecutive launches in worker order,
 // which fixes the order of the fp32 additions per element.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_scatter_add(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t total_cap, uint32_t total_n,
               const uint32_t* __restrict__ idx, const float* __restrict__ val,
               const uint32_t* __restrict__ count, float* __restrict__ out, WsHeader* hdr) {
