@@ -72,6 +72,7 @@ typedef struct gc_plan_s gc_plan_t;
 #define GC_Q_TENSOR_STRIDE      9   /* threshold mode: sampling stride used for tensor t            */
 #define GC_Q_MODE              10
 #define GC_Q_KERNEL_LAUNCHES   11   /* kernels + memsets enqueued by the library so far (host count) */
+#define GC_Q_CANDIDATE_CAPACITY 12  /* slots of the internal candidate list (top-k mode)            */
 
 /*
  * gc_plan -- describe the flat gradient once; computes k per tensor, output offsets and the
@@ -97,6 +98,24 @@ typedef struct gc_plan_s gc_plan_t;
  */
 int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *sizes,
             double density, int mode, uint32_t sample_stride, double cap_factor);
+
+/*
+ * gc_plan_set_option -- host; tune or steer a plan before it is used (never while work that
+ * uses it is in flight).  The selected set never depends on these options, only the route.
+ *   GC_OPT_PATH                  GC_PATH_AUTO (default): one-pass candidate path with the exact
+ *                                multi-pass kernels as its safety net; GC_PATH_EXACT: multi-pass only
+ *   GC_OPT_SAMPLE_RANK_PERMILLE  scales the sample rank that sets the candidate threshold
+ *                                (1000 = default; small values make the candidate set too small
+ *                                and so exercise the safety net -- a testing aid)
+ *   GC_OPT_CANDIDATE_CAPACITY    lowers the candidate-list capacity (testing aid for overflow)
+ * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
+ */
+#define GC_OPT_PATH                  0
+#define GC_OPT_SAMPLE_RANK_PERMILLE  1
+#define GC_OPT_CANDIDATE_CAPACITY    2
+#define GC_PATH_AUTO   0
+#define GC_PATH_EXACT  1
+int gc_plan_set_option(gc_plan_t *plan, int option, uint64_t value);
 
 /* gc_plan_query -- host-side lookup of plan facts; never touches the device.
  * Errors: GC_E_INVALID for an unknown key, a null pointer or tensor >= n_tensors. */
@@ -197,6 +216,10 @@ int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_stagin
 #define GC_K_DECODE_ADD     5   /* sparse set added into the dense output                  */
 #define GC_K_COPY           6   /* host<->device copies of gc_compress_host                */
 #define GC_K_OTHER          7
+#define GC_K_SAMPLE         8   /* strided sample histograms that set the candidate threshold */
+#define GC_K_FOLD_CAND      9   /* fold + candidate extraction (reads g, r; writes r, candidates) */
+#define GC_K_CAND_REFINE   10   /* radix-select levels over the candidate lists              */
+#define GC_K_CAND_COMPACT  11   /* ordered emission from the candidate lists                 */
 #define GC_K_COUNT         16
 int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
 int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);
@@ -231,6 +254,15 @@ const char *gc_kernel_name(int kernel_id);
 #define GC_NOALLOC_MAX_N (1u << 24)
 int gc_compress_noalloc(const float *grad, float *residual, uint32_t n, uint32_t k,
                         uint32_t *out_idx, float *out_val, int32_t *device_status, void *stream);
+
+/*
+ * gc_last_counters -- diagnostic twin of gc_last_status (SYNCHRONISES the stream): copies
+ * three counters of the most recent gc_compress on this workspace to the host:
+ *   counters[0] = candidates extracted by the one-pass path, counters[1] = 1 if the candidate
+ *   list overflowed (every tensor was redone by the exact kernels), counters[2] = tensors
+ *   whose candidate set was smaller than k (redone individually).
+ */
+int gc_last_counters(gc_plan_t *plan, const void *workspace, void *stream, uint32_t counters[3]);
 
 /* gc_last_cuda_error -- host; the cudaError_t value of the most recent failed runtime call
  * made on behalf of this plan (0 if none). */

@@ -23,7 +23,9 @@ GC_MAX_WORKERS = 64
 GC_K_COUNT = 16
 (GC_Q_N_TENSORS, GC_Q_TOTAL_N, GC_Q_TOTAL_CAP, GC_Q_WORKSPACE_BYTES, GC_Q_TENSOR_N, GC_Q_TENSOR_K,
  GC_Q_TENSOR_CAP, GC_Q_TENSOR_OFFSET, GC_Q_TENSOR_OUT_OFFSET, GC_Q_TENSOR_STRIDE, GC_Q_MODE,
- GC_Q_KERNEL_LAUNCHES) = range(12)
+ GC_Q_KERNEL_LAUNCHES, GC_Q_CANDIDATE_CAPACITY) = range(13)
+GC_OPT_PATH, GC_OPT_SAMPLE_RANK_PERMILLE, GC_OPT_CANDIDATE_CAPACITY = 0, 1, 2
+GC_PATH_AUTO, GC_PATH_EXACT = 0, 1
 
 _ERR = {GC_E_INVALID: "GC_E_INVALID", GC_E_UNSUPPORTED: "GC_E_UNSUPPORTED", GC_E_CUDA: "GC_E_CUDA",
         GC_E_TOO_LARGE: "GC_E_TOO_LARGE", GC_E_TIMEOUT: "GC_E_TIMEOUT"}
@@ -51,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.gc_version.argtypes = []
         L.gc_plan.restype = i32
         L.gc_plan.argtypes = [ctypes.POINTER(vp), i32, u32, vp, f64, i32, u32, f64]
+        L.gc_plan_set_option.restype = i32
+        L.gc_plan_set_option.argtypes = [vp, i32, u64]
         L.gc_plan_query.restype = i32
         L.gc_plan_query.argtypes = [vp, i32, u32, ctypes.POINTER(u64)]
         L.gc_compress.restype = i32
@@ -69,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.gc_kernel_name.argtypes = [i32]
         L.gc_compress_noalloc.restype = i32
         L.gc_compress_noalloc.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
+        L.gc_last_counters.restype = i32
+        L.gc_last_counters.argtypes = [vp, vp, vp, vp]
         L.gc_last_cuda_error.restype = i32
         L.gc_last_cuda_error.argtypes = [vp]
         L.gc_destroy.restype = i32
@@ -126,6 +132,13 @@ class Plan:
         if rc != GC_OK:
             raise GcError("gc_plan_query", rc)
         return int(v.value)
+
+    # --- gc_plan_set_option
+    def set_option(self, option: int, value: int) -> None:
+        rc = lib().gc_plan_set_option(self._h, option, value)
+        if rc != GC_OK:
+            raise GcError("gc_plan_set_option", rc)
+        self.workspace_bytes = self.query(GC_Q_WORKSPACE_BYTES)
 
     def tensor_k(self) -> List[int]:
         return [self.query(GC_Q_TENSOR_K, t) for t in range(self.n_tensors)]
@@ -218,6 +231,14 @@ class Plan:
         if rc < 0:
             raise GcError("gc_last_status", rc)
         return int(st.value), int(det.value)
+
+    def last_counters(self, workspace: torch.Tensor, stream=None):
+        """(candidates, overflowed, failed tensors) of the last compress; synchronises."""
+        c = (ctypes.c_uint32 * 3)()
+        rc = lib().gc_last_counters(self._h, _ptr(workspace), _stream_handle(stream), c)
+        if rc < 0:
+            raise GcError("gc_last_counters", rc)
+        return int(c[0]), int(c[1]), int(c[2])
 
     def launches(self) -> int:
         return self.query(GC_Q_KERNEL_LAUNCHES)

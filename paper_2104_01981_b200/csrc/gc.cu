@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "gc_kernels.cuh"
+#include "gc_fast.cuh"
 
 using namespace gc;
 
@@ -22,10 +22,16 @@ struct gc_plan_s {
     uint32_t ntiles = 0;
     std::vector<TensorDesc> desc;
     TensorDesc* d_desc = nullptr;
+    uint32_t nstiles = 0, ngroups = 0;
+    uint32_t cand_cap = 0, cand_cap_alloc = 0;
+    uint32_t n_sampled = 0;                 // tensors with a sample
+    int path = 0;                           // GC_PATH_AUTO or GC_PATH_EXACT
+    uint32_t rank_permille = 1000;          // scales the sample rank (testing aid)
     // workspace layout (byte offsets)
-    size_t off_sel = 0, off_hist = 0, off_state = 0, control_bytes = 0, ws_bytes = 0;
+    size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
+           control_bytes = 0, off_tinfo = 0, off_cidx = 0, off_cval = 0, ws_bytes = 0;
     int sm_count = 0;
-    int grid_hist = 0, grid_compact = 0;
+    int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
@@ -76,7 +82,79 @@ WsView view(const gc_plan_s* p, void* ws) {
     v.sel = reinterpret_cast<TensorSel*>(b + p->off_sel);
     v.hist = reinterpret_cast<uint32_t*>(b + p->off_hist);
     v.tile_state = reinterpret_cast<unsigned long long*>(b + p->off_state);
+    v.gate = nullptr;
     return v;
+}
+
+// Sampling parameters of the candidate path for one tensor (top-k mode).  The sample is one
+// 4-element group out of `sstride`; tau_lo is the srank-th largest sampled key, where srank
+// sits six standard deviations of the sampling noise above the expected rank density*m, so a
+// candidate set smaller than k is a < 1e-8 event for well-mixed data (and only costs a redo).
+void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap) {
+    const uint64_t n = d.n;
+    d.sstride = 0; d.srank = 0;
+    *ccap = n;
+    if (n < 131072) return;                              // small tensors: every element is a candidate
+    uint64_t target = std::max<uint64_t>(32768, n / 128);
+    uint64_t stride = std::max<uint64_t>(1, n / target);
+    uint64_t groups = (n + 3) / 4;
+    uint64_t nsg = (groups + stride - 1) / stride;
+    double m = 4.0 * (double)nsg;
+    double ks = density * m;
+    double rank = std::ceil(ks + 6.0 * std::sqrt(ks) + 8.0) * (double)rank_permille / 1000.0;
+    if (rank < 1.0) rank = 1.0;
+    if (rank >= m) return;
+    d.sstride = (uint32_t)stride;
+    d.srank = (uint32_t)rank;
+    double upper = (double)n * (rank + 6.0 * std::sqrt(rank)) / m;
+    double cap = std::ceil(1.25 * upper) + 1024.0;
+    *ccap = cap >= (double)n ? n : (uint64_t)cap;
+}
+
+// Fills the derived fields of the tensor table and the workspace layout.
+void finish_layout(gc_plan_s* p) {
+    uint64_t stile0 = 0, group0 = 0, ccap_total = 0;
+    p->n_sampled = 0;
+    for (uint32_t t = 0; t < p->T; ++t) {
+        TensorDesc& d = p->desc[t];
+        uint64_t ccap = d.n;
+        if (p->mode == GC_TOPK) sample_params(d, p->density, p->rank_permille, &ccap);
+        uint64_t nst = 0;
+        if (d.sstride) {
+            uint64_t groups = ((uint64_t)d.n + 3) / 4;
+            uint64_t nsg = (groups + d.sstride - 1) / d.sstride;
+            nst = (nsg + (uint64_t)kBlock * kVpt - 1) / ((uint64_t)kBlock * kVpt);
+            ++p->n_sampled;
+        }
+        d.stile0 = (uint32_t)stile0; d.nstiles = (uint32_t)nst;
+        d.group0 = (uint32_t)group0; d.ngroups = (d.ntiles + kWarps - 1) / kWarps;
+        stile0 += nst; group0 += d.ngroups; ccap_total += ccap;
+    }
+    p->nstiles = (uint32_t)stile0;
+    p->ngroups = (uint32_t)group0;
+    if (p->mode != GC_TOPK) ccap_total = 0;
+    if (p->cand_cap_alloc == 0) p->cand_cap_alloc = (uint32_t)ccap_total;   // fixed at plan creation
+    p->cand_cap = (uint32_t)std::min<uint64_t>(ccap_total, p->cand_cap_alloc);
+    const size_t T = p->T;
+    p->off_sel = sizeof(WsHeader);
+    p->off_ssel = p->off_sel + sizeof(TensorSel) * T;
+    p->off_gsel = p->off_ssel + sizeof(TensorSel) * T;
+    p->off_hist = align_up(p->off_gsel + sizeof(TensorSel) * T, 256);
+    p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * T, 256);
+    p->off_gstate = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
+    p->control_bytes = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
+    p->off_tinfo = p->control_bytes;
+    p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles, 256);
+    p->off_cval = align_up(p->off_cidx + sizeof(uint32_t) * (size_t)p->cand_cap_alloc, 256);
+    p->ws_bytes = align_up(p->off_cval + sizeof(float) * (size_t)p->cand_cap_alloc, 256);
+}
+
+int upload_table(gc_plan_s* p) {
+    if (p->device < 0 || p->T == 0) return GC_OK;
+    cudaError_t e = cudaMemcpy(p->d_desc, p->desc.data(), sizeof(TensorDesc) * (size_t)p->T,
+                               cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { p->last_cuda_error = (int)e; (void)cudaGetLastError(); return GC_E_CUDA; }
+    return GC_OK;
 }
 
 template <typename K>
@@ -131,15 +209,12 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         d.off = (uint32_t)off; d.n = (uint32_t)n; d.k = (uint32_t)k; d.cap = (uint32_t)cap;
         d.out_off = (uint32_t)out_off; d.tile0 = (uint32_t)tile0; d.ntiles = (uint32_t)nt;
         d.stride = n <= 65536 ? 1u : sample_stride;
+        d.pad[0] = d.pad[1] = 0;
         off += n; out_off += cap; tile0 += nt;
     }
     p->total_cap = out_off;
     p->ntiles = (uint32_t)tile0;
-    p->off_sel = sizeof(WsHeader);
-    p->off_hist = align_up(p->off_sel + sizeof(TensorSel) * (size_t)n_tensors, 256);
-    p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * n_tensors, 256);
-    p->control_bytes = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
-    p->ws_bytes = p->control_bytes;
+    finish_layout(p);
 
     if (device < 0) {            // host-only plan: answers queries, refuses compute calls
         *out = p;
@@ -159,10 +234,35 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         delete p;
         return GC_E_CUDA;
     }
-    p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, true>, kBlock);
+    p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, SRC_FOLD>, kBlock);
     p->grid_compact = p->sm_count * blocks_per_sm(k_compact, kBlock);
+    p->grid_fold = p->sm_count * blocks_per_sm(k_fold_cand, kBlock);
+    p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
+    p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
+    p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact, kBlock);
     *out = p;
     return GC_OK;
+}
+
+int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
+    if (p == nullptr) return GC_E_INVALID;
+    switch (option) {
+        case GC_OPT_PATH:
+            if (value != GC_PATH_AUTO && value != GC_PATH_EXACT) return GC_E_INVALID;
+            p->path = (int)value;
+            return GC_OK;
+        case GC_OPT_SAMPLE_RANK_PERMILLE:
+            if (value < 1 || value > 100000) return GC_E_INVALID;
+            p->rank_permille = (uint32_t)value;
+            finish_layout(p);                          // workspace size stays as planned
+            return upload_table(p);
+        case GC_OPT_CANDIDATE_CAPACITY:
+            if (value > p->cand_cap_alloc) return GC_E_INVALID;
+            p->cand_cap = (uint32_t)value;
+            return GC_OK;
+        default:
+            return GC_E_INVALID;
+    }
 }
 
 int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value) {
@@ -174,6 +274,7 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
         case GC_Q_WORKSPACE_BYTES: *value = p->ws_bytes; return GC_OK;
         case GC_Q_MODE: *value = (uint64_t)p->mode; return GC_OK;
         case GC_Q_KERNEL_LAUNCHES: *value = p->launches; return GC_OK;
+        case GC_Q_CANDIDATE_CAPACITY: *value = p->cand_cap; return GC_OK;
         default: break;
     }
     if (tensor >= p->T) return GC_E_INVALID;
@@ -214,22 +315,68 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     }
     const uint32_t nt = p->ntiles;
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
-    const int gc_ = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
+    const int gcp = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
+    char* wb = static_cast<char*>(workspace);
+    if (p->path == GC_PATH_EXACT) {
+        // exact multi-pass path on its own: fold + three histogram levels + ordered compaction
+        { Timed tm(p, s, GC_K_FOLD_HIST);
+          k_hist<0, SRC_FOLD><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws); }
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          k_hist<1, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws); }
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          k_hist<2, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws); }
+        { Timed tm(p, s, GC_K_COMPACT);
+          k_compact<<<gcp, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, ws, 0); }
+        GC_CUDA(p, cudaGetLastError());
+        return GC_OK;
+    }
+    // candidate path: sample -> fold + candidates -> refine on candidates -> compaction from
+    // candidates; then the exact kernels, gated to the tensors (normally none) it gave up on
+    WsView sws = ws;                 // sample select works on its own records
+    sws.sel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+    CandView cv;
+    cv.idx = reinterpret_cast<uint32_t*>(wb + p->off_cidx);
+    cv.val = reinterpret_cast<float*>(wb + p->off_cval);
+    cv.tile_info = reinterpret_cast<uint2*>(wb + p->off_tinfo);
+    cv.cap = p->cand_cap;
+    cv.ssel = sws.sel;
+    if (p->nstiles > 0) {
+        const int gs = (int)std::min<uint32_t>(p->nstiles, (uint32_t)p->grid_sample);
+        { Timed tm(p, s, GC_K_SAMPLE);
+          k_hist<0, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
+        { Timed tm(p, s, GC_K_SAMPLE);
+          k_hist<1, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
+    }
+    { Timed tm(p, s, GC_K_FOLD_CAND);
+      const int gf = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_fold);
+      k_fold_cand<<<gf, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
     {
-        Timed tm(p, s, GC_K_FOLD_HIST);
-        k_hist<0, true><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws);
+        const int gch = (int)std::min<uint32_t>((nt + kWarps - 1) / kWarps, (uint32_t)p->grid_chist);
+        { Timed tm(p, s, GC_K_CAND_REFINE);
+          k_cand_hist<1><<<gch, kBlock, 0, s>>>(p->d_desc, p->T, nt, ws, cv); }
+        { Timed tm(p, s, GC_K_CAND_REFINE);
+          k_cand_hist<2><<<gch, kBlock, 0, s>>>(p->d_desc, p->T, nt, ws, cv); }
     }
     {
-        Timed tm(p, s, GC_K_HIST_REFINE);
-        k_hist<1, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
+        WsView cws = ws;             // group look-back words
+        cws.tile_state = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
+        const int gcc = (int)std::min<uint32_t>(p->ngroups, (uint32_t)p->grid_ccompact);
+        Timed tm(p, s, GC_K_CAND_COMPACT);
+        k_cand_compact<<<gcc, kBlock, 0, s>>>(p->d_desc, p->T, p->ngroups, residual, out_idx, out_val,
+                                              out_count, cws, cv, 1);
     }
     {
-        Timed tm(p, s, GC_K_HIST_REFINE);
-        k_hist<2, false><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, ws);
-    }
-    {
-        Timed tm(p, s, GC_K_COMPACT);
-        k_compact<<<gc_, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, ws, 0);
+        WsView gws = ws;             // redo of failed tensors: own records, gated by the main ones
+        gws.sel = reinterpret_cast<TensorSel*>(wb + p->off_gsel);
+        gws.gate = ws.sel;
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          k_hist<0, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, gws); }
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          k_hist<1, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, gws); }
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          k_hist<2, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, gws); }
+        { Timed tm(p, s, GC_K_COMPACT);
+          k_compact<<<gcp, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, out_idx, out_val, out_count, gws, 0); }
     }
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
@@ -351,8 +498,23 @@ const char* gc_kernel_name(int id) {
         case GC_K_DECODE_CLEAR: return "decode_clear";
         case GC_K_DECODE_ADD: return "decode_add";
         case GC_K_COPY: return "copy";
+        case GC_K_SAMPLE: return "sample";
+        case GC_K_FOLD_CAND: return "fold_cand";
+        case GC_K_CAND_REFINE: return "cand_refine";
+        case GC_K_CAND_COMPACT: return "cand_compact";
         default: return "other";
     }
+}
+
+int gc_last_counters(gc_plan_t* p, const void* workspace, void* stream, uint32_t counters[3]) {
+    if (p == nullptr || workspace == nullptr || counters == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    WsHeader h;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
+    GC_CUDA(p, cudaStreamSynchronize(s));
+    counters[0] = h.cand_total; counters[1] = h.overflow; counters[2] = h.n_failed;
+    return GC_OK;
 }
 
 int gc_last_cuda_error(const gc_plan_t* p) { return p ? p->last_cuda_error : 0; }

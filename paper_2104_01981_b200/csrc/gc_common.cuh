@@ -34,7 +34,16 @@ struct TensorDesc {          // one per tensor, immutable, plan-owned device mem
     uint32_t tile0;          // first tile id
     uint32_t ntiles;         // tiles of this tensor
     uint32_t stride;         // threshold mode: sampling stride in 4-element groups
+    uint32_t sstride;        // stride (in 4-element groups) of the sample that sets the candidate
+                             // threshold; 0 = tensor is not sampled, every element is a candidate
+    uint32_t srank;          // rank taken inside the sample (k_s in threshold mode)
+    uint32_t stile0;         // first sample tile id
+    uint32_t nstiles;        // sample tiles (2048 sample groups each)
+    uint32_t group0;         // first compaction group id (a group = kWarps consecutive tiles)
+    uint32_t ngroups;        // compaction groups of this tensor
+    uint32_t pad[2];
 };
+static_assert(sizeof(TensorDesc) == 64, "tensor table entry is 64 bytes");
 
 struct TensorSel {           // one per tensor, in the workspace, rewritten every call
     uint32_t prefix;         // key bits fixed so far by the radix select
@@ -42,23 +51,44 @@ struct TensorSel {           // one per tensor, in the workspace, rewritten ever
     uint32_t T;              // k-th largest key (valid after the last level)
     uint32_t m_eq;           // how many of the entries with key == T are taken
     uint32_t done[kLevels];  // tiles histogrammed per level
-    uint32_t pad;
+    uint32_t flags;          // kSelFailed: the candidate path gave up on this tensor
 };
+constexpr uint32_t kSelFailed = 1u;
 
 struct WsHeader {            // head of the workspace, 256 bytes
     int32_t status;          // GC_OK / warning / error recorded by kernels
     uint32_t abort;          // non-zero: a bounded wait gave up, everyone leaves
     unsigned long long detail;
     uint32_t ticket[8];      // tile tickets, one per ordered kernel
-    uint32_t reserved[52];
+    uint32_t cand_total;     // candidate slots handed out so far
+    uint32_t overflow;       // candidate buffer ran out: every tensor takes the exact multi-pass path
+    uint32_t n_failed;       // tensors whose candidate set turned out too small
+    uint32_t reserved[49];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
 struct WsView {              // host-computed pointers into the workspace
     WsHeader* hdr;
-    TensorSel* sel;          // [n_tensors]
+    TensorSel* sel;          // [n_tensors] selection record the kernel works on
     uint32_t* hist;          // [n_tensors][kHistBins]
-    unsigned long long* tile_state;   // [ntiles]
+    unsigned long long* tile_state;   // [ntiles] (or [ngroups]) look-back words
+    const TensorSel* gate;   // non-null: only tensors the candidate path gave up on are processed
+};
+
+// Iteration spaces of the histogram kernels: every tile of a tensor, or its sample tiles.
+struct FullSpace {
+    __device__ static uint32_t tile0(const TensorDesc& d) { return d.tile0; }
+    __device__ static uint32_t ntiles(const TensorDesc& d) { return d.ntiles; }
+    __device__ static uint32_t rank(const TensorDesc& d) { return d.k; }
+};
+struct SampleSpace {
+    __device__ static uint32_t tile0(const TensorDesc& d) { return d.stile0; }
+    __device__ static uint32_t ntiles(const TensorDesc& d) { return d.nstiles; }
+    __device__ static uint32_t rank(const TensorDesc& d) { return d.srank; }
+};
+struct GroupSpace {
+    __device__ static uint32_t tile0(const TensorDesc& d) { return d.group0; }
+    __device__ static uint32_t ntiles(const TensorDesc& d) { return d.ngroups; }
 };
 
 // ----------------------------------------------------------------------------- small helpers
@@ -71,16 +101,23 @@ __device__ __forceinline__ void record_status(WsHeader* h, int32_t code, unsigne
     if (old > 0 && code < 0) { atomicExch(&h->status, code); h->detail = detail; }
 }
 
-// tensor that owns `tile`: last t with tile0[t] <= tile and ntiles[t] > 0 covering it
+// Tensor that owns `tile` in iteration space S: the LAST t whose first tile is <= tile.
+// Tensors without tiles share their first-tile id with their successor, so the last such t is
+// the one that actually has tiles.
+template <typename S = FullSpace>
 __device__ __forceinline__ uint32_t find_tensor(const TensorDesc* __restrict__ d, uint32_t T, uint32_t tile) {
     uint32_t lo = 0, hi = T;                 // invariant: answer in [lo, hi)
     while (hi - lo > 1) {
         uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&d[mid].tile0) <= tile) lo = mid; else hi = mid;
+        if (S::tile0(d[mid]) <= tile) lo = mid; else hi = mid;
     }
-    // tensors with zero tiles share tile0 with their successor; step back is never needed
-    // because the search keeps the LAST t with tile0 <= tile, which is the one with tiles.
     return lo;
+}
+
+__device__ __forceinline__ bool gate_open(const WsView& ws, uint32_t t) {
+    // with a gate, a tensor is processed only if the candidate path failed for it (or overall)
+    if (ws.gate == nullptr) return true;
+    return (ws.gate[t].flags & kSelFailed) != 0u || *(volatile uint32_t*)&ws.hdr->overflow != 0u;
 }
 
 struct TileGeom { uint32_t base, lo, hi; };  // aligned start, first and one-past-last valid flat index

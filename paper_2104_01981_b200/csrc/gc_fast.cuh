@@ -1,0 +1,272 @@
+// One-pass candidate path for exact top-k.
+//
+// A small strided sample of a = g + r gives, per tensor, a key tau_lo that is safely below
+// the k-th largest key.  The single full-size pass then folds the residual (12 bytes per
+// element) and copies every element with key >= tau_lo into a candidate list (a few per cent
+// of the data) while building the first radix histogram of the candidates.  The exact k-th
+// key is resolved on the candidate list alone and the final, index-ordered compaction reads
+// only candidates.  If the candidate set of a tensor turns out smaller than k, or the list
+// overflows, that tensor (or every tensor) is redone by the exact multi-pass kernels, so the
+// result never depends on the sample.
+#pragma once
+#include "gc_kernels.cuh"
+
+namespace gc {
+
+struct CandView {
+    uint32_t* idx;           // [cap] flat index of each candidate
+    float* val;              // [cap] a = g + r of each candidate
+    uint2* tile_info;        // [ntiles] (first slot, count) of the tile's candidates
+    uint32_t cap;
+    const TensorSel* ssel;   // [n_tensors] sample selection record (prefix = tau_lo >> 10)
+};
+
+// ----------------------------------------------------------------------------- fold + candidates
+// Reads g and r, writes a into r, emits candidates.  Slots are reserved with one atomic per
+// tile, so a tile's candidates are contiguous and in index order; tiles land in arbitrary
+// order and the compaction walks them by tile id.
+static __global__ void __launch_bounds__(kBlock)
+k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+            const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
+    constexpr int NB = 1 << level_bits(0);
+    __shared__ uint32_t s_hist[NB];
+    __shared__ uint32_t s_scratch[kWarps + 4];
+    __shared__ uint32_t s_tot[kWarps], s_ex[kWarps];
+    __shared__ uint32_t s_base, s_count, s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t first = blockIdx.x * per;
+    const uint32_t last = min(ntiles, first + per);
+    if (first >= last) return;
+    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    __syncthreads();
+
+    uint32_t t = find_tensor(desc, T, first);
+    TensorDesc d = desc[t];
+    uint32_t tau = d.sstride ? (cv.ssel[t].prefix << 10) : 0u;
+    uint32_t tiles_here = 0;
+
+    auto flush = [&]() {
+        if (tiles_here == 0) return;
+        __syncthreads();
+        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
+        for (int b = tid; b < NB; b += kBlock) {
+            uint32_t c = s_hist[b];
+            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t old = atomicAdd(&ws.sel[t].done[0], tiles_here);
+            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            select_step<0, true>(d.k, ws, t, s_scratch);
+        }
+        tiles_here = 0;
+    };
+
+    for (uint32_t tile = first; tile < last; ++tile) {
+        if (tile >= d.tile0 + d.ntiles) {
+            flush();
+            t = find_tensor(desc, T, tile);
+            d = desc[t];
+            tau = d.sstride ? (cv.ssel[t].prefix << 10) : 0u;
+        }
+        const TileGeom tg = tile_geom(d, tile - d.tile0);
+        Tile tl;
+        load_tile<true>(g, r, tg, warp, lane, tl);
+        uint32_t cnt[kVpt], cm = 0;
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            cnt[j] = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                bool c = ((tl.valid >> (4 * j + e)) & 1u) && key_of(tl.a[j][e]) >= tau;
+                cnt[j] += c;
+                cm |= (uint32_t)c << (4 * j + e);
+            }
+        }
+        uint32_t rk[kVpt], wtot;
+        warp_rank(cnt, lane, rk, wtot);
+        if (lane == 0) s_tot[warp] = wtot;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t v = lane < kWarps ? s_tot[lane] : 0u;
+            uint32_t inc = warp_incl_scan(v, lane);
+            if (lane < kWarps) s_ex[lane] = inc - v;
+            if (lane == 31) {
+                uint32_t base = inc ? atomicAdd(&ws.hdr->cand_total, inc) : 0u;
+                s_base = base; s_count = inc;
+                cv.tile_info[tile] = make_uint2(base, inc);
+                if (inc && (base > cv.cap || inc > cv.cap - base)) atomicExch(&ws.hdr->overflow, 1u);
+            }
+        }
+        __syncthreads();
+        const uint32_t base = s_base, count = s_count;
+        const bool fits = base <= cv.cap && count <= cv.cap - base;
+        if (cm != 0u && fits) {
+            const uint32_t wbase = base + s_ex[warp];
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                uint32_t pos = wbase + rk[j];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if ((cm >> (4 * j + e)) & 1u) {
+                        cv.idx[pos] = vec_index(tg.base, warp, lane, j) + e;
+                        cv.val[pos] = tl.a[j][e];
+                        atomicAdd(&s_hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
+                        ++pos;
+                    }
+                }
+            }
+        }
+        ++tiles_here;
+    }
+    flush();
+}
+
+// ----------------------------------------------------------------------------- candidate refinement
+// Radix-select level 1 or 2 over the candidate lists, one warp per tile.  Histogram updates
+// are warp-aggregated global atomics (only candidates under the current prefix take part);
+// the warp that completes a tensor's last tile runs the select step for it.
+template <int LEVEL>
+static __global__ void __launch_bounds__(kBlock)
+k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, WsView ws, CandView cv) {
+    constexpr int NB = 1 << level_bits(LEVEL);
+    constexpr int SH = level_shift(LEVEL);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (*(volatile uint32_t*)&ws.hdr->overflow) return;
+    for (uint32_t tile = blockIdx.x * kWarps + warp; tile < ntiles; tile += gridDim.x * kWarps) {
+        const uint32_t t = find_tensor(desc, T, tile);
+        if (ws.sel[t].flags & kSelFailed) continue;
+        const uint32_t prefix = ws.sel[t].prefix;
+        const uint2 info = cv.tile_info[tile];
+        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
+        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
+            uint32_t j = j0 + lane;
+            bool in = false;
+            uint32_t bin = 0;
+            if (j < info.y) {
+                uint32_t key = key_of(cv.val[info.x + j]);
+                in = (key >> (SH + level_bits(LEVEL))) == prefix;
+                bin = (key >> SH) & (NB - 1);
+            }
+            unsigned act = __ballot_sync(0xFFFFFFFFu, in);
+            if (in) {
+                unsigned same = __match_any_sync(act, bin);
+                if (lane == __ffs(same) - 1) atomicAdd(hist + bin, (uint32_t)__popc(same));
+            }
+        }
+        __threadfence();
+        __syncwarp();
+        uint32_t lastw = 0;
+        if (lane == 0) {
+            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], 1u);
+            lastw = (old + 1u == __ldg(&desc[t].ntiles)) ? 1u : 0u;
+        }
+        lastw = __shfl_sync(0xFFFFFFFFu, lastw, 0);
+        if (lastw) {
+            __threadfence();
+            select_step_warp<LEVEL>(ws, t, lane);
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------- candidate compaction
+// Index-ordered emission from the candidate lists.  A group is kWarps consecutive tiles of
+// one tensor, one warp per tile; groups are handed out by ticket and exchange their
+// (above-T, equal-T) counts through the look-back words, per tensor.  Sent entries are
+// written to the output and zeroed in the residual (which already holds a).
+static __global__ void __launch_bounds__(kBlock)
+k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups_total,
+               float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+               uint32_t* __restrict__ out_count, WsView ws, CandView cv, int ticket_slot) {
+    __shared__ uint32_t s_group;
+    __shared__ uint32_t s_gt_tot[kWarps], s_eq_tot[kWarps], s_gt_ex[kWarps], s_eq_ex[kWarps];
+    __shared__ uint32_t s_gt_sum, s_eq_sum;
+    __shared__ unsigned long long s_excl;
+    __shared__ int s_ok;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (*(volatile uint32_t*)&ws.hdr->overflow) return;
+    const unsigned lt_mask = (1u << lane) - 1u;
+
+    while (true) {
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t tk = atomicAdd(&ws.hdr->ticket[ticket_slot], 1u);
+            if (*(volatile uint32_t*)&ws.hdr->abort) tk = 0xFFFFFFFFu;
+            s_group = tk;
+        }
+        __syncthreads();
+        const uint32_t group = s_group;
+        if (group >= ngroups_total) break;
+        const uint32_t t = find_tensor<GroupSpace>(desc, T, group);
+        if (ws.sel[t].flags & kSelFailed) continue;
+        const TensorDesc d = desc[t];
+        const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
+        const uint32_t tile_in_t = (group - d.group0) * kWarps + warp;
+        uint2 info = make_uint2(0u, 0u);
+        if (tile_in_t < d.ntiles) info = cv.tile_info[d.tile0 + tile_in_t];
+
+        // pass 1: counts of this warp's tile
+        uint32_t ngt = 0, neq = 0;
+        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
+            uint32_t j = j0 + lane;
+            uint32_t key = j < info.y ? key_of(cv.val[info.x + j]) : 0u;
+            bool gt = j < info.y && key > Tkey, eq = j < info.y && key == Tkey;
+            ngt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
+            neq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+        }
+        if (lane == 0) { s_gt_tot[warp] = ngt; s_eq_tot[warp] = neq; }
+        __syncthreads();
+        scan_warp_totals(s_gt_tot, s_gt_ex, &s_gt_sum, warp, lane);
+        if (warp == 1) {
+            uint32_t v = lane < kWarps ? s_eq_tot[lane] : 0u;
+            uint32_t inc = warp_incl_scan(v, lane);
+            if (lane < kWarps) s_eq_ex[lane] = inc - v;
+            if (lane == 31) s_eq_sum = inc;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long agg = ((unsigned long long)s_gt_sum << 31) | (unsigned long long)s_eq_sum;
+            bool ok;
+            unsigned long long ex = lookback(ws.tile_state, group, d.group0, agg, lane, ws.hdr, ok);
+            if (lane == 0) { s_excl = ex; s_ok = ok ? 1 : 0; }
+        }
+        __syncthreads();
+        if (!s_ok) break;
+        // pass 2: emit
+        uint32_t gpos = (uint32_t)(s_excl >> 31) + s_gt_ex[warp];
+        uint32_t epos = (uint32_t)(s_excl & 0x7FFFFFFFull) + s_eq_ex[warp];
+        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
+            uint32_t j = j0 + lane;
+            float v = 0.f;
+            uint32_t f = 0;
+            if (j < info.y) { v = cv.val[info.x + j]; f = cv.idx[info.x + j]; }
+            uint32_t key = key_of(v);
+            bool gt = j < info.y && key > Tkey, eq = j < info.y && key == Tkey;
+            unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
+            uint32_t mg = gpos + __popc(gb & lt_mask), me = epos + __popc(eb & lt_mask);
+            if (gt || (eq && me < m_eq)) {
+                uint32_t slot = mg + min(me, m_eq);
+                if (slot < d.cap) {
+                    out_idx[d.out_off + slot] = f;
+                    out_val[d.out_off + slot] = v;
+                    r[f] = 0.0f;
+                } else {
+                    record_status(ws.hdr, -1 /*GC_E_INVALID*/, f);
+                }
+            }
+            gpos += __popc(gb); epos += __popc(eb);
+        }
+        if (out_count != nullptr && group == d.group0 && tid == 0) {
+            out_count[t] = d.k;
+            out_count[T + t] = d.k;
+        }
+    }
+}
+
+}  // namespace gc

@@ -1,6 +1,8 @@
 // Kernels of the exact multi-pass path: fold + radix-select histograms over the magnitude
 // key, ordered compaction with residual zeroing, and the sparse decode.
 #pragma once
+#include <type_traits>
+
 #include "gc_common.cuh"
 
 namespace gc {
@@ -73,19 +75,20 @@ __device__ __forceinline__ void scan_warp_totals(uint32_t* s_tot, uint32_t* s_ex
 // ----------------------------------------------------------------------------- select step
 // Run by the CTA that completes the last tile of a tensor at one level: scans that tensor's
 // histogram from the top bin down, finds the bin that holds the krem-th largest key, and
-// clears the histogram for the next level.  NB = bins at this level.
-template <int LEVEL>
-__device__ void select_step(const TensorDesc* __restrict__ desc, const WsView& ws, uint32_t t,
+// clears the histogram for the next level.  `rank0` is the rank wanted at level 0.  With
+// CHECK, a histogram holding fewer than krem keys marks the tensor as failed (the candidate
+// set was too small) instead of selecting anything.
+template <int LEVEL, bool CHECK>
+__device__ void select_step(uint32_t rank0, const WsView& ws, uint32_t t,
                             uint32_t* s_scratch /* >= kWarps + 4 words */) {
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int BPT = (NB + kBlock - 1) / kBlock;          // bins per thread
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* hist = ws.hist + (size_t)t * kHistBins;
     TensorSel* sel = ws.sel + t;
-    const uint32_t krem = (LEVEL == 0) ? desc[t].k : sel->krem;
+    const uint32_t krem = (LEVEL == 0) ? rank0 : sel->krem;
     const uint32_t prefix = (LEVEL == 0) ? 0u : sel->prefix;
-    // thread `tid` owns the bins [top - BPT*tid - BPT + 1 .. top - BPT*tid], i.e. it walks
-    // the histogram from the largest key downwards
+    // thread `tid` owns BPT consecutive bins, counted from the largest key downwards
     uint32_t c[BPT];
     uint32_t sum = 0;
 #pragma unroll
@@ -102,8 +105,17 @@ __device__ void select_step(const TensorDesc* __restrict__ desc, const WsView& w
         uint32_t v = lane < kWarps ? s_scratch[lane] : 0u;
         uint32_t wi = warp_incl_scan(v, lane);
         if (lane < kWarps) s_scratch[lane] = wi - v;
+        if (lane == kWarps - 1) s_scratch[kWarps] = wi;      // total keys in the histogram
     }
     __syncthreads();
+    if (CHECK && s_scratch[kWarps] < krem) {
+        if (tid == 0) {
+            sel->flags |= kSelFailed;
+            atomicAdd(&ws.hdr->n_failed, 1u);
+        }
+        __syncthreads();
+        return;
+    }
     uint32_t above = s_scratch[warp] + inc - sum;            // keys in bins above this thread's
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
@@ -119,22 +131,58 @@ __device__ void select_step(const TensorDesc* __restrict__ desc, const WsView& w
     __syncthreads();
 }
 
+// The same step run by a single warp (used where tiles are handled warp by warp).
+template <int LEVEL>
+__device__ void select_step_warp(const WsView& ws, uint32_t t, int lane) {
+    constexpr int NB = 1 << level_bits(LEVEL);
+    constexpr int BPL = NB / 32;                              // bins per lane
+    uint32_t* hist = ws.hist + (size_t)t * kHistBins;
+    TensorSel* sel = ws.sel + t;
+    const uint32_t krem = sel->krem, prefix = sel->prefix;
+    uint32_t sum = 0;
+    for (int i = 0; i < BPL; ++i) sum += __ldcg(hist + (NB - 1 - (lane * BPL + i)));
+    uint32_t inc = warp_incl_scan(sum, lane);
+    uint32_t above = inc - sum;
+    for (int i = 0; i < BPL; ++i) {
+        int b = NB - 1 - (lane * BPL + i);
+        uint32_t c = __ldcg(hist + b);
+        hist[b] = 0u;
+        if (above < krem && krem <= above + c) {
+            uint32_t np = (prefix << level_bits(LEVEL)) | (uint32_t)b;
+            sel->prefix = np;
+            sel->krem = krem - above;
+            if (LEVEL == kLevels - 1) { sel->T = np; sel->m_eq = krem - above; }
+        }
+        above += c;
+    }
+    __syncwarp();
+}
+
 // ----------------------------------------------------------------------------- histogram pass
 // One radix-select level over all tensors.  CTAs take contiguous runs of tiles, keep a
 // shared-memory histogram while the tensor stays the same, flush it with global atomics when
 // it changes, and the CTA that completes a tensor's last tile runs the select step.
-//   LEVEL 0, FOLD: reads g and r, writes a = g + r into r (12 bytes per element)
-//   otherwise:     reads a from r (4 bytes per element); only keys under the prefix count
-template <int LEVEL, bool FOLD>
+//   SRC_FOLD   (level 0): reads g and r, writes a = g + r into r (12 bytes per element)
+//   SRC_RESID:            reads a from r (4 bytes per element)
+//   SRC_SAMPLE:           walks the tensor's sample (one 4-element group out of `sstride`),
+//                         a = g + r is computed but not stored; rank = the tensor's srank
+// At levels above 0 only keys under the prefix fixed so far are counted.
+constexpr int SRC_FOLD = 0, SRC_RESID = 1, SRC_SAMPLE = 2;
+
+template <int LEVEL, int SRC>
 __global__ void __launch_bounds__(kBlock)
 k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
        const float* __restrict__ g, float* __restrict__ r, WsView ws) {
+    using S = typename std::conditional<SRC == SRC_SAMPLE, SampleSpace, FullSpace>::type;
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int SH = level_shift(LEVEL);
     __shared__ uint32_t s_hist[NB];
     __shared__ uint32_t s_scratch[kWarps + 4];
     __shared__ uint32_t s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (ws.gate != nullptr && *(volatile uint32_t*)&ws.hdr->n_failed == 0u &&
+        *(volatile uint32_t*)&ws.hdr->overflow == 0u)
+        return;
     const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
     const uint32_t first = blockIdx.x * per;
     const uint32_t last = min(ntiles, first + per);
@@ -142,12 +190,14 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
     for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
     __syncthreads();
 
-    uint32_t t = find_tensor(desc, T, first);
+    uint32_t t = find_tensor<S>(desc, T, first);
     TensorDesc d = desc[t];
+    bool active = gate_open(ws, t);
     uint32_t prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
     uint32_t tiles_here = 0;
 
     auto flush = [&]() {
+        if (!active || tiles_here == 0) return;
         __syncthreads();
         uint32_t* hist = ws.hist + (size_t)t * kHistBins;
         for (int b = tid; b < NB; b += kBlock) {
@@ -158,34 +208,59 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         __syncthreads();
         if (tid == 0) {
             uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
-            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
+            s_last = (old + tiles_here == S::ntiles(d)) ? 1u : 0u;
         }
         __syncthreads();
         if (s_last) {
             __threadfence();
-            select_step<LEVEL>(desc, ws, t, s_scratch);
+            select_step<LEVEL, false>(S::rank(d), ws, t, s_scratch);
         }
         tiles_here = 0;
     };
 
     for (uint32_t tile = first; tile < last; ++tile) {
-        if (tile >= d.tile0 + d.ntiles) {
+        if (tile >= S::tile0(d) + S::ntiles(d)) {
             flush();
-            t = find_tensor(desc, T, tile);
+            t = find_tensor<S>(desc, T, tile);
             d = desc[t];
+            active = gate_open(ws, t);
             prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
         }
-        TileGeom tg = tile_geom(d, tile - d.tile0);
-        Tile tl;
-        load_tile<FOLD>(g, r, tg, warp, lane, tl);
+        if (!active) continue;
+        if (SRC == SRC_SAMPLE) {
+            // sample tile: 2048 sample groups; thread takes groups j*kBlock + tid
+            const uint32_t ngroups = (d.n + 3u) >> 2;
+            const uint32_t sg0 = (tile - d.stile0) * (uint32_t)(kBlock * kVpt);
 #pragma unroll
-        for (int j = 0; j < kVpt; ++j) {
+            for (int j = 0; j < kVpt; ++j) {
+                uint64_t gi = (uint64_t)(sg0 + j * kBlock + tid) * d.sstride;
+                if (gi >= ngroups) continue;
+                uint32_t i0 = (uint32_t)gi * 4u;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                uint32_t key = key_of(tl.a[j][e]);
-                bool in = (tl.valid >> (4 * j + e)) & 1u;
-                if (LEVEL > 0) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
-                if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t i = i0 + e;
+                    if (i < d.n) {
+                        uint32_t f = d.off + i;
+                        uint32_t key = key_of(__fadd_rn(__ldg(g + f), r[f]));
+                        bool in = true;
+                        if (LEVEL > 0) in = ((key >> (SH + level_bits(LEVEL))) == prefix);
+                        if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                    }
+                }
+            }
+        } else {
+            TileGeom tg = tile_geom(d, tile - d.tile0);
+            Tile tl;
+            load_tile<SRC == SRC_FOLD>(g, r, tg, warp, lane, tl);
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t key = key_of(tl.a[j][e]);
+                    bool in = (tl.valid >> (4 * j + e)) & 1u;
+                    if (LEVEL > 0) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
+                    if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                }
             }
         }
         ++tiles_here;
@@ -210,6 +285,9 @@ k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
     __shared__ unsigned long long s_excl;
     __shared__ int s_ok;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (ws.gate != nullptr && *(volatile uint32_t*)&ws.hdr->n_failed == 0u &&
+        *(volatile uint32_t*)&ws.hdr->overflow == 0u)
+        return;
 
     while (true) {
         __syncthreads();
@@ -222,6 +300,7 @@ k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         const uint32_t tile = s_tile;
         if (tile >= ntiles) break;
         const uint32_t t = find_tensor(desc, T, tile);
+        if (!gate_open(ws, t)) continue;
         const TensorDesc d = desc[t];
         const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
         const TileGeom tg = tile_geom(d, tile - d.tile0);

@@ -45,6 +45,8 @@ __global__ void k_noalloc_init(unsigned char* scratch, uint32_t n, uint32_t k, u
     if (tid == 0) {
         TensorDesc d;
         d.off = 0; d.n = n; d.k = k; d.cap = k; d.out_off = 0; d.tile0 = 0; d.ntiles = ntiles; d.stride = 1;
+        d.sstride = 0; d.srank = 0; d.stile0 = 0; d.nstiles = 0; d.group0 = 0; d.ngroups = 0;
+        d.pad[0] = d.pad[1] = 0;
         *reinterpret_cast<TensorDesc*>(scratch + kOffDesc) = d;
     }
 }
@@ -80,7 +82,7 @@ extern "C" int gc_compress_noalloc(const float* grad, float* residual, uint32_t 
             int sms = 0, bh = 0, bc = 0;
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
             if (e == cudaSuccess)
-                e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bh, k_hist<0, true>, kBlock, 0);
+                e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bh, k_hist<0, SRC_FOLD>, kBlock, 0);
             if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bc, k_compact, kBlock, 0);
             if (e != cudaSuccess || ptr == nullptr || sms < 1) {
                 (void)cudaGetLastError();
@@ -98,15 +100,16 @@ extern "C" int gc_compress_noalloc(const float* grad, float* residual, uint32_t 
     ws.sel = reinterpret_cast<TensorSel*>(sc + kOffSel);
     ws.hist = reinterpret_cast<uint32_t*>(sc + kOffHist);
     ws.tile_state = reinterpret_cast<unsigned long long*>(sc + kOffState);
+    ws.gate = nullptr;
     const TensorDesc* desc = reinterpret_cast<const TensorDesc*>(sc + kOffDesc);
     const uint32_t nt = (n + kTile - 1) / kTile;
     const int gh = (int)(nt < (uint32_t)pd.grid_hist ? nt : (uint32_t)pd.grid_hist);
     const int gcp = (int)(nt < (uint32_t)pd.grid_compact ? nt : (uint32_t)pd.grid_compact);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     k_noalloc_init<<<8, 256, 0, s>>>(sc, n, k, nt);
-    k_hist<0, true><<<gh, kBlock, 0, s>>>(desc, 1u, nt, grad, residual, ws);
-    k_hist<1, false><<<gh, kBlock, 0, s>>>(desc, 1u, nt, nullptr, residual, ws);
-    k_hist<2, false><<<gh, kBlock, 0, s>>>(desc, 1u, nt, nullptr, residual, ws);
+    k_hist<0, SRC_FOLD><<<gh, kBlock, 0, s>>>(desc, 1u, nt, grad, residual, ws);
+    k_hist<1, SRC_RESID><<<gh, kBlock, 0, s>>>(desc, 1u, nt, nullptr, residual, ws);
+    k_hist<2, SRC_RESID><<<gh, kBlock, 0, s>>>(desc, 1u, nt, nullptr, residual, ws);
     k_compact<<<gcp, kBlock, 0, s>>>(desc, 1u, nt, residual, out_idx, out_val, nullptr, ws, 0);
     k_noalloc_finish<<<1, 1, 0, s>>>(sc, device_status);
     if (cudaGetLastError() != cudaSuccess) return GC_E_CUDA;

@@ -53,11 +53,14 @@ class GpuWorker:
 
 
 def check_topk_against_oracle(sizes: Sequence[int], density: float, grads: List[torch.Tensor],
-                              r0: Optional[torch.Tensor] = None, device: int = 0):
+                              r0: Optional[torch.Tensor] = None, device: int = 0, options=None,
+                              expect_counters=None):
     """Runs len(grads) consecutive steps of one worker on GPU and oracle; asserts bitwise
     equality of indices, values, counts and residual after every step.  Returns the plan
     worker (for decode tests) and the oracle's last (idx, val)."""
     plan = api.Plan(sizes, density, device=device)
+    for opt, value in (options or {}).items():
+        plan.set_option(opt, value)
     w = GpuWorker(plan)
     ks = plan.tensor_k()
     n = plan.total_n
@@ -72,6 +75,8 @@ def check_topk_against_oracle(sizes: Sequence[int], density: float, grads: List[
             g_dev = torch.cat([g_dev, torch.zeros(4 - g_dev.numel(), device=g_dev.device)])
         w.step(g_dev)
         w.check_status()
+        if expect_counters is not None:
+            expect_counters(plan.last_counters(w.ws))
         g_cpu = g.cpu().numpy()
         oi, ov = oracle.topk_compress_tensors(list(sizes), ks, g_cpu, r_cpu)
         tot = sum(ks)

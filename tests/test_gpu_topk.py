@@ -83,6 +83,43 @@ def test_config5_gpt2_medium_full_size_two_workers():
         torch.cuda.empty_cache()
 
 
+PATHS = {
+    "auto": {},
+    "exact": {api.GC_OPT_PATH: api.GC_PATH_EXACT},
+    "auto_starved": {api.GC_OPT_SAMPLE_RANK_PERMILLE: 30},      # candidate sets too small -> redo per tensor
+    "auto_overflow": {api.GC_OPT_CANDIDATE_CAPACITY: 100},      # candidate list too short -> redo everything
+}
+
+
+@pytest.mark.parametrize("path", list(PATHS))
+def test_every_route_gives_the_same_bits(path):
+    sizes = [300_000, 5, 1_500_001, 131_072, 64, 131_071, 2_000_003]
+    n = sum(sizes)
+    grads = [randn(n, 900 + s) for s in range(3)]
+    seen = []
+    for density in (0.001, 0.01):
+        check_topk_against_oracle(sizes, density, grads, options=PATHS[path], expect_counters=seen.append)
+    if path == "auto":
+        assert all(c[1] == 0 and c[2] == 0 for c in seen), seen     # the safety net stayed idle
+    if path == "auto_starved":
+        assert all(c[2] >= 1 for c in seen), seen
+    if path == "auto_overflow":
+        assert all(c[1] == 1 for c in seen), seen
+
+
+def test_sample_blind_spot_falls_back_and_stays_exact():
+    """All large values sit where the sample never looks (groups that are not a multiple of the
+    stride), so the sampled threshold is far too low or too high; the result must not care."""
+    n = 1 << 21
+    g = randn(n, 77) * 1e-3
+    grp = torch.arange(n) // 4
+    hidden = (grp % 64) != 0
+    big = hidden & (torch.rand(n, generator=torch.Generator().manual_seed(5)) < 0.02)
+    g[big] = torch.sign(g[big]) * 5.0
+    for density in (0.001, 0.01, 0.03):
+        check_topk_against_oracle([n], density, [g, -g, g])
+
+
 def test_rejects_misaligned_and_null_buffers():
     plan = api.Plan([1024], 0.1, device=0)
     wk = GpuWorker(plan)
