@@ -95,7 +95,7 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
     d.sstride = 0; d.srank = 0;
     *ccap = n;
     if (n < 131072) return;                              // small tensors: every element is a candidate
-    uint64_t target = std::max<uint64_t>(32768, n / 128);
+    uint64_t target = std::min<uint64_t>(131072, std::max<uint64_t>(32768, n / 128));
     uint64_t stride = std::max<uint64_t>(1, n / target);
     uint64_t groups = (n + 3) / 4;
     uint64_t nsg = (groups + stride - 1) / stride;
@@ -107,7 +107,7 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
     d.sstride = (uint32_t)stride;
     d.srank = (uint32_t)rank;
     double upper = (double)n * (rank + 6.0 * std::sqrt(rank)) / m;
-    double cap = std::ceil(1.25 * upper) + 1024.0;
+    double cap = std::ceil(1.25 * upper) + 4096.0;
     *ccap = cap >= (double)n ? n : (uint64_t)cap;
 }
 
@@ -132,6 +132,9 @@ void finish_layout(gc_plan_s* p) {
     }
     p->nstiles = (uint32_t)stile0;
     p->ngroups = (uint32_t)group0;
+    // every warp of the fold pass may strand part of a slab; CTAs never outnumber tiles
+    ccap_total += (uint64_t)std::min<uint32_t>(p->ntiles, 1024u) * kWarps * kSlab;
+    if (ccap_total > 0x7FFFFFFFull) ccap_total = 0x7FFFFFFFull;
     if (p->mode != GC_TOPK) ccap_total = 0;
     if (p->cand_cap_alloc == 0) p->cand_cap_alloc = (uint32_t)ccap_total;   // fixed at plan creation
     p->cand_cap = (uint32_t)std::min<uint64_t>(ccap_total, p->cand_cap_alloc);
@@ -144,7 +147,7 @@ void finish_layout(gc_plan_s* p) {
     p->off_gstate = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
     p->control_bytes = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
     p->off_tinfo = p->control_bytes;
-    p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles, 256);
+    p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
     p->off_cval = align_up(p->off_cidx + sizeof(uint32_t) * (size_t)p->cand_cap_alloc, 256);
     p->ws_bytes = align_up(p->off_cval + sizeof(float) * (size_t)p->cand_cap_alloc, 256);
 }
@@ -337,11 +340,13 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     CandView cv;
     cv.idx = reinterpret_cast<uint32_t*>(wb + p->off_cidx);
     cv.val = reinterpret_cast<float*>(wb + p->off_cval);
-    cv.tile_info = reinterpret_cast<uint2*>(wb + p->off_tinfo);
+    cv.chunk_info = reinterpret_cast<uint2*>(wb + p->off_tinfo);
     cv.cap = p->cand_cap;
     cv.ssel = sws.sel;
     if (p->nstiles > 0) {
         const int gs = (int)std::min<uint32_t>(p->nstiles, (uint32_t)p->grid_sample);
+        // two radix levels on the sample: tau_lo is the exact srank-th sampled key cut to 21 bits,
+        // so the size of the candidate set is binomial whatever the shape of the distribution
         { Timed tm(p, s, GC_K_SAMPLE);
           k_hist<0, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
         { Timed tm(p, s, GC_K_SAMPLE);
@@ -351,7 +356,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
       const int gf = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_fold);
       k_fold_cand<<<gf, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
     {
-        const int gch = (int)std::min<uint32_t>((nt + kWarps - 1) / kWarps, (uint32_t)p->grid_chist);
+        const int gch = (int)std::min<uint32_t>((nt + 2 * kWarps - 1) / (2 * kWarps), (uint32_t)p->grid_chist);
         { Timed tm(p, s, GC_K_CAND_REFINE);
           k_cand_hist<1><<<gch, kBlock, 0, s>>>(p->d_desc, p->T, nt, ws, cv); }
         { Timed tm(p, s, GC_K_CAND_REFINE);

@@ -18,7 +18,9 @@ constexpr uint32_t kKeyMask = 0x7FFFFFFFu;
 constexpr int kLevels = 3;
 __host__ __device__ constexpr int level_bits(int l) { return l == 0 ? 11 : 10; }
 __host__ __device__ constexpr int level_shift(int l) { return l == 0 ? 20 : (l == 1 ? 10 : 0); }
+__host__ __device__ constexpr bool level_is_first(int l) { return l == 0; }
 constexpr int kHistBins = 2048;             // bins reserved per tensor (largest level)
+constexpr int kSlab = 128;                  // candidate slots a warp reserves at a time
 
 // Bounded waits: a predecessor tile is always already running (tiles are handed out by an
 // atomic ticket), so these limits are a safety net, not a schedule.

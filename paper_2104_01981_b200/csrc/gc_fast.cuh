@@ -8,6 +8,11 @@
 // only candidates.  If the candidate set of a tensor turns out smaller than k, or the list
 // overflows, that tensor (or every tensor) is redone by the exact multi-pass kernels, so the
 // result never depends on the sample.
+//
+// Candidate list layout: each warp of the fold pass owns a 512-element chunk of every tile it
+// visits and appends that chunk's candidates, in index order, to a slab of kSlab slots it
+// reserved with one atomic; chunk_info[tile * kWarps + warp] = (first slot, count).  Chunks
+// land in arbitrary order in the list; readers walk them by (tile, warp), which is index order.
 #pragma once
 #include "gc_kernels.cuh"
 
@@ -16,23 +21,45 @@ namespace gc {
 struct CandView {
     uint32_t* idx;           // [cap] flat index of each candidate
     float* val;              // [cap] a = g + r of each candidate
-    uint2* tile_info;        // [ntiles] (first slot, count) of the tile's candidates
+    uint2* chunk_info;       // [ntiles * kWarps] (first slot, count) per warp chunk
     uint32_t cap;
-    const TensorSel* ssel;   // [n_tensors] sample selection record (prefix = tau_lo >> 10)
+    const TensorSel* ssel;   // [n_tensors] sample selection record (21-bit prefix = tau_lo >> 10)
 };
 
+// The candidates of one tile as seen by a warp: lane l < kWarps holds chunk l.
+struct TileCands {
+    uint32_t base, cnt, incl, total;
+};
+__device__ __forceinline__ TileCands load_tile_cands(const CandView& cv, uint32_t tile, int lane) {
+    TileCands tc;
+    uint2 info = make_uint2(0u, 0u);
+    if (lane < kWarps) info = cv.chunk_info[(size_t)tile * kWarps + lane];
+    tc.base = info.x; tc.cnt = info.y;
+    tc.incl = warp_incl_scan(tc.cnt, lane);
+    tc.total = __shfl_sync(0xFFFFFFFFu, tc.incl, 31);
+    return tc;
+}
+// slot of the j-th candidate of the tile (all lanes call; j >= total gives a harmless slot of chunk 0)
+__device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
+    uint32_t c = 0;
+#pragma unroll
+    for (int l = 0; l < kWarps; ++l) c += (j >= __shfl_sync(0xFFFFFFFFu, tc.incl, l)) ? 1u : 0u;
+    c = min(c, (uint32_t)kWarps - 1u);
+    uint32_t b = __shfl_sync(0xFFFFFFFFu, tc.base, c);
+    uint32_t ex = __shfl_sync(0xFFFFFFFFu, tc.incl - tc.cnt, c);
+    return b + (j - ex);
+}
+
 // ----------------------------------------------------------------------------- fold + candidates
-// Reads g and r, writes a into r, emits candidates.  Slots are reserved with one atomic per
-// tile, so a tile's candidates are contiguous and in index order; tiles land in arbitrary
-// order and the compaction walks them by tile id.
+// Reads g and r, writes a into r, emits candidates.  No block-wide barrier in the tile loop:
+// every warp ranks and stores the candidates of its own chunk.
 static __global__ void __launch_bounds__(kBlock)
 k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
     constexpr int NB = 1 << level_bits(0);
     __shared__ uint32_t s_hist[NB];
     __shared__ uint32_t s_scratch[kWarps + 4];
-    __shared__ uint32_t s_tot[kWarps], s_ex[kWarps];
-    __shared__ uint32_t s_base, s_count, s_last;
+    __shared__ uint32_t s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
     const uint32_t first = blockIdx.x * per;
@@ -43,8 +70,9 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
 
     uint32_t t = find_tensor(desc, T, first);
     TensorDesc d = desc[t];
-    uint32_t tau = d.sstride ? (cv.ssel[t].prefix << 10) : 0u;
+    uint32_t tau = d.sstride ? (cv.ssel[t].prefix << level_shift(1)) : 0u;
     uint32_t tiles_here = 0;
+    uint32_t slab_next = 0, slab_left = 0;       // this warp's current slab (warp-uniform)
 
     auto flush = [&]() {
         if (tiles_here == 0) return;
@@ -73,7 +101,7 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             flush();
             t = find_tensor(desc, T, tile);
             d = desc[t];
-            tau = d.sstride ? (cv.ssel[t].prefix << 10) : 0u;
+            tau = d.sstride ? (cv.ssel[t].prefix << level_shift(1)) : 0u;
         }
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;
@@ -91,27 +119,28 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         }
         uint32_t rk[kVpt], wtot;
         warp_rank(cnt, lane, rk, wtot);
-        if (lane == 0) s_tot[warp] = wtot;
-        __syncthreads();
-        if (warp == 0) {
-            uint32_t v = lane < kWarps ? s_tot[lane] : 0u;
-            uint32_t inc = warp_incl_scan(v, lane);
-            if (lane < kWarps) s_ex[lane] = inc - v;
-            if (lane == 31) {
-                uint32_t base = inc ? atomicAdd(&ws.hdr->cand_total, inc) : 0u;
-                s_base = base; s_count = inc;
-                cv.tile_info[tile] = make_uint2(base, inc);
-                if (inc && (base > cv.cap || inc > cv.cap - base)) atomicExch(&ws.hdr->overflow, 1u);
+        // reserve slots for this chunk out of the warp's slab (new slab when it runs short)
+        bool fits = true;
+        if (wtot > slab_left) {
+            uint32_t need = max(wtot, (uint32_t)kSlab);
+            uint32_t nb = 0;
+            if (lane == 0) nb = atomicAdd(&ws.hdr->cand_total, need);
+            nb = __shfl_sync(0xFFFFFFFFu, nb, 0);
+            if (nb > cv.cap || need > cv.cap - nb) {
+                fits = false;
+                if (lane == 0) atomicExch(&ws.hdr->overflow, 1u);
+                slab_left = 0;
+            } else {
+                slab_next = nb; slab_left = need;
             }
         }
-        __syncthreads();
-        const uint32_t base = s_base, count = s_count;
-        const bool fits = base <= cv.cap && count <= cv.cap - base;
+        const uint32_t cbase = slab_next;
+        if (fits) { slab_next += wtot; slab_left -= wtot; }
+        if (lane == 0) cv.chunk_info[(size_t)tile * kWarps + warp] = make_uint2(cbase, fits ? wtot : 0u);
         if (cm != 0u && fits) {
-            const uint32_t wbase = base + s_ex[warp];
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
-                uint32_t pos = wbase + rk[j];
+                uint32_t pos = cbase + rk[j];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if ((cm >> (4 * j + e)) & 1u) {
@@ -129,50 +158,82 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
 }
 
 // ----------------------------------------------------------------------------- candidate refinement
-// Radix-select level 1 or 2 over the candidate lists, one warp per tile.  Histogram updates
-// are warp-aggregated global atomics (only candidates under the current prefix take part);
-// the warp that completes a tensor's last tile runs the select step for it.
+// Radix-select level 1 or 2 over the candidate lists.  CTAs take contiguous runs of tiles and
+// walk them kWarps at a time, one warp per tile, always inside one tensor; counts go to a
+// shared-memory histogram that is flushed when the tensor changes, and the CTA that completes
+// a tensor's last tile runs the select step (same scheme as k_hist).
 template <int LEVEL>
 static __global__ void __launch_bounds__(kBlock)
 k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, WsView ws, CandView cv) {
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int SH = level_shift(LEVEL);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ uint32_t s_hist[NB];
+    __shared__ uint32_t s_scratch[kWarps + 4];
+    __shared__ uint32_t s_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (*(volatile uint32_t*)&ws.hdr->overflow) return;
-    for (uint32_t tile = blockIdx.x * kWarps + warp; tile < ntiles; tile += gridDim.x * kWarps) {
-        const uint32_t t = find_tensor(desc, T, tile);
-        if (ws.sel[t].flags & kSelFailed) continue;
-        const uint32_t prefix = ws.sel[t].prefix;
-        const uint2 info = cv.tile_info[tile];
+    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t first = blockIdx.x * per;
+    const uint32_t last = min(ntiles, first + per);
+    if (first >= last) return;
+    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    __syncthreads();
+
+    uint32_t t = find_tensor(desc, T, first);
+    TensorDesc d = desc[t];
+    bool active = (ws.sel[t].flags & kSelFailed) == 0u;
+    uint32_t prefix = ws.sel[t].prefix;
+    uint32_t tiles_here = 0;
+
+    auto flush = [&]() {
+        if (!active || tiles_here == 0) { tiles_here = 0; return; }
+        __syncthreads();
         uint32_t* hist = ws.hist + (size_t)t * kHistBins;
-        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
-            uint32_t j = j0 + lane;
-            bool in = false;
-            uint32_t bin = 0;
-            if (j < info.y) {
-                uint32_t key = key_of(cv.val[info.x + j]);
-                in = (key >> (SH + level_bits(LEVEL))) == prefix;
-                bin = (key >> SH) & (NB - 1);
-            }
-            unsigned act = __ballot_sync(0xFFFFFFFFu, in);
-            if (in) {
-                unsigned same = __match_any_sync(act, bin);
-                if (lane == __ffs(same) - 1) atomicAdd(hist + bin, (uint32_t)__popc(same));
-            }
+        for (int b = tid; b < NB; b += kBlock) {
+            uint32_t c = s_hist[b];
+            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
         }
         __threadfence();
-        __syncwarp();
-        uint32_t lastw = 0;
-        if (lane == 0) {
-            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], 1u);
-            lastw = (old + 1u == __ldg(&desc[t].ntiles)) ? 1u : 0u;
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
+            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
         }
-        lastw = __shfl_sync(0xFFFFFFFFu, lastw, 0);
-        if (lastw) {
+        __syncthreads();
+        if (s_last) {
             __threadfence();
-            select_step_warp<LEVEL>(ws, t, lane);
+            select_step<LEVEL, false>(0u, ws, t, s_scratch);
         }
+        tiles_here = 0;
+    };
+
+    uint32_t batch = first;
+    while (batch < last) {
+        if (batch >= d.tile0 + d.ntiles) {
+            flush();
+            t = find_tensor(desc, T, batch);
+            d = desc[t];
+            active = (ws.sel[t].flags & kSelFailed) == 0u;
+            prefix = ws.sel[t].prefix;
+        }
+        const uint32_t bend = min(min(last, d.tile0 + d.ntiles), batch + (uint32_t)kWarps);
+        const uint32_t tile = batch + warp;
+        if (active && tile < bend) {
+            TileCands tc = load_tile_cands(cv, tile, lane);
+            for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
+                uint32_t j = j0 + lane;
+                uint32_t slot = cand_slot(tc, j);
+                if (j < tc.total) {
+                    uint32_t key = key_of(cv.val[slot]);
+                    if ((key >> (SH + level_bits(LEVEL))) == prefix)
+                        atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                }
+            }
+        }
+        tiles_here += bend - batch;
+        batch = bend;
     }
+    flush();
 }
 
 // ----------------------------------------------------------------------------- candidate compaction
@@ -208,15 +269,17 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
         const TensorDesc d = desc[t];
         const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
         const uint32_t tile_in_t = (group - d.group0) * kWarps + warp;
-        uint2 info = make_uint2(0u, 0u);
-        if (tile_in_t < d.ntiles) info = cv.tile_info[d.tile0 + tile_in_t];
+        TileCands tc;
+        tc.base = tc.cnt = tc.incl = tc.total = 0u;
+        if (tile_in_t < d.ntiles) tc = load_tile_cands(cv, d.tile0 + tile_in_t, lane);
 
         // pass 1: counts of this warp's tile
         uint32_t ngt = 0, neq = 0;
-        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
+        for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
             uint32_t j = j0 + lane;
-            uint32_t key = j < info.y ? key_of(cv.val[info.x + j]) : 0u;
-            bool gt = j < info.y && key > Tkey, eq = j < info.y && key == Tkey;
+            uint32_t slot = cand_slot(tc, j);
+            uint32_t key = j < tc.total ? key_of(cv.val[slot]) : 0u;
+            bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
             ngt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
             neq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
         }
@@ -241,20 +304,21 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
         // pass 2: emit
         uint32_t gpos = (uint32_t)(s_excl >> 31) + s_gt_ex[warp];
         uint32_t epos = (uint32_t)(s_excl & 0x7FFFFFFFull) + s_eq_ex[warp];
-        for (uint32_t j0 = 0; j0 < info.y; j0 += 32) {
+        for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
             uint32_t j = j0 + lane;
+            uint32_t slot = cand_slot(tc, j);
             float v = 0.f;
             uint32_t f = 0;
-            if (j < info.y) { v = cv.val[info.x + j]; f = cv.idx[info.x + j]; }
+            if (j < tc.total) { v = cv.val[slot]; f = cv.idx[slot]; }
             uint32_t key = key_of(v);
-            bool gt = j < info.y && key > Tkey, eq = j < info.y && key == Tkey;
+            bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
             unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
             uint32_t mg = gpos + __popc(gb & lt_mask), me = epos + __popc(eb & lt_mask);
             if (gt || (eq && me < m_eq)) {
-                uint32_t slot = mg + min(me, m_eq);
-                if (slot < d.cap) {
-                    out_idx[d.out_off + slot] = f;
-                    out_val[d.out_off + slot] = v;
+                uint32_t slot_out = mg + min(me, m_eq);
+                if (slot_out < d.cap) {
+                    out_idx[d.out_off + slot_out] = f;
+                    out_val[d.out_off + slot_out] = v;
                     r[f] = 0.0f;
                 } else {
                     record_status(ws.hdr, -1 /*GC_E_INVALID*/, f);

@@ -86,8 +86,8 @@ __device__ void select_step(uint32_t rank0, const WsView& ws, uint32_t t,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* hist = ws.hist + (size_t)t * kHistBins;
     TensorSel* sel = ws.sel + t;
-    const uint32_t krem = (LEVEL == 0) ? rank0 : sel->krem;
-    const uint32_t prefix = (LEVEL == 0) ? 0u : sel->prefix;
+    const uint32_t krem = level_is_first(LEVEL) ? rank0 : sel->krem;
+    const uint32_t prefix = level_is_first(LEVEL) ? 0u : sel->prefix;
     // thread `tid` owns BPT consecutive bins, counted from the largest key downwards
     uint32_t c[BPT];
     uint32_t sum = 0;
@@ -193,7 +193,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
     uint32_t t = find_tensor<S>(desc, T, first);
     TensorDesc d = desc[t];
     bool active = gate_open(ws, t);
-    uint32_t prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
+    uint32_t prefix = level_is_first(LEVEL) ? 0u : ws.sel[t].prefix;
     uint32_t tiles_here = 0;
 
     auto flush = [&]() {
@@ -224,28 +224,37 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             t = find_tensor<S>(desc, T, tile);
             d = desc[t];
             active = gate_open(ws, t);
-            prefix = (LEVEL == 0) ? 0u : ws.sel[t].prefix;
+            prefix = level_is_first(LEVEL) ? 0u : ws.sel[t].prefix;
         }
         if (!active) continue;
         if (SRC == SRC_SAMPLE) {
-            // sample tile: 2048 sample groups; thread takes groups j*kBlock + tid
+            // sample tile: 2048 sample groups; thread takes groups j*kBlock + tid.  All loads
+            // are issued before any of them is used.
             const uint32_t ngroups = (d.n + 3u) >> 2;
             const uint32_t sg0 = (tile - d.stile0) * (uint32_t)(kBlock * kVpt);
+            float gv[kVpt][4], rv[kVpt][4];
+            uint32_t ok = 0;
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
                 uint64_t gi = (uint64_t)(sg0 + j * kBlock + tid) * d.sstride;
-                if (gi >= ngroups) continue;
-                uint32_t i0 = (uint32_t)gi * 4u;
+                uint32_t i0 = (uint32_t)min(gi, (uint64_t)ngroups) * 4u;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    uint32_t i = i0 + e;
-                    if (i < d.n) {
-                        uint32_t f = d.off + i;
-                        uint32_t key = key_of(__fadd_rn(__ldg(g + f), r[f]));
-                        bool in = true;
-                        if (LEVEL > 0) in = ((key >> (SH + level_bits(LEVEL))) == prefix);
-                        if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
-                    }
+                    bool v = gi < ngroups && i0 + e < d.n;
+                    uint32_t f = d.off + (v ? i0 + e : 0u);
+                    gv[j][e] = v ? __ldg(g + f) : 0.f;
+                    rv[j][e] = v ? r[f] : 0.f;
+                    ok |= (uint32_t)v << (4 * j + e);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t key = key_of(__fadd_rn(gv[j][e], rv[j][e]));
+                    bool in = (ok >> (4 * j + e)) & 1u;
+                    if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
+                    if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
                 }
             }
         } else {
@@ -258,7 +267,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                 for (int e = 0; e < 4; ++e) {
                     uint32_t key = key_of(tl.a[j][e]);
                     bool in = (tl.valid >> (4 * j + e)) & 1u;
-                    if (LEVEL > 0) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
+                    if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
                     if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
                 }
             }

@@ -107,6 +107,20 @@ def test_every_route_gives_the_same_bits(path):
         assert all(c[1] == 1 for c in seen), seen
 
 
+def test_candidate_path_needs_no_redo_in_error_feedback_steady_state():
+    """Re-using a few gradients makes unsent entries pile up just below the threshold (a cliff in
+    the magnitude distribution).  The sampled threshold is an exact order statistic, so the
+    candidate set must still come out large enough -- and small enough -- at every step."""
+    n = 3_000_000
+    base = [randn(n, 300 + s) for s in range(2)]
+    grads = [base[s % 2] for s in range(10)]
+    seen = []
+    check_topk_against_oracle([n], 0.01, grads, expect_counters=seen.append)
+    assert all(c[1] == 0 and c[2] == 0 for c in seen), seen
+    k = 30_000
+    assert all(k <= c[0] <= 4 * k + 600_000 for c in seen), seen
+
+
 def test_sample_blind_spot_falls_back_and_stays_exact():
     """All large values sit where the sample never looks (groups that are not a multiple of the
     stride), so the sampled threshold is far too low or too high; the result must not care."""
