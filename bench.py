@@ -158,6 +158,8 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     dev = f"cuda:{local_rank}"
     api.lib()                                    # no fallback: raises when libgc.so is missing
     plan = api.Plan(w.sizes, w.density, device=local_rank)
+    if args.path == "exact":
+        plan.set_option(api.GC_OPT_PATH, api.GC_PATH_EXACT)
     n, k, W = plan.total_n, plan.total_cap, w.workers
     stream = torch.cuda.current_stream()
 
@@ -324,6 +326,8 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload 0..4 (default 2: 110M BERT-base shape)")
     ap.add_argument("--impl", default="gc", choices=["gc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="auto", choices=["auto", "exact"],
+                    help="auto: one-pass candidate path (default); exact: multi-pass kernels only")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end region")
     ap.add_argument("--input-sets", type=int, default=N_INPUT_SETS,
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "gc_fast.cuh"
+#include "gc_threshold.cuh"
 
 using namespace gc;
 
@@ -31,6 +32,7 @@ struct gc_plan_s {
     size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
            control_bytes = 0, off_tinfo = 0, off_cidx = 0, off_cval = 0, ws_bytes = 0;
     int sm_count = 0;
+    int grid_thr = 0;
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
     unsigned long long launches = 0;
     int last_cuda_error = 0;
@@ -118,7 +120,20 @@ void finish_layout(gc_plan_s* p) {
     for (uint32_t t = 0; t < p->T; ++t) {
         TensorDesc& d = p->desc[t];
         uint64_t ccap = d.n;
-        if (p->mode == GC_TOPK) sample_params(d, p->density, p->rank_permille, &ccap);
+        if (p->mode == GC_TOPK) {
+            sample_params(d, p->density, p->rank_permille, &ccap);
+        } else {
+            // threshold mode: the sample is part of the definition -- one 4-element group out of
+            // `stride`, rank k_s = min(m, max(1, ceil(density * m))) over its m elements
+            d.sstride = d.n ? d.stride : 0u;
+            uint64_t groups = ((uint64_t)d.n + 3) / 4, m = 0;
+            if (d.sstride) {
+                uint64_t nsg = (groups + d.sstride - 1) / d.sstride;
+                uint64_t last_first = (nsg - 1) * (uint64_t)d.sstride * 4;     // first element of the last sampled group
+                m = (nsg - 1) * 4 + std::min<uint64_t>(4, d.n - last_first);
+            }
+            d.srank = (uint32_t)k_rule(m, p->density);
+        }
         uint64_t nst = 0;
         if (d.sstride) {
             uint64_t groups = ((uint64_t)d.n + 3) / 4;
@@ -240,6 +255,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, SRC_FOLD>, kBlock);
     p->grid_compact = p->sm_count * blocks_per_sm(k_compact, kBlock);
     p->grid_fold = p->sm_count * blocks_per_sm(k_fold_cand, kBlock);
+    p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
     p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
     p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact, kBlock);
@@ -305,7 +321,6 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         (reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(out_idx) & 3u) ||
         (reinterpret_cast<uintptr_t>(out_val) & 3u))
         return GC_E_INVALID;
-    if (p->mode != GC_TOPK) return GC_E_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
     {
@@ -320,6 +335,24 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
     const int gcp = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
     char* wb = static_cast<char*>(workspace);
+    if (p->mode == GC_THRESHOLD) {
+        // exact order statistic of the sample (three radix levels), then one fused pass
+        WsView sws = ws;
+        sws.sel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+        const int gs = (int)std::min<uint32_t>(p->nstiles, (uint32_t)p->grid_sample);
+        { Timed tm(p, s, GC_K_SAMPLE);
+          k_hist<0, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
+        { Timed tm(p, s, GC_K_SAMPLE);
+          k_hist<1, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
+        { Timed tm(p, s, GC_K_SAMPLE);
+          k_hist<2, SRC_SAMPLE><<<gs, kBlock, 0, s>>>(p->d_desc, p->T, p->nstiles, grad, residual, sws); }
+        { Timed tm(p, s, GC_K_THRESHOLD_EMIT);
+          const int gt = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_thr);
+          k_threshold_emit<<<gt, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, out_idx, out_val,
+                                                 out_count, ws, sws.sel, 0); }
+        GC_CUDA(p, cudaGetLastError());
+        return GC_OK;
+    }
     if (p->path == GC_PATH_EXACT) {
         // exact multi-pass path on its own: fold + three histogram levels + ordered compaction
         { Timed tm(p, s, GC_K_FOLD_HIST);
@@ -504,6 +537,7 @@ const char* gc_kernel_name(int id) {
         case GC_K_DECODE_ADD: return "decode_add";
         case GC_K_COPY: return "copy";
         case GC_K_SAMPLE: return "sample";
+        case GC_K_THRESHOLD_EMIT: return "threshold_emit";
         case GC_K_FOLD_CAND: return "fold_cand";
         case GC_K_CAND_REFINE: return "cand_refine";
         case GC_K_CAND_COMPACT: return "cand_compact";

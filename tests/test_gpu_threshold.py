@@ -1,0 +1,115 @@
+"""GPU parity of the threshold-estimation variant (GC_THRESHOLD) against the CPU oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_01981_b200 import api, build, synth
+from helpers import GpuWorker, bits, same_f32_bits, to_np_u32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    api.lib()
+
+
+def randn(n, seed, scale=1.0):
+    return torch.randn(n, generator=torch.Generator().manual_seed(seed)) * scale
+
+
+def check_threshold(sizes, density, grads, stride=0, cap_factor=0.0, expect_truncated=None):
+    plan = api.Plan(sizes, density, mode=api.GC_THRESHOLD, device=0, sample_stride=stride,
+                    cap_factor=cap_factor)
+    w = GpuWorker(plan)
+    T = len(sizes)
+    caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
+    strides = [plan.query(api.GC_Q_TENSOR_STRIDE, t) for t in range(T)]
+    n = plan.total_n
+    r_cpu = np.zeros(n, np.float32)
+    for step, g in enumerate(grads):
+        gd = g.cuda()
+        if gd.numel() < 4:
+            gd = torch.cat([gd, torch.zeros(4 - gd.numel(), device="cuda")])
+        w.step(gd)
+        st, det = plan.last_status(w.ws)
+        g_cpu = g.numpy()
+        cnt = w.count.cpu().numpy()
+        gi, gv = to_np_u32(w.idx), to_np_u32(w.val)
+        off, truncated = 0, False
+        for t, sz in enumerate(sizes):
+            oi, ov, hits, tau = oracle.threshold_compress(g_cpu[off:off + sz], r_cpu[off:off + sz], density,
+                                                          strides[t], caps[t], index_base=off)
+            assert cnt[t] == oi.size and cnt[T + t] == hits, (step, t, cnt[t], oi.size, cnt[T + t], hits)
+            assert np.array_equal(gi[offs[t]:offs[t] + oi.size], oi), (step, t)
+            assert same_f32_bits(gv[offs[t]:offs[t] + oi.size], bits(ov)), (step, t)
+            truncated |= hits > caps[t]
+            off += sz
+        assert same_f32_bits(to_np_u32(w.residual[:n]), bits(r_cpu)), f"step {step}: residual differs"
+        assert st == (api.GC_W_TRUNCATED if truncated else api.GC_OK), (st, det)
+        if expect_truncated is not None:
+            assert truncated == expect_truncated
+    return plan, w
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 33, 1025, 8193, 65536, 65537, 100_003, (1 << 20) + 1])
+@pytest.mark.parametrize("density", [0.001, 0.05])
+def test_threshold_single_tensor_sizes(n, density):
+    check_threshold([n], density, [randn(n, 3 * n + s) for s in range(2)])
+
+
+@pytest.mark.parametrize("stride,cap_factor", [(0, 0.0), (1, 1.0), (3, 1.5), (16, 4.0), (64, 1.0)])
+def test_threshold_many_ragged_tensors(stride, cap_factor):
+    sizes = [5, 3, 1000, 7, 8193, 64, 1, 0, 2, 70_001, 300_000, 0, 6, 131_073]
+    n = sum(sizes)
+    check_threshold(sizes, 0.01, [randn(n, 500 + s) for s in range(3)], stride=stride, cap_factor=cap_factor)
+
+
+def test_threshold_truncation_keeps_a_prefix():
+    # the sample (stride 64) only sees tiny values, so nearly everything is a hit and the
+    # capacity cuts it to the first `cap` in index order
+    n = 400_000
+    g = randn(n, 8)
+    grp = torch.arange(n) // 4
+    g[(grp % 64) == 0] *= 1e-3
+    check_threshold([n], 0.01, [g, g], expect_truncated=True)
+
+
+def test_threshold_ties_at_tau():
+    n = 300_000
+    g = synth.quantised_gradient(n, 21)
+    check_threshold([n, n // 3], 0.02, [torch.cat([g, g[:n // 3]])] * 2, cap_factor=8.0)
+
+
+def test_threshold_config4_resnet_workers_and_decode():
+    w = synth.workload(3)
+    plan = api.Plan(w.sizes, w.density, mode=api.GC_THRESHOLD, device=0)
+    T, n = len(w.sizes), plan.total_n
+    caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
+    strides = [plan.query(api.GC_Q_TENSOR_STRIDE, t) for t in range(T)]
+    workers, pairs = [GpuWorker(plan) for _ in range(3)], []
+    for i, wk in enumerate(workers):
+        g = synth.gradient(w, i, 0, device="cuda")
+        wk.step(g)
+        g_cpu, r_cpu = g.cpu().numpy(), np.zeros(n, np.float32)
+        cnt, gi, gv = wk.count.cpu().numpy(), to_np_u32(wk.idx), to_np_u32(wk.val)
+        off, all_i, all_v = 0, [], []
+        for t, sz in enumerate(w.sizes):
+            oi, ov, hits, _ = oracle.threshold_compress(g_cpu[off:off + sz], r_cpu[off:off + sz], w.density,
+                                                        strides[t], caps[t], index_base=off)
+            assert cnt[t] == oi.size and cnt[T + t] == hits
+            assert np.array_equal(gi[offs[t]:offs[t] + oi.size], oi)
+            assert np.array_equal(gv[offs[t]:offs[t] + oi.size], bits(ov))
+            all_i.append(oi); all_v.append(ov)
+            off += sz
+        assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r_cpu))
+        pairs.append((np.concatenate(all_i), np.concatenate(all_v)))
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([x.idx for x in workers], [x.val for x in workers], [x.count for x in workers],
+                               out, True, workers[0].ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
