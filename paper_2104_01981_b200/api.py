@@ -14,7 +14,7 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SO = os.path.join(_HERE, "libgc.so")
+_SO = os.environ.get("GC_LIBRARY_PATH") or os.path.join(_HERE, "libgc.so")
 
 GC_OK, GC_E_INVALID, GC_E_UNSUPPORTED, GC_E_CUDA, GC_E_TOO_LARGE, GC_E_TIMEOUT = 0, -1, -2, -3, -4, -5
 GC_W_TRUNCATED = 1

@@ -27,8 +27,8 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, defines=(), out: str = SO) -> str:
+    if not force and not _stale() and out == SO:
         return SO
     cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo",
            "-gencode", "arch=compute_100a,code=sm_100a",
@@ -36,9 +36,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", SO] + [os.path.join(CSRC, s) for s in SOURCES]
+    cmd += [f"-D{d}" for d in defines]
+    cmd += ["-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
-    return SO
+    return out
 
 
 if __name__ == "__main__":

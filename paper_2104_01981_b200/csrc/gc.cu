@@ -30,7 +30,7 @@ struct gc_plan_s {
     uint32_t rank_permille = 1000;          // scales the sample rank (testing aid)
     // workspace layout (byte offsets)
     size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
-           control_bytes = 0, off_tinfo = 0, off_cidx = 0, off_cval = 0, ws_bytes = 0;
+           control_bytes = 0, off_tinfo = 0, off_cidx = 0, ws_bytes = 0;
     int sm_count = 0;
     int grid_thr = 0;
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
@@ -163,8 +163,7 @@ void finish_layout(gc_plan_s* p) {
     p->control_bytes = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
     p->off_tinfo = p->control_bytes;
     p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
-    p->off_cval = align_up(p->off_cidx + sizeof(uint32_t) * (size_t)p->cand_cap_alloc, 256);
-    p->ws_bytes = align_up(p->off_cval + sizeof(float) * (size_t)p->cand_cap_alloc, 256);
+    p->ws_bytes = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
 }
 
 int upload_table(gc_plan_s* p) {
@@ -254,7 +253,21 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     }
     p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, SRC_FOLD>, kBlock);
     p->grid_compact = p->sm_count * blocks_per_sm(k_compact, kBlock);
-    p->grid_fold = p->sm_count * blocks_per_sm(k_fold_cand, kBlock);
+    {
+        cudaError_t ea = cudaFuncSetAttribute(k_fold_cand, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kFoldSmemBytes);
+        int nb = 0;
+        if (ea == cudaSuccess)
+            ea = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fold_cand, kBlock, kFoldSmemBytes);
+        if (ea != cudaSuccess || nb < 1) {
+            (void)cudaGetLastError();
+            p->last_cuda_error = (int)ea;
+            cudaFree(p->d_desc);
+            delete p;
+            return GC_E_CUDA;
+        }
+        p->grid_fold = p->sm_count * nb;
+    }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
     p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
@@ -371,8 +384,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     WsView sws = ws;                 // sample select works on its own records
     sws.sel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
     CandView cv;
-    cv.idx = reinterpret_cast<uint32_t*>(wb + p->off_cidx);
-    cv.val = reinterpret_cast<float*>(wb + p->off_cval);
+    cv.pair = reinterpret_cast<uint2*>(wb + p->off_cidx);
     cv.chunk_info = reinterpret_cast<uint2*>(wb + p->off_tinfo);
     cv.cap = p->cand_cap;
     cv.ssel = sws.sel;
@@ -387,7 +399,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     }
     { Timed tm(p, s, GC_K_FOLD_CAND);
       const int gf = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_fold);
-      k_fold_cand<<<gf, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
+      k_fold_cand<<<gf, kBlock, kFoldSmemBytes, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
     {
         const int gch = (int)std::min<uint32_t>((nt + 2 * kWarps - 1) / (2 * kWarps), (uint32_t)p->grid_chist);
         { Timed tm(p, s, GC_K_CAND_REFINE);

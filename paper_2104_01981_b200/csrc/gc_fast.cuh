@@ -19,8 +19,7 @@
 namespace gc {
 
 struct CandView {
-    uint32_t* idx;           // [cap] flat index of each candidate
-    float* val;              // [cap] a = g + r of each candidate
+    uint2* pair;             // [cap] (flat index, bits of a = g + r) of each candidate
     uint2* chunk_info;       // [ntiles * kWarps] (first slot, count) per warp chunk
     uint32_t cap;
     const TensorSel* ssel;   // [n_tensors] sample selection record (21-bit prefix = tau_lo >> 10)
@@ -51,19 +50,60 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
 }
 
 // ----------------------------------------------------------------------------- fold + candidates
+// Asynchronous staging: each thread copies ITS OWN four 16-byte vectors of g and of r for the
+// tiles ahead into shared memory with cp.async (no registers held, no barrier needed because a
+// thread only ever reads back what it copied itself), kFoldStages tiles deep.  Tiles that touch
+// the ragged first or last element of a tensor are loaded synchronously instead.
+#ifndef GC_FOLD_ASYNC
+#define GC_FOLD_ASYNC 1
+#endif
+#ifndef GC_FOLD_INTERLEAVE
+#define GC_FOLD_INTERLEAVE 1
+#endif
+#ifndef GC_FOLD_MINBLOCKS
+#define GC_FOLD_MINBLOCKS 1
+#endif
+constexpr int kFoldStages = GC_FOLD_ASYNC ? 3 : 0;
+constexpr int kEmitStage = 64;              // candidates of one warp chunk staged in shared memory
+constexpr size_t kFoldSmemBytes = (size_t)kFoldStages * 2 * kTile * sizeof(float);
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gptr) {
+    uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ bool tile_is_interior(const TileGeom& q) {
+    return q.lo == q.base && q.hi == q.base + (uint32_t)kTile;
+}
+
 // Reads g and r, writes a into r, emits candidates.  No block-wide barrier in the tile loop:
 // every warp ranks and stores the candidates of its own chunk.
-static __global__ void __launch_bounds__(kBlock)
+static __global__ void __launch_bounds__(kBlock, GC_FOLD_MINBLOCKS)
 k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
     constexpr int NB = 1 << level_bits(0);
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    float* const s_g = reinterpret_cast<float*>(s_dyn);
+    float* const s_r = s_g + (size_t)kFoldStages * kTile;
     __shared__ uint32_t s_hist[NB];
     __shared__ uint32_t s_scratch[kWarps + 4];
     __shared__ uint32_t s_last;
+    __shared__ uint2 s_emit[kWarps][kEmitStage];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#if GC_FOLD_INTERLEAVE
+    // tile i of this CTA = blockIdx.x + i * gridDim.x: at any time the CTAs sweep one window
+    const uint32_t tstep = gridDim.x;
+    const uint32_t first = blockIdx.x;
+    const uint32_t last = ntiles;
+#else
+    const uint32_t tstep = 1;
     const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
     const uint32_t first = blockIdx.x * per;
     const uint32_t last = min(ntiles, first + per);
+#endif
     if (first >= last) return;
     for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
     __syncthreads();
@@ -73,6 +113,32 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
     uint32_t tau = d.sstride ? (cv.ssel[t].prefix << level_shift(1)) : 0u;
     uint32_t tiles_here = 0;
     uint32_t slab_next = 0, slab_left = 0;       // this warp's current slab (warp-uniform)
+
+    // prefetch cursor
+    uint32_t pt = t;
+    TensorDesc pd = d;
+    const uint32_t my_off = warp * kWarpChunk + lane * 4;        // + j * 128 elements
+    auto issue = [&](uint32_t p, uint32_t seq) {
+#if GC_FOLD_ASYNC
+        if (p < last) {
+            if (p >= pd.tile0 + pd.ntiles) { pt = find_tensor(desc, T, p); pd = desc[pt]; }
+            const TileGeom q = tile_geom(pd, p - pd.tile0);
+            if (tile_is_interior(q)) {
+                const uint32_t st = seq % (uint32_t)kFoldStages;
+                float* dg = s_g + (size_t)st * kTile + my_off;
+                float* dr = s_r + (size_t)st * kTile + my_off;
+                const float* gg = g + q.base + my_off;
+                const float* gr = r + q.base + my_off;
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+                    cp_async16(dg + j * 128, gg + j * 128);
+                    cp_async16(dr + j * 128, gr + j * 128);
+                }
+            }
+        }
+        cp_async_commit();
+#endif
+    };
 
     auto flush = [&]() {
         if (tiles_here == 0) return;
@@ -96,7 +162,12 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         tiles_here = 0;
     };
 
-    for (uint32_t tile = first; tile < last; ++tile) {
+#pragma unroll
+    for (int s = 0; s < kFoldStages - 1; ++s) issue(first + s * tstep, s);
+
+    uint32_t seq = 0;
+    for (uint32_t tile = first; tile < last; tile += tstep, ++seq) {
+        issue(tile + (kFoldStages - 1) * tstep, seq + kFoldStages - 1);
         if (tile >= d.tile0 + d.ntiles) {
             flush();
             t = find_tensor(desc, T, tile);
@@ -105,7 +176,28 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         }
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;
-        load_tile<true>(g, r, tg, warp, lane, tl);
+#if GC_FOLD_ASYNC
+        cp_async_wait<kFoldStages - 1>();
+        if (tile_is_interior(tg)) {
+            const uint32_t st = seq % (uint32_t)kFoldStages;
+            const float* sgp = s_g + (size_t)st * kTile + my_off;
+            const float* srp = s_r + (size_t)st * kTile + my_off;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                const float4 gv = *reinterpret_cast<const float4*>(sgp + j * 128);
+                const float4 rv = *reinterpret_cast<const float4*>(srp + j * 128);
+                float4 a;
+                a.x = __fadd_rn(gv.x, rv.x); a.y = __fadd_rn(gv.y, rv.y);
+                a.z = __fadd_rn(gv.z, rv.z); a.w = __fadd_rn(gv.w, rv.w);
+                *reinterpret_cast<float4*>(r + tg.base + my_off + j * 128) = a;
+                tl.a[j][0] = a.x; tl.a[j][1] = a.y; tl.a[j][2] = a.z; tl.a[j][3] = a.w;
+            }
+            tl.valid = 0xFFFFu;
+        } else
+#endif
+        {
+            load_tile<true>(g, r, tg, warp, lane, tl);
+        }
         uint32_t cnt[kVpt], cm = 0;
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) {
@@ -136,24 +228,40 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         }
         const uint32_t cbase = slab_next;
         if (fits) { slab_next += wtot; slab_left -= wtot; }
+#ifndef GC_EXP_NO_CHUNKINFO
         if (lane == 0) cv.chunk_info[(size_t)tile * kWarps + warp] = make_uint2(cbase, fits ? wtot : 0u);
-        if (cm != 0u && fits) {
+#endif
+        // emission: candidates are first ranked into the warp's shared staging row, then written
+        // out as one contiguous run of 8-byte pairs (a chunk rarely holds more than a dozen)
+        const bool staged = wtot <= (uint32_t)kEmitStage;
+        if (fits && wtot != 0u) {
+            if (cm != 0u) {
 #pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                uint32_t pos = cbase + rk[j];
+                for (int j = 0; j < kVpt; ++j) {
+                    uint32_t pos = rk[j];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if ((cm >> (4 * j + e)) & 1u) {
-                        cv.idx[pos] = vec_index(tg.base, warp, lane, j) + e;
-                        cv.val[pos] = tl.a[j][e];
-                        atomicAdd(&s_hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
-                        ++pos;
+                    for (int e = 0; e < 4; ++e) {
+                        if ((cm >> (4 * j + e)) & 1u) {
+                            const uint2 pr = make_uint2(vec_index(tg.base, warp, lane, j) + e,
+                                                        __float_as_uint(tl.a[j][e]));
+                            if (staged) s_emit[warp][pos] = pr; else cv.pair[cbase + pos] = pr;
+                            atomicAdd(&s_hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
+                            ++pos;
+                        }
                     }
                 }
+            }
+            if (staged) {
+                __syncwarp();
+                for (uint32_t i = lane; i < wtot; i += 32) cv.pair[cbase + i] = s_emit[warp][i];
+                __syncwarp();
             }
         }
         ++tiles_here;
     }
+#if GC_FOLD_ASYNC
+    cp_async_wait<0>();
+#endif
     flush();
 }
 
@@ -224,7 +332,7 @@ k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, Ws
                 uint32_t j = j0 + lane;
                 uint32_t slot = cand_slot(tc, j);
                 if (j < tc.total) {
-                    uint32_t key = key_of(cv.val[slot]);
+                    uint32_t key = cv.pair[slot].y & kKeyMask;
                     if ((key >> (SH + level_bits(LEVEL))) == prefix)
                         atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
                 }
@@ -278,7 +386,7 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
         for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
             uint32_t j = j0 + lane;
             uint32_t slot = cand_slot(tc, j);
-            uint32_t key = j < tc.total ? key_of(cv.val[slot]) : 0u;
+            uint32_t key = j < tc.total ? (cv.pair[slot].y & kKeyMask) : 0u;
             bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
             ngt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
             neq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
@@ -309,7 +417,7 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
             uint32_t slot = cand_slot(tc, j);
             float v = 0.f;
             uint32_t f = 0;
-            if (j < tc.total) { v = cv.val[slot]; f = cv.idx[slot]; }
+            if (j < tc.total) { const uint2 pr = cv.pair[slot]; f = pr.x; v = __uint_as_float(pr.y); }
             uint32_t key = key_of(v);
             bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
             unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
