@@ -158,8 +158,8 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     dev = f"cuda:{local_rank}"
     api.lib()                                    # no fallback: raises when libgc.so is missing
     plan = api.Plan(w.sizes, w.density, device=local_rank)
-    if args.path == "exact":
-        plan.set_option(api.GC_OPT_PATH, api.GC_PATH_EXACT)
+    if args.path != "auto":
+        plan.set_option(api.GC_OPT_PATH, {"exact": api.GC_PATH_EXACT, "staged": api.GC_PATH_STAGED}[args.path])
     n, k, W = plan.total_n, plan.total_cap, w.workers
     stream = torch.cuda.current_stream()
 
@@ -206,6 +206,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     if st != api.GC_OK:
         raise RuntimeError(f"device status {st} (detail {det}) after the timed region")
     counters = plan.last_counters(ws)
+    args.phase_us = plan.last_phase_times(ws)
 
     # ---- timed region 1b: same loop without the per-kernel events (the headline value)
     barrier()
@@ -289,7 +290,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
                  for name, v in per_kernel.items()}
     dom = max(per_kernel.items(), key=lambda kv: kv[1][0])[0]
     alg_bytes = {"fold_hist": 12.0 * n, "hist_refine": 4.0 * n, "compact": 4.0 * n + 8.0 * k,
-                 "decode_clear": 4.0 * n, "decode_add": 8.0 * k, "fold_cand": 12.0 * n,
+                 "decode_clear": 4.0 * n, "decode_add": 8.0 * k, "fold_cand": 12.0 * n, "compress_fused": 12.0 * n + 8.0 * k,
                  "threshold_emit": 12.0 * n + 8.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
@@ -324,6 +325,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
                 "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps,
                 "what": "gc_compress_host: pinned host gradient -> device, compress, pairs -> pinned host; "
                         "decode stays on the device"},
+        "fused_phase_us_last_step": [round(x, 2) for x in args.phase_us],
         "gpu_launches": launches,
         "path_counters": {"candidates_last_step": counters[0], "candidate_overflow": counters[1],
                           "tensors_redone": counters[2], "k": k},
@@ -344,8 +346,9 @@ def main():
     ap.add_argument("--config", type=int, default=2, help="workload 0..4 (default 2: 110M BERT-base shape)")
     ap.add_argument("--impl", default="gc", choices=["gc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", default="auto", choices=["auto", "exact"],
-                    help="auto: one-pass candidate path (default); exact: multi-pass kernels only")
+    ap.add_argument("--path", default="auto", choices=["auto", "staged", "exact"],
+                    help="auto: one-pass candidate path in one cooperative launch (default); staged: the "
+                         "same phases as separate launches; exact: multi-pass kernels only")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end region")
     ap.add_argument("--input-sets", type=int, default=N_INPUT_SETS,
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")

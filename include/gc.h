@@ -103,7 +103,9 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  * gc_plan_set_option -- host; tune or steer a plan before it is used (never while work that
  * uses it is in flight).  The selected set never depends on these options, only the route.
  *   GC_OPT_PATH                  GC_PATH_AUTO (default): one-pass candidate path with the exact
- *                                multi-pass kernels as its safety net; GC_PATH_EXACT: multi-pass only
+ *                                multi-pass kernels as its safety net, all in one cooperative launch;
+ *                                GC_PATH_STAGED: the same phases as separate launches;
+ *                                GC_PATH_EXACT: multi-pass kernels only
  *   GC_OPT_SAMPLE_RANK_PERMILLE  scales the sample rank that sets the candidate threshold
  *                                (1000 = default; small values make the candidate set too small
  *                                and so exercise the safety net -- a testing aid)
@@ -115,6 +117,7 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
 #define GC_OPT_CANDIDATE_CAPACITY    2
 #define GC_PATH_AUTO   0
 #define GC_PATH_EXACT  1
+#define GC_PATH_STAGED 2
 int gc_plan_set_option(gc_plan_t *plan, int option, uint64_t value);
 
 /* gc_plan_query -- host-side lookup of plan facts; never touches the device.
@@ -221,6 +224,7 @@ int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_stagin
 #define GC_K_CAND_REFINE   10   /* radix-select levels over the candidate lists              */
 #define GC_K_CAND_COMPACT  11   /* ordered emission from the candidate lists                 */
 #define GC_K_THRESHOLD_EMIT 12  /* threshold mode: fold + send everything at or above tau    */
+#define GC_K_FUSED         13   /* whole top-k compress as one cooperative launch            */
 #define GC_K_COUNT         16
 int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
 int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);
@@ -264,6 +268,14 @@ int gc_compress_noalloc(const float *grad, float *residual, uint32_t n, uint32_t
  *   whose candidate set was smaller than k (redone individually).
  */
 int gc_last_counters(gc_plan_t *plan, const void *workspace, void *stream, uint32_t counters[3]);
+
+/*
+ * gc_last_phase_times -- diagnostic (SYNCHRONISES the stream): durations in nanoseconds of the
+ * phases of the most recent fused top-k launch on this workspace, as stamped by its first CTA
+ * (phase i ends at barrier i).  *n_phases receives how many of ns[0..19] are valid.
+ */
+int gc_last_phase_times(gc_plan_t *plan, const void *workspace, void *stream, uint64_t ns[20],
+                        uint32_t *n_phases);
 
 /* gc_last_cuda_error -- host; the cudaError_t value of the most recent failed runtime call
  * made on behalf of this plan (0 if none). */

@@ -25,7 +25,7 @@ GC_K_COUNT = 16
  GC_Q_TENSOR_CAP, GC_Q_TENSOR_OFFSET, GC_Q_TENSOR_OUT_OFFSET, GC_Q_TENSOR_STRIDE, GC_Q_MODE,
  GC_Q_KERNEL_LAUNCHES, GC_Q_CANDIDATE_CAPACITY) = range(13)
 GC_OPT_PATH, GC_OPT_SAMPLE_RANK_PERMILLE, GC_OPT_CANDIDATE_CAPACITY = 0, 1, 2
-GC_PATH_AUTO, GC_PATH_EXACT = 0, 1
+GC_PATH_AUTO, GC_PATH_EXACT, GC_PATH_STAGED = 0, 1, 2
 
 _ERR = {GC_E_INVALID: "GC_E_INVALID", GC_E_UNSUPPORTED: "GC_E_UNSUPPORTED", GC_E_CUDA: "GC_E_CUDA",
         GC_E_TOO_LARGE: "GC_E_TOO_LARGE", GC_E_TIMEOUT: "GC_E_TIMEOUT"}
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.gc_compress_noalloc.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
         L.gc_last_counters.restype = i32
         L.gc_last_counters.argtypes = [vp, vp, vp, vp]
+        L.gc_last_phase_times.restype = i32
+        L.gc_last_phase_times.argtypes = [vp, vp, vp, vp, vp]
         L.gc_last_cuda_error.restype = i32
         L.gc_last_cuda_error.argtypes = [vp]
         L.gc_destroy.restype = i32
@@ -239,6 +241,15 @@ class Plan:
         if rc < 0:
             raise GcError("gc_last_counters", rc)
         return int(c[0]), int(c[1]), int(c[2])
+
+    def last_phase_times(self, workspace: torch.Tensor, stream=None):
+        """Phase durations (microseconds) of the last fused top-k launch; synchronises."""
+        ns = (ctypes.c_uint64 * 20)()
+        n = ctypes.c_uint32(0)
+        rc = lib().gc_last_phase_times(self._h, _ptr(workspace), _stream_handle(stream), ns, ctypes.byref(n))
+        if rc < 0:
+            raise GcError("gc_last_phase_times", rc)
+        return [ns[i] / 1e3 for i in range(n.value)]
 
     def launches(self) -> int:
         return self.query(GC_Q_KERNEL_LAUNCHES)

@@ -34,6 +34,7 @@ struct gc_plan_s {
     int sm_count = 0;
     int grid_thr = 0;
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
+    int grid_fused = 0;                     // CTAs of the cooperative launch (0 = not available)
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
@@ -253,25 +254,19 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     }
     p->grid_hist = p->sm_count * blocks_per_sm(k_hist<0, SRC_FOLD>, kBlock);
     p->grid_compact = p->sm_count * blocks_per_sm(k_compact, kBlock);
+    p->grid_fold = p->sm_count * blocks_per_sm(k_fold_cand, kBlock);
     {
-        cudaError_t ea = cudaFuncSetAttribute(k_fold_cand, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kFoldSmemBytes);
-        int nb = 0;
-        if (ea == cudaSuccess)
-            ea = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_fold_cand, kBlock, kFoldSmemBytes);
-        if (ea != cudaSuccess || nb < 1) {
+        int coop = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess) {
             (void)cudaGetLastError();
-            p->last_cuda_error = (int)ea;
-            cudaFree(p->d_desc);
-            delete p;
-            return GC_E_CUDA;
+            coop = 0;
         }
-        p->grid_fold = p->sm_count * nb;
+        p->grid_fused = coop ? p->sm_count * blocks_per_sm(k_compress_fused, kBlock) : 0;
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
     p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
-    p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact, kBlock);
+    p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact<true>, kBlock);
     *out = p;
     return GC_OK;
 }
@@ -280,7 +275,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
     if (p == nullptr) return GC_E_INVALID;
     switch (option) {
         case GC_OPT_PATH:
-            if (value != GC_PATH_AUTO && value != GC_PATH_EXACT) return GC_E_INVALID;
+            if (value != GC_PATH_AUTO && value != GC_PATH_EXACT && value != GC_PATH_STAGED) return GC_E_INVALID;
             p->path = (int)value;
             return GC_OK;
         case GC_OPT_SAMPLE_RANK_PERMILLE:
@@ -383,11 +378,28 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     // candidates; then the exact kernels, gated to the tensors (normally none) it gave up on
     WsView sws = ws;                 // sample select works on its own records
     sws.sel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+    WsView gws = ws;                 // redo of failed tensors: own records, gated by the main ones
+    gws.sel = reinterpret_cast<TensorSel*>(wb + p->off_gsel);
+    gws.gate = ws.sel;
     CandView cv;
     cv.pair = reinterpret_cast<uint2*>(wb + p->off_cidx);
     cv.chunk_info = reinterpret_cast<uint2*>(wb + p->off_tinfo);
+    cv.group_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
     cv.cap = p->cand_cap;
     cv.ssel = sws.sel;
+    if (p->path == GC_PATH_AUTO && p->grid_fused > 0) {
+        // everything in one cooperative launch
+        FusedArgs fa;
+        fa.desc = p->d_desc; fa.T = p->T; fa.ntiles = nt; fa.nstiles = p->nstiles; fa.ngroups = p->ngroups;
+        fa.g = grad; fa.r = residual; fa.out_idx = out_idx; fa.out_val = out_val; fa.out_count = out_count;
+        fa.ws = ws; fa.sws = sws; fa.gws = gws; fa.cv = cv;
+        void* args[] = {&fa};
+        const uint32_t want = std::max<uint32_t>(std::max<uint32_t>(nt, p->nstiles), 1u);
+        const int gf = (int)std::min<uint32_t>(want, (uint32_t)p->grid_fused);
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_compress_fused, dim3(gf), dim3(kBlock), args, 0, s));
+        return GC_OK;
+    }
     if (p->nstiles > 0) {
         const int gs = (int)std::min<uint32_t>(p->nstiles, (uint32_t)p->grid_sample);
         // two radix levels on the sample: tau_lo is the exact srank-th sampled key cut to 21 bits,
@@ -399,7 +411,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     }
     { Timed tm(p, s, GC_K_FOLD_CAND);
       const int gf = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_fold);
-      k_fold_cand<<<gf, kBlock, kFoldSmemBytes, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
+      k_fold_cand<<<gf, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws, cv); }
     {
         const int gch = (int)std::min<uint32_t>((nt + 2 * kWarps - 1) / (2 * kWarps), (uint32_t)p->grid_chist);
         { Timed tm(p, s, GC_K_CAND_REFINE);
@@ -408,17 +420,15 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
           k_cand_hist<2><<<gch, kBlock, 0, s>>>(p->d_desc, p->T, nt, ws, cv); }
     }
     {
-        WsView cws = ws;             // group look-back words
-        cws.tile_state = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
         const int gcc = (int)std::min<uint32_t>(p->ngroups, (uint32_t)p->grid_ccompact);
-        Timed tm(p, s, GC_K_CAND_COMPACT);
-        k_cand_compact<<<gcc, kBlock, 0, s>>>(p->d_desc, p->T, p->ngroups, residual, out_idx, out_val,
-                                              out_count, cws, cv, 1);
+        { Timed tm(p, s, GC_K_CAND_COMPACT);
+          k_cand_compact<false><<<gcc, kBlock, 0, s>>>(p->d_desc, p->T, p->ngroups, residual, out_idx, out_val,
+                                                       out_count, ws, cv); }
+        { Timed tm(p, s, GC_K_CAND_COMPACT);
+          k_cand_compact<true><<<gcc, kBlock, 0, s>>>(p->d_desc, p->T, p->ngroups, residual, out_idx, out_val,
+                                                      out_count, ws, cv); }
     }
     {
-        WsView gws = ws;             // redo of failed tensors: own records, gated by the main ones
-        gws.sel = reinterpret_cast<TensorSel*>(wb + p->off_gsel);
-        gws.gate = ws.sel;
         { Timed tm(p, s, GC_K_HIST_REFINE);
           k_hist<0, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, gws); }
         { Timed tm(p, s, GC_K_HIST_REFINE);
@@ -550,6 +560,7 @@ const char* gc_kernel_name(int id) {
         case GC_K_COPY: return "copy";
         case GC_K_SAMPLE: return "sample";
         case GC_K_THRESHOLD_EMIT: return "threshold_emit";
+        case GC_K_FUSED: return "compress_fused";
         case GC_K_FOLD_CAND: return "fold_cand";
         case GC_K_CAND_REFINE: return "cand_refine";
         case GC_K_CAND_COMPACT: return "cand_compact";
@@ -565,6 +576,19 @@ int gc_last_counters(gc_plan_t* p, const void* workspace, void* stream, uint32_t
     GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
     GC_CUDA(p, cudaStreamSynchronize(s));
     counters[0] = h.cand_total; counters[1] = h.overflow; counters[2] = h.n_failed;
+    return GC_OK;
+}
+
+int gc_last_phase_times(gc_plan_t* p, const void* workspace, void* stream, uint64_t ns[20], uint32_t* n_phases) {
+    if (p == nullptr || workspace == nullptr || ns == nullptr || n_phases == nullptr) return GC_E_INVALID;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    WsHeader h;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
+    GC_CUDA(p, cudaStreamSynchronize(s));
+    uint32_t n = h.n_stamps > 20u ? 20u : h.n_stamps;
+    *n_phases = n > 0 ? n - 1 : 0;
+    for (uint32_t i = 0; i + 1 < n; ++i) ns[i] = h.stamp[i + 1] - h.stamp[i];
     return GC_OK;
 }
 

@@ -65,7 +65,11 @@ struct WsHeader {            // head of the workspace, 256 bytes
     uint32_t cand_total;     // candidate slots handed out so far
     uint32_t overflow;       // candidate buffer ran out: every tensor takes the exact multi-pass path
     uint32_t n_failed;       // tensors whose candidate set turned out too small
-    uint32_t reserved[49];
+    uint32_t barrier;        // arrivals at the grid barriers of the fused kernel (monotonic)
+    uint32_t n_stamps;       // phase time stamps recorded by CTA 0 of the fused kernel
+    uint32_t pad0[3];
+    unsigned long long stamp[20];   // %globaltimer (ns) at the start and after each phase
+    uint32_t reserved[4];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -96,6 +100,29 @@ struct GroupSpace {
 // ----------------------------------------------------------------------------- small helpers
 __device__ __forceinline__ uint32_t key_of(float a) { return __float_as_uint(a) & kKeyMask; }
 
+// Loads of data that another CTA may have written earlier in the SAME launch (the fused kernel
+// runs all phases in one grid) must not be served from this SM's L1: read them at L2.
+__device__ __forceinline__ uint32_t ld_cg(const uint32_t* p) { return __ldcg(p); }
+__device__ __forceinline__ float ld_cg(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ld_cg(const float4* p) { return __ldcg(p); }
+__device__ __forceinline__ uint2 ld_cg(const uint2* p) { return __ldcg(p); }
+__device__ __forceinline__ unsigned long long ld_cg(const unsigned long long* p) { return __ldcg(p); }
+
+constexpr int kEmitStage = 64;               // candidates of one warp chunk staged in shared memory
+
+// Static shared memory of every streaming kernel (one instance per CTA, reused by all phases).
+struct BlockSmem {
+    uint32_t hist[2048];
+    uint32_t scratch[kWarps + 4];
+    uint32_t last, tile;
+    uint32_t gt_tot[kWarps], eq_tot[kWarps], gt_ex[kWarps], eq_ex[kWarps];
+    uint32_t gt_sum, eq_sum;
+    unsigned long long excl;
+    unsigned long long red[kWarps];
+    int ok;
+    uint2 emit[kWarps][kEmitStage];
+};
+
 __device__ __forceinline__ void record_status(WsHeader* h, int32_t code, unsigned long long detail) {
     // errors (negative) win over warnings; first writer of a kind keeps its detail
     int32_t old = atomicCAS(&h->status, 0, code);
@@ -119,7 +146,10 @@ __device__ __forceinline__ uint32_t find_tensor(const TensorDesc* __restrict__ d
 __device__ __forceinline__ bool gate_open(const WsView& ws, uint32_t t) {
     // with a gate, a tensor is processed only if the candidate path failed for it (or overall)
     if (ws.gate == nullptr) return true;
-    return (ws.gate[t].flags & kSelFailed) != 0u || *(volatile uint32_t*)&ws.hdr->overflow != 0u;
+    return (ld_cg(&ws.gate[t].flags) & kSelFailed) != 0u || ld_cg(&ws.hdr->overflow) != 0u;
+}
+__device__ __forceinline__ bool nothing_to_redo(const WsView& ws) {
+    return ws.gate != nullptr && ld_cg(&ws.hdr->n_failed) == 0u && ld_cg(&ws.hdr->overflow) == 0u;
 }
 
 struct TileGeom { uint32_t base, lo, hi; };  // aligned start, first and one-past-last valid flat index
@@ -242,6 +272,43 @@ __device__ __forceinline__ unsigned long long lookback(unsigned long long* state
     }
     if (lane == 0) st_state(state + tile, kFlagPre | ((excl + agg) & kValMask));
     return excl;
+}
+
+__device__ __forceinline__ void phase_stamp(WsHeader* hdr) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long ts;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
+        uint32_t i = hdr->n_stamps;
+        if (i < 20u) { hdr->stamp[i] = ts; hdr->n_stamps = i + 1u; }
+    }
+}
+
+// ----------------------------------------------------------------------------- grid barrier
+// Barrier across all CTAs of a cooperative launch (all of them are resident).  The counter
+// only grows: the b-th barrier waits for b * gridDim.x arrivals.  The wait is bounded; if it
+// runs out the abort flag is raised, GC_E_TIMEOUT is recorded and every CTA leaves.
+__device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        __threadfence();
+        const uint32_t target = (passed + 1u) * gridDim.x;
+        atomicAdd(&hdr->barrier, 1u);
+        uint32_t spins = 0;
+        while (ld_cg(&hdr->barrier) < target) {
+            if (++spins > kSpinLimit || ld_cg(&hdr->abort) != 0u) { ok = 0; break; }
+            if (spins > 32) __nanosleep(spins > 4096 ? 400 : 60);
+        }
+        if (!ok) {
+            record_status(hdr, -5 /*GC_E_TIMEOUT*/, 0xB0000000ull + passed);
+            atomicExch(&hdr->abort, 1u);
+        }
+        __threadfence();
+        *s_ok = ok;
+    }
+    __syncthreads();
+    ++passed;
+    return *s_ok != 0;
 }
 
 }  // namespace gc

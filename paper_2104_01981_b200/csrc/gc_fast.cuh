@@ -13,6 +13,10 @@
 // visits and appends that chunk's candidates, in index order, to a slab of kSlab slots it
 // reserved with one atomic; chunk_info[tile * kWarps + warp] = (first slot, count).  Chunks
 // land in arbitrary order in the list; readers walk them by (tile, warp), which is index order.
+//
+// All phases exist as __device__ bodies.  k_compress_fused runs them back to back in ONE
+// cooperative launch with grid barriers in between; the k_* wrappers run them as separate
+// launches (same results, used when a cooperative launch is not wanted).
 #pragma once
 #include "gc_kernels.cuh"
 
@@ -21,6 +25,7 @@ namespace gc {
 struct CandView {
     uint2* pair;             // [cap] (flat index, bits of a = g + r) of each candidate
     uint2* chunk_info;       // [ntiles * kWarps] (first slot, count) per warp chunk
+    unsigned long long* group_cnt;   // [ngroups] (above-T << 31 | equal-T) counts per compaction group
     uint32_t cap;
     const TensorSel* ssel;   // [n_tensors] sample selection record (21-bit prefix = tau_lo >> 10)
 };
@@ -32,13 +37,13 @@ struct TileCands {
 __device__ __forceinline__ TileCands load_tile_cands(const CandView& cv, uint32_t tile, int lane) {
     TileCands tc;
     uint2 info = make_uint2(0u, 0u);
-    if (lane < kWarps) info = cv.chunk_info[(size_t)tile * kWarps + lane];
+    if (lane < kWarps) info = ld_cg(&cv.chunk_info[(size_t)tile * kWarps + lane]);
     tc.base = info.x; tc.cnt = info.y;
     tc.incl = warp_incl_scan(tc.cnt, lane);
     tc.total = __shfl_sync(0xFFFFFFFFu, tc.incl, 31);
     return tc;
 }
-// slot of the j-th candidate of the tile (all lanes call; j >= total gives a harmless slot of chunk 0)
+// slot of the j-th candidate of the tile (all lanes call; j >= total gives a harmless slot)
 __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
     uint32_t c = 0;
 #pragma unroll
@@ -50,154 +55,36 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
 }
 
 // ----------------------------------------------------------------------------- fold + candidates
-// Asynchronous staging: each thread copies ITS OWN four 16-byte vectors of g and of r for the
-// tiles ahead into shared memory with cp.async (no registers held, no barrier needed because a
-// thread only ever reads back what it copied itself), kFoldStages tiles deep.  Tiles that touch
-// the ragged first or last element of a tensor are loaded synchronously instead.
-#ifndef GC_FOLD_ASYNC
-#define GC_FOLD_ASYNC 1
-#endif
-#ifndef GC_FOLD_INTERLEAVE
-#define GC_FOLD_INTERLEAVE 1
-#endif
-#ifndef GC_FOLD_MINBLOCKS
-#define GC_FOLD_MINBLOCKS 1
-#endif
-constexpr int kFoldStages = GC_FOLD_ASYNC ? 3 : 0;
-constexpr int kEmitStage = 64;              // candidates of one warp chunk staged in shared memory
-constexpr size_t kFoldSmemBytes = (size_t)kFoldStages * 2 * kTile * sizeof(float);
-
-__device__ __forceinline__ void cp_async16(void* smem, const void* gptr) {
-    uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gptr) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ bool tile_is_interior(const TileGeom& q) {
-    return q.lo == q.base && q.hi == q.base + (uint32_t)kTile;
-}
-
-// Reads g and r, writes a into r, emits candidates.  No block-wide barrier in the tile loop:
-// every warp ranks and stores the candidates of its own chunk.
-static __global__ void __launch_bounds__(kBlock, GC_FOLD_MINBLOCKS)
-k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
-            const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
+// Reads g and r, writes a into r, emits candidates.  Tile i of a CTA is blockIdx.x + i *
+// gridDim.x, so at any moment the CTAs sweep one contiguous window of memory.  No block-wide
+// barrier in the tile loop: every warp ranks and stores the candidates of its own chunk.
+static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
+                               uint32_t ntiles, const float* __restrict__ g, float* __restrict__ r,
+                               const WsView& ws, const CandView& cv) {
     constexpr int NB = 1 << level_bits(0);
-    extern __shared__ __align__(16) unsigned char s_dyn[];
-    float* const s_g = reinterpret_cast<float*>(s_dyn);
-    float* const s_r = s_g + (size_t)kFoldStages * kTile;
-    __shared__ uint32_t s_hist[NB];
-    __shared__ uint32_t s_scratch[kWarps + 4];
-    __shared__ uint32_t s_last;
-    __shared__ uint2 s_emit[kWarps][kEmitStage];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-#if GC_FOLD_INTERLEAVE
-    // tile i of this CTA = blockIdx.x + i * gridDim.x: at any time the CTAs sweep one window
-    const uint32_t tstep = gridDim.x;
-    const uint32_t first = blockIdx.x;
-    const uint32_t last = ntiles;
-#else
-    const uint32_t tstep = 1;
-    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
-    const uint32_t first = blockIdx.x * per;
-    const uint32_t last = min(ntiles, first + per);
-#endif
-    if (first >= last) return;
-    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    const uint32_t first = blockIdx.x, tstep = gridDim.x;
+    if (first >= ntiles) return;
+    for (int b = tid; b < NB; b += kBlock) sm.hist[b] = 0u;
     __syncthreads();
 
     uint32_t t = find_tensor(desc, T, first);
     TensorDesc d = desc[t];
-    uint32_t tau = d.sstride ? (cv.ssel[t].prefix << level_shift(1)) : 0u;
+    uint32_t tau = d.sstride ? (ld_cg(&cv.ssel[t].prefix) << level_shift(1)) : 0u;
     uint32_t tiles_here = 0;
     uint32_t slab_next = 0, slab_left = 0;       // this warp's current slab (warp-uniform)
 
-    // prefetch cursor
-    uint32_t pt = t;
-    TensorDesc pd = d;
-    const uint32_t my_off = warp * kWarpChunk + lane * 4;        // + j * 128 elements
-    auto issue = [&](uint32_t p, uint32_t seq) {
-#if GC_FOLD_ASYNC
-        if (p < last) {
-            if (p >= pd.tile0 + pd.ntiles) { pt = find_tensor(desc, T, p); pd = desc[pt]; }
-            const TileGeom q = tile_geom(pd, p - pd.tile0);
-            if (tile_is_interior(q)) {
-                const uint32_t st = seq % (uint32_t)kFoldStages;
-                float* dg = s_g + (size_t)st * kTile + my_off;
-                float* dr = s_r + (size_t)st * kTile + my_off;
-                const float* gg = g + q.base + my_off;
-                const float* gr = r + q.base + my_off;
-#pragma unroll
-                for (int j = 0; j < kVpt; ++j) {
-                    cp_async16(dg + j * 128, gg + j * 128);
-                    cp_async16(dr + j * 128, gr + j * 128);
-                }
-            }
-        }
-        cp_async_commit();
-#endif
-    };
-
-    auto flush = [&]() {
-        if (tiles_here == 0) return;
-        __syncthreads();
-        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
-        for (int b = tid; b < NB; b += kBlock) {
-            uint32_t c = s_hist[b];
-            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t old = atomicAdd(&ws.sel[t].done[0], tiles_here);
-            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
-        }
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            select_step<0, true>(d.k, ws, t, s_scratch);
-        }
-        tiles_here = 0;
-    };
-
-#pragma unroll
-    for (int s = 0; s < kFoldStages - 1; ++s) issue(first + s * tstep, s);
-
-    uint32_t seq = 0;
-    for (uint32_t tile = first; tile < last; tile += tstep, ++seq) {
-        issue(tile + (kFoldStages - 1) * tstep, seq + kFoldStages - 1);
+    for (uint32_t tile = first; tile < ntiles; tile += tstep) {
         if (tile >= d.tile0 + d.ntiles) {
-            flush();
+            if (tiles_here) flush_and_select<0, true>(sm, ws, t, tiles_here, d.ntiles, d.k);
+            tiles_here = 0;
             t = find_tensor(desc, T, tile);
             d = desc[t];
-            tau = d.sstride ? (cv.ssel[t].prefix << level_shift(1)) : 0u;
+            tau = d.sstride ? (ld_cg(&cv.ssel[t].prefix) << level_shift(1)) : 0u;
         }
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;
-#if GC_FOLD_ASYNC
-        cp_async_wait<kFoldStages - 1>();
-        if (tile_is_interior(tg)) {
-            const uint32_t st = seq % (uint32_t)kFoldStages;
-            const float* sgp = s_g + (size_t)st * kTile + my_off;
-            const float* srp = s_r + (size_t)st * kTile + my_off;
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                const float4 gv = *reinterpret_cast<const float4*>(sgp + j * 128);
-                const float4 rv = *reinterpret_cast<const float4*>(srp + j * 128);
-                float4 a;
-                a.x = __fadd_rn(gv.x, rv.x); a.y = __fadd_rn(gv.y, rv.y);
-                a.z = __fadd_rn(gv.z, rv.z); a.w = __fadd_rn(gv.w, rv.w);
-                *reinterpret_cast<float4*>(r + tg.base + my_off + j * 128) = a;
-                tl.a[j][0] = a.x; tl.a[j][1] = a.y; tl.a[j][2] = a.z; tl.a[j][3] = a.w;
-            }
-            tl.valid = 0xFFFFu;
-        } else
-#endif
-        {
-            load_tile<true>(g, r, tg, warp, lane, tl);
-        }
+        load_tile<true>(g, r, tg, warp, lane, tl);
         uint32_t cnt[kVpt], cm = 0;
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) {
@@ -228,9 +115,7 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         }
         const uint32_t cbase = slab_next;
         if (fits) { slab_next += wtot; slab_left -= wtot; }
-#ifndef GC_EXP_NO_CHUNKINFO
         if (lane == 0) cv.chunk_info[(size_t)tile * kWarps + warp] = make_uint2(cbase, fits ? wtot : 0u);
-#endif
         // emission: candidates are first ranked into the warp's shared staging row, then written
         // out as one contiguous run of 8-byte pairs (a chunk rarely holds more than a dozen)
         const bool staged = wtot <= (uint32_t)kEmitStage;
@@ -244,8 +129,8 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                         if ((cm >> (4 * j + e)) & 1u) {
                             const uint2 pr = make_uint2(vec_index(tg.base, warp, lane, j) + e,
                                                         __float_as_uint(tl.a[j][e]));
-                            if (staged) s_emit[warp][pos] = pr; else cv.pair[cbase + pos] = pr;
-                            atomicAdd(&s_hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
+                            if (staged) sm.emit[warp][pos] = pr; else cv.pair[cbase + pos] = pr;
+                            atomicAdd(&sm.hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
                             ++pos;
                         }
                     }
@@ -253,76 +138,48 @@ k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             }
             if (staged) {
                 __syncwarp();
-                for (uint32_t i = lane; i < wtot; i += 32) cv.pair[cbase + i] = s_emit[warp][i];
+                for (uint32_t i = lane; i < wtot; i += 32) cv.pair[cbase + i] = sm.emit[warp][i];
                 __syncwarp();
             }
         }
         ++tiles_here;
     }
-#if GC_FOLD_ASYNC
-    cp_async_wait<0>();
-#endif
-    flush();
+    if (tiles_here) flush_and_select<0, true>(sm, ws, t, tiles_here, d.ntiles, d.k);
 }
 
 // ----------------------------------------------------------------------------- candidate refinement
 // Radix-select level 1 or 2 over the candidate lists.  CTAs take contiguous runs of tiles and
-// walk them kWarps at a time, one warp per tile, always inside one tensor; counts go to a
+// walk them kWarps at a time, one warp per tile, always inside one tensor; counts go to the
 // shared-memory histogram that is flushed when the tensor changes, and the CTA that completes
-// a tensor's last tile runs the select step (same scheme as k_hist).
+// a tensor's last tile runs the select step (same scheme as hist_body).
 template <int LEVEL>
-static __global__ void __launch_bounds__(kBlock)
-k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, WsView ws, CandView cv) {
+__device__ void cand_hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
+                               uint32_t ntiles, const WsView& ws, const CandView& cv) {
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int SH = level_shift(LEVEL);
-    __shared__ uint32_t s_hist[NB];
-    __shared__ uint32_t s_scratch[kWarps + 4];
-    __shared__ uint32_t s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (*(volatile uint32_t*)&ws.hdr->overflow) return;
     const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
     const uint32_t first = blockIdx.x * per;
     const uint32_t last = min(ntiles, first + per);
     if (first >= last) return;
-    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    for (int b = tid; b < NB; b += kBlock) sm.hist[b] = 0u;
     __syncthreads();
 
     uint32_t t = find_tensor(desc, T, first);
     TensorDesc d = desc[t];
-    bool active = (ws.sel[t].flags & kSelFailed) == 0u;
-    uint32_t prefix = ws.sel[t].prefix;
+    bool active = (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
+    uint32_t prefix = ld_cg(&ws.sel[t].prefix);
     uint32_t tiles_here = 0;
-
-    auto flush = [&]() {
-        if (!active || tiles_here == 0) { tiles_here = 0; return; }
-        __syncthreads();
-        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
-        for (int b = tid; b < NB; b += kBlock) {
-            uint32_t c = s_hist[b];
-            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
-            s_last = (old + tiles_here == d.ntiles) ? 1u : 0u;
-        }
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            select_step<LEVEL, false>(0u, ws, t, s_scratch);
-        }
-        tiles_here = 0;
-    };
 
     uint32_t batch = first;
     while (batch < last) {
         if (batch >= d.tile0 + d.ntiles) {
-            flush();
+            if (active && tiles_here) flush_and_select<LEVEL, false>(sm, ws, t, tiles_here, d.ntiles, 0u);
+            tiles_here = 0;
             t = find_tensor(desc, T, batch);
             d = desc[t];
-            active = (ws.sel[t].flags & kSelFailed) == 0u;
-            prefix = ws.sel[t].prefix;
+            active = (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
+            prefix = ld_cg(&ws.sel[t].prefix);
         }
         const uint32_t bend = min(min(last, d.tile0 + d.ntiles), batch + (uint32_t)kWarps);
         const uint32_t tile = batch + warp;
@@ -332,92 +189,93 @@ k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, Ws
                 uint32_t j = j0 + lane;
                 uint32_t slot = cand_slot(tc, j);
                 if (j < tc.total) {
-                    uint32_t key = cv.pair[slot].y & kKeyMask;
+                    uint32_t key = ld_cg(&cv.pair[slot]).y & kKeyMask;
                     if ((key >> (SH + level_bits(LEVEL))) == prefix)
-                        atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                        atomicAdd(&sm.hist[(key >> SH) & (NB - 1)], 1u);
                 }
             }
         }
         tiles_here += bend - batch;
         batch = bend;
     }
-    flush();
+    if (active && tiles_here) flush_and_select<LEVEL, false>(sm, ws, t, tiles_here, d.ntiles, 0u);
 }
 
 // ----------------------------------------------------------------------------- candidate compaction
-// Index-ordered emission from the candidate lists.  A group is kWarps consecutive tiles of
-// one tensor, one warp per tile; groups are handed out by ticket and exchange their
-// (above-T, equal-T) counts through the look-back words, per tensor.  Sent entries are
-// written to the output and zeroed in the residual (which already holds a).
-static __global__ void __launch_bounds__(kBlock)
-k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups_total,
-               float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
-               uint32_t* __restrict__ out_count, WsView ws, CandView cv, int ticket_slot) {
-    __shared__ uint32_t s_group;
-    __shared__ uint32_t s_gt_tot[kWarps], s_eq_tot[kWarps], s_gt_ex[kWarps], s_eq_ex[kWarps];
-    __shared__ uint32_t s_gt_sum, s_eq_sum;
-    __shared__ unsigned long long s_excl;
-    __shared__ int s_ok;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (*(volatile uint32_t*)&ws.hdr->overflow) return;
-    const unsigned lt_mask = (1u << lane) - 1u;
+// Index-ordered emission from the candidate lists in two steps.  A group is kWarps consecutive
+// tiles of one tensor, one warp per tile; group i of a CTA is blockIdx.x + i * gridDim.x.
+//   count: every group stores its (above-T, equal-T) totals;
+//   emit:  a group adds up the totals of the groups before it in its tensor, ranks its own
+//          candidates, writes the sent ones to the output and zeroes them in the residual
+//          (which already holds a).
+// An element is sent iff key > T, or key == T and fewer than m_eq equal keys precede it.
+__device__ __forceinline__ void group_tile_counts(const CandView& cv, const TileCands& tc, uint32_t Tkey,
+                                                  int lane, uint32_t& ngt, uint32_t& neq) {
+    ngt = 0; neq = 0;
+    for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
+        uint32_t j = j0 + lane;
+        uint32_t slot = cand_slot(tc, j);
+        uint32_t key = j < tc.total ? (ld_cg(&cv.pair[slot]).y & kKeyMask) : 0u;
+        bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
+        ngt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
+        neq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+    }
+}
 
-    while (true) {
+template <bool EMIT>
+__device__ void cand_compact_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
+                                  uint32_t ngroups_total, float* __restrict__ r,
+                                  uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                  uint32_t* __restrict__ out_count, const WsView& ws, const CandView& cv) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    for (uint32_t group = blockIdx.x; group < ngroups_total; group += gridDim.x) {
         __syncthreads();
-        if (tid == 0) {
-            uint32_t tk = atomicAdd(&ws.hdr->ticket[ticket_slot], 1u);
-            if (*(volatile uint32_t*)&ws.hdr->abort) tk = 0xFFFFFFFFu;
-            s_group = tk;
-        }
-        __syncthreads();
-        const uint32_t group = s_group;
-        if (group >= ngroups_total) break;
         const uint32_t t = find_tensor<GroupSpace>(desc, T, group);
-        if (ws.sel[t].flags & kSelFailed) continue;
+        if (ld_cg(&ws.sel[t].flags) & kSelFailed) continue;
         const TensorDesc d = desc[t];
-        const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
+        const uint32_t Tkey = ld_cg(&ws.sel[t].T), m_eq = ld_cg(&ws.sel[t].m_eq);
         const uint32_t tile_in_t = (group - d.group0) * kWarps + warp;
         TileCands tc;
         tc.base = tc.cnt = tc.incl = tc.total = 0u;
         if (tile_in_t < d.ntiles) tc = load_tile_cands(cv, d.tile0 + tile_in_t, lane);
-
-        // pass 1: counts of this warp's tile
-        uint32_t ngt = 0, neq = 0;
-        for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
-            uint32_t j = j0 + lane;
-            uint32_t slot = cand_slot(tc, j);
-            uint32_t key = j < tc.total ? (cv.pair[slot].y & kKeyMask) : 0u;
-            bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
-            ngt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
-            neq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+        uint32_t ngt, neq;
+        group_tile_counts(cv, tc, Tkey, lane, ngt, neq);
+        if (lane == 0) { sm.gt_tot[warp] = ngt; sm.eq_tot[warp] = neq; }
+        if (EMIT) {
+            // totals of the groups before this one in the tensor
+            unsigned long long part = 0;
+            for (uint32_t q = d.group0 + tid; q < group; q += kBlock) part += ld_cg(&cv.group_cnt[q]);
+            part = warp_sum64(part);
+            if (lane == 0) sm.red[warp] = part;
         }
-        if (lane == 0) { s_gt_tot[warp] = ngt; s_eq_tot[warp] = neq; }
         __syncthreads();
-        scan_warp_totals(s_gt_tot, s_gt_ex, &s_gt_sum, warp, lane);
+        scan_warp_totals(sm.gt_tot, sm.gt_ex, &sm.gt_sum, warp, lane);
         if (warp == 1) {
-            uint32_t v = lane < kWarps ? s_eq_tot[lane] : 0u;
+            uint32_t v = lane < kWarps ? sm.eq_tot[lane] : 0u;
             uint32_t inc = warp_incl_scan(v, lane);
-            if (lane < kWarps) s_eq_ex[lane] = inc - v;
-            if (lane == 31) s_eq_sum = inc;
+            if (lane < kWarps) sm.eq_ex[lane] = inc - v;
+            if (lane == 31) sm.eq_sum = inc;
+        }
+        if (EMIT && warp == 2) {
+            unsigned long long v = lane < kWarps ? sm.red[lane] : 0ull;
+            v = warp_sum64(v);
+            if (lane == 0) sm.excl = v;
         }
         __syncthreads();
-        if (warp == 0) {
-            unsigned long long agg = ((unsigned long long)s_gt_sum << 31) | (unsigned long long)s_eq_sum;
-            bool ok;
-            unsigned long long ex = lookback(ws.tile_state, group, d.group0, agg, lane, ws.hdr, ok);
-            if (lane == 0) { s_excl = ex; s_ok = ok ? 1 : 0; }
+        if (!EMIT) {
+            if (tid == 0)
+                cv.group_cnt[group] = ((unsigned long long)sm.gt_sum << 31) | (unsigned long long)sm.eq_sum;
+            continue;
         }
-        __syncthreads();
-        if (!s_ok) break;
-        // pass 2: emit
-        uint32_t gpos = (uint32_t)(s_excl >> 31) + s_gt_ex[warp];
-        uint32_t epos = (uint32_t)(s_excl & 0x7FFFFFFFull) + s_eq_ex[warp];
+        uint32_t gpos = (uint32_t)(sm.excl >> 31) + sm.gt_ex[warp];
+        uint32_t epos = (uint32_t)(sm.excl & 0x7FFFFFFFull) + sm.eq_ex[warp];
         for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
             uint32_t j = j0 + lane;
             uint32_t slot = cand_slot(tc, j);
             float v = 0.f;
             uint32_t f = 0;
-            if (j < tc.total) { const uint2 pr = cv.pair[slot]; f = pr.x; v = __uint_as_float(pr.y); }
+            if (j < tc.total) { const uint2 pr = ld_cg(&cv.pair[slot]); f = pr.x; v = __uint_as_float(pr.y); }
             uint32_t key = key_of(v);
             bool gt = j < tc.total && key > Tkey, eq = j < tc.total && key == Tkey;
             unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
@@ -439,6 +297,101 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
             out_count[T + t] = d.k;
         }
     }
+}
+
+// ----------------------------------------------------------------------------- separate launches
+static __global__ void __launch_bounds__(kBlock)
+k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+            const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
+    __shared__ BlockSmem sm;
+    fold_cand_body(sm, desc, T, ntiles, g, r, ws, cv);
+}
+
+template <int LEVEL>
+static __global__ void __launch_bounds__(kBlock)
+k_cand_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, WsView ws, CandView cv) {
+    __shared__ BlockSmem sm;
+    if (ld_cg(&ws.hdr->overflow)) return;
+    cand_hist_body<LEVEL>(sm, desc, T, ntiles, ws, cv);
+}
+
+template <bool EMIT>
+static __global__ void __launch_bounds__(kBlock)
+k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups_total,
+               float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+               uint32_t* __restrict__ out_count, WsView ws, CandView cv) {
+    __shared__ BlockSmem sm;
+    if (ld_cg(&ws.hdr->overflow)) return;
+    cand_compact_body<EMIT>(sm, desc, T, ngroups_total, r, out_idx, out_val, out_count, ws, cv);
+}
+
+// ----------------------------------------------------------------------------- one launch
+struct FusedArgs {
+    const TensorDesc* desc;
+    uint32_t T, ntiles, nstiles, ngroups;
+    const float* g;
+    float* r;
+    uint32_t* out_idx;
+    float* out_val;
+    uint32_t* out_count;
+    WsView ws;               // main selection records, tile look-back words
+    WsView sws;              // sample selection records
+    WsView gws;              // records of the redo, gated by the main ones
+    CandView cv;
+};
+
+// Whole top-k compress of one call in a single cooperative launch (one CTA per SM):
+//   sample level 0 | sample level 1 | fold + candidates | candidate level 1 | candidate level 2
+//   | group counts | emit, and -- only if a tensor's candidate set was too small or the list
+//   overflowed -- the exact multi-pass redo of those tensors.
+// Phases are separated by grid barriers; every decision taken after a barrier reads values
+// that were final before it, so all CTAs take the same route.
+static __global__ void __launch_bounds__(kBlock, 1)
+k_compress_fused(FusedArgs a) {
+    __shared__ BlockSmem sm;
+    uint32_t passed = 0;
+    WsHeader* hdr = a.ws.hdr;
+    phase_stamp(hdr);
+    if (a.nstiles) {
+        hist_body<0, SRC_SAMPLE>(sm, a.desc, a.T, a.nstiles, a.g, a.r, a.sws);
+        if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+        hist_body<1, SRC_SAMPLE>(sm, a.desc, a.T, a.nstiles, a.g, a.r, a.sws);
+        if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    }
+    fold_cand_body(sm, a.desc, a.T, a.ntiles, a.g, a.r, a.ws, a.cv);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    const bool overflow = ld_cg(&hdr->overflow) != 0u;
+    if (!overflow) {
+        cand_hist_body<1>(sm, a.desc, a.T, a.ntiles, a.ws, a.cv);
+        if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+        cand_hist_body<2>(sm, a.desc, a.T, a.ntiles, a.ws, a.cv);
+        if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+        cand_compact_body<false>(sm, a.desc, a.T, a.ngroups, a.r, a.out_idx, a.out_val, a.out_count, a.ws, a.cv);
+        if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+        cand_compact_body<true>(sm, a.desc, a.T, a.ngroups, a.r, a.out_idx, a.out_val, a.out_count, a.ws, a.cv);
+        __syncthreads();
+        phase_stamp(hdr);
+    }
+    if (!overflow && ld_cg(&hdr->n_failed) == 0u) return;
+    // redo (rare): r already holds a for every element
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    compact_body(sm, a.desc, a.T, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
 }
 
 }  // namespace gc

@@ -1,5 +1,7 @@
 // Kernels of the exact multi-pass path: fold + radix-select histograms over the magnitude
-// key, ordered compaction with residual zeroing, and the sparse decode.
+// key, ordered compaction with residual zeroing, and the sparse decode.  Every kernel is a
+// thin __global__ wrapper around a __device__ body so that the fused kernel can run the same
+// bodies as phases of one launch.
 #pragma once
 #include <type_traits>
 
@@ -16,6 +18,7 @@ struct Tile {
 // Loads the thread's vectors of one tile.  FOLD: a = g + r (one rounded fp32 add) and a is
 // stored to r; otherwise a is read from r.  Interior vectors use 128-bit accesses; vectors
 // that straddle the tensor's first or last element fall back to guarded scalar accesses.
+// r is read at L2 (it may have been written by another CTA earlier in the same launch).
 template <bool FOLD>
 __device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __restrict__ r,
                                           const TileGeom& tg, int warp, int lane, Tile& t) {
@@ -27,7 +30,7 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __
         uint32_t f0 = vec_index(tg.base, warp, lane, j);
         full[j] = (f0 >= tg.lo) && (f0 + 4 <= tg.hi);
         if (full[j]) {
-            rv[j] = *reinterpret_cast<const float4*>(r + f0);
+            rv[j] = ld_cg(reinterpret_cast<const float4*>(r + f0));
             if (FOLD) gv[j] = __ldg(reinterpret_cast<const float4*>(g + f0));
         }
     }
@@ -50,7 +53,7 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __
                 uint32_t f = f0 + e;
                 float v = 0.0f;
                 if (f >= tg.lo && f < tg.hi) {
-                    v = r[f];
+                    v = ld_cg(r + f);
                     if (FOLD) { v = __fadd_rn(__ldg(g + f), v); r[f] = v; }
                     t.valid |= 1u << (4 * j + e);
                 }
@@ -86,15 +89,15 @@ __device__ void select_step(uint32_t rank0, const WsView& ws, uint32_t t,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* hist = ws.hist + (size_t)t * kHistBins;
     TensorSel* sel = ws.sel + t;
-    const uint32_t krem = level_is_first(LEVEL) ? rank0 : sel->krem;
-    const uint32_t prefix = level_is_first(LEVEL) ? 0u : sel->prefix;
+    const uint32_t krem = level_is_first(LEVEL) ? rank0 : ld_cg(&sel->krem);
+    const uint32_t prefix = level_is_first(LEVEL) ? 0u : ld_cg(&sel->prefix);
     // thread `tid` owns BPT consecutive bins, counted from the largest key downwards
     uint32_t c[BPT];
     uint32_t sum = 0;
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
         int b = NB - 1 - (tid * BPT + i);
-        c[i] = (b >= 0) ? __ldcg(hist + b) : 0u;
+        c[i] = (b >= 0) ? ld_cg(hist + b) : 0u;
         if (b >= 0) hist[b] = 0u;
         sum += c[i];
     }
@@ -110,7 +113,7 @@ __device__ void select_step(uint32_t rank0, const WsView& ws, uint32_t t,
     __syncthreads();
     if (CHECK && s_scratch[kWarps] < krem) {
         if (tid == 0) {
-            sel->flags |= kSelFailed;
+            sel->flags = kSelFailed;
             atomicAdd(&ws.hdr->n_failed, 1u);
         }
         __syncthreads();
@@ -131,31 +134,32 @@ __device__ void select_step(uint32_t rank0, const WsView& ws, uint32_t t,
     __syncthreads();
 }
 
-// The same step run by a single warp (used where tiles are handled warp by warp).
-template <int LEVEL>
-__device__ void select_step_warp(const WsView& ws, uint32_t t, int lane) {
+// Shared tail of every histogram phase: add the CTA's shared-memory histogram of tensor t to
+// the global one, count the tiles it covered, and let the CTA that completes the tensor run
+// the select step.
+template <int LEVEL, bool CHECK>
+__device__ __forceinline__ void flush_and_select(BlockSmem& sm, const WsView& ws, uint32_t t,
+                                                 uint32_t tiles_here, uint32_t tiles_of_tensor,
+                                                 uint32_t rank0) {
     constexpr int NB = 1 << level_bits(LEVEL);
-    constexpr int BPL = NB / 32;                              // bins per lane
+    const int tid = threadIdx.x;
+    __syncthreads();
     uint32_t* hist = ws.hist + (size_t)t * kHistBins;
-    TensorSel* sel = ws.sel + t;
-    const uint32_t krem = sel->krem, prefix = sel->prefix;
-    uint32_t sum = 0;
-    for (int i = 0; i < BPL; ++i) sum += __ldcg(hist + (NB - 1 - (lane * BPL + i)));
-    uint32_t inc = warp_incl_scan(sum, lane);
-    uint32_t above = inc - sum;
-    for (int i = 0; i < BPL; ++i) {
-        int b = NB - 1 - (lane * BPL + i);
-        uint32_t c = __ldcg(hist + b);
-        hist[b] = 0u;
-        if (above < krem && krem <= above + c) {
-            uint32_t np = (prefix << level_bits(LEVEL)) | (uint32_t)b;
-            sel->prefix = np;
-            sel->krem = krem - above;
-            if (LEVEL == kLevels - 1) { sel->T = np; sel->m_eq = krem - above; }
-        }
-        above += c;
+    for (int b = tid; b < NB; b += kBlock) {
+        uint32_t c = sm.hist[b];
+        if (c) { atomicAdd(hist + b, c); sm.hist[b] = 0u; }
     }
-    __syncwarp();
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
+        sm.last = (old + tiles_here == tiles_of_tensor) ? 1u : 0u;
+    }
+    __syncthreads();
+    if (sm.last) {
+        __threadfence();
+        select_step<LEVEL, CHECK>(rank0, ws, t, sm.scratch);
+    }
 }
 
 // ----------------------------------------------------------------------------- histogram pass
@@ -170,61 +174,35 @@ __device__ void select_step_warp(const WsView& ws, uint32_t t, int lane) {
 constexpr int SRC_FOLD = 0, SRC_RESID = 1, SRC_SAMPLE = 2;
 
 template <int LEVEL, int SRC>
-__global__ void __launch_bounds__(kBlock)
-k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
-       const float* __restrict__ g, float* __restrict__ r, WsView ws) {
+__device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                          const float* __restrict__ g, float* __restrict__ r, const WsView& ws) {
     using S = typename std::conditional<SRC == SRC_SAMPLE, SampleSpace, FullSpace>::type;
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int SH = level_shift(LEVEL);
-    __shared__ uint32_t s_hist[NB];
-    __shared__ uint32_t s_scratch[kWarps + 4];
-    __shared__ uint32_t s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (ws.gate != nullptr && *(volatile uint32_t*)&ws.hdr->n_failed == 0u &&
-        *(volatile uint32_t*)&ws.hdr->overflow == 0u)
-        return;
+    if (nothing_to_redo(ws)) return;
     const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
     const uint32_t first = blockIdx.x * per;
     const uint32_t last = min(ntiles, first + per);
     if (first >= last) return;
-    for (int b = tid; b < NB; b += kBlock) s_hist[b] = 0u;
+    for (int b = tid; b < NB; b += kBlock) sm.hist[b] = 0u;
     __syncthreads();
 
     uint32_t t = find_tensor<S>(desc, T, first);
     TensorDesc d = desc[t];
     bool active = gate_open(ws, t);
-    uint32_t prefix = level_is_first(LEVEL) ? 0u : ws.sel[t].prefix;
+    uint32_t prefix = level_is_first(LEVEL) ? 0u : ld_cg(&ws.sel[t].prefix);
     uint32_t tiles_here = 0;
-
-    auto flush = [&]() {
-        if (!active || tiles_here == 0) return;
-        __syncthreads();
-        uint32_t* hist = ws.hist + (size_t)t * kHistBins;
-        for (int b = tid; b < NB; b += kBlock) {
-            uint32_t c = s_hist[b];
-            if (c) { atomicAdd(hist + b, c); s_hist[b] = 0u; }
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t old = atomicAdd(&ws.sel[t].done[LEVEL], tiles_here);
-            s_last = (old + tiles_here == S::ntiles(d)) ? 1u : 0u;
-        }
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            select_step<LEVEL, false>(S::rank(d), ws, t, s_scratch);
-        }
-        tiles_here = 0;
-    };
 
     for (uint32_t tile = first; tile < last; ++tile) {
         if (tile >= S::tile0(d) + S::ntiles(d)) {
-            flush();
+            if (active && tiles_here)
+                flush_and_select<LEVEL, false>(sm, ws, t, tiles_here, S::ntiles(d), S::rank(d));
+            tiles_here = 0;
             t = find_tensor<S>(desc, T, tile);
             d = desc[t];
             active = gate_open(ws, t);
-            prefix = level_is_first(LEVEL) ? 0u : ws.sel[t].prefix;
+            prefix = level_is_first(LEVEL) ? 0u : ld_cg(&ws.sel[t].prefix);
         }
         if (!active) continue;
         if (SRC == SRC_SAMPLE) {
@@ -243,7 +221,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                     bool v = gi < ngroups && i0 + e < d.n;
                     uint32_t f = d.off + (v ? i0 + e : 0u);
                     gv[j][e] = v ? __ldg(g + f) : 0.f;
-                    rv[j][e] = v ? r[f] : 0.f;
+                    rv[j][e] = v ? ld_cg(r + f) : 0.f;
                     ok |= (uint32_t)v << (4 * j + e);
                 }
             }
@@ -254,7 +232,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                     uint32_t key = key_of(__fadd_rn(gv[j][e], rv[j][e]));
                     bool in = (ok >> (4 * j + e)) & 1u;
                     if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
-                    if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                    if (in) atomicAdd(&sm.hist[(key >> SH) & (NB - 1)], 1u);
                 }
             }
         } else {
@@ -268,13 +246,21 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                     uint32_t key = key_of(tl.a[j][e]);
                     bool in = (tl.valid >> (4 * j + e)) & 1u;
                     if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
-                    if (in) atomicAdd(&s_hist[(key >> SH) & (NB - 1)], 1u);
+                    if (in) atomicAdd(&sm.hist[(key >> SH) & (NB - 1)], 1u);
                 }
             }
         }
         ++tiles_here;
     }
-    flush();
+    if (active && tiles_here) flush_and_select<LEVEL, false>(sm, ws, t, tiles_here, S::ntiles(d), S::rank(d));
+}
+
+template <int LEVEL, int SRC>
+__global__ void __launch_bounds__(kBlock)
+k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+       const float* __restrict__ g, float* __restrict__ r, WsView ws) {
+    __shared__ BlockSmem sm;
+    hist_body<LEVEL, SRC>(sm, desc, T, ntiles, g, r, ws);
 }
 
 // ----------------------------------------------------------------------------- compaction
@@ -284,34 +270,27 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
 // exchange.  An element is sent iff key > T, or key == T and fewer than m_eq equal keys
 // precede it in the tensor.  Sent elements are written as (flat index, value) at their rank
 // and zeroed in the residual.
-static __global__ void __launch_bounds__(kBlock)
-k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
-          float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
-          uint32_t* __restrict__ out_count, WsView ws, int ticket_slot) {
-    __shared__ uint32_t s_tile;
-    __shared__ uint32_t s_gt_tot[kWarps], s_eq_tot[kWarps], s_gt_ex[kWarps], s_eq_ex[kWarps];
-    __shared__ uint32_t s_gt_sum, s_eq_sum;
-    __shared__ unsigned long long s_excl;
-    __shared__ int s_ok;
+static __device__ void compact_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                             float* __restrict__ r, uint32_t* __restrict__ out_idx,
+                             float* __restrict__ out_val, uint32_t* __restrict__ out_count,
+                             const WsView& ws, int ticket_slot) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (ws.gate != nullptr && *(volatile uint32_t*)&ws.hdr->n_failed == 0u &&
-        *(volatile uint32_t*)&ws.hdr->overflow == 0u)
-        return;
+    if (nothing_to_redo(ws)) return;
 
     while (true) {
         __syncthreads();
         if (tid == 0) {
             uint32_t tk = atomicAdd(&ws.hdr->ticket[ticket_slot], 1u);
-            if (*(volatile uint32_t*)&ws.hdr->abort) tk = 0xFFFFFFFFu;
-            s_tile = tk;
+            if (ld_cg(&ws.hdr->abort)) tk = 0xFFFFFFFFu;
+            sm.tile = tk;
         }
         __syncthreads();
-        const uint32_t tile = s_tile;
+        const uint32_t tile = sm.tile;
         if (tile >= ntiles) break;
         const uint32_t t = find_tensor(desc, T, tile);
         if (!gate_open(ws, t)) continue;
         const TensorDesc d = desc[t];
-        const uint32_t Tkey = ws.sel[t].T, m_eq = ws.sel[t].m_eq;
+        const uint32_t Tkey = ld_cg(&ws.sel[t].T), m_eq = ld_cg(&ws.sel[t].m_eq);
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;
         load_tile<false>(nullptr, r, tg, warp, lane, tl);
@@ -333,26 +312,26 @@ k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
         uint32_t rg[kVpt], re[kVpt], wg, we;
         warp_rank(cg, lane, rg, wg);
         warp_rank(ce, lane, re, we);
-        if (lane == 0) { s_gt_tot[warp] = wg; s_eq_tot[warp] = we; }
+        if (lane == 0) { sm.gt_tot[warp] = wg; sm.eq_tot[warp] = we; }
         __syncthreads();
-        scan_warp_totals(s_gt_tot, s_gt_ex, &s_gt_sum, warp, lane);
+        scan_warp_totals(sm.gt_tot, sm.gt_ex, &sm.gt_sum, warp, lane);
         if (warp == 1) {
-            uint32_t v = lane < kWarps ? s_eq_tot[lane] : 0u;
+            uint32_t v = lane < kWarps ? sm.eq_tot[lane] : 0u;
             uint32_t inc = warp_incl_scan(v, lane);
-            if (lane < kWarps) s_eq_ex[lane] = inc - v;
-            if (lane == 31) s_eq_sum = inc;
+            if (lane < kWarps) sm.eq_ex[lane] = inc - v;
+            if (lane == 31) sm.eq_sum = inc;
         }
         __syncthreads();
         if (warp == 0) {
-            unsigned long long agg = ((unsigned long long)s_gt_sum << 31) | (unsigned long long)s_eq_sum;
+            unsigned long long agg = ((unsigned long long)sm.gt_sum << 31) | (unsigned long long)sm.eq_sum;
             bool ok;
             unsigned long long ex = lookback(ws.tile_state, tile, d.tile0, agg, lane, ws.hdr, ok);
-            if (lane == 0) { s_excl = ex; s_ok = ok ? 1 : 0; }
+            if (lane == 0) { sm.excl = ex; sm.ok = ok ? 1 : 0; }
         }
         __syncthreads();
-        if (!s_ok) break;
-        const uint32_t gt_before = (uint32_t)(s_excl >> 31) + s_gt_ex[warp];
-        const uint32_t eq_before = (uint32_t)(s_excl & 0x7FFFFFFFull) + s_eq_ex[warp];
+        if (!sm.ok) break;
+        const uint32_t gt_before = (uint32_t)(sm.excl >> 31) + sm.gt_ex[warp];
+        const uint32_t eq_before = (uint32_t)(sm.excl & 0x7FFFFFFFull) + sm.eq_ex[warp];
         if ((gtm | eqm) != 0u) {
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
@@ -363,14 +342,14 @@ k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                     if (gt || (eq && epos < m_eq)) {
                         uint32_t slot = gpos + min(epos, m_eq);
                         uint32_t f = vec_index(tg.base, warp, lane, j) + e;
-                        if (slot >= d.cap) {          // cannot happen with a correct select; never write outside
+                        if (slot < d.cap) {
+                            uint32_t pos = d.out_off + slot;
+                            out_idx[pos] = f;
+                            out_val[pos] = tl.a[j][e];
+                            r[f] = 0.0f;
+                        } else {      // cannot happen with a correct select; never write outside
                             record_status(ws.hdr, -1 /*GC_E_INVALID*/, f);
-                            continue;
                         }
-                        uint32_t pos = d.out_off + slot;
-                        out_idx[pos] = f;
-                        out_val[pos] = tl.a[j][e];
-                        r[f] = 0.0f;
                     }
                     gpos += gt; epos += eq;
                 }
@@ -383,13 +362,15 @@ k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
     }
 }
 
-// ----------------------------------------------------------------------------- decode
-struct DecodeArgs {
-    const uint32_t* idx[64];
-    const float* val[64];
-    const uint32_t* count[64];
-};
+static __global__ void __launch_bounds__(kBlock)
+k_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+          float* __restrict__ r, uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+          uint32_t* __restrict__ out_count, WsView ws, int ticket_slot) {
+    __shared__ BlockSmem sm;
+    compact_body(sm, desc, T, ntiles, r, out_idx, out_val, out_count, ws, ticket_slot);
+}
 
+// ----------------------------------------------------------------------------- decode
 // One sparse set added into the dense buffer.  Indices of one set are distinct, so plain
 // read-modify-write is race free; sets are applied by consecutive launches in worker order,
 // which fixes the order of the fp32 additions per element.

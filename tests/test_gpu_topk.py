@@ -86,6 +86,9 @@ def test_config5_gpt2_medium_full_size_two_workers():
 PATHS = {
     "auto": {},
     "exact": {api.GC_OPT_PATH: api.GC_PATH_EXACT},
+    "staged": {api.GC_OPT_PATH: api.GC_PATH_STAGED},
+    "staged_starved": {api.GC_OPT_PATH: api.GC_PATH_STAGED, api.GC_OPT_SAMPLE_RANK_PERMILLE: 30},
+    "staged_overflow": {api.GC_OPT_PATH: api.GC_PATH_STAGED, api.GC_OPT_CANDIDATE_CAPACITY: 100},
     "auto_starved": {api.GC_OPT_SAMPLE_RANK_PERMILLE: 30},      # candidate sets too small -> redo per tensor
     "auto_overflow": {api.GC_OPT_CANDIDATE_CAPACITY: 100},      # candidate list too short -> redo everything
 }
@@ -99,11 +102,11 @@ def test_every_route_gives_the_same_bits(path):
     seen = []
     for density in (0.001, 0.01):
         check_topk_against_oracle(sizes, density, grads, options=PATHS[path], expect_counters=seen.append)
-    if path == "auto":
+    if path in ("auto", "staged"):
         assert all(c[1] == 0 and c[2] == 0 for c in seen), seen     # the safety net stayed idle
-    if path == "auto_starved":
+    if path.endswith("_starved"):
         assert all(c[2] >= 1 for c in seen), seen
-    if path == "auto_overflow":
+    if path.endswith("_overflow"):
         assert all(c[1] == 1 for c in seen), seen
 
 
