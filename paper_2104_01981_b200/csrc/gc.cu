@@ -139,7 +139,7 @@ void finish_layout(gc_plan_s* p) {
         if (d.sstride) {
             uint64_t groups = ((uint64_t)d.n + 3) / 4;
             uint64_t nsg = (groups + d.sstride - 1) / d.sstride;
-            nst = (nsg + (uint64_t)kBlock * kVpt - 1) / ((uint64_t)kBlock * kVpt);
+            nst = (nsg + (uint64_t)kSampleTile - 1) / (uint64_t)kSampleTile;
             ++p->n_sampled;
         }
         d.stile0 = (uint32_t)stile0; d.nstiles = (uint32_t)nst;
@@ -429,6 +429,9 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
                                                       out_count, ws, cv); }
     }
     {
+        { Timed tm(p, s, GC_K_HIST_REFINE);
+          const int gr = (int)std::min<uint32_t>((nt + kWarps - 1) / kWarps, (uint32_t)p->grid_chist);
+          k_cand_restore<<<gr, kBlock, 0, s>>>(p->d_desc, p->T, nt, residual, ws, cv); }
         { Timed tm(p, s, GC_K_HIST_REFINE);
           k_hist<0, SRC_RESID><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, nullptr, residual, gws); }
         { Timed tm(p, s, GC_K_HIST_REFINE);

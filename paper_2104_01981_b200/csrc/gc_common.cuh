@@ -7,11 +7,12 @@
 namespace gc {
 
 // ----------------------------------------------------------------------------- geometry
-constexpr int kBlock = 512;                 // threads per CTA for the streaming kernels
+constexpr int kBlock = 256;                 // threads per CTA for the streaming kernels
 constexpr int kWarps = kBlock / 32;
 constexpr int kVpt = 4;                     // 128-bit vectors per thread per tile
 constexpr int kTile = kBlock * kVpt * 4;    // 8192 elements per tile
 constexpr int kWarpChunk = 32 * kVpt * 4;   // contiguous elements owned by one warp
+constexpr int kSampleTile = kBlock;         // sample groups (of 4 elements) per sample tile: one per thread
 constexpr uint32_t kKeyMask = 0x7FFFFFFFu;
 
 // radix-select levels over the 31-bit magnitude key: 11 + 10 + 10 bits
@@ -40,7 +41,7 @@ struct TensorDesc {          // one per tensor, immutable, plan-owned device mem
                              // threshold; 0 = tensor is not sampled, every element is a candidate
     uint32_t srank;          // rank taken inside the sample (k_s in threshold mode)
     uint32_t stile0;         // first sample tile id
-    uint32_t nstiles;        // sample tiles (2048 sample groups each)
+    uint32_t nstiles;        // sample tiles (kSampleTile sample groups each)
     uint32_t group0;         // first compaction group id (a group = kWarps consecutive tiles)
     uint32_t ngroups;        // compaction groups of this tensor
     uint32_t pad[2];

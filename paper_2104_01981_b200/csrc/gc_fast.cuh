@@ -55,12 +55,16 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
 }
 
 // ----------------------------------------------------------------------------- fold + candidates
-// Reads g and r, writes a into r, emits candidates.  Tile i of a CTA is blockIdx.x + i *
-// gridDim.x, so at any moment the CTAs sweep one contiguous window of memory.  No block-wide
-// barrier in the tile loop: every warp ranks and stores the candidates of its own chunk.
+// Reads g and r, computes a = g + r, emits candidates and writes the residual back with the
+// candidates ALREADY zeroed (their values live in the candidate list): after the selection
+// only the few candidates that were not sent need their value restored, instead of every
+// sent entry needing a scattered zero.  A chunk whose candidates did not fit in the list keeps
+// its values in r.  Tile i of a CTA is blockIdx.x + i * gridDim.x, so at any moment the CTAs
+// sweep one contiguous window of memory.  No block-wide barrier in the tile loop: every warp
+// ranks and stores the candidates of its own chunk.
 static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
-                               uint32_t ntiles, const float* __restrict__ g, float* __restrict__ r,
-                               const WsView& ws, const CandView& cv) {
+                                      uint32_t ntiles, const float* __restrict__ g, float* __restrict__ r,
+                                      const WsView& ws, const CandView& cv) {
     constexpr int NB = 1 << level_bits(0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t first = blockIdx.x, tstep = gridDim.x;
@@ -73,6 +77,7 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
     uint32_t tau = d.sstride ? (ld_cg(&cv.ssel[t].prefix) << level_shift(1)) : 0u;
     uint32_t tiles_here = 0;
     uint32_t slab_next = 0, slab_left = 0;       // this warp's current slab (warp-uniform)
+    const uint32_t my_off = warp * kWarpChunk + lane * 4;
 
     for (uint32_t tile = first; tile < ntiles; tile += tstep) {
         if (tile >= d.tile0 + d.ntiles) {
@@ -83,15 +88,45 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
             tau = d.sstride ? (ld_cg(&cv.ssel[t].prefix) << level_shift(1)) : 0u;
         }
         const TileGeom tg = tile_geom(d, tile - d.tile0);
-        Tile tl;
-        load_tile<true>(g, r, tg, warp, lane, tl);
+        const bool interior = tg.lo == tg.base && tg.hi == tg.base + (uint32_t)kTile;
+        float a[kVpt][4];
+        uint32_t valid = 0xFFFFu;
+        if (interior) {
+            float4 gv[kVpt], rv[kVpt];
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                gv[j] = __ldg(reinterpret_cast<const float4*>(g + tg.base + my_off + j * 128));
+                rv[j] = ld_cg(reinterpret_cast<const float4*>(r + tg.base + my_off + j * 128));
+            }
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                a[j][0] = __fadd_rn(gv[j].x, rv[j].x); a[j][1] = __fadd_rn(gv[j].y, rv[j].y);
+                a[j][2] = __fadd_rn(gv[j].z, rv[j].z); a[j][3] = __fadd_rn(gv[j].w, rv[j].w);
+            }
+        } else {
+            valid = 0u;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t f = tg.base + my_off + j * 128 + e;
+                    float v = 0.0f;
+                    if (f >= tg.lo && f < tg.hi) {
+                        v = __fadd_rn(__ldg(g + f), ld_cg(r + f));
+                        valid |= 1u << (4 * j + e);
+                    }
+                    a[j][e] = v;
+                }
+            }
+        }
         uint32_t cnt[kVpt], cm = 0;
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) {
             cnt[j] = 0;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                bool c = ((tl.valid >> (4 * j + e)) & 1u) && key_of(tl.a[j][e]) >= tau;
+                bool c = key_of(a[j][e]) >= tau;
+                if (!interior) c = c && ((valid >> (4 * j + e)) & 1u);
                 cnt[j] += c;
                 cm |= (uint32_t)c << (4 * j + e);
             }
@@ -116,6 +151,28 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
         const uint32_t cbase = slab_next;
         if (fits) { slab_next += wtot; slab_left -= wtot; }
         if (lane == 0) cv.chunk_info[(size_t)tile * kWarps + warp] = make_uint2(cbase, fits ? wtot : 0u);
+        // residual write-back: a, with +0 where the element went into the candidate list
+        const uint32_t zm = fits ? cm : 0u;
+        if (interior) {
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                float4 o;
+                o.x = ((zm >> (4 * j + 0)) & 1u) ? 0.0f : a[j][0];
+                o.y = ((zm >> (4 * j + 1)) & 1u) ? 0.0f : a[j][1];
+                o.z = ((zm >> (4 * j + 2)) & 1u) ? 0.0f : a[j][2];
+                o.w = ((zm >> (4 * j + 3)) & 1u) ? 0.0f : a[j][3];
+                *reinterpret_cast<float4*>(r + tg.base + my_off + j * 128) = o;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if ((valid >> (4 * j + e)) & 1u)
+                        r[tg.base + my_off + j * 128 + e] = ((zm >> (4 * j + e)) & 1u) ? 0.0f : a[j][e];
+                }
+            }
+        }
         // emission: candidates are first ranked into the warp's shared staging row, then written
         // out as one contiguous run of 8-byte pairs (a chunk rarely holds more than a dozen)
         const bool staged = wtot <= (uint32_t)kEmitStage;
@@ -127,10 +184,9 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if ((cm >> (4 * j + e)) & 1u) {
-                            const uint2 pr = make_uint2(vec_index(tg.base, warp, lane, j) + e,
-                                                        __float_as_uint(tl.a[j][e]));
+                            const uint2 pr = make_uint2(tg.base + my_off + j * 128 + e, __float_as_uint(a[j][e]));
                             if (staged) sm.emit[warp][pos] = pr; else cv.pair[cbase + pos] = pr;
-                            atomicAdd(&sm.hist[key_of(tl.a[j][e]) >> level_shift(0)], 1u);
+                            atomicAdd(&sm.hist[key_of(a[j][e]) >> level_shift(0)], 1u);
                             ++pos;
                         }
                     }
@@ -145,6 +201,28 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
         ++tiles_here;
     }
     if (tiles_here) flush_and_select<0, true>(sm, ws, t, tiles_here, d.ntiles, d.k);
+}
+
+// Puts the value of every listed candidate back into the residual, for the tensors that are
+// about to be redone by the exact kernels (those need r = a everywhere).
+static __device__ void cand_restore_body(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                                         float* __restrict__ r, const WsView& ws, const CandView& cv) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool all = ld_cg(&ws.hdr->overflow) != 0u;
+    if (!all && ld_cg(&ws.hdr->n_failed) == 0u) return;
+    for (uint32_t tile = blockIdx.x * kWarps + warp; tile < ntiles; tile += gridDim.x * kWarps) {
+        const uint32_t t = find_tensor(desc, T, tile);
+        if (!all && (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u) continue;
+        TileCands tc = load_tile_cands(cv, tile, lane);
+        for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
+            uint32_t j = j0 + lane;
+            uint32_t slot = cand_slot(tc, j);
+            if (j < tc.total) {
+                const uint2 pr = ld_cg(&cv.pair[slot]);
+                r[pr.x] = __uint_as_float(pr.y);
+            }
+        }
+    }
 }
 
 // ----------------------------------------------------------------------------- candidate refinement
@@ -206,8 +284,8 @@ __device__ void cand_hist_body(BlockSmem& sm, const TensorDesc* __restrict__ des
 // tiles of one tensor, one warp per tile; group i of a CTA is blockIdx.x + i * gridDim.x.
 //   count: every group stores its (above-T, equal-T) totals;
 //   emit:  a group adds up the totals of the groups before it in its tensor, ranks its own
-//          candidates, writes the sent ones to the output and zeroes them in the residual
-//          (which already holds a).
+//          candidates, writes the sent ones to the output (their residual is already +0) and
+//          restores the value of the others in the residual.
 // An element is sent iff key > T, or key == T and fewer than m_eq equal keys precede it.
 __device__ __forceinline__ void group_tile_counts(const CandView& cv, const TileCands& tc, uint32_t Tkey,
                                                   int lane, uint32_t& ngt, uint32_t& neq) {
@@ -282,13 +360,14 @@ __device__ void cand_compact_body(BlockSmem& sm, const TensorDesc* __restrict__ 
             uint32_t mg = gpos + __popc(gb & lt_mask), me = epos + __popc(eb & lt_mask);
             if (gt || (eq && me < m_eq)) {
                 uint32_t slot_out = mg + min(me, m_eq);
-                if (slot_out < d.cap) {
+                if (slot_out < d.cap) {          // the residual already holds +0 for this entry
                     out_idx[d.out_off + slot_out] = f;
                     out_val[d.out_off + slot_out] = v;
-                    r[f] = 0.0f;
                 } else {
                     record_status(ws.hdr, -1 /*GC_E_INVALID*/, f);
                 }
+            } else if (j < tc.total) {
+                r[f] = v;                        // candidate that is not sent: give its value back
             }
             gpos += __popc(gb); epos += __popc(eb);
         }
@@ -300,11 +379,17 @@ __device__ void cand_compact_body(BlockSmem& sm, const TensorDesc* __restrict__ 
 }
 
 // ----------------------------------------------------------------------------- separate launches
-static __global__ void __launch_bounds__(kBlock)
+static __global__ void __launch_bounds__(kBlock, 4)
 k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
     __shared__ BlockSmem sm;
     fold_cand_body(sm, desc, T, ntiles, g, r, ws, cv);
+}
+
+static __global__ void __launch_bounds__(kBlock)
+k_cand_restore(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles, float* __restrict__ r,
+               WsView ws, CandView cv) {
+    cand_restore_body(desc, T, ntiles, r, ws, cv);
 }
 
 template <int LEVEL>
@@ -346,7 +431,7 @@ struct FusedArgs {
 //   overflowed -- the exact multi-pass redo of those tensors.
 // Phases are separated by grid barriers; every decision taken after a barrier reads values
 // that were final before it, so all CTAs take the same route.
-static __global__ void __launch_bounds__(kBlock, 1)
+static __global__ void __launch_bounds__(kBlock, 4)
 k_compress_fused(FusedArgs a) {
     __shared__ BlockSmem sm;
     uint32_t passed = 0;
@@ -379,7 +464,11 @@ k_compress_fused(FusedArgs a) {
         phase_stamp(hdr);
     }
     if (!overflow && ld_cg(&hdr->n_failed) == 0u) return;
-    // redo (rare): r already holds a for every element
+    // redo (rare): first give the listed candidates of those tensors their values back, so that
+    // r holds a for every element again
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    cand_restore_body(a.desc, a.T, a.ntiles, a.r, a.ws, a.cv);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     phase_stamp(hdr);
     hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);

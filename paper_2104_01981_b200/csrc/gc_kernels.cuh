@@ -206,34 +206,27 @@ __device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, ui
         }
         if (!active) continue;
         if (SRC == SRC_SAMPLE) {
-            // sample tile: 2048 sample groups; thread takes groups j*kBlock + tid.  All loads
-            // are issued before any of them is used.
+            // sample tile: kSampleTile sample groups, one per thread; all loads are issued
+            // before any of them is used
             const uint32_t ngroups = (d.n + 3u) >> 2;
-            const uint32_t sg0 = (tile - d.stile0) * (uint32_t)(kBlock * kVpt);
-            float gv[kVpt][4], rv[kVpt][4];
+            const uint64_t gi = (uint64_t)((tile - d.stile0) * (uint32_t)kSampleTile + tid) * d.sstride;
+            const uint32_t i0 = (uint32_t)min(gi, (uint64_t)ngroups) * 4u;
+            float gv[4], rv[4];
             uint32_t ok = 0;
 #pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                uint64_t gi = (uint64_t)(sg0 + j * kBlock + tid) * d.sstride;
-                uint32_t i0 = (uint32_t)min(gi, (uint64_t)ngroups) * 4u;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    bool v = gi < ngroups && i0 + e < d.n;
-                    uint32_t f = d.off + (v ? i0 + e : 0u);
-                    gv[j][e] = v ? __ldg(g + f) : 0.f;
-                    rv[j][e] = v ? ld_cg(r + f) : 0.f;
-                    ok |= (uint32_t)v << (4 * j + e);
-                }
+            for (int e = 0; e < 4; ++e) {
+                bool v = gi < ngroups && i0 + e < d.n;
+                uint32_t f = d.off + (v ? i0 + e : 0u);
+                gv[e] = v ? __ldg(g + f) : 0.f;
+                rv[e] = v ? ld_cg(r + f) : 0.f;
+                ok |= (uint32_t)v << e;
             }
 #pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    uint32_t key = key_of(__fadd_rn(gv[j][e], rv[j][e]));
-                    bool in = (ok >> (4 * j + e)) & 1u;
-                    if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
-                    if (in) atomicAdd(&sm.hist[(key >> SH) & (NB - 1)], 1u);
-                }
+            for (int e = 0; e < 4; ++e) {
+                uint32_t key = key_of(__fadd_rn(gv[e], rv[e]));
+                bool in = (ok >> e) & 1u;
+                if (!level_is_first(LEVEL)) in = in && ((key >> (SH + level_bits(LEVEL))) == prefix);
+                if (in) atomicAdd(&sm.hist[(key >> SH) & (NB - 1)], 1u);
             }
         } else {
             TileGeom tg = tile_geom(d, tile - d.tile0);
