@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "gc_fast.cuh"
+#include "gc_single.cuh"
 #include "gc_threshold.cuh"
 
 using namespace gc;
@@ -35,6 +35,11 @@ struct gc_plan_s {
     int grid_thr = 0;
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
     int grid_fused = 0;                     // CTAs of the cooperative launch (0 = not available)
+    // single-tensor shared-memory-pool kernel
+    int grid_single_max = 0;                // resident CTAs (0 = not available)
+    uint32_t single_grid = 0, single_maxt = 0, single_pool = 0;   // 0 = plan does not qualify
+    size_t single_smem = 0;
+    size_t off_hist5 = 0;
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
@@ -161,10 +166,32 @@ void finish_layout(gc_plan_s* p) {
     p->off_hist = align_up(p->off_gsel + sizeof(TensorSel) * T, 256);
     p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * T, 256);
     p->off_gstate = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
-    p->control_bytes = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
+    p->off_hist5 = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
+    p->control_bytes = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 5 * (size_t)kHistBins : 0), 256);
     p->off_tinfo = p->control_bytes;
     p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
     p->ws_bytes = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
+}
+
+
+// Decides whether the plan can use the single-tensor kernel and with which geometry.
+void plan_single(gc_plan_s* p) {
+    p->single_grid = 0;
+    if (p->mode != GC_TOPK || p->T != 1 || p->grid_single_max <= 0) return;
+    const TensorDesc& d = p->desc[0];
+    if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
+    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
+    const uint32_t maxt = (d.ntiles + G - 1) / G;
+    const size_t rec_bytes = (size_t)maxt * (2 * kWarps * sizeof(uint32_t) + sizeof(unsigned long long));
+    if (rec_bytes > 24576) return;                                   // chunk records must stay small
+    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, (1u << 22) - 1u);   // region per CTA
+    // expected candidates per CTA (sample rank over sample size, times n), with head-room
+    const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
+    if (nsg > (uint64_t)2 * G * kBlock) return;                     // a thread owns at most two sample groups
+    const double expect = (double)d.n * (double)d.srank / (4.0 * (double)nsg) / (double)G;
+    if ((double)pool < 1.5 * expect + 512.0) return;
+    if ((uint64_t)maxt > p->ngroups) return;                         // row totals live in the group array
+    p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
 }
 
 int upload_table(gc_plan_s* p) {
@@ -262,6 +289,15 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
             coop = 0;
         }
         p->grid_fused = coop ? p->sm_count * blocks_per_sm(k_compress_fused, kBlock) : 0;
+        p->grid_single_max = 0;
+        if (coop) {
+            int nb = 0;       // sized for the largest chunk-record block the kernel may be given
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, 24576) ==
+                    cudaSuccess && nb >= 1)
+                p->grid_single_max = p->sm_count * nb;
+        }
+        (void)cudaGetLastError();
+        plan_single(p);
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
@@ -282,6 +318,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
             if (value < 1 || value > 100000) return GC_E_INVALID;
             p->rank_permille = (uint32_t)value;
             finish_layout(p);                          // workspace size stays as planned
+            plan_single(p);
             return upload_table(p);
         case GC_OPT_CANDIDATE_CAPACITY:
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
@@ -387,6 +424,23 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     cv.group_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
     cv.cap = p->cand_cap;
     cv.ssel = sws.sel;
+    if (p->path == GC_PATH_AUTO && p->single_grid > 0) {
+        // one large tensor: candidates stay in shared memory
+        SingleArgs sa;
+        sa.d = p->desc[0]; sa.desc = p->d_desc; sa.ntiles = nt; sa.maxt = p->single_maxt;
+        sa.pool_cap = std::min<uint32_t>(p->single_pool, p->cand_cap);
+        sa.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+        sa.g = grad; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;
+        sa.hist5 = reinterpret_cast<uint32_t*>(wb + p->off_hist5);
+        sa.tile_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_tinfo);
+        sa.row_tot = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
+        sa.ws = ws; sa.gws = gws;
+        void* args[] = {&sa};
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_single, dim3(p->single_grid), dim3(kBlock),
+                                               args, p->single_smem, s));
+        return GC_OK;
+    }
     if (p->path == GC_PATH_AUTO && p->grid_fused > 0) {
         // everything in one cooperative launch
         FusedArgs fa;
