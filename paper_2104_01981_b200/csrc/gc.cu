@@ -646,6 +646,10 @@ int gc_last_phase_times(gc_plan_t* p, const void* workspace, void* stream, uint6
     uint32_t n = h.n_stamps > 20u ? 20u : h.n_stamps;
     *n_phases = n > 0 ? n - 1 : 0;
     for (uint32_t i = 0; i + 1 < n; ++i) ns[i] = h.stamp[i + 1] - h.stamp[i];
+    if (n > 0 && n < 20 && h.t_last_exit > h.stamp[n - 1]) {       // tail: last CTA out after CTA 0's last stamp
+        ns[n - 1] = h.t_last_exit - h.stamp[n - 1];
+        *n_phases = n;
+    }
     return GC_OK;
 }
 

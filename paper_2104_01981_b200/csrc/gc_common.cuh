@@ -70,7 +70,8 @@ struct WsHeader {            // head of the workspace, 256 bytes
     uint32_t n_stamps;       // phase time stamps recorded by CTA 0 of the fused kernel
     uint32_t pad0[3];
     unsigned long long stamp[20];   // %globaltimer (ns) at the start and after each phase
-    uint32_t reserved[4];
+    unsigned long long t_last_exit; // latest exit of any CTA of the fused kernel (ns)
+    uint32_t reserved[2];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -281,6 +282,14 @@ __device__ __forceinline__ void phase_stamp(WsHeader* hdr) {
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
         uint32_t i = hdr->n_stamps;
         if (i < 20u) { hdr->stamp[i] = ts; hdr->n_stamps = i + 1u; }
+    }
+}
+
+__device__ __forceinline__ void exit_stamp(WsHeader* hdr) {
+    if (threadIdx.x == 0) {
+        unsigned long long ts;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
+        atomicMax(&hdr->t_last_exit, ts);
     }
 }
 
