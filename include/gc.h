@@ -225,6 +225,7 @@ int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_stagin
 #define GC_K_CAND_COMPACT  11   /* ordered emission from the candidate lists                 */
 #define GC_K_THRESHOLD_EMIT 12  /* threshold mode: fold + send everything at or above tau    */
 #define GC_K_FUSED         13   /* whole top-k compress as one cooperative launch            */
+#define GC_K_SMALL         14   /* small tensors, each selected exactly by one CTA           */
 #define GC_K_COUNT         16
 int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
 int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);

@@ -23,6 +23,8 @@ struct gc_plan_s {
     uint32_t ntiles = 0;
     std::vector<TensorDesc> desc;
     TensorDesc* d_desc = nullptr;
+    uint32_t* d_small = nullptr;            // ids of the small tensors (device), n_small entries
+    std::vector<uint32_t> small_ids;
     uint32_t nstiles = 0, ngroups = 0;
     uint32_t cand_cap = 0, cand_cap_alloc = 0;
     uint32_t n_sampled = 0;                 // tensors with a sample
@@ -102,8 +104,8 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
     const uint64_t n = d.n;
     d.sstride = 0; d.srank = 0;
     *ccap = n;
-    if (n < 131072) return;                              // small tensors: every element is a candidate
-    uint64_t target = std::min<uint64_t>(131072, std::max<uint64_t>(32768, n / 128));
+    if (n < kSmallMax) { d.kind = kKindSmall; *ccap = 0; return; }   // one CTA does the whole tensor
+    uint64_t target = std::min<uint64_t>(131072, std::max<uint64_t>(n / 128, std::min<uint64_t>(8192, n / 2)));
     uint64_t stride = std::max<uint64_t>(1, n / target);
     uint64_t groups = (n + 3) / 4;
     uint64_t nsg = (groups + stride - 1) / stride;
@@ -123,8 +125,10 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
 void finish_layout(gc_plan_s* p) {
     uint64_t stile0 = 0, group0 = 0, ccap_total = 0;
     p->n_sampled = 0;
+    p->small_ids.clear();
     for (uint32_t t = 0; t < p->T; ++t) {
         TensorDesc& d = p->desc[t];
+        d.kind = kKindRegular; d.pad = 0;
         uint64_t ccap = d.n;
         if (p->mode == GC_TOPK) {
             sample_params(d, p->density, p->rank_permille, &ccap);
@@ -149,6 +153,7 @@ void finish_layout(gc_plan_s* p) {
         }
         d.stile0 = (uint32_t)stile0; d.nstiles = (uint32_t)nst;
         d.group0 = (uint32_t)group0; d.ngroups = (d.ntiles + kWarps - 1) / kWarps;
+        if (d.kind == kKindSmall && d.n > 0) p->small_ids.push_back(t);
         stile0 += nst; group0 += d.ngroups; ccap_total += ccap;
     }
     p->nstiles = (uint32_t)stile0;
@@ -198,6 +203,9 @@ int upload_table(gc_plan_s* p) {
     if (p->device < 0 || p->T == 0) return GC_OK;
     cudaError_t e = cudaMemcpy(p->d_desc, p->desc.data(), sizeof(TensorDesc) * (size_t)p->T,
                                cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !p->small_ids.empty())
+        e = cudaMemcpy(p->d_small, p->small_ids.data(), sizeof(uint32_t) * p->small_ids.size(),
+                       cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; (void)cudaGetLastError(); return GC_E_CUDA; }
     return GC_OK;
 }
@@ -254,7 +262,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         d.off = (uint32_t)off; d.n = (uint32_t)n; d.k = (uint32_t)k; d.cap = (uint32_t)cap;
         d.out_off = (uint32_t)out_off; d.tile0 = (uint32_t)tile0; d.ntiles = (uint32_t)nt;
         d.stride = n <= 65536 ? 1u : sample_stride;
-        d.pad[0] = d.pad[1] = 0;
+        d.kind = kKindRegular; d.pad = 0;
         off += n; out_off += cap; tile0 += nt;
     }
     p->total_cap = out_off;
@@ -270,12 +278,13 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     if (e == cudaSuccess && n_tensors > 0) {
         e = cudaMalloc(reinterpret_cast<void**>(&p->d_desc), sizeof(TensorDesc) * (size_t)n_tensors);
         if (e == cudaSuccess)
-            e = cudaMemcpy(p->d_desc, p->desc.data(), sizeof(TensorDesc) * (size_t)n_tensors,
-                           cudaMemcpyHostToDevice);
+            e = cudaMalloc(reinterpret_cast<void**>(&p->d_small), sizeof(uint32_t) * (size_t)n_tensors);
+        if (e == cudaSuccess) e = upload_table(p) == GC_OK ? cudaSuccess : cudaErrorUnknown;
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         if (p->d_desc) cudaFree(p->d_desc);
+        if (p->d_small) cudaFree(p->d_small);
         delete p;
         return GC_E_CUDA;
     }
@@ -445,14 +454,21 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         // everything in one cooperative launch
         FusedArgs fa;
         fa.desc = p->d_desc; fa.T = p->T; fa.ntiles = nt; fa.nstiles = p->nstiles; fa.ngroups = p->ngroups;
+        fa.small_ids = p->d_small; fa.n_small = (uint32_t)p->small_ids.size();
         fa.g = grad; fa.r = residual; fa.out_idx = out_idx; fa.out_val = out_val; fa.out_count = out_count;
         fa.ws = ws; fa.sws = sws; fa.gws = gws; fa.cv = cv;
         void* args[] = {&fa};
-        const uint32_t want = std::max<uint32_t>(std::max<uint32_t>(nt, p->nstiles), 1u);
+        const uint32_t want = std::max<uint32_t>(std::max<uint32_t>(nt, p->nstiles), 1u);   // nt >= #small tensors
         const int gf = (int)std::min<uint32_t>(want, (uint32_t)p->grid_fused);
         Timed tm(p, s, GC_K_FUSED);
         GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_compress_fused, dim3(gf), dim3(kBlock), args, 0, s));
         return GC_OK;
+    }
+    if (!p->small_ids.empty()) {
+        Timed tm(p, s, GC_K_SMALL);
+        const int gsm = (int)std::min<uint32_t>((uint32_t)p->small_ids.size(), (uint32_t)p->grid_hist);
+        k_small_tensors<<<gsm, kBlock, 0, s>>>(p->d_desc, p->T, p->d_small, (uint32_t)p->small_ids.size(), grad,
+                                               residual, out_idx, out_val, out_count);
     }
     if (p->nstiles > 0) {
         const int gs = (int)std::min<uint32_t>(p->nstiles, (uint32_t)p->grid_sample);
@@ -618,6 +634,7 @@ const char* gc_kernel_name(int id) {
         case GC_K_SAMPLE: return "sample";
         case GC_K_THRESHOLD_EMIT: return "threshold_emit";
         case GC_K_FUSED: return "compress_fused";
+        case GC_K_SMALL: return "small_tensors";
         case GC_K_FOLD_CAND: return "fold_cand";
         case GC_K_CAND_REFINE: return "cand_refine";
         case GC_K_CAND_COMPACT: return "cand_compact";
@@ -659,6 +676,7 @@ int gc_destroy(gc_plan_t* p) {
     if (p == nullptr) return GC_OK;
     int rc = GC_OK;
     for (auto& r : p->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    if (p->d_small) { (void)cudaSetDevice(p->device); (void)cudaFree(p->d_small); }
     if (p->d_desc) {
         (void)cudaSetDevice(p->device);
         if (cudaFree(p->d_desc) != cudaSuccess) { (void)cudaGetLastError(); rc = GC_E_CUDA; }

@@ -44,8 +44,12 @@ struct TensorDesc {          // one per tensor, immutable, plan-owned device mem
     uint32_t nstiles;        // sample tiles (kSampleTile sample groups each)
     uint32_t group0;         // first compaction group id (a group = kWarps consecutive tiles)
     uint32_t ngroups;        // compaction groups of this tensor
-    uint32_t pad[2];
+    uint32_t kind;           // kKindRegular, or kKindSmall: the candidate path hands the whole tensor
+                             // to one CTA that selects exactly on its own (no sample, no candidates)
+    uint32_t pad;
 };
+constexpr uint32_t kKindRegular = 0u, kKindSmall = 1u;
+constexpr uint32_t kSmallMax = 16384;        // tensors below this many elements are "small"
 static_assert(sizeof(TensorDesc) == 64, "tensor table entry is 64 bytes");
 
 struct TensorSel {           // one per tensor, in the workspace, rewritten every call
@@ -145,9 +149,11 @@ __device__ __forceinline__ uint32_t find_tensor(const TensorDesc* __restrict__ d
     return lo;
 }
 
-__device__ __forceinline__ bool gate_open(const WsView& ws, uint32_t t) {
-    // with a gate, a tensor is processed only if the candidate path failed for it (or overall)
+__device__ __forceinline__ bool gate_open(const WsView& ws, uint32_t t, const TensorDesc& d) {
+    // with a gate, a tensor is processed only if the candidate path failed for it (or overall);
+    // small tensors were finished by their own CTA and are never redone
     if (ws.gate == nullptr) return true;
+    if (d.kind == kKindSmall) return false;
     return (ld_cg(&ws.gate[t].flags) & kSelFailed) != 0u || ld_cg(&ws.hdr->overflow) != 0u;
 }
 __device__ __forceinline__ bool nothing_to_redo(const WsView& ws) {

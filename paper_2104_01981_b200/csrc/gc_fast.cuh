@@ -54,21 +54,136 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
     return b + (j - ex);
 }
 
+// ----------------------------------------------------------------------------- small tensors
+// Exact top-k of one small tensor (fewer than kSmallMax elements) by ONE CTA, start to finish:
+// fold + level-0 histogram, two refinement passes and the ordered emission all stay inside the
+// CTA (shared-memory histograms, __syncthreads only), so hundreds of tiny tensors cost no global
+// atomics, no completion counters and no grid barriers.
+static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const TensorDesc& d, uint32_t t, uint32_t T,
+                                         const float* __restrict__ g, float* __restrict__ r,
+                                         uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                         uint32_t* __restrict__ out_count) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t prefix = 0, krem = d.k;
+#pragma unroll 1
+    for (int level = 0; level < kLevels; ++level) {
+        const int bits = level_bits(level), sh = level_shift(level);
+        __syncthreads();
+        for (int b = tid; b < (1 << level_bits(0)); b += kBlock) sm.hist[b] = 0u;
+        __syncthreads();
+        for (uint32_t ti = 0; ti < d.ntiles; ++ti) {
+            const TileGeom tg = tile_geom(d, ti);
+            Tile tl;
+            if (level == 0) load_tile<true>(g, r, tg, warp, lane, tl); else load_tile<false>(nullptr, r, tg, warp, lane, tl);
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t key = key_of(tl.a[j][e]);
+                    bool in = (tl.valid >> (4 * j + e)) & 1u;
+                    if (level > 0) in = in && ((key >> (sh + bits)) == prefix);
+                    if (in) atomicAdd(&sm.hist[(key >> sh) & ((1u << bits) - 1u)], 1u);
+                }
+            }
+        }
+        __syncthreads();
+        uint32_t bin, above;
+        if (level == 0) block_select<(1 << level_bits(0)), true>(sm, sm.hist, krem, bin, above);
+        else block_select<(1 << level_bits(1)), true>(sm, sm.hist, krem, bin, above);
+        prefix = (prefix << bits) | bin;
+        krem -= above;
+    }
+    const uint32_t Tkey = prefix, m_eq = krem;
+    // ordered emission, tile after tile, with running counts
+    uint32_t gt_run = 0, eq_run = 0;
+    for (uint32_t ti = 0; ti < d.ntiles; ++ti) {
+        const TileGeom tg = tile_geom(d, ti);
+        Tile tl;
+        load_tile<false>(nullptr, r, tg, warp, lane, tl);
+        uint32_t cg[kVpt], ce[kVpt], gtm = 0, eqm = 0;
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            cg[j] = 0; ce[j] = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t key = key_of(tl.a[j][e]);
+                const bool v = (tl.valid >> (4 * j + e)) & 1u;
+                const bool gt = v && key > Tkey, eq = v && key == Tkey;
+                cg[j] += gt; ce[j] += eq;
+                gtm |= (uint32_t)gt << (4 * j + e);
+                eqm |= (uint32_t)eq << (4 * j + e);
+            }
+        }
+        uint32_t rg[kVpt], re[kVpt], wg, we;
+        warp_rank(cg, lane, rg, wg);
+        warp_rank(ce, lane, re, we);
+        __syncthreads();
+        if (lane == 0) { sm.gt_tot[warp] = wg; sm.eq_tot[warp] = we; }
+        __syncthreads();
+        scan_warp_totals(sm.gt_tot, sm.gt_ex, &sm.gt_sum, warp, lane);
+        if (warp == 1) {
+            uint32_t v = lane < kWarps ? sm.eq_tot[lane] : 0u;
+            uint32_t inc = warp_incl_scan(v, lane);
+            if (lane < kWarps) sm.eq_ex[lane] = inc - v;
+            if (lane == 31) sm.eq_sum = inc;
+        }
+        __syncthreads();
+        if ((gtm | eqm) != 0u) {
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                uint32_t gpos = gt_run + sm.gt_ex[warp] + rg[j], epos = eq_run + sm.eq_ex[warp] + re[j];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool gt = (gtm >> (4 * j + e)) & 1u, eq = (eqm >> (4 * j + e)) & 1u;
+                    if (gt || (eq && epos < m_eq)) {
+                        const uint32_t slot = gpos + min(epos, m_eq);
+                        const uint32_t f = vec_index(tg.base, warp, lane, j) + e;
+                        if (slot < d.cap) {
+                            out_idx[d.out_off + slot] = f;
+                            out_val[d.out_off + slot] = tl.a[j][e];
+                            r[f] = 0.0f;
+                        }
+                    }
+                    gpos += gt; epos += eq;
+                }
+            }
+        }
+        gt_run += sm.gt_sum; eq_run += sm.eq_sum;
+    }
+    if (out_count != nullptr && tid == 0) { out_count[t] = d.k; out_count[T + t] = d.k; }
+    __syncthreads();
+}
+
+// All small tensors of the plan, dealt out to the CTAs round-robin.
+static __device__ void small_tensors_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
+                                          const uint32_t* __restrict__ small_ids, uint32_t n_small,
+                                          const float* __restrict__ g, float* __restrict__ r,
+                                          uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                          uint32_t* __restrict__ out_count) {
+    for (uint32_t q = blockIdx.x; q < n_small; q += gridDim.x) {
+        const uint32_t t = small_ids[q];
+        const TensorDesc d = desc[t];
+        small_tensor_body(sm, d, t, T, g, r, out_idx, out_val, out_count);
+    }
+}
+
 // ----------------------------------------------------------------------------- fold + candidates
 // Reads g and r, computes a = g + r, emits candidates and writes the residual back with the
 // candidates ALREADY zeroed (their values live in the candidate list): after the selection
 // only the few candidates that were not sent need their value restored, instead of every
 // sent entry needing a scattered zero.  A chunk whose candidates did not fit in the list keeps
-// its values in r.  Tile i of a CTA is blockIdx.x + i * gridDim.x, so at any moment the CTAs
-// sweep one contiguous window of memory.  No block-wide barrier in the tile loop: every warp
-// ranks and stores the candidates of its own chunk.
+// its values in r.  CTAs take contiguous runs of tiles (plans with many tensors then change
+// tensor -- and flush their histogram -- as rarely as possible).  No block-wide barrier in the
+// tile loop: every warp ranks and stores the candidates of its own chunk.
 static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
                                       uint32_t ntiles, const float* __restrict__ g, float* __restrict__ r,
                                       const WsView& ws, const CandView& cv) {
     constexpr int NB = 1 << level_bits(0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t first = blockIdx.x, tstep = gridDim.x;
-    if (first >= ntiles) return;
+    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t first = blockIdx.x * per;
+    const uint32_t last = min(ntiles, first + per);
+    if (first >= last) return;
     for (int b = tid; b < NB; b += kBlock) sm.hist[b] = 0u;
     __syncthreads();
 
@@ -79,7 +194,7 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
     uint32_t slab_next = 0, slab_left = 0;       // this warp's current slab (warp-uniform)
     const uint32_t my_off = warp * kWarpChunk + lane * 4;
 
-    for (uint32_t tile = first; tile < ntiles; tile += tstep) {
+    for (uint32_t tile = first; tile < last; ++tile) {
         if (tile >= d.tile0 + d.ntiles) {
             if (tiles_here) flush_and_select<0, true>(sm, ws, t, tiles_here, d.ntiles, d.k);
             tiles_here = 0;
@@ -87,6 +202,7 @@ static __device__ void fold_cand_body(BlockSmem& sm, const TensorDesc* __restric
             d = desc[t];
             tau = d.sstride ? (ld_cg(&cv.ssel[t].prefix) << level_shift(1)) : 0u;
         }
+        if (d.kind == kKindSmall) continue;      // finished by its own CTA
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         const bool interior = tg.lo == tg.base && tg.hi == tg.base + (uint32_t)kTile;
         float a[kVpt][4];
@@ -212,6 +328,7 @@ static __device__ void cand_restore_body(const TensorDesc* __restrict__ desc, ui
     if (!all && ld_cg(&ws.hdr->n_failed) == 0u) return;
     for (uint32_t tile = blockIdx.x * kWarps + warp; tile < ntiles; tile += gridDim.x * kWarps) {
         const uint32_t t = find_tensor(desc, T, tile);
+        if (desc[t].kind == kKindSmall) continue;
         if (!all && (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u) continue;
         TileCands tc = load_tile_cands(cv, tile, lane);
         for (uint32_t j0 = 0; j0 < tc.total; j0 += 32) {
@@ -245,7 +362,7 @@ __device__ void cand_hist_body(BlockSmem& sm, const TensorDesc* __restrict__ des
 
     uint32_t t = find_tensor(desc, T, first);
     TensorDesc d = desc[t];
-    bool active = (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
+    bool active = d.kind != kKindSmall && (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
     uint32_t prefix = ld_cg(&ws.sel[t].prefix);
     uint32_t tiles_here = 0;
 
@@ -256,7 +373,7 @@ __device__ void cand_hist_body(BlockSmem& sm, const TensorDesc* __restrict__ des
             tiles_here = 0;
             t = find_tensor(desc, T, batch);
             d = desc[t];
-            active = (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
+            active = d.kind != kKindSmall && (ld_cg(&ws.sel[t].flags) & kSelFailed) == 0u;
             prefix = ld_cg(&ws.sel[t].prefix);
         }
         const uint32_t bend = min(min(last, d.tile0 + d.ntiles), batch + (uint32_t)kWarps);
@@ -310,8 +427,8 @@ __device__ void cand_compact_body(BlockSmem& sm, const TensorDesc* __restrict__ 
     for (uint32_t group = blockIdx.x; group < ngroups_total; group += gridDim.x) {
         __syncthreads();
         const uint32_t t = find_tensor<GroupSpace>(desc, T, group);
-        if (ld_cg(&ws.sel[t].flags) & kSelFailed) continue;
         const TensorDesc d = desc[t];
+        if (d.kind == kKindSmall || (ld_cg(&ws.sel[t].flags) & kSelFailed)) continue;
         const uint32_t Tkey = ld_cg(&ws.sel[t].T), m_eq = ld_cg(&ws.sel[t].m_eq);
         const uint32_t tile_in_t = (group - d.group0) * kWarps + warp;
         TileCands tc;
@@ -379,6 +496,14 @@ __device__ void cand_compact_body(BlockSmem& sm, const TensorDesc* __restrict__ 
 }
 
 // ----------------------------------------------------------------------------- separate launches
+static __global__ void __launch_bounds__(kBlock)
+k_small_tensors(const TensorDesc* __restrict__ desc, uint32_t T, const uint32_t* __restrict__ small_ids,
+                uint32_t n_small, const float* __restrict__ g, float* __restrict__ r,
+                uint32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t* __restrict__ out_count) {
+    __shared__ BlockSmem sm;
+    small_tensors_body(sm, desc, T, small_ids, n_small, g, r, out_idx, out_val, out_count);
+}
+
 static __global__ void __launch_bounds__(kBlock, 4)
 k_fold_cand(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
             const float* __restrict__ g, float* __restrict__ r, WsView ws, CandView cv) {
@@ -414,6 +539,8 @@ k_cand_compact(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ngroups
 struct FusedArgs {
     const TensorDesc* desc;
     uint32_t T, ntiles, nstiles, ngroups;
+    const uint32_t* small_ids;
+    uint32_t n_small;
     const float* g;
     float* r;
     uint32_t* out_idx;
@@ -437,6 +564,8 @@ k_compress_fused(FusedArgs a) {
     uint32_t passed = 0;
     WsHeader* hdr = a.ws.hdr;
     phase_stamp(hdr);
+    // small tensors need nothing from anyone: run them first, no barrier of their own
+    small_tensors_body(sm, a.desc, a.T, a.small_ids, a.n_small, a.g, a.r, a.out_idx, a.out_val, a.out_count);
     if (a.nstiles) {
         hist_body<0, SRC_SAMPLE>(sm, a.desc, a.T, a.nstiles, a.g, a.r, a.sws);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;

@@ -162,6 +162,48 @@ __device__ __forceinline__ void flush_and_select(BlockSmem& sm, const WsView& ws
     }
 }
 
+// ----------------------------------------------------------------------------- CTA-wide select
+// Every thread of the CTA: find the bin of `hist` (NB bins; in global memory and complete, or in
+// this CTA's shared memory) that holds the krem-th largest key.  Returns false if the histogram
+// holds fewer than krem keys.  All threads get the same result.
+template <int NB, bool IN_SMEM>
+__device__ bool block_select(BlockSmem& sm, const uint32_t* hist, uint32_t krem, uint32_t& bin,
+                             uint32_t& above_out) {
+    constexpr int BPT = (NB + kBlock - 1) / kBlock;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t c[BPT], sum = 0;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        int b = NB - 1 - (tid * BPT + i);
+        c[i] = (b >= 0) ? (IN_SMEM ? hist[b] : ld_cg(hist + b)) : 0u;
+        sum += c[i];
+    }
+    uint32_t inc = warp_incl_scan(sum, lane);
+    __syncthreads();
+    if (lane == 31) sm.scratch[warp] = inc;
+    if (tid == 0) { sm.gt_sum = 0xFFFFFFFFu; sm.eq_sum = 0u; }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t v = lane < kWarps ? sm.scratch[lane] : 0u;
+        uint32_t wi = warp_incl_scan(v, lane);
+        if (lane < kWarps) sm.scratch[lane] = wi - v;
+        if (lane == kWarps - 1) sm.scratch[kWarps] = wi;
+    }
+    __syncthreads();
+    uint32_t above = sm.scratch[warp] + inc - sum;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        int b = NB - 1 - (tid * BPT + i);
+        if (b >= 0 && above < krem && krem <= above + c[i]) { sm.gt_sum = (uint32_t)b; sm.eq_sum = above; }
+        above += c[i];
+    }
+    __syncthreads();
+    bin = sm.gt_sum; above_out = sm.eq_sum;
+    const bool ok = sm.scratch[kWarps] >= krem && bin != 0xFFFFFFFFu;
+    __syncthreads();
+    return ok;
+}
+
 // ----------------------------------------------------------------------------- histogram pass
 // One radix-select level over all tensors.  CTAs take contiguous runs of tiles, keep a
 // shared-memory histogram while the tensor stays the same, flush it with global atomics when
@@ -190,7 +232,7 @@ __device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, ui
 
     uint32_t t = find_tensor<S>(desc, T, first);
     TensorDesc d = desc[t];
-    bool active = gate_open(ws, t);
+    bool active = gate_open(ws, t, d);
     uint32_t prefix = level_is_first(LEVEL) ? 0u : ld_cg(&ws.sel[t].prefix);
     uint32_t tiles_here = 0;
 
@@ -201,7 +243,7 @@ __device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, ui
             tiles_here = 0;
             t = find_tensor<S>(desc, T, tile);
             d = desc[t];
-            active = gate_open(ws, t);
+            active = gate_open(ws, t, d);
             prefix = level_is_first(LEVEL) ? 0u : ld_cg(&ws.sel[t].prefix);
         }
         if (!active) continue;
@@ -263,7 +305,7 @@ k_hist(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
 // exchange.  An element is sent iff key > T, or key == T and fewer than m_eq equal keys
 // precede it in the tensor.  Sent elements are written as (flat index, value) at their rank
 // and zeroed in the residual.
-static __device__ void compact_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+static __device__ __noinline__ void compact_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                              float* __restrict__ r, uint32_t* __restrict__ out_idx,
                              float* __restrict__ out_val, uint32_t* __restrict__ out_count,
                              const WsView& ws, int ticket_slot) {
@@ -281,8 +323,8 @@ static __device__ void compact_body(BlockSmem& sm, const TensorDesc* __restrict_
         const uint32_t tile = sm.tile;
         if (tile >= ntiles) break;
         const uint32_t t = find_tensor(desc, T, tile);
-        if (!gate_open(ws, t)) continue;
         const TensorDesc d = desc[t];
+        if (!gate_open(ws, t, d)) continue;
         const uint32_t Tkey = ld_cg(&ws.sel[t].T), m_eq = ld_cg(&ws.sel[t].m_eq);
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;

@@ -46,7 +46,7 @@ __global__ void k_noalloc_init(unsigned char* scratch, uint32_t n, uint32_t k, u
         TensorDesc d;
         d.off = 0; d.n = n; d.k = k; d.cap = k; d.out_off = 0; d.tile0 = 0; d.ntiles = ntiles; d.stride = 1;
         d.sstride = 0; d.srank = 0; d.stile0 = 0; d.nstiles = 0; d.group0 = 0; d.ngroups = 0;
-        d.pad[0] = d.pad[1] = 0;
+        d.kind = kKindRegular; d.pad = 0;
         *reinterpret_cast<TensorDesc*>(scratch + kOffDesc) = d;
     }
 }

@@ -34,46 +34,6 @@ struct SingleArgs {
     WsView ws, gws;
 };
 
-// Every CTA: find the bin of `hist` (NB bins, global, complete) that holds the krem-th largest
-// key.  Returns false if the histogram holds fewer than krem keys.  All threads get the result.
-template <int NB>
-__device__ bool block_select(BlockSmem& sm, const uint32_t* hist, uint32_t krem, uint32_t& bin,
-                             uint32_t& above_out) {
-    constexpr int BPT = (NB + kBlock - 1) / kBlock;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t c[BPT], sum = 0;
-#pragma unroll
-    for (int i = 0; i < BPT; ++i) {
-        int b = NB - 1 - (tid * BPT + i);
-        c[i] = (b >= 0) ? ld_cg(hist + b) : 0u;
-        sum += c[i];
-    }
-    uint32_t inc = warp_incl_scan(sum, lane);
-    __syncthreads();
-    if (lane == 31) sm.scratch[warp] = inc;
-    if (tid == 0) { sm.gt_sum = 0xFFFFFFFFu; sm.eq_sum = 0u; }
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t v = lane < kWarps ? sm.scratch[lane] : 0u;
-        uint32_t wi = warp_incl_scan(v, lane);
-        if (lane < kWarps) sm.scratch[lane] = wi - v;
-        if (lane == kWarps - 1) sm.scratch[kWarps] = wi;
-    }
-    __syncthreads();
-    uint32_t above = sm.scratch[warp] + inc - sum;
-#pragma unroll
-    for (int i = 0; i < BPT; ++i) {
-        int b = NB - 1 - (tid * BPT + i);
-        if (b >= 0 && above < krem && krem <= above + c[i]) { sm.gt_sum = (uint32_t)b; sm.eq_sum = above; }
-        above += c[i];
-    }
-    __syncthreads();
-    bin = sm.gt_sum; above_out = sm.eq_sum;
-    const bool ok = sm.scratch[kWarps] >= krem && bin != 0xFFFFFFFFu;
-    __syncthreads();
-    return ok;
-}
-
 __device__ __forceinline__ void flush_hist(BlockSmem& sm, uint32_t* hist, int nb) {
     __syncthreads();
     for (int b = threadIdx.x; b < nb; b += kBlock) {
@@ -140,7 +100,7 @@ k_topk_single(SingleArgs a) {
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
         uint32_t bin0, above0;
-        const bool ok0 = block_select<(1 << level_bits(0))>(sm, a.hist5 + 0 * kHistBins, d.srank, bin0, above0);
+        const bool ok0 = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 0 * kHistBins, d.srank, bin0, above0);
         if (ok0) {
 #pragma unroll
             for (int q = 0; q < kMaxOwn; ++q)
@@ -154,7 +114,7 @@ k_topk_single(SingleArgs a) {
         phase_stamp(hdr);
         if (ok0) {
             uint32_t bin1, above1;
-            if (block_select<(1 << level_bits(1))>(sm, a.hist5 + 1 * kHistBins, d.srank - above0, bin1, above1))
+            if (block_select<(1 << level_bits(1)), false>(sm, a.hist5 + 1 * kHistBins, d.srank - above0, bin1, above1))
                 tau = ((bin0 << level_bits(1)) | bin1) << level_shift(1);
         }
         // tau == 0 (sample too small for the rank): every element becomes a candidate, the pool
@@ -279,7 +239,7 @@ k_topk_single(SingleArgs a) {
     if (good) {
         // ------------------------------------------------------------ radix select on the candidates
         uint32_t bin0, above0, bin1 = 0, above1 = 0, bin2 = 0, above2 = 0;
-        good = block_select<(1 << level_bits(0))>(sm, a.hist5 + 2 * kHistBins, d.k, bin0, above0);
+        good = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 2 * kHistBins, d.k, bin0, above0);
         if (good) {
             for (uint32_t i = tid; i < used; i += kBlock) {
                 const uint32_t key = ld_cg(&pool[i]).y & kKeyMask;
@@ -290,7 +250,7 @@ k_topk_single(SingleArgs a) {
         flush_hist(sm, a.hist5 + 3 * kHistBins, 1 << level_bits(1));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
-        if (good) good = block_select<(1 << level_bits(1))>(sm, a.hist5 + 3 * kHistBins, d.k - above0, bin1, above1);
+        if (good) good = block_select<(1 << level_bits(1)), false>(sm, a.hist5 + 3 * kHistBins, d.k - above0, bin1, above1);
         const uint32_t p1 = (bin0 << level_bits(1)) | bin1;
         if (good) {
             for (uint32_t i = tid; i < used; i += kBlock) {
@@ -302,7 +262,7 @@ k_topk_single(SingleArgs a) {
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
         if (good)
-            good = block_select<(1 << level_bits(2))>(sm, a.hist5 + 4 * kHistBins, d.k - above0 - above1, bin2, above2);
+            good = block_select<(1 << level_bits(2)), false>(sm, a.hist5 + 4 * kHistBins, d.k - above0 - above1, bin2, above2);
         Tkey = (p1 << level_bits(2)) | bin2;
         m_eq = d.k - above0 - above1 - above2;
     }
