@@ -168,7 +168,11 @@ int gc_compress(gc_plan_t *plan, const float *grad, float *residual,
  *   workspace  device, GC_Q_WORKSPACE_BYTES bytes, 256-byte aligned; either one that
  *              gc_compress has used (ordered before this call on the stream) or zero-filled
  *              by the caller -- this call does not reset the status word
- * An index >= total_n is skipped and GC_E_INVALID is recorded in the device status.
+ * With count = NULL every list must be exactly as gc_compress wrote it in top-k mode (total_cap
+ * pairs, ascending index): the dense buffer is then built tile by tile in shared memory and
+ * written once.  With count arrays the sets are applied one launch per worker instead.
+ * An index >= total_n (or a list that is not ascending) is skipped and GC_E_INVALID is recorded
+ * in the device status.
  * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_CUDA.  Asynchronous.
  */
 int gc_decompress_accumulate(gc_plan_t *plan, uint32_t W,
@@ -226,6 +230,7 @@ int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_stagin
 #define GC_K_THRESHOLD_EMIT 12  /* threshold mode: fold + send everything at or above tau    */
 #define GC_K_FUSED         13   /* whole top-k compress as one cooperative launch            */
 #define GC_K_SMALL         14   /* small tensors, each selected exactly by one CTA           */
+#define GC_K_DECODE_TILES  15   /* tiled decode: W sorted lists summed into the dense buffer */
 #define GC_K_COUNT         16
 int gc_profile_enable(gc_plan_t *plan, uint32_t max_records);
 int gc_profile_read(gc_plan_t *plan, float *total_ms, uint32_t *launches);

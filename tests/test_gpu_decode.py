@@ -62,6 +62,34 @@ def test_decode_matches_oracle_bitwise(W, sizes, density):
     assert st == api.GC_OK
 
 
+@pytest.mark.parametrize("W", [3, 16, 33, 64])
+def test_decode_many_workers_and_unaligned_output(W):
+    """Worker counts that are not powers of two, more than one pass of 32 workers, duplicate
+    indices across workers (same seed for some workers), and a dense buffer that is only
+    4-byte aligned (no bulk copies)."""
+    sizes = [70_001, 9, 20_000]
+    plan = api.Plan(sizes, 0.03, device=0)
+    n = plan.total_n
+    workers = [GpuWorker(plan) for _ in range(W)]
+    for w, wk in enumerate(workers):
+        gen = torch.Generator().manual_seed(5 + w // 3)              # groups of 3 workers share indices
+        g = torch.randn(n, generator=gen) * (10.0 ** (w % 5 - 2))
+        wk.step(g.cuda())
+    pairs = oracle_pairs(workers, plan)
+    for shift in (0, 1):
+        backing = torch.full((n + 8,), 3.0, device="cuda")
+        out = backing[shift:shift + n]
+        for zero_first in (True, False):
+            before = out.cpu().numpy().copy()
+            plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out,
+                                       zero_first, workers[0].ws)
+            want = oracle.decode_accumulate(pairs, before, zero_first)
+            assert np.array_equal(to_np_u32(out), bits(want)), (W, shift, zero_first)
+        assert backing[shift + n:].eq(3.0).all() and backing[:shift].eq(3.0).all()
+    st, _ = plan.last_status(workers[0].ws)
+    assert st == api.GC_OK
+
+
 def test_density_one_reproduces_the_dense_sum():
     sizes, W = [9, 30_000, 4097], 5
     plan, workers, grads = run_workers(sizes, 1.0, W, seed=11, dist_scale=[1.0, 1e3, 1e-3, 50.0, 0.1])
@@ -93,12 +121,19 @@ def test_worker_order_is_observable_and_fixed():
 def test_out_of_range_index_is_skipped_and_reported():
     plan = api.Plan([100], 0.04, device=0)          # k = 4
     ws = plan.alloc_workspace()
-    idx = torch.tensor([1, 50, 100, 99], dtype=torch.int32, device="cuda")
+    idx = torch.tensor([1, 50, 99, 100], dtype=torch.int32, device="cuda")
     val = torch.ones(4, device="cuda")
     out = torch.empty(100, device="cuda")
     plan.decompress_accumulate([idx], [val], None, out, True, ws)
     st, det = plan.last_status(ws)
-    assert st == api.GC_E_INVALID and det == 2
+    assert st == api.GC_E_INVALID and det == 3          # position of the bad entry in the list
+    assert out.sum().item() == 3.0
+    # the per-worker launch path (count arrays given) reports the same
+    ws.zero_()
+    cnt = torch.tensor([4, 4], dtype=torch.int32, device="cuda")
+    plan.decompress_accumulate([idx], [val], [cnt], out, True, ws)
+    st, det = plan.last_status(ws)
+    assert st == api.GC_E_INVALID and det == 3
     assert out.sum().item() == 3.0
 
 
