@@ -15,6 +15,7 @@ namespace gc {
 constexpr int kDecTile = 1024;               // floats per warp tile
 constexpr int kDecBlock = 256;
 constexpr int kDecWarps = kDecBlock / 32;
+constexpr int kDecRounds = 4;                // entries a lane pre-loads per worker and tile
 
 struct DecodeLists {
     const uint32_t* idx[64];
@@ -114,25 +115,37 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         for (int ps = 0; ps < passes; ++ps) {
             const uint32_t w = (uint32_t)(ps * Wp + lane / E);
             const bool live = w < W;
-            // fast path: the first E entries at the cursor of every worker, loaded together
-            const uint32_t p = cur[ps] + (uint32_t)sub;
-            uint32_t ix = 0xFFFFFFFFu;
-            float v = 0.f;
-            if (live && p < cnt) { ix = __ldg(ls.idx[w] + p); v = __ldg(ls.val[w] + p); }
-            const bool in = ix < hi;                      // lists are sorted: the ins of a worker are a prefix
-            // a worker whose E entries all fall inside may have more: then this tile takes the
-            // strictly sequential path below so that worker order is kept for every element
-            const bool maybe_more = in && sub == E - 1;
+            // fast path: the first kDecRounds * E entries at the cursor of every worker, loaded together
+            uint32_t ix[kDecRounds];
+            float v[kDecRounds];
+            uint32_t nin = 0;
+#pragma unroll
+            for (int rd = 0; rd < kDecRounds; ++rd) {
+                const uint32_t p = cur[ps] + (uint32_t)(rd * E + sub);
+                ix[rd] = 0xFFFFFFFFu; v[rd] = 0.f;
+                if (live && p < cnt) { ix[rd] = __ldg(ls.idx[w] + p); v[rd] = __ldg(ls.val[w] + p); }
+            }
+#pragma unroll
+            for (int rd = 0; rd < kDecRounds; ++rd) nin += ix[rd] < hi;   // sorted lists: the ins are a prefix
+            // a worker whose loaded entries all fall inside may have more: then this tile takes
+            // the strictly sequential path below so that worker order is kept for every element
+            const bool maybe_more = (ix[kDecRounds - 1] < hi) && sub == E - 1;
             if (!__any_sync(0xFFFFFFFFu, maybe_more)) {
                 for (int q = 0; q < Wp; ++q) {            // apply in worker order
-                    if (lane / E == q && in) {
-                        if (ix >= lo) tilebuf[ix - lo] = __fadd_rn(tilebuf[ix - lo], v);
-                        else record_status(hdr, -1 /*GC_E_INVALID*/, p);      // unsorted input
+                    if (lane / E == q) {
+#pragma unroll
+                        for (int rd = 0; rd < kDecRounds; ++rd) {
+                            if (ix[rd] < hi) {
+                                if (ix[rd] >= lo) tilebuf[ix[rd] - lo] = __fadd_rn(tilebuf[ix[rd] - lo], v[rd]);
+                                else record_status(hdr, -1 /*GC_E_INVALID*/, cur[ps]);      // unsorted input
+                            }
+                        }
                     }
                     __syncwarp();
                 }
-                const unsigned inb = __ballot_sync(0xFFFFFFFFu, in) & gmask;
-                cur[ps] += (uint32_t)__popc(inb);
+                uint32_t tot = nin;                       // sum over the E lanes of the group
+                for (int o = 1; o < E; o <<= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, o);
+                cur[ps] += tot;
             } else {
                 for (int q = 0; q < Wp; ++q) {
                     const uint32_t wq = (uint32_t)(ps * Wp + q);

@@ -51,7 +51,9 @@ k_topk_single(SingleArgs a) {
     uint32_t* const rec = reinterpret_cast<uint32_t*>(s_dyn);                  // [maxt*kWarps] off<<10 | cnt
     uint32_t* const rec2 = rec + (size_t)a.maxt * kWarps;                      // [maxt*kWarps] gt<<16 | eq
     unsigned long long* const tile_base = reinterpret_cast<unsigned long long*>(rec2 + (size_t)a.maxt * kWarps);
-    uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;              // this CTA's region
+    // This CTA's region.  Only this CTA (hence only this SM) ever writes or reads it, and it is
+    // never read before it is written, so the later phases may read it through L1.
+    uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t G = gridDim.x, b = blockIdx.x;
@@ -242,7 +244,7 @@ k_topk_single(SingleArgs a) {
         good = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 2 * kHistBins, d.k, bin0, above0);
         if (good) {
             for (uint32_t i = tid; i < used; i += kBlock) {
-                const uint32_t key = ld_cg(&pool[i]).y & kKeyMask;
+                const uint32_t key = pool[i].y & kKeyMask;
                 if ((key >> level_shift(0)) == bin0)
                     atomicAdd(&sm.hist[(key >> level_shift(1)) & ((1u << level_bits(1)) - 1u)], 1u);
             }
@@ -254,7 +256,7 @@ k_topk_single(SingleArgs a) {
         const uint32_t p1 = (bin0 << level_bits(1)) | bin1;
         if (good) {
             for (uint32_t i = tid; i < used; i += kBlock) {
-                const uint32_t key = ld_cg(&pool[i]).y & kKeyMask;
+                const uint32_t key = pool[i].y & kKeyMask;
                 if ((key >> level_shift(1)) == p1) atomicAdd(&sm.hist[key & ((1u << level_bits(2)) - 1u)], 1u);
             }
         }
@@ -274,7 +276,7 @@ k_topk_single(SingleArgs a) {
             const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
             uint32_t ngt = 0, neq = 0;
             for (uint32_t j = 0; j < cnt; ++j) {
-                const uint32_t key = ld_cg(&pool[off + j]).y & kKeyMask;
+                const uint32_t key = pool[off + j].y & kKeyMask;
                 ngt += key > Tkey; neq += key == Tkey;
             }
             rec2[c] = (ngt << 16) | neq;
@@ -324,7 +326,7 @@ k_topk_single(SingleArgs a) {
                 gpos += v >> 16; epos += v & 0xFFFFu;
             }
             for (uint32_t j = 0; j < cnt; ++j) {
-                const uint2 pr = ld_cg(&pool[off + j]);
+                const uint2 pr = pool[off + j];
                 const uint32_t key = pr.y & kKeyMask;
                 const bool gt = key > Tkey, eq = key == Tkey;
                 if (gt || (eq && epos < m_eq)) {
@@ -354,7 +356,7 @@ k_topk_single(SingleArgs a) {
     for (uint32_t c = tid; c < n_own * kWarps; c += kBlock) {      // only chunks that were stored
         const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
         for (uint32_t j = 0; j < cnt; ++j) {
-            const uint2 pr = ld_cg(&pool[off + j]);
+            const uint2 pr = pool[off + j];
             a.r[pr.x] = __uint_as_float(pr.y);
         }
     }
