@@ -294,6 +294,8 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
                  "threshold_emit": 12.0 * n + 8.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
+    # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
+    ncu_traffic = {("c3_bert_base_110m_student_t", "compress_fused"): 1326.3e6}.get((w.name, dom))
 
     # CPU baseline: the oracle on a bounded sample of the same workload
     cpu = None
@@ -317,7 +319,8 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
         "ms_per_step_with_kernel_events": ms / args.steps,
         "kernels": breakdown,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                     "frac": achieved / peak, "traffic": ncu_traffic, "peak_source": peak_src,
+                     "traffic_source": "profiles/k_topk_single_c3_bert110m.md" if ncu_traffic else None,
                      "algorithmic_bytes_per_launch": alg_bytes.get(dom)},
         "cpu_baseline": cpu,
         "e2e": None if not e2e_steps else {"value": grad_bytes_step * e2e_steps / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
