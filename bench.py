@@ -151,6 +151,23 @@ def run_reference(args, w: synth.Workload, rank: int):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- ranks
+def reduce_max_over_ranks(values, world: int, device) -> list:
+    """Replicas only: every rank runs the same workload on its own GPU and the job's time is the
+    slowest rank's.  Returns the element-wise maximum over ranks (identity for one rank)."""
+    if world <= 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    t = torch.nan_to_num(t, nan=-1.0)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float("nan") if x < 0 else x for x in t.tolist()]
+
+
+def whole_job_value(n: int, workers: int, world: int, steps: int, ms: float) -> float:
+    """Gradient GB/s of the whole job: bytes of gradient all ranks consumed / slowest rank's time."""
+    return 4.0 * n * workers * world * steps / (ms * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------- GPU arm
 def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     from paper_2104_01981_b200 import api
@@ -270,16 +287,13 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
 
 def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e, e2e_steps,
             per_kernel, launches, clocks, counters):
-    if world > 1:
-        t = torch.tensor([ms, ms_plain, ms_e2e], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms, ms_plain, ms_e2e = t.tolist()
+    ms, ms_plain, ms_e2e = reduce_max_over_ranks([ms, ms_plain, ms_e2e], world, dev)
     if rank != 0:
         return
 
     from paper_2104_01981_b200 import api
     grad_bytes_step = 4.0 * n * W * world
-    value = grad_bytes_step * args.steps / (ms_plain * 1e-3) / 1e9
+    value = whole_job_value(n, W, world, args.steps, ms_plain)
     cb, db = min_bytes(n, k, W)
     t_step = ms_plain * 1e-3 / args.steps
     peak, peak_src = measured_peak_gbs()
