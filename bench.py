@@ -174,7 +174,8 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     api.lib()                                    # no fallback: raises when libgc.so is missing
-    plan = api.Plan(w.sizes, w.density, device=local_rank)
+    mode = api.GC_THRESHOLD if args.mode == "threshold" else api.GC_TOPK
+    plan = api.Plan(w.sizes, w.density, mode=mode, device=local_rank)
     if args.path != "auto":
         plan.set_option(api.GC_OPT_PATH, {"exact": api.GC_PATH_EXACT, "staged": api.GC_PATH_STAGED}[args.path])
     n, k, W = plan.total_n, plan.total_cap, w.workers
@@ -189,10 +190,14 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     ws = plan.alloc_workspace()
     dense = torch.empty(n, dtype=torch.float32, device=dev)
 
+    thr = mode == api.GC_THRESHOLD          # threshold mode: variable counts travel with the pairs
+    cnts = [o[2] for o in outs] if thr else None
+
     def step(i: int):
         for wk in range(W):
-            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], None, ws, stream)
-        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], None, dense, True, ws, stream)
+            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
+                          ws, stream)
+        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], cnts, dense, True, ws, stream)
 
     def barrier():
         if world > 1:
@@ -220,7 +225,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     launches = plan.launches() - launches0
     plan.profile_enable(0)
     st, det = plan.last_status(ws)
-    if st != api.GC_OK:
+    if st not in (api.GC_OK, api.GC_W_TRUNCATED):
         raise RuntimeError(f"device status {st} (detail {det}) after the timed region")
     counters = plan.last_counters(ws)
     args.phase_us = plan.last_phase_times(ws)
@@ -237,10 +242,11 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     # ---- timed regions 1c/1d: the two halves on their own (no per-kernel events)
     def compress_only(i: int):
         for wk in range(W):
-            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], None, ws, stream)
+            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
+                          ws, stream)
 
     def decode_only(i: int):
-        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], None, dense, True, ws, stream)
+        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], cnts, dense, True, ws, stream)
 
     halves = []
     for fn in (compress_only, decode_only):
@@ -305,7 +311,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     dom = max(per_kernel.items(), key=lambda kv: kv[1][0])[0]
     alg_bytes = {"fold_hist": 12.0 * n, "hist_refine": 4.0 * n, "compact": 4.0 * n + 8.0 * k,
                  "decode_clear": 4.0 * n, "decode_add": 8.0 * k, "fold_cand": 12.0 * n, "compress_fused": 12.0 * n + 8.0 * k,
-                 "threshold_emit": 12.0 * n + 8.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
+                 "threshold_emit": 12.0 * n + 4.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
     # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
@@ -323,7 +329,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_plain / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "elements": n, "k": k, "density": w.density, "workers": W,
+        "config": {"workload": w.name, "mode": args.mode, "elements": n, "k": k, "density": w.density, "workers": W,
                    "tensors": len(w.sizes), "input_sets": sets,
                    "l2": "inputs larger than L2 (no flush): each gradient and residual is %d MB" % (4 * n >> 20)},
         "elements_per_s": n * W * world * args.steps / (ms_plain * 1e-3),
@@ -366,6 +372,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "exact"],
                     help="auto: one-pass candidate path in one cooperative launch (default); staged: the "
                          "same phases as separate launches; exact: multi-pass kernels only")
+    ap.add_argument("--mode", default="topk", choices=["topk", "threshold"],
+                    help="selection mode (threshold = the sampled-threshold variant)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end region")
     ap.add_argument("--input-sets", type=int, default=N_INPUT_SETS,
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")

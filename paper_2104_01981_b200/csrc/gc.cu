@@ -35,7 +35,7 @@ struct gc_plan_s {
     size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
            control_bytes = 0, off_tinfo = 0, off_cidx = 0, ws_bytes = 0;
     int sm_count = 0;
-    int grid_thr = 0, grid_decode = 0;
+    int grid_thr = 0, grid_decode[2] = {0, 0};
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
     int grid_fused = 0;                     // CTAs of the cooperative launch (0 = not available)
     // single-tensor shared-memory-pool kernel
@@ -310,7 +310,18 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         plan_single(p);
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
-    p->grid_decode = p->sm_count * blocks_per_sm(k_decode_tiles, kDecBlock);
+    {
+        cudaError_t ed = cudaFuncSetAttribute(k_decode_tiles, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)(2 * kDecTileBytes));
+        for (int nbuf = 1; nbuf <= 2; ++nbuf) {
+            int nb = 0;
+            if (ed == cudaSuccess)
+                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_tiles, kDecBlock,
+                                                                   nbuf * kDecTileBytes);
+            if (ed != cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
+            p->grid_decode[nbuf - 1] = p->sm_count * nb;     // 0: fall back to one launch per worker
+        }
+    }
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
     p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
     p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact<true>, kBlock);
@@ -533,17 +544,19 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return GC_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
-    if (count == nullptr && W > 0 && p->total_cap > 0 && p->path != GC_PATH_EXACT) {
+    const int nbuf = W <= 2 ? 2 : 1;      // few workers per tile: overlap the tile's way out with the next tile
+    if (count == nullptr && W > 0 && p->total_cap > 0 && p->path != GC_PATH_EXACT && p->grid_decode[nbuf - 1] > 0) {
         // every list holds exactly total_cap pairs in ascending index: tiled decode, dense buffer
         // written once (and not read at all when it is cleared first)
         DecodeLists ls;
         for (uint32_t w = 0; w < 64; ++w) { ls.idx[w] = idx[w < W ? w : 0]; ls.val[w] = val[w < W ? w : 0]; }
         const uint32_t ntl = (uint32_t)((p->total_n + kDecTile - 1) / kDecTile);
-        const int grid = (int)std::min<uint32_t>((ntl + kDecWarps - 1) / kDecWarps, (uint32_t)p->grid_decode);
+        const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[nbuf - 1]);
         const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;
         Timed tm(p, s, GC_K_DECODE_TILES);
-        k_decode_tiles<<<grid, kDecBlock, 0, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, dense_out,
-                                                  zero_first ? 1 : 0, use_bulk, ws.hdr);
+        k_decode_tiles<<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap,
+                                                                     (uint32_t)p->total_n, dense_out,
+                                                                     zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr);
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
