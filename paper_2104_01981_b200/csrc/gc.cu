@@ -42,7 +42,7 @@ struct gc_plan_s {
     int grid_single_max = 0;                // resident CTAs (0 = not available)
     uint32_t single_grid = 0, single_maxt = 0, single_pool = 0;   // 0 = plan does not qualify
     size_t single_smem = 0;
-    size_t off_hist5 = 0;
+    size_t off_hist5 = 0, off_rowseg = 0;
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
@@ -54,6 +54,8 @@ struct gc_plan_s {
 namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+constexpr size_t kSingleMaxT = 341;          // most tiles one CTA of k_topk_single may own
 
 inline uint64_t k_rule(uint64_t n, double density) {
     if (n == 0) return 0;
@@ -173,7 +175,9 @@ void finish_layout(gc_plan_s* p) {
     p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * T, 256);
     p->off_gstate = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
     p->off_hist5 = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
-    p->control_bytes = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 5 * (size_t)kHistBins : 0), 256);
+    // single-tensor kernel: five histograms, then row totals and 32-CTA segment totals
+    p->off_rowseg = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 5 * (size_t)kHistBins : 0), 256);
+    p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(unsigned long long) * kSingleMaxT * 21 : 0), 256);
     p->off_tinfo = p->control_bytes;
     p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
     p->ws_bytes = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
@@ -189,14 +193,13 @@ void plan_single(gc_plan_s* p) {
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
     const uint32_t maxt = (d.ntiles + G - 1) / G;
     const size_t rec_bytes = (size_t)maxt * (2 * kWarps * sizeof(uint32_t) + sizeof(unsigned long long));
-    if (rec_bytes > 24576) return;                                   // chunk records must stay small
+    if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, (1u << 22) - 1u);   // region per CTA
     // expected candidates per CTA (sample rank over sample size, times n), with head-room
     const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
     if (nsg > (uint64_t)2 * G * kBlock) return;                     // a thread owns at most two sample groups
     const double expect = (double)d.n * (double)d.srank / (4.0 * (double)nsg) / (double)G;
     if ((double)pool < 1.5 * expect + 512.0) return;
-    if ((uint64_t)maxt > p->ngroups) return;                         // row totals live in the group array
     p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
 }
 
@@ -302,7 +305,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_single_max = 0;
         if (coop) {
             int nb = 0;       // sized for the largest chunk-record block the kernel may be given
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, 24576) ==
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, kSingleMaxT * 72) ==
                     cudaSuccess && nb >= 1)
                 p->grid_single_max = p->sm_count * nb;
         }
@@ -455,7 +458,8 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         sa.g = grad; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;
         sa.hist5 = reinterpret_cast<uint32_t*>(wb + p->off_hist5);
         sa.tile_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_tinfo);
-        sa.row_tot = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
+        sa.row_tot = reinterpret_cast<unsigned long long*>(wb + p->off_rowseg);
+        sa.seg_tot = sa.row_tot + p->single_maxt;
         sa.ws = ws; sa.gws = gws;
         void* args[] = {&sa};
         Timed tm(p, s, GC_K_FUSED);

@@ -31,6 +31,7 @@ struct SingleArgs {
     uint32_t* hist5;                 // [5][kHistBins] sample L0, sample L1, candidates L0, L1, L2 (zeroed)
     unsigned long long* tile_cnt;    // [ntiles] (above-T << 31 | equal-T) per tile
     unsigned long long* row_tot;     // [maxt] the same summed over each row of tiles (zeroed)
+    unsigned long long* seg_tot;     // [maxt][ceil(G/32)] ... and over each run of 32 CTAs of a row (zeroed)
     WsView ws, gws;
 };
 
@@ -291,6 +292,7 @@ k_topk_single(SingleArgs a) {
             }
             a.tile_cnt[b + i * G] = tot;
             atomicAdd(a.row_tot + i, tot);
+            atomicAdd(a.seg_tot + (size_t)i * ((G + 31u) / 32u) + b / 32u, tot);
         }
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
@@ -308,10 +310,14 @@ k_topk_single(SingleArgs a) {
             }
         }
         __syncthreads();
+        // tiles of row i owned by lower CTAs = whole 32-CTA segments below this CTA's segment
+        // + the lower CTAs inside it: at most two loads per lane whatever b is
         for (uint32_t i = warp; i < n_own; i += kWarps) {
+            const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
             unsigned long long part = 0;
-            const unsigned long long* row = a.tile_cnt + (size_t)i * G;
-            for (uint32_t q = lane; q < b; q += 32) part += ld_cg(row + q);
+            if ((uint32_t)lane < myseg) part += ld_cg(a.seg_tot + (size_t)i * nseg + lane);
+            const uint32_t q = myseg * 32u + (uint32_t)lane;
+            if (q < b) part += ld_cg(a.tile_cnt + (size_t)i * G + q);
             part = warp_sum64(part);
             if (lane == 0) tile_base[i] += part;
         }
