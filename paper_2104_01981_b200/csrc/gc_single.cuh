@@ -272,7 +272,9 @@ k_topk_single(SingleArgs a) {
     // `good` is the same in every CTA: it only depends on global histograms read after a barrier
 
     if (good) {
-        // ------------------------------------------------------------ counts per chunk, tile, row
+        // ------------------------------------------------------------ counts per chunk, tile, row, segment
+        // (one thread per chunk here: a chunk holds a handful of candidates and there are
+        // hundreds of chunks per CTA; the warp-per-tile form measured twice as slow)
         for (uint32_t c = tid; c < n_own * kWarps; c += kBlock) {
             const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
             uint32_t ngt = 0, neq = 0;
@@ -310,43 +312,47 @@ k_topk_single(SingleArgs a) {
             }
         }
         __syncthreads();
-        // tiles of row i owned by lower CTAs = whole 32-CTA segments below this CTA's segment
-        // + the lower CTAs inside it: at most two loads per lane whatever b is
+        const unsigned lt_mask = (1u << lane) - 1u;
         for (uint32_t i = warp; i < n_own; i += kWarps) {
+            // tiles of row i owned by lower CTAs = whole 32-CTA segments below this CTA's segment
+            // + the lower CTAs inside it: at most two loads per lane whatever b is
             const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
             unsigned long long part = 0;
             if ((uint32_t)lane < myseg) part += ld_cg(a.seg_tot + (size_t)i * nseg + lane);
             const uint32_t q = myseg * 32u + (uint32_t)lane;
             if (q < b) part += ld_cg(a.tile_cnt + (size_t)i * G + q);
-            part = warp_sum64(part);
-            if (lane == 0) tile_base[i] += part;
-        }
-        __syncthreads();
-        for (uint32_t c = tid; c < n_own * kWarps; c += kBlock) {
-            const uint32_t i = c / kWarps, w = c % kWarps;
-            const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
-            if (cnt == 0u) continue;
-            uint32_t gpos = (uint32_t)(tile_base[i] >> 31), epos = (uint32_t)(tile_base[i] & 0x7FFFFFFFull);
-            for (uint32_t w2 = 0; w2 < w; ++w2) {
-                const uint32_t v = rec2[i * kWarps + w2];
-                gpos += v >> 16; epos += v & 0xFFFFu;
-            }
-            for (uint32_t j = 0; j < cnt; ++j) {
-                const uint2 pr = pool[off + j];
+            const unsigned long long base = tile_base[i] + warp_sum64(part);
+            uint32_t gpos = (uint32_t)(base >> 31), epos = (uint32_t)(base & 0x7FFFFFFFull);
+            const uint32_t rc = lane < kWarps ? rec[i * kWarps + lane] : 0u;
+            const uint32_t cnt = rc & 1023u, off = rc >> 10;
+            const uint32_t incl = warp_incl_scan(cnt, lane);
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            for (uint32_t j0 = 0; j0 < total; j0 += 32) {
+                const uint32_t j = j0 + lane;
+                uint32_t c = 0;
+#pragma unroll
+                for (int l = 0; l < kWarps; ++l) c += (j >= __shfl_sync(0xFFFFFFFFu, incl, l)) ? 1u : 0u;
+                c = min(c, (uint32_t)kWarps - 1u);
+                const uint32_t src = __shfl_sync(0xFFFFFFFFu, off, c) + (j - __shfl_sync(0xFFFFFFFFu, incl - cnt, c));
+                const bool valid = j < total;
+                uint2 pr = make_uint2(0u, 0u);
+                if (valid) pr = pool[src];
                 const uint32_t key = pr.y & kKeyMask;
-                const bool gt = key > Tkey, eq = key == Tkey;
-                if (gt || (eq && epos < m_eq)) {
-                    const uint32_t slot = gpos + min(epos, m_eq);
+                const bool gt = valid && key > Tkey, eq = valid && key == Tkey;
+                const unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
+                const uint32_t mg = gpos + __popc(gb & lt_mask), me = epos + __popc(eb & lt_mask);
+                if (gt || (eq && me < m_eq)) {
+                    const uint32_t slot = mg + min(me, m_eq);
                     if (slot < d.cap) {          // the residual already holds +0 for this entry
                         a.out_idx[d.out_off + slot] = pr.x;
                         a.out_val[d.out_off + slot] = __uint_as_float(pr.y);
                     } else {
                         record_status(hdr, -1 /*GC_E_INVALID*/, pr.x);
                     }
-                } else {
+                } else if (valid) {
                     a.r[pr.x] = __uint_as_float(pr.y);   // candidate that is not sent: value goes back
                 }
-                gpos += gt; epos += eq;
+                gpos += __popc(gb); epos += __popc(eb);
             }
         }
         if (a.out_count != nullptr && b == 0 && tid == 0) { a.out_count[0] = d.k; a.out_count[1] = d.k; }
