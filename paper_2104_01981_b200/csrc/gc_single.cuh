@@ -358,6 +358,7 @@ k_topk_single(SingleArgs a) {
         if (a.out_count != nullptr && b == 0 && tid == 0) { a.out_count[0] = d.k; a.out_count[1] = d.k; }
         __syncthreads();
         phase_stamp(hdr);
+        exit_stamp(hdr);
         return;
     }
 
