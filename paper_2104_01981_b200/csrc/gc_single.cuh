@@ -244,10 +244,17 @@ k_topk_single(SingleArgs a) {
         uint32_t bin0, above0, bin1 = 0, above1 = 0, bin2 = 0, above2 = 0;
         good = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 2 * kHistBins, d.k, bin0, above0);
         if (good) {
-            for (uint32_t i = tid; i < used; i += kBlock) {
-                const uint32_t key = pool[i].y & kKeyMask;
-                if ((key >> level_shift(0)) == bin0)
-                    atomicAdd(&sm.hist[(key >> level_shift(1)) & ((1u << level_bits(1)) - 1u)], 1u);
+            for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {      // four loads in flight per thread
+                uint32_t key[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock;
+                    key[u] = i < used ? (pool[i].y & kKeyMask) : 0xFFFFFFFFu;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if ((key[u] >> level_shift(0)) == bin0)
+                        atomicAdd(&sm.hist[(key[u] >> level_shift(1)) & ((1u << level_bits(1)) - 1u)], 1u);
             }
         }
         flush_hist(sm, a.hist5 + 3 * kHistBins, 1 << level_bits(1));
@@ -256,9 +263,16 @@ k_topk_single(SingleArgs a) {
         if (good) good = block_select<(1 << level_bits(1)), false>(sm, a.hist5 + 3 * kHistBins, d.k - above0, bin1, above1);
         const uint32_t p1 = (bin0 << level_bits(1)) | bin1;
         if (good) {
-            for (uint32_t i = tid; i < used; i += kBlock) {
-                const uint32_t key = pool[i].y & kKeyMask;
-                if ((key >> level_shift(1)) == p1) atomicAdd(&sm.hist[key & ((1u << level_bits(2)) - 1u)], 1u);
+            for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {
+                uint32_t key[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock;
+                    key[u] = i < used ? (pool[i].y & kKeyMask) : 0xFFFFFFFFu;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if ((key[u] >> level_shift(1)) == p1) atomicAdd(&sm.hist[key[u] & ((1u << level_bits(2)) - 1u)], 1u);
             }
         }
         flush_hist(sm, a.hist5 + 4 * kHistBins, 1 << level_bits(2));
