@@ -174,3 +174,37 @@ def quantised_gradient(n: int, seed: int, step: float = 0.125,
     gen.manual_seed(seed)
     g = torch.empty(n, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
     return torch.round(g / step) * step
+
+
+# --------------------------------------------------------------------------- sparse sets
+def _distinct_sorted(rng, n: int, k: int):
+    """k distinct integers of [0, n), ascending (numpy, no permutation of n)."""
+    import numpy as np
+    if k >= n:
+        return np.arange(n, dtype=np.int64)
+    if k > n // 2:
+        drop = _distinct_sorted(rng, n, n - k)
+        keep = np.ones(n, dtype=bool)
+        keep[drop] = False
+        return np.nonzero(keep)[0]
+    got = np.unique(rng.integers(0, n, size=int(k * 1.1) + 16))
+    while got.size < k:
+        got = np.unique(np.concatenate([got, rng.integers(0, n, size=k - got.size + 16)]))
+    if got.size > k:
+        got = np.sort(rng.choice(got, size=k, replace=False))
+    return got
+
+
+def sparse_set(sizes, ks, seed: int, scale: float = 1.0):
+    """A seeded sparse set laid out like a top-k output: for every tensor t, ks[t] distinct flat
+    indices inside the tensor, ascending, with N(0, scale^2) values.  Returns numpy arrays
+    (uint32 indices, float32 values).  Input generator only: nothing here selects anything."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    idx, off = [], 0
+    for n, k in zip(sizes, ks):
+        idx.append(_distinct_sorted(rng, int(n), int(k)) + off)
+        off += int(n)
+    idx = np.concatenate(idx).astype(np.uint32) if idx else np.zeros(0, np.uint32)
+    val = (rng.standard_normal(idx.size) * scale).astype(np.float32)
+    return idx, val

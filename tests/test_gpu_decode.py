@@ -31,62 +31,83 @@ def run_workers(sizes, density, W, seed, steps=1, dist_scale=None):
     return plan, workers, grads
 
 
-def oracle_pairs(workers, plan):
-    tot = plan.total_cap
-    return [(to_np_u32(w.idx[:tot]).copy(), w.val[:tot].cpu().numpy().copy()) for w in workers]
+def synthetic_sets(plan, sizes, W, seed, share_every=0):
+    """W seeded sparse sets shaped like this plan's top-k output, as numpy pairs and as device
+    tensors.  They come from the input generator, never from the CUDA compress path.  With
+    share_every = s, groups of s consecutive workers use the same indices (collisions)."""
+    ks = plan.tensor_k()
+    pairs, d_idx, d_val = [], [], []
+    for w in range(W):
+        iseed = seed + (w // share_every if share_every else w)
+        idx, _ = synth.sparse_set(sizes, ks, iseed)
+        _, val = synth.sparse_set(sizes, ks, 7919 * seed + w, scale=10.0 ** (w % 5 - 2))
+        pairs.append((idx, val))
+        d_idx.append(torch.from_numpy(idx.view(np.int32)).cuda())
+        d_val.append(torch.from_numpy(val).cuda())
+    return pairs, d_idx, d_val
 
 
 @pytest.mark.parametrize("W", [1, 2, 8])
 @pytest.mark.parametrize("sizes,density", [([100_000], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02),
                                            ([40_000], 0.5)])
 def test_decode_matches_oracle_bitwise(W, sizes, density):
-    plan, workers, _ = run_workers(sizes, density, W, seed=3, steps=2,
-                                   dist_scale=[10.0 ** (w % 4 - 2) for w in range(W)])
+    plan = api.Plan(sizes, density, device=0)
+    ws = plan.alloc_workspace()
+    pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=3, share_every=2)
     n = plan.total_n
     out = torch.full((n,), 7.0, device="cuda")
-    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out, True,
-                               workers[0].ws)
-    want = oracle.decode_accumulate(oracle_pairs(workers, plan), np.empty(n, np.float32), True)
+    plan.decompress_accumulate(d_idx, d_val, None, out, True, ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
     assert np.array_equal(to_np_u32(out), bits(want))
-    # with explicit count arrays the result is the same
+    # with explicit count arrays (one launch per worker) the result is the same
+    T = len(sizes)
+    cnt = torch.tensor(plan.tensor_k() * 2, dtype=torch.int32, device="cuda")
     out2 = torch.full((n,), 7.0, device="cuda")
-    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers],
-                               [w.count for w in workers], out2, True, workers[0].ws)
+    plan.decompress_accumulate(d_idx, d_val, [cnt] * W, out2, True, ws)
     assert torch.equal(out, out2)
     # accumulate mode adds on top of the existing content
-    plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out2, False,
-                               workers[0].ws)
-    want2 = oracle.decode_accumulate(oracle_pairs(workers, plan), want.copy(), False)
+    plan.decompress_accumulate(d_idx, d_val, None, out2, False, ws)
+    want2 = oracle.decode_accumulate(pairs, want.copy(), False)
     assert np.array_equal(to_np_u32(out2), bits(want2))
-    st, _ = plan.last_status(workers[0].ws)
+    st, _ = plan.last_status(ws)
     assert st == api.GC_OK
 
 
 @pytest.mark.parametrize("W", [3, 16, 33, 64])
 def test_decode_many_workers_and_unaligned_output(W):
-    """Worker counts that are not powers of two, more than one pass of 32 workers, duplicate
-    indices across workers (same seed for some workers), and a dense buffer that is only
-    4-byte aligned (no bulk copies)."""
+    """Worker counts that are not powers of two, more than 32 workers, duplicate indices across
+    workers, and a dense buffer that is only 4-byte aligned (no bulk copies)."""
     sizes = [70_001, 9, 20_000]
     plan = api.Plan(sizes, 0.03, device=0)
+    ws = plan.alloc_workspace()
     n = plan.total_n
-    workers = [GpuWorker(plan) for _ in range(W)]
-    for w, wk in enumerate(workers):
-        gen = torch.Generator().manual_seed(5 + w // 3)              # groups of 3 workers share indices
-        g = torch.randn(n, generator=gen) * (10.0 ** (w % 5 - 2))
-        wk.step(g.cuda())
-    pairs = oracle_pairs(workers, plan)
+    pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=5, share_every=3)
     for shift in (0, 1):
         backing = torch.full((n + 8,), 3.0, device="cuda")
         out = backing[shift:shift + n]
         for zero_first in (True, False):
             before = out.cpu().numpy().copy()
-            plan.decompress_accumulate([w.idx for w in workers], [w.val for w in workers], None, out,
-                                       zero_first, workers[0].ws)
+            plan.decompress_accumulate(d_idx, d_val, None, out, zero_first, ws)
             want = oracle.decode_accumulate(pairs, before, zero_first)
             assert np.array_equal(to_np_u32(out), bits(want)), (W, shift, zero_first)
         assert backing[shift + n:].eq(3.0).all() and backing[:shift].eq(3.0).all()
-    st, _ = plan.last_status(workers[0].ws)
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_OK
+
+
+def test_config5_sixteen_workers_full_size_decode():
+    """The 355M-element workload: 16 seeded sparse sets of k = 354,824 pairs each, decoded in one
+    call; every element is checked against the oracle."""
+    w = synth.workload(4)
+    plan = api.Plan(w.sizes, w.density, device=0)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    pairs, d_idx, d_val = synthetic_sets(plan, w.sizes, w.workers, seed=11, share_every=4)
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate(d_idx, d_val, None, out, True, ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
+    st, _ = plan.last_status(ws)
     assert st == api.GC_OK
 
 
