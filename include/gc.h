@@ -215,7 +215,7 @@ int gc_compress_host(gc_plan_t *plan, const float *host_grad, float *grad_stagin
  * and frees the events.  gc_profile_read synchronises the device, sums the elapsed time and
  * the launches per kernel id (GC_K_*; arrays of GC_K_COUNT entries) and clears the records.
  */
-#define GC_K_CLEAR_CTRL     0   /* memset of the workspace control block                  */
+#define GC_K_CLEAR_CTRL     0   /* zeroing of the workspace control block (and of out_count) */
 #define GC_K_FOLD_HIST      1   /* fold + level-0 histogram (reads g, r; writes r)        */
 #define GC_K_HIST_REFINE    2   /* level-1 / level-2 histogram over r                      */
 #define GC_K_COMPACT        3   /* ordered compaction + residual zeroing                   */

@@ -42,7 +42,9 @@ struct gc_plan_s {
     int grid_single_max = 0;                // resident CTAs (0 = not available)
     uint32_t single_grid = 0, single_maxt = 0, single_pool = 0;   // 0 = plan does not qualify
     size_t single_smem = 0;
-    size_t off_hist5 = 0, off_rowseg = 0;
+    size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0;
+    uint32_t single_srank_hi = 0, single_srank_mid = 0;
+    uint32_t n_empty = 0;                   // tensors without elements
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
@@ -55,6 +57,11 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+constexpr size_t kSingleMidCap = 8192;       // short list of k_topk_single (candidates in the band bin of the threshold)
+constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tensor
+constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
+constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
+constexpr size_t kSingleRowBytes = (2 * kWarps + 3) * sizeof(uint32_t);   // shared memory per owned tile
 constexpr size_t kSingleMaxT = 341;          // most tiles one CTA of k_topk_single may own
 
 inline uint64_t k_rule(uint64_t n, double density) {
@@ -103,12 +110,12 @@ WsView view(const gc_plan_s* p, void* ws) {
 // 4-element group out of `sstride`; tau_lo is the srank-th largest sampled key, where srank
 // sits six standard deviations of the sampling noise above the expected rank density*m, so a
 // candidate set smaller than k is a < 1e-8 event for well-mixed data (and only costs a redo).
-void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap) {
+void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap, uint64_t target_max) {
     const uint64_t n = d.n;
     d.sstride = 0; d.srank = 0;
     *ccap = n;
     if (n < kSmallMax) { d.kind = kKindSmall; *ccap = 0; return; }   // one CTA does the whole tensor
-    uint64_t target = std::min<uint64_t>(131072, std::max<uint64_t>(n / 128, std::min<uint64_t>(8192, n / 2)));
+    uint64_t target = std::min<uint64_t>(target_max, std::max<uint64_t>(n / 128, std::min<uint64_t>(8192, n / 2)));
     uint64_t stride = std::max<uint64_t>(1, n / target);
     uint64_t groups = (n + 3) / 4;
     uint64_t nsg = (groups + stride - 1) / stride;
@@ -134,7 +141,7 @@ void finish_layout(gc_plan_s* p) {
         d.kind = kKindRegular; d.pad = 0;
         uint64_t ccap = d.n;
         if (p->mode == GC_TOPK) {
-            sample_params(d, p->density, p->rank_permille, &ccap);
+            sample_params(d, p->density, p->rank_permille, &ccap, p->T == 1 ? kSampleMaxSingle : kSampleMax);
         } else {
             // threshold mode: the sample is part of the definition -- one 4-element group out of
             // `stride`, rank k_s = min(m, max(1, ceil(density * m))) over its m elements
@@ -177,10 +184,13 @@ void finish_layout(gc_plan_s* p) {
     p->off_hist5 = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
     // single-tensor kernel: five histograms, then row totals and 32-CTA segment totals
     p->off_rowseg = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 5 * (size_t)kHistBins : 0), 256);
-    p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(unsigned long long) * kSingleMaxT * 21 : 0), 256);
+    p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(uint32_t) * kSingleMaxT * 20 : 0), 256);
+    p->off_fine = p->control_bytes;
+    p->control_bytes = align_up(p->off_fine + (T == 1 ? sizeof(uint32_t) * (size_t)kFineBins : 0), 256);
     p->off_tinfo = p->control_bytes;
     p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
-    p->ws_bytes = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
+    p->off_mid = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
+    p->ws_bytes = align_up(p->off_mid + (T == 1 ? sizeof(uint2) * (size_t)kSingleMidCap : 0), 256);
 }
 
 
@@ -192,14 +202,20 @@ void plan_single(gc_plan_s* p) {
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
     const uint32_t maxt = (d.ntiles + G - 1) / G;
-    const size_t rec_bytes = (size_t)maxt * (2 * kWarps * sizeof(uint32_t) + sizeof(unsigned long long));
     if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
-    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, (1u << 22) - 1u);   // region per CTA
+    // region per CTA; one bit per slot has to fit in shared memory beside the chunk records
+    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
+    const size_t rec_bytes = (size_t)maxt * kSingleRowBytes + sizeof(uint32_t) * ((pool + 31) / 32);
     // expected candidates per CTA (sample rank over sample size, times n), with head-room
     const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
     if (nsg > (uint64_t)2 * G * kBlock) return;                     // a thread owns at most two sample groups
     const double expect = (double)d.n * (double)d.srank / (4.0 * (double)nsg) / (double)G;
     if ((double)pool < 1.5 * expect + 512.0) return;
+    // upper bracket: the sample rank that stays below the expected one by the same margin
+    const double ks = p->density * 4.0 * (double)nsg;
+    const double hi = std::floor(ks - 6.0 * std::sqrt(ks) - 8.0);
+    p->single_srank_hi = hi >= 1.0 ? (uint32_t)hi : 0u;
+    p->single_srank_mid = (uint32_t)std::max(1.0, std::ceil(ks));
     p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
 }
 
@@ -255,6 +271,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     for (uint32_t t = 0; t < n_tensors; ++t) {
         TensorDesc& d = p->desc[t];
         uint64_t n = sizes[t];
+        if (n == 0) ++p->n_empty;
         uint64_t k = k_rule(n, density);
         uint64_t cap = k;
         if (mode == GC_THRESHOLD) {
@@ -305,7 +322,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_single_max = 0;
         if (coop) {
             int nb = 0;       // sized for the largest chunk-record block the kernel may be given
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, kSingleMaxT * 72) ==
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, kSingleMaxT * kSingleRowBytes + kSinglePoolMax / 8) ==
                     cudaSuccess && nb >= 1)
                 p->grid_single_max = p->sm_count * nb;
         }
@@ -395,9 +412,11 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     WsView ws = view(p, workspace);
     {
         Timed tm(p, s, GC_K_CLEAR_CTRL);
-        GC_CUDA(p, cudaMemsetAsync(workspace, 0, p->control_bytes, s));
+        const size_t n16 = p->control_bytes / 16;             // control_bytes is a multiple of 256
+        const int gc = (int)std::min<size_t>((n16 + 4 * kBlock - 1) / (4 * kBlock), (size_t)p->sm_count * 4);
+        k_clear<<<gc, kBlock, 0, s>>>(reinterpret_cast<uint4*>(workspace), n16);
     }
-    if (out_count != nullptr) {
+    if (out_count != nullptr && p->n_empty > 0) {       // every tensor with elements gets its counts written
         Timed tm(p, s, GC_K_CLEAR_CTRL);
         GC_CUDA(p, cudaMemsetAsync(out_count, 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
     }
@@ -457,9 +476,11 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         sa.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
         sa.g = grad; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;
         sa.hist5 = reinterpret_cast<uint32_t*>(wb + p->off_hist5);
-        sa.tile_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_tinfo);
-        sa.row_tot = reinterpret_cast<unsigned long long*>(wb + p->off_rowseg);
-        sa.seg_tot = sa.row_tot + p->single_maxt;
+        sa.srank_hi = p->single_srank_hi; sa.srank_mid = p->single_srank_mid; sa.mid_cap = (uint32_t)kSingleMidCap;
+        sa.mid = reinterpret_cast<uint2*>(wb + p->off_mid);
+        sa.fine = reinterpret_cast<uint32_t*>(wb + p->off_fine);
+        sa.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+        sa.seg_tot = reinterpret_cast<uint32_t*>(wb + p->off_rowseg);
         sa.ws = ws; sa.gws = gws;
         void* args[] = {&sa};
         Timed tm(p, s, GC_K_FUSED);

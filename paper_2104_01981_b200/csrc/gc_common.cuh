@@ -312,7 +312,7 @@ __device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, in
         atomicAdd(&hdr->barrier, 1u);
         uint32_t spins = 0;
         while (ld_cg(&hdr->barrier) < target) {
-            if (++spins > kSpinLimit || ld_cg(&hdr->abort) != 0u) { ok = 0; break; }
+            if (++spins > kSpinLimit || ((spins & 15u) == 0u && ld_cg(&hdr->abort) != 0u)) { ok = 0; break; }
             if (spins > 32) __nanosleep(spins > 4096 ? 400 : 60);
         }
         if (!ok) {

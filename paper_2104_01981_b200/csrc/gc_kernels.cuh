@@ -204,6 +204,12 @@ __device__ bool block_select(BlockSmem& sm, const uint32_t* hist, uint32_t krem,
     return ok;
 }
 
+// Zeroes n16 16-byte words (the control block of a workspace).
+static __global__ void __launch_bounds__(kBlock) k_clear(uint4* __restrict__ p, size_t n16) {
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t i = (size_t)blockIdx.x * kBlock + threadIdx.x; i < n16; i += (size_t)gridDim.x * kBlock) p[i] = z;
+}
+
 // ----------------------------------------------------------------------------- histogram pass
 // One radix-select level over all tensors.  CTAs take contiguous runs of tiles, keep a
 // shared-memory histogram while the tensor stays the same, flush it with global atomics when

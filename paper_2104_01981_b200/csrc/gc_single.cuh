@@ -1,37 +1,69 @@
-// Exact top-k of ONE large tensor in one cooperative launch with the candidates held in
-// shared memory ("global top-k" workloads: the whole model is one flat tensor).
+// Exact top-k of ONE large tensor in one cooperative launch ("global top-k" workloads: the
+// whole model is one flat tensor).
 //
-// Same idea as the general candidate path (sample -> fold + candidates -> radix select on the
+// Same idea as the general candidate path (sample -> fold + candidates -> select on the
 // candidates -> index-ordered emission, exact multi-pass redo as the safety net), specialised:
 //   * CTA b owns tiles b, b + G, b + 2G, ... (G = grid size): every CTA sees every region of
 //     the tensor, so candidate counts stay balanced even when magnitudes differ between layers;
 //   * a CTA appends the candidates of its own tiles to a private, contiguous region of the
-//     candidate list (L2-resident) and keeps the per-chunk records in shared memory, so the
-//     selection phases stream that region linearly with no indirection.  (Holding the
-//     candidates themselves in shared memory was measured slower: the large carve-out leaves
-//     too little L1 for the streaming loads of the fold pass.);
-//   * each histogram level is flushed to global memory, and after the grid barrier EVERY CTA
-//     scans it and derives the same prefix -- no completion counters, no designated CTA;
+//     candidate list (L2-resident) and keeps the per-chunk records in shared memory.  (Holding
+//     the candidates themselves in shared memory was measured slower: the large carve-out
+//     leaves too little L1 for the streaming loads of the fold pass.);
+//   * the sample brackets the threshold from both sides: tau_lo (every element at or above it
+//     becomes a candidate) and tau_hi (elements at or above it are almost surely sent).  The
+//     fold pass histograms the candidates over [tau_lo, tau_hi) in 2047 equal steps, so after
+//     ONE grid barrier every CTA knows the step ("band bin") the k-th largest key lies in;
+//   * the few candidates inside that bin go to a short list which every CTA ranks on its own
+//     (no further barrier): that gives the exact threshold key and the tie cut;
+//   * the fold pass writes +0 into the residual only for candidates at or above tau_z, the
+//     sample's estimate of the threshold itself, and a = g + r for the others; the emission
+//     then has to touch the residual only where that guess was wrong (a sent candidate below
+//     tau_z, an unsent one above it) -- few scattered stores instead of one per unsent candidate;
+//   * counting and emission are passes over the CTA's own candidate list, one candidate per
+//     thread: the chunk a candidate came from follows from its index, and its output slot is
+//     the first slot of that chunk + the sent candidates before it in the chunk (a bit mask in
+//     shared memory);
+//   * every histogram is flushed to global memory and, after the grid barrier, EVERY CTA scans
+//     it and derives the same result -- no completion counters, no designated CTA;
 //   * output slots come from per-row totals: row i is the i-th tile of every CTA.
+// Nothing here is probabilistic in its result: the counts decide, and whenever the bracket
+// misses (or a list overflows) the exact multi-pass kernels redo the tensor.
 #pragma once
 #include "gc_fast.cuh"
 
 namespace gc {
 
+// Fine sample bins per coarse bin, log2.  7 gives tau 18 significant bits; measured on the
+// 110M-element workload the step got faster from 5 to 7 bits (fewer collisions between the
+// sample's global atomics) and no faster beyond.
+constexpr int kFineBits = 7;
+constexpr int kFineShift = 31 - 11 - kFineBits;        // key >> kFineShift = fine bin
+constexpr uint32_t kFineBins = 1u << (11 + kFineBits);
+// Neighbouring fine bins are the hot ones (most samples fall into a few binades), so their
+// counters are spread over distinct cache lines: slot = bin * odd constant mod kFineBins.
+__device__ __forceinline__ uint32_t fine_slot(uint32_t bin) { return (bin * 40503u) & (kFineBins - 1u); }
+constexpr uint32_t kMidRegs = 4;                       // short-list entries a thread keeps in registers
+constexpr uint32_t kMidFast = kMidRegs * kBlock;       // short lists up to this size are read once
+
 struct SingleArgs {
     TensorDesc d;                    // the tensor (by value)
     const TensorDesc* desc;          // device table (for the redo phases)
     uint32_t ntiles, maxt, pool_cap; // tiles, max tiles per CTA, pool slots per CTA
+    uint32_t srank_hi;               // sample rank of the upper bracket (0 = none)
+    uint32_t srank_mid;              // sample rank that estimates the threshold itself
+    uint32_t mid_cap;                // capacity of the short list
     const float* g;
     float* r;
     uint32_t* out_idx;
     float* out_val;
     uint32_t* out_count;
     uint2* cand;                     // [gridDim.x * pool_cap] candidate list, one region per CTA
-    uint32_t* hist5;                 // [5][kHistBins] sample L0, sample L1, candidates L0, L1, L2 (zeroed)
-    unsigned long long* tile_cnt;    // [ntiles] (above-T << 31 | equal-T) per tile
-    unsigned long long* row_tot;     // [maxt] the same summed over each row of tiles (zeroed)
-    unsigned long long* seg_tot;     // [maxt][ceil(G/32)] ... and over each run of 32 CTAs of a row (zeroed)
+    uint2* mid;                      // [mid_cap] candidates inside the band bin of the threshold
+    uint32_t* hist5;                 // [0] coarse sample histogram, [2] band histogram,
+                                     // [3][0] short-list length (all zeroed)
+    uint32_t* fine;                  // [kFineBins] fine sample histogram (zeroed)
+    uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
+    uint32_t* seg_tot;               // [maxt][ceil(G/32)] the same summed over each run of 32 CTAs of a row (zeroed)
     WsView ws, gws;
 };
 
@@ -43,15 +75,107 @@ __device__ __forceinline__ void flush_hist(BlockSmem& sm, uint32_t* hist, int nb
     }
 }
 
+// NR ranks (1 = largest; 0 = not wanted) in one histogram of NB bins that is read once from
+// global memory.  For each: the bin that holds the rank, the count above the bin and the count
+// inside it; ok = the histogram holds at least that many entries.
+struct Picked { uint32_t bin, above, count; bool ok; };
+template <int NB, int NR>
+__device__ void block_select_multi(BlockSmem& sm, const uint32_t* hist, const uint32_t (&k)[NR], Picked (&p)[NR]) {
+    static_assert(NR <= kWarps, "results live in per-warp slots");
+    constexpr int BPT = (NB + kBlock - 1) / kBlock;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t c[BPT], sum = 0;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        const int b = NB - 1 - (tid * BPT + i);
+        c[i] = b >= 0 ? ld_cg(hist + b) : 0u;
+        sum += c[i];
+    }
+    const uint32_t inc = warp_incl_scan(sum, lane);
+    __syncthreads();
+    if (lane == 31) sm.scratch[warp] = inc;
+    if (tid < NR) sm.gt_tot[tid] = 0xFFFFFFFFu;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = lane < kWarps ? sm.scratch[lane] : 0u;
+        const uint32_t wi = warp_incl_scan(v, lane);
+        if (lane < kWarps) sm.scratch[lane] = wi - v;
+        if (lane == kWarps - 1) sm.scratch[kWarps] = wi;
+    }
+    __syncthreads();
+    uint32_t above = sm.scratch[warp] + inc - sum;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        const int b = NB - 1 - (tid * BPT + i);
+        if (b >= 0) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r)
+                if (above < k[r] && k[r] <= above + c[i]) { sm.gt_tot[r] = (uint32_t)b; sm.eq_tot[r] = above; sm.gt_ex[r] = c[i]; }
+        }
+        above += c[i];
+    }
+    __syncthreads();
+    const uint32_t total = sm.scratch[kWarps];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+        p[r].bin = sm.gt_tot[r]; p[r].above = sm.eq_tot[r]; p[r].count = sm.gt_ex[r];
+        p[r].ok = k[r] != 0u && total >= k[r] && p[r].bin != 0xFFFFFFFFu;
+    }
+    __syncthreads();
+}
+
+// Rank `rank` (1 = largest) among the values f(entry) of the short-list entries that f accepts,
+// by radix select over `nbits` bits, 11 at a time from the top, with the histogram in shared
+// memory.  Every CTA runs this on the same list and gets the same answer.  Entries come from
+// registers (e[], the first kMidFast) and from global memory beyond them.  Returns false if
+// fewer than `rank` entries are accepted; `above` = accepted entries with a larger value,
+// `at` = accepted entries with exactly the selected value.  sm.hist must be zero on entry and
+// is zero again on return.
+template <typename F>
+__device__ bool short_list_select(BlockSmem& sm, const uint2 (&e)[kMidRegs], const uint2* mid, uint32_t m,
+                                  int nbits, uint32_t rank, F f, uint32_t& value, uint32_t& above,
+                                  uint32_t& at) {
+    const int tid = threadIdx.x;
+    uint32_t prefix = 0, krem = rank;
+    above = 0; at = 0;
+    bool ok = true;
+    for (int hi = nbits; hi > 0 && ok; hi -= 11) {
+        const int lo = hi > 11 ? hi - 11 : 0, w = hi - lo;          // this level: bits [lo, hi)
+        auto count = [&](const uint2& pr) {
+            uint32_t v;
+            if (!f(pr, v)) return;
+            if (hi < 32 && (v >> hi) != prefix) return;
+            atomicAdd(&sm.hist[(v >> lo) & ((1u << w) - 1u)], 1u);
+        };
+#pragma unroll
+        for (uint32_t u = 0; u < kMidRegs; ++u)
+            if (u * kBlock + tid < m) count(e[u]);
+        for (uint32_t i = kMidFast + tid; i < m; i += kBlock) count(ld_cg(mid + i));
+        __syncthreads();
+        uint32_t bin, ab;
+        ok = block_select<2048, true>(sm, sm.hist, krem, bin, ab);
+        at = ok ? sm.hist[bin] : 0u;
+        __syncthreads();
+        for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
+        __syncthreads();
+        if (ok) { prefix = (prefix << w) | bin; krem -= ab; above += ab; }
+    }
+    value = prefix;
+    return ok;
+}
+
 static __global__ void __launch_bounds__(kBlock, 4)
 k_topk_single(SingleArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used;
     extern __shared__ __align__(16) unsigned char s_dyn[];
-    // dynamic shared memory: chunk records, chunk select counts, tile bases
+    // dynamic shared memory: chunk records, per-chunk counts, output slot of every own tile
     uint32_t* const rec = reinterpret_cast<uint32_t*>(s_dyn);                  // [maxt*kWarps] off<<10 | cnt
-    uint32_t* const rec2 = rec + (size_t)a.maxt * kWarps;                      // [maxt*kWarps] gt<<16 | eq
-    unsigned long long* const tile_base = reinterpret_cast<unsigned long long*>(rec2 + (size_t)a.maxt * kWarps);
+    uint32_t* const rec2 = rec + (size_t)a.maxt * kWarps;                      // [maxt*kWarps] above the band bin
+    uint32_t* const tile_base = rec2 + (size_t)a.maxt * kWarps;                // [maxt]
+    uint32_t* const row_sum = tile_base + a.maxt;                              // [maxt]
+    uint32_t* const row_mid = row_sum + a.maxt;                                // [maxt]
+    uint32_t* const sent_bits = row_mid + a.maxt;                              // [ceil(pool_cap / 32)]
     // This CTA's region.  Only this CTA (hence only this SM) ever writes or reads it, and it is
     // never read before it is written, so the later phases may read it through L1.
     uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
@@ -63,13 +187,18 @@ k_topk_single(SingleArgs a) {
     uint32_t passed = 0;
     const uint32_t n_own = b < a.ntiles ? (a.ntiles - b + G - 1) / G : 0u;
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
+    for (uint32_t i = tid; i < n_own * kWarps; i += kBlock) rec2[i] = 0u;
+    for (uint32_t i = tid; i < n_own; i += kBlock) row_mid[i] = 0u;
+    const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
     if (tid == 0) s_used = 0u;
     phase_stamp(hdr);
 
-    // ---------------------------------------------------------------- sample (two radix levels)
-    // One 4-element group out of d.sstride; a thread keeps the keys of its groups in registers
-    // between the two levels.  tau_lo = the srank-th largest sampled key, cut to 21 bits.
-    uint32_t tau = 0;
+    // ---------------------------------------------------------------- sample
+    // One 4-element group out of d.sstride.  Two histograms of the sampled keys are built in one
+    // pass: a coarse one (top 11 bits, via shared memory) and a fine one (top 16 bits, straight
+    // into global memory; few samples share a fine bin).  tau = the srank-th largest sampled
+    // key cut to 16 bits; tau_hi = upper edge of the 16-bit cell of the srank_hi-th largest.
+    uint32_t tau = 0, tau_hi = 0x80000000u, tau_z = 0;
     {
         const uint32_t ngroups = (d.n + 3u) >> 2;
         const uint32_t nsg = (ngroups + d.sstride - 1) / d.sstride;
@@ -98,31 +227,55 @@ k_topk_single(SingleArgs a) {
         for (int q = 0; q < kMaxOwn; ++q)
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                if ((sok >> (4 * q + e)) & 1u) atomicAdd(&sm.hist[skey[q][e] >> level_shift(0)], 1u);
+                if ((sok >> (4 * q + e)) & 1u) {
+                    atomicAdd(&sm.hist[skey[q][e] >> level_shift(0)], 1u);
+                    atomicAdd(a.fine + fine_slot(skey[q][e] >> kFineShift), 1u);
+                }
         flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
-        uint32_t bin0, above0;
-        const bool ok0 = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 0 * kHistBins, d.srank, bin0, above0);
-        if (ok0) {
+        // both brackets from one read of the coarse histogram, then the kFineBits finer bits of
+        // each from the 2^kFineBits fine bins under its coarse bin (one warp per bracket)
+        const uint32_t want[3] = {d.srank, a.srank_hi, a.srank_mid};
+        Picked pk[3];
+        block_select_multi<(1 << level_bits(0)), 3>(sm, a.hist5 + 0 * kHistBins, want, pk);
+        if (warp < 3) {
+            const Picked& p = pk[warp];
+            uint32_t res = 0xFFFFFFFFu;
+            if (p.ok) {
+                // lane l holds the PER fine bins [top - (l+1) PER, top - l PER) of the coarse bin, highest first
+                constexpr uint32_t PER = 1u << (kFineBits - 5);
+                const uint32_t first = (p.bin << kFineBits) + (1u << kFineBits) - 1u - (uint32_t)lane * PER;
+                uint32_t v[PER], sum = 0;
 #pragma unroll
-            for (int q = 0; q < kMaxOwn; ++q)
+                for (uint32_t j = 0; j < PER; ++j) { v[j] = ld_cg(a.fine + fine_slot(first - j)); sum += v[j]; }
+                const uint32_t inc = warp_incl_scan(sum, lane);
+                const uint32_t krem = want[warp] - p.above;
+                uint32_t mine = 0xFFFFFFFFu, run = inc - sum;
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (((sok >> (4 * q + e)) & 1u) && (skey[q][e] >> level_shift(0)) == bin0)
-                        atomicAdd(&sm.hist[(skey[q][e] >> level_shift(1)) & ((1u << level_bits(1)) - 1u)], 1u);
+                for (uint32_t j = 0; j < PER; ++j) {
+                    if (run < krem && krem <= run + v[j]) mine = first - j;
+                    run += v[j];
+                }
+                const unsigned hit = __ballot_sync(0xFFFFFFFFu, mine != 0xFFFFFFFFu);
+                if (hit != 0u) res = __shfl_sync(0xFFFFFFFFu, mine, __ffs(hit) - 1);
+            }
+            if (lane == 0) sm.gt_tot[warp] = res;
         }
-        flush_hist(sm, a.hist5 + 1 * kHistBins, 1 << level_bits(1));
-        if (!grid_barrier(hdr, passed, &sm.ok)) return;
-        phase_stamp(hdr);
-        if (ok0) {
-            uint32_t bin1, above1;
-            if (block_select<(1 << level_bits(1)), false>(sm, a.hist5 + 1 * kHistBins, d.srank - above0, bin1, above1))
-                tau = ((bin0 << level_bits(1)) | bin1) << level_shift(1);
-        }
+        __syncthreads();
+        if (sm.gt_tot[0] != 0xFFFFFFFFu) tau = sm.gt_tot[0] << kFineShift;
+        if (sm.gt_tot[1] != 0xFFFFFFFFu) tau_hi = (sm.gt_tot[1] + 1u) << kFineShift;
+        if (sm.gt_tot[2] != 0xFFFFFFFFu) tau_z = sm.gt_tot[2] << kFineShift;
+        __syncthreads();
         // tau == 0 (sample too small for the rank): every element becomes a candidate, the pool
         // overflows and the exact redo takes over
     }
+    if (tau_z < tau) tau_z = tau;
+    // Band histogram: bin(key) = min((key - tau) >> shift, 2047), monotonic in the key; bins
+    // 0..2046 cover [tau, tau_hi) and bin 2047 takes everything above.
+    if (tau_hi <= tau) tau_hi = 0x80000000u;
+    int shift = 0;
+    while (((tau_hi - tau) >> shift) > 2046u) ++shift;
 
     // ---------------------------------------------------------------- fold + candidates
     const uint32_t my_off = warp * kWarpChunk + lane * 4;
@@ -161,16 +314,18 @@ k_topk_single(SingleArgs a) {
                 }
             }
         }
-        uint32_t cnt[kVpt], cm = 0;
+        uint32_t cnt[kVpt], cm = 0, hm = 0;      // candidates; candidates that are zeroed right away
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) {
             cnt[j] = 0;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                bool c = key_of(av[j][e]) >= tau;
+                const uint32_t key = key_of(av[j][e]);
+                bool c = key >= tau;
                 if (!interior) c = c && ((valid >> (4 * j + e)) & 1u);
                 cnt[j] += c;
                 cm |= (uint32_t)c << (4 * j + e);
+                hm |= (uint32_t)(key >= tau_z) << (4 * j + e);      // tau_z >= tau > 0: implies c
             }
         }
         uint32_t rk[kVpt], wtot;
@@ -181,7 +336,8 @@ k_topk_single(SingleArgs a) {
         const bool fits = off + wtot <= a.pool_cap;
         if (!fits) block_overflow = true;
         if (lane == 0) rec[i * kWarps + warp] = fits ? ((off << 10) | wtot) : 0u;
-        const uint32_t zm = fits ? cm : 0u;
+        const uint32_t em = fits ? cm : 0u;      // goes to the candidate list
+        const uint32_t zm = fits ? (hm & cm) : 0u;      // ... and leaves +0 in the residual (probably sent)
         if (interior) {
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
@@ -206,16 +362,16 @@ k_topk_single(SingleArgs a) {
         // contiguous run of 8-byte pairs
         const bool staged = wtot <= (uint32_t)kEmitStage;
         if (fits && wtot != 0u) {
-            if (zm != 0u) {
+            if (em != 0u) {
 #pragma unroll
                 for (int j = 0; j < kVpt; ++j) {
                     uint32_t pos = rk[j];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        if ((zm >> (4 * j + e)) & 1u) {
+                        if ((em >> (4 * j + e)) & 1u) {
                             const uint2 pr = make_uint2(tg.base + my_off + j * 128 + e, __float_as_uint(av[j][e]));
                             if (staged) sm.emit[warp][pos] = pr; else pool[off + pos] = pr;
-                            atomicAdd(&sm.hist[key_of(av[j][e]) >> level_shift(0)], 1u);
+                            atomicAdd(&sm.hist[min((key_of(av[j][e]) - tau) >> shift, 2047u)], 1u);
                             ++pos;
                         }
                     }
@@ -233,147 +389,234 @@ k_topk_single(SingleArgs a) {
     }
     if (tid == 0) atomicAdd(&hdr->cand_total, min(s_used, a.pool_cap));
     const uint32_t used = s_used;      // read linearly only when no chunk anywhere overflowed
-    flush_hist(sm, a.hist5 + 2 * kHistBins, 1 << level_bits(0));
+    flush_hist(sm, a.hist5 + 2 * kHistBins, 2048);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     phase_stamp(hdr);
 
-    bool good = ld_cg(&hdr->overflow) == 0u;
-    uint32_t Tkey = 0, m_eq = 0;
-    if (good) {
-        // ------------------------------------------------------------ radix select on the candidates
-        uint32_t bin0, above0, bin1 = 0, above1 = 0, bin2 = 0, above2 = 0;
-        good = block_select<(1 << level_bits(0)), false>(sm, a.hist5 + 2 * kHistBins, d.k, bin0, above0);
-        if (good) {
-            for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {      // four loads in flight per thread
-                uint32_t key[4];
+    // ---------------------------------------------------------------- band bin of the threshold
+    // `good` is the same in every CTA: it only depends on global data read after a barrier
+    // the first candidates of the count pass are fetched while the histogram is being read
+    constexpr uint32_t kPre = 8;
+    uint2 pre[kPre];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t i = i0 + u * kBlock;
-                    key[u] = i < used ? (pool[i].y & kKeyMask) : 0xFFFFFFFFu;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if ((key[u] >> level_shift(0)) == bin0)
-                        atomicAdd(&sm.hist[(key[u] >> level_shift(1)) & ((1u << level_bits(1)) - 1u)], 1u);
-            }
-        }
-        flush_hist(sm, a.hist5 + 3 * kHistBins, 1 << level_bits(1));
-        if (!grid_barrier(hdr, passed, &sm.ok)) return;
-        phase_stamp(hdr);
-        if (good) good = block_select<(1 << level_bits(1)), false>(sm, a.hist5 + 3 * kHistBins, d.k - above0, bin1, above1);
-        const uint32_t p1 = (bin0 << level_bits(1)) | bin1;
-        if (good) {
-            for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {
-                uint32_t key[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t i = i0 + u * kBlock;
-                    key[u] = i < used ? (pool[i].y & kKeyMask) : 0xFFFFFFFFu;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if ((key[u] >> level_shift(1)) == p1) atomicAdd(&sm.hist[key[u] & ((1u << level_bits(2)) - 1u)], 1u);
-            }
-        }
-        flush_hist(sm, a.hist5 + 4 * kHistBins, 1 << level_bits(2));
-        if (!grid_barrier(hdr, passed, &sm.ok)) return;
-        phase_stamp(hdr);
-        if (good)
-            good = block_select<(1 << level_bits(2)), false>(sm, a.hist5 + 4 * kHistBins, d.k - above0 - above1, bin2, above2);
-        Tkey = (p1 << level_bits(2)) | bin2;
-        m_eq = d.k - above0 - above1 - above2;
-    }
-    // `good` is the same in every CTA: it only depends on global histograms read after a barrier
+    for (uint32_t u = 0; u < kPre; ++u) pre[u] = u * kBlock + tid < used ? pool[u * kBlock + tid] : make_uint2(0u, 0u);
+    const uint32_t overflowed = ld_cg(&hdr->overflow);
+    const uint32_t want_k[1] = {d.k};
+    Picked pa[1];
+    block_select_multi<2048, 1>(sm, a.hist5 + 2 * kHistBins, want_k, pa);
+    const uint32_t A = pa[0].bin, aboveA = pa[0].above, m = pa[0].count;      // m = candidates inside the band bin
+    bool good = overflowed == 0u && pa[0].ok && m <= a.mid_cap;
 
     if (good) {
-        // ------------------------------------------------------------ counts per chunk, tile, row, segment
-        // (one thread per chunk here: a chunk holds a handful of candidates and there are
-        // hundreds of chunks per CTA; the warp-per-tile form measured twice as slow)
-        for (uint32_t c = tid; c < n_own * kWarps; c += kBlock) {
-            const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
-            uint32_t ngt = 0, neq = 0;
-            for (uint32_t j = 0; j < cnt; ++j) {
-                const uint32_t key = pool[off + j].y & kKeyMask;
-                ngt += key > Tkey; neq += key == Tkey;
+        // ------------------------------------------------------------ counts above the band bin
+        // One linear pass over the CTA's candidates: those above the bin are counted per chunk
+        // (the chunk follows from the index), those inside it go to the short list.
+        const uint32_t base0 = d.off & ~3u;
+        auto classify = [&](const uint2& pr) {
+            const uint32_t bin = min(((pr.y & kKeyMask) - tau) >> shift, 2047u);
+            if (bin > A) {
+                const uint32_t rel = pr.x - base0;
+                atomicAdd(&rec2[((rel >> 12) / G) * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
+            } else if (bin == A) {
+                const uint32_t slot = atomicAdd(a.hist5 + 3 * kHistBins, 1u);
+                if (slot < a.mid_cap) a.mid[slot] = pr;
             }
-            rec2[c] = (ngt << 16) | neq;
+        };
+#pragma unroll
+        for (uint32_t u = 0; u < kPre; ++u)
+            if (u * kBlock + tid < used) classify(pre[u]);
+        for (uint32_t i0 = kPre * kBlock + tid; i0 < used; i0 += 4 * kBlock) {      // four loads in flight per thread
+            uint2 pr[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * kBlock;
+                pr[u] = i < used ? pool[i] : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * kBlock < used) classify(pr[u]);
         }
         __syncthreads();
         for (uint32_t i = tid; i < n_own; i += kBlock) {
-            unsigned long long tot = 0;
+            uint32_t tot = 0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) {
-                const uint32_t v = rec2[i * kWarps + w];
-                tot += ((unsigned long long)(v >> 16) << 31) | (unsigned long long)(v & 0xFFFFu);
-            }
+            for (int w = 0; w < kWarps; ++w) tot += rec2[i * kWarps + w];
             a.tile_cnt[b + i * G] = tot;
-            atomicAdd(a.row_tot + i, tot);
-            atomicAdd(a.seg_tot + (size_t)i * ((G + 31u) / 32u) + b / 32u, tot);
+            atomicAdd(a.seg_tot + (size_t)i * nseg + myseg, tot);
         }
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr);
 
-        // ------------------------------------------------------------ slot of every own tile, emission
-        // tile_base[i] = sum of the rows before row i + the tiles of row i owned by lower CTAs
-        if (warp == 0) {
-            unsigned long long run = 0;
-            for (uint32_t i0 = 0; i0 < n_own; i0 += 32) {
-                const uint32_t i = i0 + lane;
-                const unsigned long long v = i < n_own ? ld_cg(a.row_tot + i) : 0ull;
-                const unsigned long long inc = warp_incl_scan64(v, lane);
-                if (i < n_own) tile_base[i] = run + inc - v;
-                run += __shfl_sync(0xFFFFFFFFu, inc, 31);
-            }
-        }
-        __syncthreads();
-        const unsigned lt_mask = (1u << lane) - 1u;
-        for (uint32_t i = warp; i < n_own; i += kWarps) {
-            // tiles of row i owned by lower CTAs = whole 32-CTA segments below this CTA's segment
-            // + the lower CTAs inside it: at most two loads per lane whatever b is
-            const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
-            unsigned long long part = 0;
-            if ((uint32_t)lane < myseg) part += ld_cg(a.seg_tot + (size_t)i * nseg + lane);
-            const uint32_t q = myseg * 32u + (uint32_t)lane;
-            if (q < b) part += ld_cg(a.tile_cnt + (size_t)i * G + q);
-            const unsigned long long base = tile_base[i] + warp_sum64(part);
-            uint32_t gpos = (uint32_t)(base >> 31), epos = (uint32_t)(base & 0x7FFFFFFFull);
-            const uint32_t rc = lane < kWarps ? rec[i * kWarps + lane] : 0u;
-            const uint32_t cnt = rc & 1023u, off = rc >> 10;
-            const uint32_t incl = warp_incl_scan(cnt, lane);
-            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            for (uint32_t j0 = 0; j0 < total; j0 += 32) {
-                const uint32_t j = j0 + lane;
-                uint32_t c = 0;
+        // ------------------------------------------------------------ exact threshold from the short list
+        // Every CTA ranks the same m entries: Tkey = the (k - aboveA)-th largest key among them.
+        // If more entries equal Tkey than are still wanted, the lowest indices win: idx_cut is
+        // the largest index that is still sent.
+        uint2 e[kMidRegs];
 #pragma unroll
-                for (int l = 0; l < kWarps; ++l) c += (j >= __shfl_sync(0xFFFFFFFFu, incl, l)) ? 1u : 0u;
-                c = min(c, (uint32_t)kWarps - 1u);
-                const uint32_t src = __shfl_sync(0xFFFFFFFFu, off, c) + (j - __shfl_sync(0xFFFFFFFFu, incl - cnt, c));
-                const bool valid = j < total;
-                uint2 pr = make_uint2(0u, 0u);
-                if (valid) pr = pool[src];
-                const uint32_t key = pr.y & kKeyMask;
-                const bool gt = valid && key > Tkey, eq = valid && key == Tkey;
-                const unsigned gb = __ballot_sync(0xFFFFFFFFu, gt), eb = __ballot_sync(0xFFFFFFFFu, eq);
-                const uint32_t mg = gpos + __popc(gb & lt_mask), me = epos + __popc(eb & lt_mask);
-                if (gt || (eq && me < m_eq)) {
-                    const uint32_t slot = mg + min(me, m_eq);
-                    if (slot < d.cap) {          // the residual already holds +0 for this entry
-                        a.out_idx[d.out_off + slot] = pr.x;
-                        a.out_val[d.out_off + slot] = __uint_as_float(pr.y);
-                    } else {
-                        record_status(hdr, -1 /*GC_E_INVALID*/, pr.x);
-                    }
-                } else if (valid) {
-                    a.r[pr.x] = __uint_as_float(pr.y);   // candidate that is not sent: value goes back
-                }
-                gpos += __popc(gb); epos += __popc(eb);
+        for (uint32_t u = 0; u < kMidRegs; ++u)
+            e[u] = u * kBlock + tid < m ? ld_cg(a.mid + u * kBlock + tid) : make_uint2(0u, 0u);
+        // while those loads fly: per row, the candidates above the bin in the whole row and in
+        // the tiles of lower CTAs (whole 32-CTA segments below this CTA's + the lower CTAs of
+        // its own segment): two loads per lane and row, two rows per step
+        for (uint32_t i0 = warp * 2u; i0 < n_own; i0 += kWarps * 2u) {
+            uint32_t sv[2], tv[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t i = i0 + u, q = myseg * 32u + (uint32_t)lane;
+                sv[u] = (i < n_own && (uint32_t)lane < nseg) ? ld_cg(a.seg_tot + (size_t)i * nseg + lane) : 0u;
+                tv[u] = (i < n_own && q < b) ? ld_cg(a.tile_cnt + (size_t)i * G + q) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t row = __reduce_add_sync(0xFFFFFFFFu, sv[u]);
+                const uint32_t low = __reduce_add_sync(0xFFFFFFFFu, tv[u] + ((uint32_t)lane < myseg ? sv[u] : 0u));
+                if (lane == 0 && i0 + u < n_own) { row_sum[i0 + u] = row; tile_base[i0 + u] = low; }
             }
         }
-        if (a.out_count != nullptr && b == 0 && tid == 0) { a.out_count[0] = d.k; a.out_count[1] = d.k; }
-        __syncthreads();
-        phase_stamp(hdr);
-        exit_stamp(hdr);
-        return;
+        const uint32_t binlo = tau + (A << shift);
+        uint32_t v_sel, mid_gt, n_eq, idx_cut = 0xFFFFFFFFu;
+        good = short_list_select(sm, e, a.mid, m, A == 2047u ? 31 : max(shift, 1), d.k - aboveA,
+                                 [&](const uint2& pr, uint32_t& v) { v = (pr.y & kKeyMask) - binlo; return true; },
+                                 v_sel, mid_gt, n_eq);
+        const uint32_t Tkey = binlo + v_sel;
+        const uint32_t m_eq = d.k - aboveA - mid_gt;      // entries equal to Tkey that are sent
+        if (good && n_eq > m_eq && n_eq <= (uint32_t)kBlock) {
+            // a few entries tie at the threshold: list their indices, rank them directly
+            auto note = [&](const uint2& pr) {
+                if ((pr.y & kKeyMask) == Tkey) sm.hist[atomicAdd(&sm.hist[2047], 1u)] = pr.x;
+            };
+#pragma unroll
+            for (uint32_t u = 0; u < kMidRegs; ++u)
+                if (u * kBlock + tid < m) note(e[u]);
+            for (uint32_t i = kMidFast + tid; i < m; i += kBlock) note(ld_cg(a.mid + i));
+            __syncthreads();
+            if ((uint32_t)tid < n_eq) {
+                const uint32_t mine = sm.hist[tid];
+                uint32_t lower = 0;
+                for (uint32_t j = 0; j < n_eq; ++j) lower += sm.hist[j] < mine;
+                if (lower == m_eq - 1u) sm.scratch[0] = mine;
+            }
+            __syncthreads();
+            idx_cut = sm.scratch[0];
+            __syncthreads();
+            if ((uint32_t)tid < n_eq) sm.hist[tid] = 0u;
+            if (tid == 0) sm.hist[2047] = 0u;
+            __syncthreads();
+        } else if (good && n_eq > m_eq) {
+            uint32_t v_idx, x0, x1;
+            good = short_list_select(sm, e, a.mid, m, 32, m_eq,
+                                     [&](const uint2& pr, uint32_t& v) { v = ~pr.x; return (pr.y & kKeyMask) == Tkey; },
+                                     v_idx, x0, x1);
+            idx_cut = ~v_idx;
+        }
+        // (a failure here would mean the short list changed under us; all CTAs see the same)
+        if (good) {
+            // -------------------------------------------------------- output slots
+            // A sent short-list entry in tile t raises the slot of every own tile after t, i.e.
+            // of the rows from t / G on (one later unless t belongs to a lower CTA); in an own
+            // tile it also raises the count of its chunk.
+            auto sent_key = [&](const uint2& pr) {
+                const uint32_t key = pr.y & kKeyMask;
+                return key > Tkey || (key == Tkey && pr.x <= idx_cut);
+            };
+            auto below = [&](const uint2& pr) {
+                if (!sent_key(pr)) return;
+                const uint32_t rel = pr.x - base0, t = rel >> 12, row = t / G, owner = t - row * G;
+                const uint32_t first = row + (owner < b ? 0u : 1u);
+                if (first < n_own) atomicAdd(&row_mid[first], 1u);
+                if (owner == b) atomicAdd(&rec2[row * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
+            };
+#pragma unroll
+            for (uint32_t u = 0; u < kMidRegs; ++u)
+                if (u * kBlock + tid < m) below(e[u]);
+            for (uint32_t i = kMidFast + tid; i < m; i += kBlock) below(ld_cg(a.mid + i));
+            __syncthreads();
+            if (warp == 0) {
+                // tile_base[i] = rows before i + lower CTAs of row i + sent short-list entries before the tile
+                uint32_t run = 0;
+                for (uint32_t i0 = 0; i0 < n_own; i0 += 32) {
+                    const uint32_t i = i0 + lane;
+                    const uint32_t v = i < n_own ? row_sum[i] : 0u;
+                    const uint32_t w = i < n_own ? row_mid[i] : 0u;
+                    const uint32_t inc = warp_incl_scan(v + w, lane);
+                    if (i < n_own) tile_base[i] += run + inc - v;
+                    run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+                }
+            }
+            __syncthreads();
+            // rec2[c] = output slot of the first sent candidate of chunk c
+            for (uint32_t i = tid; i < n_own; i += kBlock) {
+                uint32_t pos = tile_base[i];
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) {
+                    const uint32_t c = rec2[i * kWarps + w];
+                    rec2[i * kWarps + w] = pos;
+                    pos += c;
+                }
+            }
+            phase_stamp(hdr);      // threshold and output slots known
+            // sent flags of the CTA's candidates in list order, one bit each
+            const uint32_t nwords = (used + 31u) >> 5;
+            for (uint32_t i0 = 0; i0 < nwords * 32u; i0 += 4 * kBlock) {
+                uint2 pr[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock + tid;
+                    pr[u] = i < used ? pool[i] : make_uint2(0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock + tid;
+                    if (i0 + u * kBlock + (tid & ~31) >= nwords * 32u) continue;          // whole warp past the end
+                    const unsigned sb = __ballot_sync(0xFFFFFFFFu, i < used && sent_key(pr[u]));
+                    if (lane == 0) sent_bits[i >> 5] = sb;
+                }
+            }
+            __syncthreads();
+            // emission: slot = first slot of the chunk + sent candidates before this one in the chunk
+            for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {
+                uint2 pr[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock;
+                    pr[u] = i < used ? pool[i] : make_uint2(0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t i = i0 + u * kBlock;
+                    if (i >= used) continue;
+                    // the fold pass left +0 in the residual iff the key reached tau_z
+                    const bool zeroed = (pr[u].y & kKeyMask) >= tau_z;
+                    if (!sent_key(pr[u])) {
+                        if (zeroed) a.r[pr[u].x] = __uint_as_float(pr[u].y);     // value goes back
+                        continue;
+                    }
+                    if (!zeroed) a.r[pr[u].x] = 0.0f;
+                    const uint32_t rel = pr[u].x - base0;
+                    const uint32_t c = ((rel >> 12) / G) * kWarps + ((rel >> 9) & (kWarps - 1u));
+                    const uint32_t s = rec[c] >> 10;                   // first list position of the chunk
+                    uint32_t before;
+                    if ((s >> 5) == (i >> 5)) {
+                        before = __popc((sent_bits[i >> 5] & ((1u << (i & 31u)) - 1u)) >> (s & 31u));
+                    } else {
+                        before = __popc(sent_bits[s >> 5] >> (s & 31u)) + __popc(sent_bits[i >> 5] & ((1u << (i & 31u)) - 1u));
+                        for (uint32_t w = (s >> 5) + 1u; w < (i >> 5); ++w) before += __popc(sent_bits[w]);
+                    }
+                    const uint32_t slot = rec2[c] + before;
+                    if (slot < d.cap) {
+                        a.out_idx[d.out_off + slot] = pr[u].x;
+                        a.out_val[d.out_off + slot] = __uint_as_float(pr[u].y);
+                    } else {
+                        record_status(hdr, -1 /*GC_E_INVALID*/, pr[u].x);
+                    }
+                }
+            }
+            if (a.out_count != nullptr && b == 0 && tid == 0) { a.out_count[0] = d.k; a.out_count[1] = d.k; }
+            __syncthreads();
+            phase_stamp(hdr);
+            exit_stamp(hdr);
+            return;
+        }
     }
 
     // ---------------------------------------------------------------- safety net (rare)

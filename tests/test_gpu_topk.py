@@ -45,6 +45,20 @@ def test_tie_stress_quantised_values():
         check_topk_against_oracle([100_000, 100_000, 100_000], density, grads)
 
 
+@pytest.mark.parametrize("step,expect_no_redo", [(2.0 ** -12, True), (2.0 ** -8, True), (2.0 ** -6, True),
+                                                   (2.0 ** -4, False)])
+def test_one_tensor_ties_at_the_threshold(step, expect_no_redo):
+    """One large tensor whose values sit on a grid: from a dozen to thousands of elements share the
+    threshold magnitude, so the tie cut (lowest indices win) decides; up to a few thousand ties the
+    one-tensor kernel has to settle it without the exact redo."""
+    n = 2_000_000
+    grads = [synth.quantised_gradient(n, 70 + s, step=step) for s in range(2)]
+    seen = []
+    check_topk_against_oracle([n], 0.01, grads, expect_counters=seen.append)
+    if expect_no_redo:
+        assert all(c[1] == 0 and c[2] == 0 for c in seen), seen
+
+
 def test_degenerate_values():
     n = 20_000
     for g in (torch.zeros(n), torch.full((n,), -2.5), torch.cat([torch.ones(n // 2), -torch.ones(n // 2)])):
