@@ -10,7 +10,7 @@ namespace gc {
 constexpr int kBlock = 256;                 // threads per CTA for the streaming kernels
 constexpr int kWarps = kBlock / 32;
 constexpr int kVpt = 4;                     // 128-bit vectors per thread per tile
-constexpr int kTile = kBlock * kVpt * 4;    // 8192 elements per tile
+constexpr int kTile = kBlock * kVpt * 4;    // 4096 elements per tile
 constexpr int kWarpChunk = 32 * kVpt * 4;   // contiguous elements owned by one warp
 constexpr int kSampleTile = kBlock;         // sample groups (of 4 elements) per sample tile: one per thread
 constexpr uint32_t kKeyMask = 0x7FFFFFFFu;
@@ -49,7 +49,8 @@ struct TensorDesc {          // one per tensor, immutable, plan-owned device mem
     uint32_t pad;
 };
 constexpr uint32_t kKindRegular = 0u, kKindSmall = 1u;
-constexpr uint32_t kSmallMax = 16384;        // tensors below this many elements are "small"
+constexpr uint32_t kSmallMax = kTile - 3;     // tensors below this many elements are "small": whatever
+                                              // their offset, they lie inside one tile
 static_assert(sizeof(TensorDesc) == 64, "tensor table entry is 64 bytes");
 
 struct TensorSel {           // one per tensor, in the workspace, rewritten every call

@@ -55,15 +55,19 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
 }
 
 // ----------------------------------------------------------------------------- small tensors
-// Exact top-k of one small tensor (fewer than kSmallMax elements) by ONE CTA, start to finish:
-// fold + level-0 histogram, two refinement passes and the ordered emission all stay inside the
-// CTA (shared-memory histograms, __syncthreads only), so hundreds of tiny tensors cost no global
-// atomics, no completion counters and no grid barriers.
+// Exact top-k of one small tensor (fewer than kSmallMax elements: it fits one tile) by ONE CTA,
+// start to finish: the tile is read once and stays in registers through the three histogram
+// levels (shared memory, __syncthreads only) and the ordered emission, so hundreds of tiny
+// tensors cost one memory round trip each, no global atomics, no completion counters and no
+// grid barriers.
 static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const TensorDesc& d, uint32_t t, uint32_t T,
                                          const float* __restrict__ g, float* __restrict__ r,
                                          uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
                                          uint32_t* __restrict__ out_count) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const TileGeom tg = tile_geom(d, 0u);
+    Tile tl;
+    load_tile<true>(g, r, tg, warp, lane, tl);           // r = a = g + r; sent entries get +0 below
     uint32_t prefix = 0, krem = d.k;
 #pragma unroll 1
     for (int level = 0; level < kLevels; ++level) {
@@ -71,19 +75,14 @@ static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const Tenso
         __syncthreads();
         for (int b = tid; b < (1 << level_bits(0)); b += kBlock) sm.hist[b] = 0u;
         __syncthreads();
-        for (uint32_t ti = 0; ti < d.ntiles; ++ti) {
-            const TileGeom tg = tile_geom(d, ti);
-            Tile tl;
-            if (level == 0) load_tile<true>(g, r, tg, warp, lane, tl); else load_tile<false>(nullptr, r, tg, warp, lane, tl);
 #pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
+        for (int j = 0; j < kVpt; ++j) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t key = key_of(tl.a[j][e]);
-                    bool in = (tl.valid >> (4 * j + e)) & 1u;
-                    if (level > 0) in = in && ((key >> (sh + bits)) == prefix);
-                    if (in) atomicAdd(&sm.hist[(key >> sh) & ((1u << bits) - 1u)], 1u);
-                }
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t key = key_of(tl.a[j][e]);
+                bool in = (tl.valid >> (4 * j + e)) & 1u;
+                if (level > 0) in = in && ((key >> (sh + bits)) == prefix);
+                if (in) atomicAdd(&sm.hist[(key >> sh) & ((1u << bits) - 1u)], 1u);
             }
         }
         __syncthreads();
@@ -94,61 +93,54 @@ static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const Tenso
         krem -= above;
     }
     const uint32_t Tkey = prefix, m_eq = krem;
-    // ordered emission, tile after tile, with running counts
-    uint32_t gt_run = 0, eq_run = 0;
-    for (uint32_t ti = 0; ti < d.ntiles; ++ti) {
-        const TileGeom tg = tile_geom(d, ti);
-        Tile tl;
-        load_tile<false>(nullptr, r, tg, warp, lane, tl);
-        uint32_t cg[kVpt], ce[kVpt], gtm = 0, eqm = 0;
+    // ordered emission
+    uint32_t cg[kVpt], ce[kVpt], gtm = 0, eqm = 0;
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) {
+        cg[j] = 0; ce[j] = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t key = key_of(tl.a[j][e]);
+            const bool v = (tl.valid >> (4 * j + e)) & 1u;
+            const bool gt = v && key > Tkey, eq = v && key == Tkey;
+            cg[j] += gt; ce[j] += eq;
+            gtm |= (uint32_t)gt << (4 * j + e);
+            eqm |= (uint32_t)eq << (4 * j + e);
+        }
+    }
+    uint32_t rg[kVpt], re[kVpt], wg, we;
+    warp_rank(cg, lane, rg, wg);
+    warp_rank(ce, lane, re, we);
+    __syncthreads();
+    if (lane == 0) { sm.gt_tot[warp] = wg; sm.eq_tot[warp] = we; }
+    __syncthreads();
+    scan_warp_totals(sm.gt_tot, sm.gt_ex, &sm.gt_sum, warp, lane);
+    if (warp == 1) {
+        uint32_t v = lane < kWarps ? sm.eq_tot[lane] : 0u;
+        uint32_t inc = warp_incl_scan(v, lane);
+        if (lane < kWarps) sm.eq_ex[lane] = inc - v;
+        if (lane == 31) sm.eq_sum = inc;
+    }
+    __syncthreads();
+    if ((gtm | eqm) != 0u) {
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) {
-            cg[j] = 0; ce[j] = 0;
+            uint32_t gpos = sm.gt_ex[warp] + rg[j], epos = sm.eq_ex[warp] + re[j];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const uint32_t key = key_of(tl.a[j][e]);
-                const bool v = (tl.valid >> (4 * j + e)) & 1u;
-                const bool gt = v && key > Tkey, eq = v && key == Tkey;
-                cg[j] += gt; ce[j] += eq;
-                gtm |= (uint32_t)gt << (4 * j + e);
-                eqm |= (uint32_t)eq << (4 * j + e);
-            }
-        }
-        uint32_t rg[kVpt], re[kVpt], wg, we;
-        warp_rank(cg, lane, rg, wg);
-        warp_rank(ce, lane, re, we);
-        __syncthreads();
-        if (lane == 0) { sm.gt_tot[warp] = wg; sm.eq_tot[warp] = we; }
-        __syncthreads();
-        scan_warp_totals(sm.gt_tot, sm.gt_ex, &sm.gt_sum, warp, lane);
-        if (warp == 1) {
-            uint32_t v = lane < kWarps ? sm.eq_tot[lane] : 0u;
-            uint32_t inc = warp_incl_scan(v, lane);
-            if (lane < kWarps) sm.eq_ex[lane] = inc - v;
-            if (lane == 31) sm.eq_sum = inc;
-        }
-        __syncthreads();
-        if ((gtm | eqm) != 0u) {
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                uint32_t gpos = gt_run + sm.gt_ex[warp] + rg[j], epos = eq_run + sm.eq_ex[warp] + re[j];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const bool gt = (gtm >> (4 * j + e)) & 1u, eq = (eqm >> (4 * j + e)) & 1u;
-                    if (gt || (eq && epos < m_eq)) {
-                        const uint32_t slot = gpos + min(epos, m_eq);
-                        const uint32_t f = vec_index(tg.base, warp, lane, j) + e;
-                        if (slot < d.cap) {
-                            out_idx[d.out_off + slot] = f;
-                            out_val[d.out_off + slot] = tl.a[j][e];
-                            r[f] = 0.0f;
-                        }
+                const bool gt = (gtm >> (4 * j + e)) & 1u, eq = (eqm >> (4 * j + e)) & 1u;
+                if (gt || (eq && epos < m_eq)) {
+                    const uint32_t slot = gpos + min(epos, m_eq);
+                    const uint32_t f = vec_index(tg.base, warp, lane, j) + e;
+                    if (slot < d.cap) {
+                        out_idx[d.out_off + slot] = f;
+                        out_val[d.out_off + slot] = tl.a[j][e];
+                        r[f] = 0.0f;
                     }
-                    gpos += gt; epos += eq;
                 }
+                gpos += gt; epos += eq;
             }
         }
-        gt_run += sm.gt_sum; eq_run += sm.eq_sum;
     }
     if (out_count != nullptr && tid == 0) { out_count[t] = d.k; out_count[T + t] = d.k; }
     __syncthreads();
