@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "gc_single.cuh"
+#include "gc_multi.cuh"
 #include "gc_threshold.cuh"
 #include "gc_decode.cuh"
 
@@ -44,6 +45,10 @@ struct gc_plan_s {
     size_t single_smem = 0;
     size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0;
     uint32_t single_srank_hi = 0, single_srank_mid = 0;
+    int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
+    uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0;       // 0 = plan does not qualify
+    size_t multi_smem = 0;
+    size_t off_shist = 0, off_bhist = 0, off_midn = 0, off_mmid = 0, off_skeys = 0;
     uint32_t n_empty = 0;                   // tensors without elements
     unsigned long long launches = 0;
     int last_cuda_error = 0;
@@ -62,6 +67,8 @@ constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tenso
 constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
 constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
 constexpr size_t kSingleRowBytes = (2 * kWarps + 3) * sizeof(uint32_t);   // shared memory per owned tile
+constexpr size_t kMultiMaxPer = 224;         // most tiles one CTA of k_topk_multi may own
+constexpr size_t kMultiRowBytes = (2 * kWarps + kSegWords) * sizeof(uint32_t);   // shared memory per owned tile
 constexpr size_t kSingleMaxT = 341;          // most tiles one CTA of k_topk_single may own
 
 inline uint64_t k_rule(uint64_t n, double density) {
@@ -110,7 +117,8 @@ WsView view(const gc_plan_s* p, void* ws) {
 // 4-element group out of `sstride`; tau_lo is the srank-th largest sampled key, where srank
 // sits six standard deviations of the sampling noise above the expected rank density*m, so a
 // candidate set smaller than k is a < 1e-8 event for well-mixed data (and only costs a redo).
-void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap, uint64_t target_max) {
+void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap, uint64_t target_max,
+                   double coarse_factor) {
     const uint64_t n = d.n;
     d.sstride = 0; d.srank = 0;
     *ccap = n;
@@ -127,7 +135,7 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
     d.sstride = (uint32_t)stride;
     d.srank = (uint32_t)rank;
     double upper = (double)n * (rank + 6.0 * std::sqrt(rank)) / m;
-    double cap = std::ceil(1.25 * upper) + 4096.0;
+    double cap = std::ceil(coarse_factor * 1.25 * upper) + 4096.0;
     *ccap = cap >= (double)n ? n : (uint64_t)cap;
 }
 
@@ -141,7 +149,9 @@ void finish_layout(gc_plan_s* p) {
         d.kind = kKindRegular; d.pad = 0;
         uint64_t ccap = d.n;
         if (p->mode == GC_TOPK) {
-            sample_params(d, p->density, p->rank_permille, &ccap, p->T == 1 ? kSampleMaxSingle : kSampleMax);
+            // (many tensors: the bracket is a histogram bin edge, up to twice the candidates)
+            sample_params(d, p->density, p->rank_permille, &ccap, p->T == 1 ? kSampleMaxSingle : kSampleMax,
+                          p->T == 1 ? 1.0 : 2.0);
         } else {
             // threshold mode: the sample is part of the definition -- one 4-element group out of
             // `stride`, rank k_s = min(m, max(1, ceil(density * m))) over its m elements
@@ -187,10 +197,18 @@ void finish_layout(gc_plan_s* p) {
     p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(uint32_t) * kSingleMaxT * 20 : 0), 256);
     p->off_fine = p->control_bytes;
     p->control_bytes = align_up(p->off_fine + (T == 1 ? sizeof(uint32_t) * (size_t)kFineBins : 0), 256);
+    // many-tensor kernel: sample and band histogram per tensor, short-list lengths
+    const size_t multi_hist = (T >= 2 && p->mode == GC_TOPK) ? sizeof(uint32_t) * (size_t)kHistBins * T : 0;
+    p->off_shist = p->control_bytes;
+    p->off_bhist = align_up(p->off_shist + multi_hist, 256);
+    p->off_midn = align_up(p->off_bhist + multi_hist, 256);
+    p->control_bytes = align_up(p->off_midn + (multi_hist ? sizeof(uint32_t) * T : 0), 256);
     p->off_tinfo = p->control_bytes;
     p->off_cidx = align_up(p->off_tinfo + sizeof(uint2) * (size_t)p->ntiles * kWarps, 256);
     p->off_mid = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
-    p->ws_bytes = align_up(p->off_mid + (T == 1 ? sizeof(uint2) * (size_t)kSingleMidCap : 0), 256);
+    p->off_mmid = align_up(p->off_mid + (T == 1 ? sizeof(uint2) * (size_t)kSingleMidCap : 0), 256);
+    p->off_skeys = align_up(p->off_mmid + (multi_hist ? sizeof(uint2) * (size_t)kMultiMidCap * T : 0), 256);
+    p->ws_bytes = align_up(p->off_skeys + (multi_hist ? sizeof(uint4) * (size_t)kBlock * p->nstiles : 0), 256);
 }
 
 
@@ -214,9 +232,42 @@ void plan_single(gc_plan_s* p) {
     // upper bracket: the sample rank that stays below the expected one by the same margin
     const double ks = p->density * 4.0 * (double)nsg;
     const double hi = std::floor(ks - 6.0 * std::sqrt(ks) - 8.0);
-    p->single_srank_hi = hi >= 1.0 ? (uint32_t)hi : 0u;
+    p->single_srank_hi = hi >= 1.0 ? (uint32_t)hi : 1u;    // small sample: the largest sampled key bounds the band
     p->single_srank_mid = (uint32_t)std::max(1.0, std::ceil(ks));
     p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
+}
+
+// Decides whether the plan can use the many-tensor kernel and with which geometry.
+void plan_multi(gc_plan_s* p) {
+    p->multi_grid = 0;
+    if (p->mode != GC_TOPK || p->T < 2 || p->grid_multi_max <= 0 || p->ntiles == 0) return;
+    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_multi_max, p->ntiles);
+    const uint32_t per = (p->ntiles + G - 1) / G;
+    if (per > kMultiMaxPer) return;
+    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
+    // expected candidates of the busiest CTA (bracket rank over sample size, times two for the
+    // bin edge), with head-room
+    std::vector<double> per_tile(p->T, 0.0);
+    for (uint32_t t = 0; t < p->T; ++t) {
+        const TensorDesc& d = p->desc[t];
+        if (d.kind == kKindSmall || d.ntiles == 0) continue;
+        if (d.sstride == 0) { per_tile[t] = (double)kTile; continue; }
+        const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
+        per_tile[t] = std::min<double>(kTile, 2.0 * (double)kTile * (double)d.srank / (4.0 * (double)nsg));
+    }
+    double worst = 0.0;
+    uint32_t t = 0;
+    for (uint32_t b = 0; b < G; ++b) {
+        double e = 0.0;
+        for (uint32_t tile = b * per; tile < std::min<uint32_t>(p->ntiles, (b + 1) * per); ++tile) {
+            while (t + 1 < p->T && (p->desc[t].ntiles == 0 || tile >= p->desc[t].tile0 + p->desc[t].ntiles)) ++t;
+            e += per_tile[t];
+        }
+        worst = std::max(worst, e);
+    }
+    if ((double)pool < 1.5 * worst + 512.0) return;
+    p->multi_grid = G; p->multi_per = per; p->multi_pool = pool;
+    p->multi_smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32);
 }
 
 int upload_table(gc_plan_s* p) {
@@ -328,6 +379,17 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         }
         (void)cudaGetLastError();
         plan_single(p);
+        p->grid_multi_max = 0;
+        if (coop) {
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi, kBlock,
+                                                              kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8) ==
+                    cudaSuccess && nb >= 1)
+                p->grid_multi_max = p->sm_count * nb;
+            else
+                (void)cudaGetLastError();
+        }
+        plan_multi(p);
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     {
@@ -361,6 +423,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
             p->rank_permille = (uint32_t)value;
             finish_layout(p);                          // workspace size stays as planned
             plan_single(p);
+            plan_multi(p);
             return upload_table(p);
         case GC_OPT_CANDIDATE_CAPACITY:
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
@@ -486,6 +549,28 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         Timed tm(p, s, GC_K_FUSED);
         GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_single, dim3(p->single_grid), dim3(kBlock),
                                                args, p->single_smem, s));
+        return GC_OK;
+    }
+    if (p->path == GC_PATH_AUTO && p->multi_grid > 0) {
+        // many tensors: one cooperative launch, three grid barriers
+        MultiArgs ma;
+        ma.desc = p->d_desc; ma.T = p->T; ma.ntiles = nt; ma.nstiles = p->nstiles;
+        ma.per = p->multi_per;
+        ma.pool_cap = std::min<uint32_t>(p->multi_pool, p->cand_cap / p->multi_grid);     // each CTA's share
+        ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();
+        ma.g = grad; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
+        ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+        ma.mid = reinterpret_cast<uint2*>(wb + p->off_mmid);
+        ma.mid_n = reinterpret_cast<uint32_t*>(wb + p->off_midn);
+        ma.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
+        ma.bhist = reinterpret_cast<uint32_t*>(wb + p->off_bhist);
+        ma.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+        ma.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
+        ma.ws = ws; ma.gws = gws;
+        void* args[] = {&ma};
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_multi, dim3(p->multi_grid), dim3(kBlock),
+                                               args, p->multi_smem, s));
         return GC_OK;
     }
     if (p->path == GC_PATH_AUTO && p->grid_fused > 0) {

@@ -113,6 +113,7 @@ __device__ __forceinline__ uint32_t ld_cg(const uint32_t* p) { return __ldcg(p);
 __device__ __forceinline__ float ld_cg(const float* p) { return __ldcg(p); }
 __device__ __forceinline__ float4 ld_cg(const float4* p) { return __ldcg(p); }
 __device__ __forceinline__ uint2 ld_cg(const uint2* p) { return __ldcg(p); }
+__device__ __forceinline__ uint4 ld_cg(const uint4* p) { return __ldcg(p); }
 __device__ __forceinline__ unsigned long long ld_cg(const unsigned long long* p) { return __ldcg(p); }
 
 constexpr int kEmitStage = 64;               // candidates of one warp chunk staged in shared memory

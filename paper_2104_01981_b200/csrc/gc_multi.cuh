@@ -1,0 +1,578 @@
+// Exact top-k of MANY tensors (layer-wise plans) in one cooperative launch.
+//
+// The scheme of the one-tensor kernel, applied per tensor: sample -> bracket [tau, tau_hi) and a
+// guess tau_z of the threshold -> fold + candidates + band histogram -> band bin of the k-th
+// key -> short list ranked by every CTA that needs it -> index-ordered emission; three grid
+// barriers.  What differs:
+//   * CTA b owns a contiguous run of tiles, so it sees one to a few tensors ("segments") and
+//     keeps one small record per segment in shared memory;
+//   * all histograms and short lists exist once per tensor in global memory; a CTA only looks
+//     at those of its own segments;
+//   * the sample is a coarse histogram only (top 11 key bits), so tau and tau_hi are bin edges:
+//     up to twice the candidates of an exact bracket, which is still a few per mille of the
+//     tensor; tau_z is interpolated inside its bin (it is only a guess);
+//   * the slot of a segment's first entry = what the tensor's earlier tiles send: the sum of
+//     their published counts + the sent short-list entries that lie before the segment;
+//   * tensors that fit one tile ("small") are finished by one CTA each between the arrival at
+//     and the wait on the first barrier, dealt to the CTAs from the top (those have no sample
+//     tiles);
+//   * a tensor whose bracket missed, or whose band bin holds more than kMultiMidCap candidates,
+//     is flagged and redone by the exact multi-pass kernels at the end (the others are not);
+//     if a CTA's candidate region overflows, everything is redone.
+#pragma once
+#include "gc_single.cuh"
+
+namespace gc {
+
+constexpr uint32_t kMultiMidCap = kMidFast;      // short list per tensor (entries stay in registers)
+constexpr uint32_t kSegWords = 16;               // shared-memory words per segment record
+constexpr uint32_t kRefineTiles = 32;            // samples of up to this many sample tiles are ranked a second time
+
+struct MultiArgs {
+    const TensorDesc* desc;
+    uint32_t T, ntiles, nstiles;
+    uint32_t per;                    // tiles per CTA (contiguous run)
+    uint32_t pool_cap;               // candidate slots per CTA
+    const uint32_t* small_ids;
+    uint32_t n_small;
+    const float* g;
+    float* r;
+    uint32_t* out_idx;
+    float* out_val;
+    uint32_t* out_count;
+    uint2* cand;                     // [gridDim.x * pool_cap]
+    uint2* mid;                      // [T][kMultiMidCap] candidates inside the band bin of the threshold
+    uint32_t* mid_n;                 // [T] their number (zeroed)
+    uint32_t* shist;                 // [T][kHistBins] coarse sample histogram (zeroed)
+    uint32_t* bhist;                 // [T][kHistBins] band histogram (zeroed)
+    uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
+    uint4* skeys;                    // [nstiles * kBlock] the sampled keys, one group of four per entry
+    WsView ws, gws;
+};
+
+// segment record (one per tensor a CTA's tile run touches), kSegWords words in shared memory
+enum : uint32_t {
+    SG_T = 0, SG_TILE0, SG_NTILE, SG_BASE0, SG_BEGIN, SG_TAU, SG_TAUZ, SG_SHIFT,
+    SG_A, SG_ABOVE, SG_M, SG_TKEY, SG_CUT, SG_OK, SG_OUT, SG_K
+};
+
+__device__ __forceinline__ void grid_arrive(WsHeader* hdr) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&hdr->barrier, 1u);
+    }
+}
+// second half of a barrier whose arrival was signalled with grid_arrive
+__device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        const uint32_t target = (passed + 1u) * gridDim.x;
+        uint32_t spins = 0;
+        while (ld_cg(&hdr->barrier) < target) {
+            if (++spins > kSpinLimit || ((spins & 15u) == 0u && ld_cg(&hdr->abort) != 0u)) { ok = 0; break; }
+            if (spins > 32) __nanosleep(spins > 4096 ? 400 : 60);
+        }
+        if (!ok) {
+            record_status(hdr, -5 /*GC_E_TIMEOUT*/, 0xB0000000ull + passed);
+            atomicExch(&hdr->abort, 1u);
+        }
+        __threadfence();
+        *s_ok = ok;
+    }
+    __syncthreads();
+    ++passed;
+    return *s_ok != 0;
+}
+
+static __global__ void __launch_bounds__(kBlock, 4)
+k_topk_multi(MultiArgs a) {
+    __shared__ BlockSmem sm;
+    __shared__ uint32_t s_used, s_cnt;
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    uint32_t* const rec = reinterpret_cast<uint32_t*>(s_dyn);                  // [per*kWarps] off<<10 | cnt
+    uint32_t* const rec2 = rec + (size_t)a.per * kWarps;                       // [per*kWarps] counts, later slots
+    uint32_t* const seg = rec2 + (size_t)a.per * kWarps;                       // [per][kSegWords]
+    uint32_t* const sent_bits = seg + (size_t)a.per * kSegWords;               // [ceil(pool_cap / 32)]
+    uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t G = gridDim.x, b = blockIdx.x;
+    WsHeader* hdr = a.ws.hdr;
+    uint32_t passed = 0;
+    const uint32_t first = min(a.ntiles, b * a.per), last = min(a.ntiles, first + a.per);
+    const uint32_t ntl = last - first;                                         // own tiles
+    for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
+    for (uint32_t i = tid; i < ntl * kWarps; i += kBlock) { rec[i] = 0u; rec2[i] = 0u; }
+    if (tid == 0) { s_used = 0u; s_cnt = 0u; }
+    phase_stamp(hdr);
+    __syncthreads();
+
+    // ---------------------------------------------------------------- sample: coarse histogram per tensor
+    if (a.nstiles) {
+        const uint32_t sper = (a.nstiles + G - 1) / G;
+        const uint32_t sfirst = min(a.nstiles, b * sper), slast = min(a.nstiles, sfirst + sper);
+        uint32_t t = 0xFFFFFFFFu;
+        TensorDesc d;
+        for (uint32_t st = sfirst; st < slast; ++st) {
+            if (t == 0xFFFFFFFFu || st >= d.stile0 + d.nstiles) {
+                if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));
+                __syncthreads();
+                t = find_tensor<SampleSpace>(a.desc, a.T, st);
+                d = a.desc[t];
+            }
+            const uint32_t ngroups = (d.n + 3u) >> 2;
+            const uint32_t nsg = (ngroups + d.sstride - 1) / d.sstride;
+            const uint64_t sg = (uint64_t)(st - d.stile0) * kBlock + tid;
+            const uint64_t gi = sg * d.sstride;
+            uint32_t key[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};     // = not a sample
+            if (sg < nsg && gi < ngroups) {
+                const uint32_t i0 = (uint32_t)gi * 4u;
+                float gv[4], rv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool v = i0 + e < d.n;
+                    const uint32_t f = d.off + (v ? i0 + e : 0u);
+                    gv[e] = v ? __ldg(a.g + f) : 0.f;
+                    rv[e] = v ? ld_cg(a.r + f) : 0.f;
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (i0 + e < d.n) {
+                        key[e] = key_of(__fadd_rn(gv[e], rv[e]));
+                        atomicAdd(&sm.hist[key[e] >> level_shift(0)], 1u);
+                    }
+            }
+            // the keys are kept: the fold pass ranks them a second time, and by then the residual
+            // they were computed from has been overwritten
+            if (d.nstiles <= kRefineTiles) a.skeys[(size_t)st * kBlock + tid] = make_uint4(key[0], key[1], key[2], key[3]);
+        }
+        if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));
+    }
+    grid_arrive(hdr);
+    // small tensors need nothing from anyone: they fill the wait (CTAs from the top take them)
+    for (uint32_t q = G - 1u - b; q < a.n_small; q += G) {
+        const uint32_t t = a.small_ids[q];
+        const TensorDesc d = a.desc[t];
+        small_tensor_body(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
+    }
+    __syncthreads();
+    for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
+    if (!grid_wait(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+
+    // ---------------------------------------------------------------- fold + candidates, segment by segment
+    uint32_t nseg = 0;
+    {
+        const uint32_t my_off = warp * kWarpChunk + lane * 4;
+        bool block_overflow = false, open = false;
+        uint32_t cur = 0xFFFFFFFFu, tau = 0, tau_z = 0;
+        int shift = 0;
+        TensorDesc d;
+        for (uint32_t tile = first; tile < last; ++tile) {
+            const uint32_t i = tile - first;
+            if (cur == 0xFFFFFFFFu || tile >= d.tile0 + d.ntiles) {
+                if (open) flush_hist(sm, a.bhist + (size_t)cur * kHistBins, 2048);
+                open = false;
+                cur = find_tensor(a.desc, a.T, tile);
+                d = a.desc[cur];
+                if (d.kind != kKindSmall) {
+                    // bracket of this tensor from its sample histogram: tau = lower edge of the bin of
+                    // the srank-th largest sampled key, tau_hi = upper edge of the bin of the one that
+                    // stays below the expected rank by the same margin, tau_z inside the bin of the
+                    // expected rank itself
+                    uint32_t tau_hi = 0x80000000u;
+                    tau = 0; tau_z = 0;
+                    if (d.sstride != 0u) {
+                        const uint32_t ngroups = (d.n + 3u) >> 2;
+                        const float msamp = 4.0f * (float)((ngroups + d.sstride - 1) / d.sstride);
+                        const float ks = (float)d.k * msamp / (float)d.n;
+                        const float hi = floorf(ks - 6.0f * sqrtf(ks) - 8.0f);
+                        // (a sample too small for that margin: the largest sampled key bounds the band instead)
+                        const uint32_t want[3] = {d.srank, hi >= 1.0f ? (uint32_t)hi : 1u, max(1u, (uint32_t)ceilf(ks))};
+                        Picked pk[3];
+                        block_select_multi<(1 << level_bits(0)), 3>(sm, a.shist + (size_t)cur * kHistBins, want, pk);
+                        if (pk[0].ok) tau = pk[0].bin << level_shift(0);
+                        if (pk[0].ok && d.nstiles <= kRefineTiles) {
+                            // second radix level of the lower bracket over the kept sample keys:
+                            // tau gets 22 significant bits (sm.hist is free between segments)
+                            const uint4* sk = a.skeys + (size_t)d.stile0 * kBlock;
+                            const uint32_t nk = d.nstiles * kBlock, bin0 = pk[0].bin;
+                            for (uint32_t q0 = tid; q0 < nk; q0 += 4 * kBlock) {
+                                uint4 kv[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)
+                                    kv[u] = q0 + u * kBlock < nk ? ld_cg(sk + q0 + u * kBlock)
+                                                                 : make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const uint32_t kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e)
+                                        if ((kk[e] >> level_shift(0)) == bin0)
+                                            atomicAdd(&sm.hist[(kk[e] >> (level_shift(0) - 11)) & 2047u], 1u);
+                                }
+                            }
+                            __syncthreads();
+                            uint32_t bin1, above1;
+                            const bool ok1 = block_select<2048, true>(sm, sm.hist, d.srank - pk[0].above, bin1, above1);
+                            for (int i2 = tid; i2 < 2048; i2 += kBlock) sm.hist[i2] = 0u;
+                            __syncthreads();
+                            if (ok1) tau |= bin1 << (level_shift(0) - 11);
+                        }
+                        if (pk[1].ok) tau_hi = (pk[1].bin + 1u) << level_shift(0);
+                        if (pk[2].ok) {
+                            const float pos = ((float)(want[2] - pk[2].above) - 0.5f) / (float)pk[2].count;   // from the top of the bin
+                            tau_z = (pk[2].bin << level_shift(0)) +
+                                    (uint32_t)((1.0f - pos) * (float)((1u << level_shift(0)) - 1u));
+                        }
+                    }
+                    if (tau_z < tau) tau_z = tau;
+                    if (tau_hi <= tau) tau_hi = 0x80000000u;
+                    shift = 0;
+                    while (((tau_hi - tau) >> shift) > 2046u) ++shift;
+                    if (tid == 0) {
+                        uint32_t* s = seg + (size_t)nseg * kSegWords;
+                        const TileGeom tg0 = tile_geom(d, tile - d.tile0);
+                        s[SG_T] = cur; s[SG_TILE0] = i; s[SG_NTILE] = min(last, d.tile0 + d.ntiles) - tile;
+                        s[SG_BASE0] = (d.off & ~3u) + (tile - d.tile0) * (uint32_t)kTile; s[SG_BEGIN] = tg0.lo;
+                        s[SG_TAU] = tau; s[SG_TAUZ] = tau_z; s[SG_SHIFT] = (uint32_t)shift;
+                        s[SG_OK] = 1u; s[SG_OUT] = d.out_off; s[SG_K] = d.k;
+                    }
+                    ++nseg;
+                    open = true;
+                }
+            }
+            if (d.kind == kKindSmall) continue;          // finished by its own CTA
+            const TileGeom tg = tile_geom(d, tile - d.tile0);
+            const bool interior = tg.lo == tg.base && tg.hi == tg.base + (uint32_t)kTile;
+            float av[kVpt][4];
+            uint32_t valid = 0xFFFFu;
+            if (interior) {
+                float4 gv[kVpt], rv[kVpt];
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+                    gv[j] = __ldg(reinterpret_cast<const float4*>(a.g + tg.base + my_off + j * 128));
+                    rv[j] = ld_cg(reinterpret_cast<const float4*>(a.r + tg.base + my_off + j * 128));
+                }
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+                    av[j][0] = __fadd_rn(gv[j].x, rv[j].x); av[j][1] = __fadd_rn(gv[j].y, rv[j].y);
+                    av[j][2] = __fadd_rn(gv[j].z, rv[j].z); av[j][3] = __fadd_rn(gv[j].w, rv[j].w);
+                }
+            } else {
+                valid = 0u;
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t f = tg.base + my_off + j * 128 + e;
+                        float v = 0.0f;
+                        if (f >= tg.lo && f < tg.hi) {
+                            v = __fadd_rn(__ldg(a.g + f), ld_cg(a.r + f));
+                            valid |= 1u << (4 * j + e);
+                        }
+                        av[j][e] = v;
+                    }
+                }
+            }
+            uint32_t cnt[kVpt], cm = 0, hm = 0;      // candidates; candidates that are zeroed right away
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                cnt[j] = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t key = key_of(av[j][e]);
+                    bool c = key >= tau;
+                    if (!interior) c = c && ((valid >> (4 * j + e)) & 1u);
+                    cnt[j] += c;
+                    cm |= (uint32_t)c << (4 * j + e);
+                    hm |= (uint32_t)(key >= tau_z) << (4 * j + e);
+                }
+            }
+            uint32_t rk[kVpt], wtot;
+            warp_rank(cnt, lane, rk, wtot);
+            uint32_t off = 0;
+            if (lane == 0 && wtot) off = atomicAdd(&s_used, wtot);
+            off = __shfl_sync(0xFFFFFFFFu, off, 0);
+            const bool fits = off + wtot <= a.pool_cap;
+            if (!fits) block_overflow = true;
+            if (lane == 0) rec[i * kWarps + warp] = fits ? ((off << 10) | wtot) : 0u;
+            const uint32_t em = fits ? cm : 0u;             // goes to the candidate list
+            const uint32_t zm = fits ? (hm & cm) : 0u;      // ... and leaves +0 in the residual (probably sent)
+            if (interior) {
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+                    float4 o;
+                    o.x = ((zm >> (4 * j + 0)) & 1u) ? 0.0f : av[j][0];
+                    o.y = ((zm >> (4 * j + 1)) & 1u) ? 0.0f : av[j][1];
+                    o.z = ((zm >> (4 * j + 2)) & 1u) ? 0.0f : av[j][2];
+                    o.w = ((zm >> (4 * j + 3)) & 1u) ? 0.0f : av[j][3];
+                    *reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128) = o;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if ((valid >> (4 * j + e)) & 1u)
+                            a.r[tg.base + my_off + j * 128 + e] = ((zm >> (4 * j + e)) & 1u) ? 0.0f : av[j][e];
+                    }
+                }
+            }
+            const bool staged = wtot <= (uint32_t)kEmitStage;
+            if (fits && wtot != 0u) {
+                if (em != 0u) {
+#pragma unroll
+                    for (int j = 0; j < kVpt; ++j) {
+                        uint32_t pos = rk[j];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if ((em >> (4 * j + e)) & 1u) {
+                                const uint2 pr = make_uint2(tg.base + my_off + j * 128 + e, __float_as_uint(av[j][e]));
+                                if (staged) sm.emit[warp][pos] = pr; else pool[off + pos] = pr;
+                                atomicAdd(&sm.hist[min((key_of(av[j][e]) - tau) >> shift, 2047u)], 1u);
+                                ++pos;
+                            }
+                        }
+                    }
+                }
+                if (staged) {
+                    __syncwarp();
+                    for (uint32_t q = lane; q < wtot; q += 32) pool[off + q] = sm.emit[warp][q];
+                    __syncwarp();
+                }
+            }
+        }
+        if (open) flush_hist(sm, a.bhist + (size_t)cur * kHistBins, 2048);
+        if (__syncthreads_or(block_overflow ? 1 : 0)) {
+            if (tid == 0) atomicExch(&hdr->overflow, 1u);
+        }
+        if (tid == 0) atomicAdd(&hdr->cand_total, min(s_used, a.pool_cap));
+    }
+    const uint32_t used = s_used;      // read linearly only when no chunk anywhere overflowed
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+
+    // segment of a candidate: the last one that begins at or before its index
+    auto seg_of = [&](uint32_t idx) -> uint32_t* {
+        uint32_t s = nseg - 1u;
+        while (s > 0u && seg[(size_t)s * kSegWords + SG_BEGIN] > idx) --s;
+        return seg + (size_t)s * kSegWords;
+    };
+    auto chunk_of = [&](const uint32_t* s, uint32_t idx) -> uint32_t {
+        const uint32_t rel = idx - s[SG_BASE0];
+        return (s[SG_TILE0] + (rel >> 12)) * kWarps + ((rel >> 9) & (kWarps - 1u));
+    };
+
+    const bool overflowed = ld_cg(&hdr->overflow) != 0u;
+    if (!overflowed && nseg != 0u) {
+        // ------------------------------------------------------------ band bin per segment, counts above it
+        for (uint32_t sidx = 0; sidx < nseg; ++sidx) {
+            uint32_t* s = seg + (size_t)sidx * kSegWords;
+            const uint32_t t = s[SG_T];
+            const uint32_t want_k[1] = {s[SG_K]};
+            Picked pa[1];
+            block_select_multi<2048, 1>(sm, a.bhist + (size_t)t * kHistBins, want_k, pa);
+            const bool ok = pa[0].ok && pa[0].count <= kMultiMidCap;
+            if (tid == 0) {
+                s[SG_A] = pa[0].bin; s[SG_ABOVE] = pa[0].above; s[SG_M] = pa[0].count; s[SG_OK] = ok ? 1u : 0u;
+                if (!ok) {          // every CTA that sees this tensor decides the same; count it once
+                    const uint32_t old = atomicOr(&a.ws.sel[t].flags, kSelFailed);
+                    if ((old & kSelFailed) == 0u) atomicAdd(&hdr->n_failed, 1u);
+                }
+            }
+        }
+        __syncthreads();
+        auto classify = [&](const uint2& pr) {
+            const uint32_t* s = seg_of(pr.x);
+            if (s[SG_OK] == 0u) return;
+            const uint32_t bin = min(((pr.y & kKeyMask) - s[SG_TAU]) >> s[SG_SHIFT], 2047u);
+            if (bin > s[SG_A]) {
+                atomicAdd(&rec2[chunk_of(s, pr.x)], 1u);
+            } else if (bin == s[SG_A]) {
+                const uint32_t slot = atomicAdd(a.mid_n + s[SG_T], 1u);
+                if (slot < kMultiMidCap) a.mid[(size_t)s[SG_T] * kMultiMidCap + slot] = pr;
+            }
+        };
+        for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {      // four loads in flight per thread
+            uint2 pr[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * kBlock;
+                pr[u] = i < used ? pool[i] : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * kBlock < used) classify(pr[u]);
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < ntl; i += kBlock) {
+            uint32_t tot = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) tot += rec2[i * kWarps + w];
+            a.tile_cnt[first + i] = tot;
+        }
+    }
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+
+    if (!overflowed) {
+        if (nseg != 0u) {
+            // -------------------------------------------------------- threshold, tie cut and slots per segment
+            for (uint32_t sidx = 0; sidx < nseg; ++sidx) {
+                uint32_t* s = seg + (size_t)sidx * kSegWords;
+                if (s[SG_OK] == 0u) continue;
+                const uint32_t t = s[SG_T], m = s[SG_M];
+                const TensorDesc d = a.desc[t];
+                const uint2* mid = a.mid + (size_t)t * kMultiMidCap;
+                uint2 e[kMidRegs];
+#pragma unroll
+                for (uint32_t u = 0; u < kMidRegs; ++u)
+                    e[u] = u * kBlock + tid < m ? ld_cg(mid + u * kBlock + tid) : make_uint2(0u, 0u);
+                // candidates above the band bin in the tensor's tiles before this segment
+                const uint32_t nbefore = first + s[SG_TILE0] - d.tile0;
+                uint32_t part = 0;
+                for (uint32_t q = tid; q < nbefore; q += kBlock) part += ld_cg(a.tile_cnt + d.tile0 + q);
+                part = __reduce_add_sync(0xFFFFFFFFu, part);
+                if (tid == 0) s_cnt = 0u;
+                __syncthreads();
+                if (lane == 0 && part) atomicAdd(&s_cnt, part);
+                const uint32_t shift = s[SG_SHIFT], A = s[SG_A];
+                const uint32_t binlo = s[SG_TAU] + (A << shift);
+                uint32_t v_sel, mid_gt, n_eq, idx_cut = 0xFFFFFFFFu;
+                const uint32_t krem = s[SG_K] - s[SG_ABOVE];
+                bool good = short_list_select(sm, e, mid, m, A == 2047u ? 31 : max((int)shift, 1), krem,
+                                              [&](const uint2& pr, uint32_t& v) { v = (pr.y & kKeyMask) - binlo; return true; },
+                                              v_sel, mid_gt, n_eq);
+                const uint32_t Tkey = binlo + v_sel;
+                const uint32_t m_eq = krem - mid_gt;
+                if (good && n_eq > m_eq) {
+                    uint32_t v_idx, x0, x1;
+                    good = short_list_select(sm, e, mid, m, 32, m_eq,
+                                             [&](const uint2& pr, uint32_t& v) { v = ~pr.x; return (pr.y & kKeyMask) == Tkey; },
+                                             v_idx, x0, x1);
+                    idx_cut = ~v_idx;
+                }
+                // sent short-list entries: before the segment they shift its first slot, inside it
+                // they join the count of their chunk
+                const uint32_t seg_end = s[SG_BASE0] + s[SG_NTILE] * (uint32_t)kTile;
+#pragma unroll
+                for (uint32_t u = 0; u < kMidRegs; ++u) {
+                    if (!(good && u * kBlock + tid < m)) continue;
+                    const uint32_t key = e[u].y & kKeyMask;
+                    if (!(key > Tkey || (key == Tkey && e[u].x <= idx_cut))) continue;
+                    if (e[u].x < s[SG_BEGIN]) atomicAdd(&s_cnt, 1u);
+                    else if (e[u].x < seg_end) atomicAdd(&rec2[chunk_of(s, e[u].x)], 1u);
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    s[SG_TKEY] = Tkey; s[SG_CUT] = idx_cut;
+                    s[SG_OUT] = d.out_off + s_cnt;                     // slot of the segment's first sent entry
+                    if (!good) {        // cannot happen unless the list changed under us: report, send nothing
+                        s[SG_OK] = 0u;
+                        record_status(hdr, -1 /*GC_E_INVALID*/, 0xE0000000ull + t);
+                    } else if (a.out_count != nullptr && first + s[SG_TILE0] == d.tile0) {
+                        a.out_count[t] = d.k; a.out_count[a.T + t] = d.k;
+                    }
+                }
+                __syncthreads();
+            }
+            // rec2[c] = output slot of the first sent candidate of chunk c (one warp walks each segment)
+            for (uint32_t sidx = warp; sidx < nseg; sidx += kWarps) {
+                const uint32_t* s = seg + (size_t)sidx * kSegWords;
+                if (s[SG_OK] == 0u) continue;
+                uint32_t run = s[SG_OUT];
+                const uint32_t c0 = s[SG_TILE0] * kWarps, nc = s[SG_NTILE] * kWarps;
+                for (uint32_t q0 = 0; q0 < nc; q0 += 32) {
+                    const uint32_t q = q0 + lane;
+                    const uint32_t v = q < nc ? rec2[c0 + q] : 0u;
+                    const uint32_t inc = warp_incl_scan(v, lane);
+                    if (q < nc) rec2[c0 + q] = run + inc - v;
+                    run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+                }
+            }
+            __syncthreads();
+        }
+        phase_stamp(hdr);
+        // sent flags of the CTA's candidates in list order, one bit each
+        auto sent_of = [&](const uint32_t* s, const uint2& pr) {
+            const uint32_t key = pr.y & kKeyMask;
+            return s[SG_OK] != 0u && (key > s[SG_TKEY] || (key == s[SG_TKEY] && pr.x <= s[SG_CUT]));
+        };
+        const uint32_t nwords = (used + 31u) >> 5;
+        for (uint32_t i0 = 0; i0 < nwords * 32u; i0 += kBlock) {
+            const uint32_t i = i0 + tid;
+            if (i0 + (tid & ~31) >= nwords * 32u) continue;          // whole warp past the end
+            bool sent = false;
+            if (i < used) {
+                const uint2 pr = pool[i];
+                sent = sent_of(seg_of(pr.x), pr);
+            }
+            const unsigned sb = __ballot_sync(0xFFFFFFFFu, sent);
+            if (lane == 0) sent_bits[i >> 5] = sb;
+        }
+        __syncthreads();
+        // emission: slot = first slot of the chunk + sent candidates before this one in the chunk
+        for (uint32_t i0 = tid; i0 < used; i0 += 4 * kBlock) {
+            uint2 pr[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * kBlock;
+                pr[u] = i < used ? pool[i] : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * kBlock;
+                if (i >= used) continue;
+                const uint32_t* s = seg_of(pr[u].x);
+                // the fold pass left +0 in the residual iff the key reached tau_z
+                const bool zeroed = (pr[u].y & kKeyMask) >= s[SG_TAUZ];
+                if (!sent_of(s, pr[u])) {          // also every candidate of a tensor that is redone
+                    if (zeroed) a.r[pr[u].x] = __uint_as_float(pr[u].y);     // value goes back
+                    continue;
+                }
+                if (!zeroed) a.r[pr[u].x] = 0.0f;
+                const uint32_t c = chunk_of(s, pr[u].x);
+                const uint32_t p0 = rec[c] >> 10;                  // first list position of the chunk
+                uint32_t before;
+                if ((p0 >> 5) == (i >> 5)) {
+                    before = __popc((sent_bits[i >> 5] & ((1u << (i & 31u)) - 1u)) >> (p0 & 31u));
+                } else {
+                    before = __popc(sent_bits[p0 >> 5] >> (p0 & 31u)) + __popc(sent_bits[i >> 5] & ((1u << (i & 31u)) - 1u));
+                    for (uint32_t w = (p0 >> 5) + 1u; w < (i >> 5); ++w) before += __popc(sent_bits[w]);
+                }
+                const uint32_t slot = rec2[c] + before;
+                a.out_idx[slot] = pr[u].x;
+                a.out_val[slot] = __uint_as_float(pr[u].y);
+            }
+        }
+        __syncthreads();
+        phase_stamp(hdr);
+        exit_stamp(hdr);
+        if (ld_cg(&hdr->n_failed) == 0u) return;
+    } else {
+        // a candidate region overflowed: every recorded candidate gets its value back
+        for (uint32_t c = tid; c < ntl * kWarps; c += kBlock) {
+            const uint32_t rc = rec[c], off = rc >> 10, cnt = rc & 1023u;
+            for (uint32_t j = 0; j < cnt; ++j) {
+                const uint2 pr = pool[off + j];
+                a.r[pr.x] = __uint_as_float(pr.y);
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- exact redo (rare)
+    // of the flagged tensors, or of all of them after an overflow: r holds a = g + r for them again
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr);
+    hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    compact_body(sm, a.desc, a.T, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
+}
+
+}  // namespace gc

@@ -49,7 +49,7 @@ struct SingleArgs {
     TensorDesc d;                    // the tensor (by value)
     const TensorDesc* desc;          // device table (for the redo phases)
     uint32_t ntiles, maxt, pool_cap; // tiles, max tiles per CTA, pool slots per CTA
-    uint32_t srank_hi;               // sample rank of the upper bracket (0 = none)
+    uint32_t srank_hi;               // sample rank of the upper bracket (at least 1)
     uint32_t srank_mid;              // sample rank that estimates the threshold itself
     uint32_t mid_cap;                // capacity of the short list
     const float* g;
