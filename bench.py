@@ -315,7 +315,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
     # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
-    ncu_traffic = {("c3_bert_base_110m_student_t", "compress_fused"): 1380.6e6}.get((w.name, dom))
+    ncu_traffic = {("c3_bert_base_110m_student_t", "compress_fused"): 1390.4e6}.get((w.name, dom))
 
     # CPU baseline: the oracle on a bounded sample of the same workload
     cpu = None
