@@ -104,7 +104,8 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  * uses it is in flight).  The selected set never depends on these options, only the route.
  *   GC_OPT_PATH                  GC_PATH_AUTO (default): one-pass candidate path with the exact
  *                                multi-pass kernels as its safety net, all in one cooperative launch;
- *                                GC_PATH_STAGED: the same phases as separate launches;
+ *                                GC_PATH_STAGED: sample, candidate extraction, candidate select and
+ *                                emission as separate launches (global histograms per level);
  *                                GC_PATH_EXACT: multi-pass kernels only
  *   GC_OPT_SAMPLE_RANK_PERMILLE  scales the sample rank that sets the candidate threshold
  *                                (1000 = default; small values make the candidate set too small
