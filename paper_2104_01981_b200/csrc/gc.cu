@@ -476,7 +476,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     {
         Timed tm(p, s, GC_K_CLEAR_CTRL);
         const size_t n16 = p->control_bytes / 16;             // control_bytes is a multiple of 256
-        const int gc = (int)std::min<size_t>((n16 + 4 * kBlock - 1) / (4 * kBlock), (size_t)p->sm_count * 4);
+        const int gc = (int)std::min<size_t>((n16 + kBlock - 1) / kBlock, (size_t)p->sm_count * 8);
         k_clear<<<gc, kBlock, 0, s>>>(reinterpret_cast<uint4*>(workspace), n16);
     }
     if (out_count != nullptr && p->n_empty > 0) {       // every tensor with elements gets its counts written

@@ -284,13 +284,17 @@ __device__ __forceinline__ unsigned long long lookback(unsigned long long* state
     return excl;
 }
 
-__device__ __forceinline__ void phase_stamp(WsHeader* hdr) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+// Phase time stamp by CTA 0 (diagnostic).  The running index lives in a register of the caller
+// so that the stamp is two stores and no load: a load here would sit on CTA 0's path to the
+// next grid barrier, and every other CTA waits for that one.
+__device__ __forceinline__ void phase_stamp(WsHeader* hdr, uint32_t& n) {
+    if (blockIdx.x == 0 && threadIdx.x == 0 && n < 20u) {
         unsigned long long ts;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
-        uint32_t i = hdr->n_stamps;
-        if (i < 20u) { hdr->stamp[i] = ts; hdr->n_stamps = i + 1u; }
+        hdr->stamp[n] = ts;
+        hdr->n_stamps = n + 1u;
     }
+    ++n;
 }
 
 __device__ __forceinline__ void exit_stamp(WsHeader* hdr) {

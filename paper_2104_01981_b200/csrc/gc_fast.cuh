@@ -553,54 +553,54 @@ struct FusedArgs {
 static __global__ void __launch_bounds__(kBlock, 4)
 k_compress_fused(FusedArgs a) {
     __shared__ BlockSmem sm;
-    uint32_t passed = 0;
+    uint32_t passed = 0, n_stamp = 0;
     WsHeader* hdr = a.ws.hdr;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     // small tensors need nothing from anyone: run them first, no barrier of their own
     small_tensors_body(sm, a.desc, a.T, a.small_ids, a.n_small, a.g, a.r, a.out_idx, a.out_val, a.out_count);
     if (a.nstiles) {
         hist_body<0, SRC_SAMPLE>(sm, a.desc, a.T, a.nstiles, a.g, a.r, a.sws);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
         hist_body<1, SRC_SAMPLE>(sm, a.desc, a.T, a.nstiles, a.g, a.r, a.sws);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     }
     fold_cand_body(sm, a.desc, a.T, a.ntiles, a.g, a.r, a.ws, a.cv);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     const bool overflow = ld_cg(&hdr->overflow) != 0u;
     if (!overflow) {
         cand_hist_body<1>(sm, a.desc, a.T, a.ntiles, a.ws, a.cv);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
         cand_hist_body<2>(sm, a.desc, a.T, a.ntiles, a.ws, a.cv);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
         cand_compact_body<false>(sm, a.desc, a.T, a.ngroups, a.r, a.out_idx, a.out_val, a.out_count, a.ws, a.cv);
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
         cand_compact_body<true>(sm, a.desc, a.T, a.ngroups, a.r, a.out_idx, a.out_val, a.out_count, a.ws, a.cv);
         __syncthreads();
-        phase_stamp(hdr);
+        phase_stamp(hdr, n_stamp);
     }
     if (!overflow && ld_cg(&hdr->n_failed) == 0u) return;
     // redo (rare): first give the listed candidates of those tensors their values back, so that
     // r holds a for every element again
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     cand_restore_body(a.desc, a.T, a.ntiles, a.r, a.ws, a.cv);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     compact_body(sm, a.desc, a.T, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
 }
 

@@ -99,13 +99,13 @@ k_topk_multi(MultiArgs a) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t G = gridDim.x, b = blockIdx.x;
     WsHeader* hdr = a.ws.hdr;
-    uint32_t passed = 0;
+    uint32_t passed = 0, n_stamp = 0;
     const uint32_t first = min(a.ntiles, b * a.per), last = min(a.ntiles, first + a.per);
     const uint32_t ntl = last - first;                                         // own tiles
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     for (uint32_t i = tid; i < ntl * kWarps; i += kBlock) { rec[i] = 0u; rec2[i] = 0u; }
     if (tid == 0) { s_used = 0u; s_cnt = 0u; }
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     __syncthreads();
 
     // ---------------------------------------------------------------- sample: coarse histogram per tensor
@@ -159,7 +159,7 @@ k_topk_multi(MultiArgs a) {
     __syncthreads();
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     if (!grid_wait(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
 
     // ---------------------------------------------------------------- fold + candidates, segment by segment
     uint32_t nseg = 0;
@@ -352,7 +352,7 @@ k_topk_multi(MultiArgs a) {
     }
     const uint32_t used = s_used;      // read linearly only when no chunk anywhere overflowed
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
 
     // segment of a candidate: the last one that begins at or before its index
     auto seg_of = [&](uint32_t idx) -> uint32_t* {
@@ -415,7 +415,7 @@ k_topk_multi(MultiArgs a) {
         }
     }
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
 
     if (!overflowed) {
         if (nseg != 0u) {
@@ -494,7 +494,7 @@ k_topk_multi(MultiArgs a) {
             }
             __syncthreads();
         }
-        phase_stamp(hdr);
+        phase_stamp(hdr, n_stamp);
         // sent flags of the CTA's candidates in list order, one bit each
         auto sent_of = [&](const uint32_t* s, const uint2& pr) {
             const uint32_t key = pr.y & kKeyMask;
@@ -548,7 +548,7 @@ k_topk_multi(MultiArgs a) {
             }
         }
         __syncthreads();
-        phase_stamp(hdr);
+        phase_stamp(hdr, n_stamp);
         exit_stamp(hdr);
         if (ld_cg(&hdr->n_failed) == 0u) return;
     } else {
@@ -565,7 +565,7 @@ k_topk_multi(MultiArgs a) {
     // ---------------------------------------------------------------- exact redo (rare)
     // of the flagged tensors, or of all of them after an overflow: r holds a = g + r for them again
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);

@@ -184,14 +184,14 @@ k_topk_single(SingleArgs a) {
     const uint32_t G = gridDim.x, b = blockIdx.x;
     const TensorDesc& d = a.d;
     WsHeader* hdr = a.ws.hdr;
-    uint32_t passed = 0;
+    uint32_t passed = 0, n_stamp = 0;
     const uint32_t n_own = b < a.ntiles ? (a.ntiles - b + G - 1) / G : 0u;
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     for (uint32_t i = tid; i < n_own * kWarps; i += kBlock) rec2[i] = 0u;
     for (uint32_t i = tid; i < n_own; i += kBlock) row_mid[i] = 0u;
     const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
     if (tid == 0) s_used = 0u;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
 
     // ---------------------------------------------------------------- sample
     // One 4-element group out of d.sstride.  Two histograms of the sampled keys are built in one
@@ -231,9 +231,20 @@ k_topk_single(SingleArgs a) {
                     atomicAdd(&sm.hist[skey[q][e] >> level_shift(0)], 1u);
                     atomicAdd(a.fine + fine_slot(skey[q][e] >> kFineShift), 1u);
                 }
+        // the first own tile is asked into L2 while the sample is being settled
+        if (n_own) {
+            const uint32_t pb = (d.off & ~3u) + b * (uint32_t)kTile + warp * kWarpChunk + lane * 4;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                if (pb + j * 128 + 4 <= d.off + d.n) {
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.g + pb + j * 128));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.r + pb + j * 128));
+                }
+            }
+        }
         flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-        phase_stamp(hdr);
+        phase_stamp(hdr, n_stamp);
         // both brackets from one read of the coarse histogram, then the kFineBits finer bits of
         // each from the 2^kFineBits fine bins under its coarse bin (one warp per bracket)
         const uint32_t want[3] = {d.srank, a.srank_hi, a.srank_mid};
@@ -346,7 +357,7 @@ k_topk_single(SingleArgs a) {
                 o.y = ((zm >> (4 * j + 1)) & 1u) ? 0.0f : av[j][1];
                 o.z = ((zm >> (4 * j + 2)) & 1u) ? 0.0f : av[j][2];
                 o.w = ((zm >> (4 * j + 3)) & 1u) ? 0.0f : av[j][3];
-                *reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128) = o;
+                __stcs(reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128), o);    // streaming: evict first
             }
         } else {
 #pragma unroll
@@ -391,7 +402,7 @@ k_topk_single(SingleArgs a) {
     const uint32_t used = s_used;      // read linearly only when no chunk anywhere overflowed
     flush_hist(sm, a.hist5 + 2 * kHistBins, 2048);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
 
     // ---------------------------------------------------------------- band bin of the threshold
     // `good` is the same in every CTA: it only depends on global data read after a barrier
@@ -445,7 +456,7 @@ k_topk_single(SingleArgs a) {
             atomicAdd(a.seg_tot + (size_t)i * nseg + myseg, tot);
         }
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
-        phase_stamp(hdr);
+        phase_stamp(hdr, n_stamp);
 
         // ------------------------------------------------------------ exact threshold from the short list
         // Every CTA ranks the same m entries: Tkey = the (k - aboveA)-th largest key among them.
@@ -554,7 +565,7 @@ k_topk_single(SingleArgs a) {
                     pos += c;
                 }
             }
-            phase_stamp(hdr);      // threshold and output slots known
+            phase_stamp(hdr, n_stamp);      // threshold and output slots known
             // sent flags of the CTA's candidates in list order, one bit each
             const uint32_t nwords = (used + 31u) >> 5;
             for (uint32_t i0 = 0; i0 < nwords * 32u; i0 += 4 * kBlock) {
@@ -604,8 +615,8 @@ k_topk_single(SingleArgs a) {
                     }
                     const uint32_t slot = rec2[c] + before;
                     if (slot < d.cap) {
-                        a.out_idx[d.out_off + slot] = pr[u].x;
-                        a.out_val[d.out_off + slot] = __uint_as_float(pr[u].y);
+                        __stcs(a.out_idx + d.out_off + slot, pr[u].x);
+                        __stcs(a.out_val + d.out_off + slot, __uint_as_float(pr[u].y));
                     } else {
                         record_status(hdr, -1 /*GC_E_INVALID*/, pr[u].x);
                     }
@@ -613,7 +624,7 @@ k_topk_single(SingleArgs a) {
             }
             if (a.out_count != nullptr && b == 0 && tid == 0) { a.out_count[0] = d.k; a.out_count[1] = d.k; }
             __syncthreads();
-            phase_stamp(hdr);
+            phase_stamp(hdr, n_stamp);
             exit_stamp(hdr);
             return;
         }
@@ -631,7 +642,7 @@ k_topk_single(SingleArgs a) {
         }
     }
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr);
+    phase_stamp(hdr, n_stamp);
     hist_body<0, SRC_RESID>(sm, a.desc, 1u, a.ntiles, nullptr, a.r, a.gws);
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     hist_body<1, SRC_RESID>(sm, a.desc, 1u, a.ntiles, nullptr, a.r, a.gws);
