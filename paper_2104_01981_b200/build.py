@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 SO = os.path.join(_HERE, "libgc.so")
-SOURCES = ["gc.cu", "gc_noalloc.cu"]
+SOURCES = ["gc.cu", "gc_noalloc.cu", "ecrm.cu"]
 
 
 def _nvcc() -> str:
@@ -23,7 +23,8 @@ def _stale() -> bool:
     if not os.path.exists(SO):
         return True
     t = os.path.getmtime(SO)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(_ROOT, "include", "gc.h")]
+    inc = os.path.join(_ROOT, "include")
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(inc, f) for f in os.listdir(inc)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

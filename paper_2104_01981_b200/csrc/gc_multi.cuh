@@ -308,7 +308,7 @@ k_topk_multi(MultiArgs a) {
                     o.y = ((zm >> (4 * j + 1)) & 1u) ? 0.0f : av[j][1];
                     o.z = ((zm >> (4 * j + 2)) & 1u) ? 0.0f : av[j][2];
                     o.w = ((zm >> (4 * j + 3)) & 1u) ? 0.0f : av[j][3];
-                    *reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128) = o;
+                    __stcs(reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128), o);    // streaming: evict first
                 }
             } else {
 #pragma unroll

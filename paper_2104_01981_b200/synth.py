@@ -208,3 +208,32 @@ def sparse_set(sizes, ks, seed: int, scale: float = 1.0):
     idx = np.concatenate(idx).astype(np.uint32) if idx else np.zeros(0, np.uint32)
     val = (rng.standard_normal(idx.size) * scale).astype(np.float32)
     return idx, val
+
+
+# --------------------------------------------------------------------------- embedding-table batches
+def ecrm_tables(n_rows: int, dim: int, k: int, seed: int, device: str | torch.device = "cpu",
+                integer_valued: bool = False):
+    """k embedding-table shards [n_rows][dim] with N(0, 0.01^2)-like entries (or small integers,
+    for cases that must be exact) and zero optimizer state.  Input generator only."""
+    gen = torch.Generator(device=torch.device(device))
+    gen.manual_seed(seed)
+    shards = []
+    for _ in range(k):
+        e = torch.empty(n_rows, dim, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+        shards.append(torch.round(e * 8.0) if integer_valued else e * 0.01)
+    return shards
+
+
+def ecrm_batch(n_rows: int, m: int, dim: int, seed: int, device: str | torch.device = "cpu",
+               integer_valued: bool = False):
+    """One batch's aggregated sparse gradient for a shard: m distinct row numbers (random order,
+    as a hash-based unique leaves them) and their gradient rows."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    rows = _distinct_sorted(rng, n_rows, m)
+    rng.shuffle(rows)
+    gen = torch.Generator(device=torch.device(device))
+    gen.manual_seed(seed + 17)
+    g = torch.empty(m, dim, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+    g = torch.round(g * 4.0) if integer_valued else g * 0.05
+    return torch.from_numpy(rows.astype(np.uint32).view(np.int32)).to(device), g

@@ -20,14 +20,20 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "gc.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(gc_[a-z_0-9]+)\s*\(", text)))
+    syms = set()
+    inc = os.path.join(ROOT, "include")
+    for name in sorted(os.listdir(inc)):
+        text = open(os.path.join(inc, name)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        syms |= set(re.findall(r"\b((?:gc|ecrm)_[a-z_0-9]+)\s*\(", text))
+    return sorted(syms)
 
 
 def test_every_declared_symbol_is_exported(lib):
     syms = declared_symbols()
     assert {"gc_plan", "gc_compress", "gc_decompress_accumulate", "gc_destroy"} <= set(syms)
+    assert {"ecrm_encode", "ecrm_decode", "ecrm_rows_step", "ecrm_parity_add", "ecrm_degraded_read",
+            "ecrm_placement"} <= set(syms)
     for s in syms:
         assert hasattr(lib, s), s
     assert lib.gc_version() >= 1
@@ -87,3 +93,15 @@ def test_host_only_plan_refuses_compute(lib):
     p = api.Plan([16], 0.5, device=-1)
     assert p.compress_ptr(16, 16, 16, 16, None, 256, 0) == api.GC_E_UNSUPPORTED
     assert lib.gc_destroy(None) == api.GC_OK
+
+
+def test_ecrm_placement_matches_the_oracle_rule(lib):
+    from oracle import ecrm_oracle
+    from paper_2104_01981_b200 import ecrm
+    for k in (1, 3, 4, 32):
+        for group in (0, 1, k, k + 1, 12345678901):
+            assert ecrm.placement(k, group) == ecrm_oracle.placement(k, group)
+    with pytest.raises(ecrm.EcrmError):
+        ecrm.placement(0, 1)
+    with pytest.raises(ecrm.EcrmError):
+        ecrm.placement(33, 1)
