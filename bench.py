@@ -20,6 +20,7 @@ import os
 import statistics
 import subprocess
 import sys
+import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -361,6 +362,129 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- erasure-coded embedding tables
+def run_ecrm(args, rank: int, world: int, local_rank: int):
+    """Second workload (`--workload ecrm`): the server-side work of erasure-coded embedding-table
+    training on one GPU that plays data server and parity host.  A step = optimizer on the m rows
+    a batch touched (differences out) + the parity host adding them; the encoder, the full-shard
+    decoder and degraded reads are timed beside it.  Prints its own JSON line."""
+    from paper_2104_01981_b200 import ecrm
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    n_rows, p_rows, m, dim, k = args.ecrm_rows, args.ecrm_rows // 4, args.ecrm_batch, 128, 4
+    peak, peak_src = measured_peak_gbs()
+    entry = synth.ecrm_tables(n_rows, dim, 1, seed=1, device=dev)[0]
+    state = torch.zeros(n_rows, dim, device=dev)
+    p_entry = torch.zeros(p_rows, dim, device=dev)
+    p_state = torch.zeros(p_rows, dim, device=dev)
+    sets = []
+    for sidx in range(4):                                  # distinct batches cycled through (each 0.5 GB: larger than L2)
+        rows, g = synth.ecrm_batch(n_rows, m, dim, seed=10 + sidx, device="cpu")
+        prow = torch.from_numpy((rows.numpy().view(np.uint32) % np.uint32(p_rows)).astype(np.uint32).view(np.int32))
+        # parity rows must be distinct inside one call: keep the first occurrence of each
+        _, first = np.unique(prow.numpy(), return_index=True)
+        keep = torch.from_numpy(np.sort(first))
+        sets.append((rows[keep].to(dev), g[keep].to(dev), prow[keep].to(dev)))
+    m_eff = min(s[0].numel() for s in sets)
+    sets = [(r[:m_eff].contiguous(), g[:m_eff].contiguous(), pr[:m_eff].contiguous()) for r, g, pr in sets]
+    de = torch.empty(m_eff, dim, device=dev)
+    ds = torch.empty(m_eff, dim, device=dev)
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        for i in range(args.warmup):
+            fn(i)
+        barrier()
+        e0.record(stream)
+        for i in range(steps):
+            fn(args.warmup + i)
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    def step(i):
+        rows, g, prow = sets[i % len(sets)]
+        ecrm.rows_step(ecrm.ECRM_MOMENTUM, rows, g, entry, state, 0.01, 0.9, de, ds, None, stream)
+        ecrm.parity_add(prow, de, ds, p_entry, p_state, None, stream)
+
+    def only_step(i):
+        rows, g, _ = sets[i % len(sets)]
+        ecrm.rows_step(ecrm.ECRM_MOMENTUM, rows, g, entry, state, 0.01, 0.9, de, ds, None, stream)
+
+    def only_add(i):
+        ecrm.parity_add(sets[i % len(sets)][2], de, ds, p_entry, p_state, None, stream)
+
+    clocks = ClockSampler(local_rank, os.path.join(tempfile.gettempdir(), f"gc_clocks_ecrm_{rank}.csv"))
+    ms = timed(step, args.steps)
+    ms_step = timed(only_step, args.steps)
+    ms_add = timed(only_add, args.steps)
+    # encoder / decoder over whole shards (k = 4 shards of 1 GiB), degraded reads of m rows
+    shard_n = min(n_rows, 2 * 1024 * 1024) * dim
+    shards = [entry.view(-1)[:shard_n]] + [torch.randn(shard_n, device=dev) for _ in range(k - 1)]
+    parity = torch.empty(shard_n, device=dev)
+    out = torch.empty(shard_n, device=dev)
+    n_cd = max(3, args.steps // 10)
+    ms_enc = timed(lambda i: ecrm.encode(shards, parity, stream), n_cd)
+    ms_dec = timed(lambda i: ecrm.decode(shards[1:], parity, out, stream), n_cd)
+    rd_rows = (sets[0][0].view(torch.int32) % (shard_n // dim)).contiguous()
+    rd_out = torch.empty(m_eff, dim, device=dev)
+    sh2 = [x.view(-1, dim) for x in shards]
+    ms_rd = timed(lambda i: ecrm.degraded_read(rd_rows, None, sh2[1:], parity.view(-1, dim), rd_out, None, stream), n_cd)
+    clk = clocks.stop()
+    ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd = reduce_max_over_ranks([ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd],
+                                                                        world, dev)
+    if rank != 0:
+        return
+    row_b = dim * 4
+    bytes_step = m_eff * (7 * row_b + 4)          # g, e, s read; e, s, de, ds written; row number
+    bytes_add = m_eff * (6 * row_b + 4)           # de, ds read; parity entry and state read + written
+    upd_gbs = (bytes_step + bytes_add) * world * args.steps / (ms * 1e-3) / 1e9
+    step_gbs = bytes_step / (ms_step / args.steps * 1e-3) / 1e9
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import ecrm_oracle as eo
+        srows, sg, sprow = (t[:20000].cpu() for t in sets[0])
+        he, hs = entry[:].cpu().numpy(), np.zeros((n_rows, dim), np.float32)
+        hp, hps = np.zeros((p_rows, dim), np.float32), np.zeros((p_rows, dim), np.float32)
+        t0 = time.perf_counter()
+        d1, d2 = eo.rows_step(eo.MOMENTUM, srows.numpy().view(np.uint32), sg.numpy(), he, hs, 0.01, 0.9)
+        eo.parity_add(sprow.numpy().view(np.uint32), d1, d2, hp, hps)
+        dt = time.perf_counter() - t0
+        cpu = {"value": 20000 * (13 * row_b + 8) / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "sample": "20000 rows of one batch: optimizer step + parity add, numpy row by row"}
+    line = {
+        "metric": "ecrm_update_traffic_GB_per_s", "value": upd_gbs, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "ecrm_embedding_rows", "rows": n_rows, "parity_rows": p_rows, "dim": dim,
+                   "rows_per_batch": m_eff, "optimizer": "momentum", "k": k,
+                   "l2": "four batches of 0.5 GB cycled; tables of several GB (no flush)"},
+        "rows_per_s": m_eff * world * args.steps / (ms * 1e-3),
+        "kernels": {
+            "rows_step": {"ms_per_launch": ms_step / args.steps, "GB_per_s": step_gbs},
+            "parity_add": {"ms_per_launch": ms_add / args.steps,
+                           "GB_per_s": bytes_add / (ms_add / args.steps * 1e-3) / 1e9},
+            "encode_k4": {"ms_per_launch": ms_enc / n_cd, "GB_per_s": (k + 1) * 4 * shard_n / (ms_enc / n_cd * 1e-3) / 1e9},
+            "decode_k4": {"ms_per_launch": ms_dec / n_cd, "GB_per_s": (k + 1) * 4 * shard_n / (ms_dec / n_cd * 1e-3) / 1e9},
+            "degraded_read_k4": {"ms_per_launch": ms_rd / n_cd,
+                                 "GB_per_s": m_eff * ((k + 1) * row_b + 4) / (ms_rd / n_cd * 1e-3) / 1e9},
+        },
+        "roofline": {"bound": "hbm", "kernel": "rows_step", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": step_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": bytes_step},
+        "cpu_baseline": cpu, "e2e": None, "gpu_launches": 2 * args.steps, "clocks": clk,
+    }
+    print(json.dumps(line))
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -377,6 +501,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end region")
     ap.add_argument("--input-sets", type=int, default=N_INPUT_SETS,
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")
+    ap.add_argument("--workload", default="gc", choices=["gc", "ecrm"],
+                    help="gc: gradient compression (the headline line); ecrm: erasure-coded embedding-table rows")
+    ap.add_argument("--ecrm-rows", type=int, default=8 * 1024 * 1024, help="rows of the embedding-table shard")
+    ap.add_argument("--ecrm-batch", type=int, default=1024 * 1024, help="distinct rows one batch updates")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "gc" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -389,7 +517,10 @@ def main():
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
     try:
-        run_gpu(args, w, rank, world, local_rank)
+        if args.workload == "ecrm":
+            run_ecrm(args, rank, world, local_rank)
+        else:
+            run_gpu(args, w, rank, world, local_rank)
     finally:
         if world > 1:
             torch.distributed.destroy_process_group()
