@@ -477,7 +477,8 @@ def run_ecrm(args, rank: int, world: int, local_rank: int):
                                  "GB_per_s": m_eff * ((k + 1) * row_b + 4) / (ms_rd / n_cd * 1e-3) / 1e9},
         },
         "roofline": {"bound": "hbm", "kernel": "rows_step", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": step_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "frac": step_gbs / peak, "traffic": m_eff * 3430.4, "peak_source": peak_src,
+                     "traffic_source": "profiles/k_ecrm_rows_step_2m_rows_dim128.md (3430 B per row, scaled by rows)",
                      "algorithmic_bytes_per_launch": bytes_step},
         "cpu_baseline": cpu, "e2e": None, "gpu_launches": 2 * args.steps, "clocks": clk,
     }
