@@ -10,6 +10,7 @@
 #include "gc_single.cuh"
 #include "gc_multi.cuh"
 #include "gc_threshold.cuh"
+#include "gc_thr_single.cuh"
 #include "gc_decode.cuh"
 
 using namespace gc;
@@ -45,6 +46,9 @@ struct gc_plan_s {
     size_t single_smem = 0;
     size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0;
     uint32_t single_srank_hi = 0, single_srank_mid = 0;
+    int grid_thr_single_max = 0;
+    uint32_t thr_grid = 0, thr_maxt = 0, thr_pool = 0, thr_rounds = 0;    // one-tensor threshold kernel (0 = no)
+    size_t thr_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
     uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0;       // 0 = plan does not qualify
     size_t multi_smem = 0;
@@ -181,7 +185,13 @@ void finish_layout(gc_plan_s* p) {
     // every warp of the fold pass may strand part of a slab; CTAs never outnumber tiles
     ccap_total += (uint64_t)std::min<uint32_t>(p->ntiles, 1024u) * kWarps * kSlab;
     if (ccap_total > 0x7FFFFFFFull) ccap_total = 0x7FFFFFFFull;
-    if (p->mode != GC_TOPK) ccap_total = 0;
+    if (p->mode != GC_TOPK) {
+        // one-tensor threshold plans keep a hit list: about k hits are expected (the sample says so),
+        // up to the capacity factor are sent; the rest is slack for up to 1024 CTA regions
+        ccap_total = 0;
+        if (p->T == 1 && p->desc[0].n > 0)
+            ccap_total = std::min<uint64_t>(0x7FFFFFFFull, (uint64_t)(2.5 * (double)p->desc[0].cap) + (1u << 20));
+    }
     if (p->cand_cap_alloc == 0) p->cand_cap_alloc = (uint32_t)ccap_total;   // fixed at plan creation
     p->cand_cap = (uint32_t)std::min<uint64_t>(ccap_total, p->cand_cap_alloc);
     const size_t T = p->T;
@@ -192,8 +202,8 @@ void finish_layout(gc_plan_s* p) {
     p->off_state = align_up(p->off_hist + sizeof(uint32_t) * (size_t)kHistBins * T, 256);
     p->off_gstate = align_up(p->off_state + sizeof(unsigned long long) * (size_t)p->ntiles, 256);
     p->off_hist5 = align_up(p->off_gstate + sizeof(unsigned long long) * (size_t)p->ngroups, 256);
-    // single-tensor kernel: five histograms, then row totals and 32-CTA segment totals
-    p->off_rowseg = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 5 * (size_t)kHistBins : 0), 256);
+    // one-tensor kernels: six 2048-bin histogram slots, then 32-CTA segment totals
+    p->off_rowseg = align_up(p->off_hist5 + (T == 1 ? sizeof(uint32_t) * 6 * (size_t)kHistBins : 0), 256);
     p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(uint32_t) * kSingleMaxT * 20 : 0), 256);
     p->off_fine = p->control_bytes;
     p->control_bytes = align_up(p->off_fine + (T == 1 ? sizeof(uint32_t) * (size_t)kFineBins : 0), 256);
@@ -208,7 +218,8 @@ void finish_layout(gc_plan_s* p) {
     p->off_mid = align_up(p->off_cidx + sizeof(uint2) * (size_t)p->cand_cap_alloc, 256);
     p->off_mmid = align_up(p->off_mid + (T == 1 ? sizeof(uint2) * (size_t)kSingleMidCap : 0), 256);
     p->off_skeys = align_up(p->off_mmid + (multi_hist ? sizeof(uint2) * (size_t)kMultiMidCap * T : 0), 256);
-    p->ws_bytes = align_up(p->off_skeys + (multi_hist ? sizeof(uint4) * (size_t)kBlock * p->nstiles : 0), 256);
+    const bool keep_keys = multi_hist != 0 || (T == 1 && p->mode == GC_THRESHOLD);
+    p->ws_bytes = align_up(p->off_skeys + (keep_keys ? sizeof(uint4) * (size_t)kBlock * p->nstiles : 0), 256);
 }
 
 
@@ -235,6 +246,24 @@ void plan_single(gc_plan_s* p) {
     p->single_srank_hi = hi >= 1.0 ? (uint32_t)hi : 1u;    // small sample: the largest sampled key bounds the band
     p->single_srank_mid = (uint32_t)std::max(1.0, std::ceil(ks));
     p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
+}
+
+// Decides whether a threshold plan can use the one-tensor kernel and with which geometry.
+void plan_thr_single(gc_plan_s* p) {
+    p->thr_grid = 0;
+    if (p->mode != GC_THRESHOLD || p->T != 1 || p->grid_thr_single_max <= 0) return;
+    const TensorDesc& d = p->desc[0];
+    if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
+    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_thr_single_max, d.ntiles);
+    const uint32_t maxt = (d.ntiles + G - 1) / G;
+    if (maxt > kSingleMaxT || G > 640) return;
+    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
+    if ((double)pool < 1.25 * (double)d.k / (double)G + 256.0) return;
+    const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
+    const uint64_t rounds = (nsg + (uint64_t)G * kBlock - 1) / ((uint64_t)G * kBlock);
+    if (rounds > 64) return;
+    p->thr_grid = G; p->thr_maxt = maxt; p->thr_pool = pool; p->thr_rounds = (uint32_t)rounds;
+    p->thr_smem = (size_t)maxt * (2 * kWarps + 2) * sizeof(uint32_t);
 }
 
 // Decides whether the plan can use the many-tensor kernel and with which geometry.
@@ -379,6 +408,17 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         }
         (void)cudaGetLastError();
         plan_single(p);
+        p->grid_thr_single_max = 0;
+        if (coop) {
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_threshold_single, kBlock,
+                                                              kSingleMaxT * (2 * kWarps + 2) * sizeof(uint32_t)) ==
+                    cudaSuccess && nb >= 1)
+                p->grid_thr_single_max = p->sm_count * nb;
+            else
+                (void)cudaGetLastError();
+        }
+        plan_thr_single(p);
         p->grid_multi_max = 0;
         if (coop) {
             int nb = 0;
@@ -487,6 +527,27 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
     const int gcp = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
     char* wb = static_cast<char*>(workspace);
+    if (p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thr_grid > 0) {
+        // one large tensor: sample, exact threshold, fold + hits and emission in one cooperative launch
+        ThrSingleArgs ta;
+        ta.d = p->desc[0]; ta.desc = p->d_desc; ta.ntiles = nt; ta.maxt = p->thr_maxt; ta.pool_cap = p->thr_pool;
+        ta.sample_rounds = p->thr_rounds;
+        ta.g = grad; ta.r = residual; ta.out_idx = out_idx; ta.out_val = out_val; ta.out_count = out_count;
+        ta.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+        ta.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
+        ta.hist5 = reinterpret_cast<uint32_t*>(wb + p->off_hist5);
+        ta.hist13 = ta.hist5 + 2 * kHistBins;          // slots 2..5 of the six
+        ta.mid = reinterpret_cast<uint2*>(wb + p->off_mid); ta.mid_cap = (uint32_t)kSingleMidCap;
+        ta.fine = reinterpret_cast<uint32_t*>(wb + p->off_fine);
+        ta.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+        ta.seg_tot = reinterpret_cast<uint32_t*>(wb + p->off_rowseg);
+        ta.ws = ws;
+        void* args[] = {&ta};
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_threshold_single, dim3(p->thr_grid), dim3(kBlock),
+                                               args, p->thr_smem, s));
+        return GC_OK;
+    }
     if (p->mode == GC_THRESHOLD) {
         // exact order statistic of the sample (three radix levels), then one fused pass
         WsView sws = ws;

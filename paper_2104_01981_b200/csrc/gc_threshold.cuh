@@ -8,13 +8,14 @@ namespace gc {
 
 // Ticket-ordered tiles; the number of hits before a tile (within its tensor) comes from the
 // look-back exchange, so output slots are index-ordered and a truncated tensor keeps exactly
-// its first `cap` hits.  `ssel[t].T` holds tau.
-static __global__ void __launch_bounds__(kBlock)
-k_threshold_emit(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
-                 const float* __restrict__ g, float* __restrict__ r,
-                 uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
-                 uint32_t* __restrict__ out_count, WsView ws, const TensorSel* __restrict__ ssel,
-                 int ticket_slot) {
+// its first `cap` hits.  tau of tensor t = ssel[t].T, or `tau_fixed` when ssel is null.
+// FOLD: a = g + r is computed here (and stored); otherwise r already holds a.
+template <bool FOLD>
+static __device__ void threshold_emit_body(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                                           const float* __restrict__ g, float* __restrict__ r,
+                                           uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                           uint32_t* __restrict__ out_count, const WsView& ws,
+                                           const TensorSel* __restrict__ ssel, uint32_t tau_fixed, int ticket_slot) {
     __shared__ uint32_t s_tile;
     __shared__ uint32_t s_tot[kWarps], s_ex[kWarps];
     __shared__ uint32_t s_sum;
@@ -34,10 +35,10 @@ k_threshold_emit(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntile
         if (tile >= ntiles) break;
         const uint32_t t = find_tensor(desc, T, tile);
         const TensorDesc d = desc[t];
-        const uint32_t tau = ssel[t].T;
+        const uint32_t tau = ssel != nullptr ? ssel[t].T : tau_fixed;
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;
-        load_tile<true>(g, r, tg, warp, lane, tl);
+        load_tile<FOLD>(g, r, tg, warp, lane, tl);
 
         uint32_t cnt[kVpt], hm = 0;
 #pragma unroll
@@ -92,6 +93,15 @@ k_threshold_emit(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntile
             if (hits > d.cap) record_status(ws.hdr, 1 /*GC_W_TRUNCATED*/, t);
         }
     }
+}
+
+static __global__ void __launch_bounds__(kBlock)
+k_threshold_emit(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                 const float* __restrict__ g, float* __restrict__ r,
+                 uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                 uint32_t* __restrict__ out_count, WsView ws, const TensorSel* __restrict__ ssel,
+                 int ticket_slot) {
+    threshold_emit_body<true>(desc, T, ntiles, g, r, out_idx, out_val, out_count, ws, ssel, 0u, ticket_slot);
 }
 
 }  // namespace gc

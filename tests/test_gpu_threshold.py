@@ -113,3 +113,19 @@ def test_threshold_config4_resnet_workers_and_decode():
                                out, True, workers[0].ws)
     want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
     assert np.array_equal(to_np_u32(out), bits(want))
+
+
+def test_threshold_one_tensor_mild_truncation_and_two_valued_input():
+    """One large tensor (the fused one-tensor kernel).  cap_factor 1.0: the hits exceed the
+    capacity by a little in some steps, so the kernel itself cuts the tail and puts those
+    values back.  Two-valued input: tens of thousands of sampled keys are equal to tau (the
+    8192-bin route of the sample select) and every element is a hit (the hit list overflows,
+    the look-back pass takes over)."""
+    n = 2_000_003
+    grads = [randn(n, 900 + s) for s in range(4)]
+    check_threshold([n], 0.01, grads, cap_factor=1.0)
+    check_threshold([n], 0.02, grads[:2], stride=16, cap_factor=1.25)
+    g = torch.ones(n)
+    g[torch.rand(n, generator=torch.Generator().manual_seed(3)) < 0.1] = -3.0
+    check_threshold([n], 0.5, [g, g])
+    check_threshold([n], 0.05, [g])
