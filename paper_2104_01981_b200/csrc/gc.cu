@@ -50,6 +50,7 @@ struct gc_plan_s {
     uint32_t thr_grid = 0, thr_maxt = 0, thr_pool = 0, thr_rounds = 0;    // one-tensor threshold kernel (0 = no)
     size_t thr_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
+    uint32_t multi_ntab = 0;
     uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0;       // 0 = plan does not qualify
     size_t multi_smem = 0;
     size_t off_shist = 0, off_bhist = 0, off_midn = 0, off_mmid = 0, off_skeys = 0;
@@ -71,7 +72,8 @@ constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tenso
 constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
 constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
 constexpr size_t kSingleRowBytes = (2 * kWarps + 3) * sizeof(uint32_t);   // shared memory per owned tile
-constexpr size_t kMultiMaxPer = 224;         // most tiles one CTA of k_topk_multi may own
+constexpr uint32_t kMultiMaxTab = 1024;      // tensors whose tile tables k_topk_multi keeps in shared memory
+constexpr size_t kMultiMaxPer = 160;         // most tiles one CTA of k_topk_multi may own
 constexpr size_t kMultiRowBytes = (2 * kWarps + kSegWords) * sizeof(uint32_t);   // shared memory per owned tile
 constexpr size_t kSingleMaxT = 341;          // most tiles one CTA of k_topk_single may own
 
@@ -296,7 +298,9 @@ void plan_multi(gc_plan_s* p) {
     }
     if ((double)pool < 1.5 * worst + 512.0) return;
     p->multi_grid = G; p->multi_per = per; p->multi_pool = pool;
-    p->multi_smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32);
+    p->multi_ntab = p->T <= kMultiMaxTab ? p->T : 0u;
+    p->multi_smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32) +
+                    2 * sizeof(uint32_t) * (size_t)p->multi_ntab;
 }
 
 int upload_table(gc_plan_s* p) {
@@ -423,7 +427,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         if (coop) {
             int nb = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi, kBlock,
-                                                              kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8) ==
+                                                              kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8 + 8 * kMultiMaxTab) ==
                     cudaSuccess && nb >= 1)
                 p->grid_multi_max = p->sm_count * nb;
             else
@@ -618,6 +622,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         ma.desc = p->d_desc; ma.T = p->T; ma.ntiles = nt; ma.nstiles = p->nstiles;
         ma.per = p->multi_per;
         ma.pool_cap = std::min<uint32_t>(p->multi_pool, p->cand_cap / p->multi_grid);     // each CTA's share
+        ma.pool_smem_words = (p->multi_pool + 31) / 32; ma.ntab = p->multi_ntab;
         ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();
         ma.g = grad; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
         ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);

@@ -33,6 +33,8 @@ struct MultiArgs {
     uint32_t T, ntiles, nstiles;
     uint32_t per;                    // tiles per CTA (contiguous run)
     uint32_t pool_cap;               // candidate slots per CTA
+    uint32_t pool_smem_words;        // words of shared memory reserved for one bit per candidate slot
+    uint32_t ntab;                   // T if the tile tables fit in shared memory, else 0
     const uint32_t* small_ids;
     uint32_t n_small;
     const float* g;
@@ -94,6 +96,8 @@ k_topk_multi(MultiArgs a) {
     uint32_t* const rec2 = rec + (size_t)a.per * kWarps;                       // [per*kWarps] counts, later slots
     uint32_t* const seg = rec2 + (size_t)a.per * kWarps;                       // [per][kSegWords]
     uint32_t* const sent_bits = seg + (size_t)a.per * kSegWords;               // [ceil(pool_cap / 32)]
+    uint32_t* const tab_tile0 = sent_bits + (a.pool_smem_words);               // [ntab] first tile of every tensor
+    uint32_t* const tab_stile0 = tab_tile0 + a.ntab;                           // [ntab] first sample tile
     uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -105,8 +109,22 @@ k_topk_multi(MultiArgs a) {
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     for (uint32_t i = tid; i < ntl * kWarps; i += kBlock) { rec[i] = 0u; rec2[i] = 0u; }
     if (tid == 0) { s_used = 0u; s_cnt = 0u; }
+    // first tile / first sample tile of every tensor, so that "which tensor owns this tile" is a
+    // binary search in shared memory instead of a chain of dependent global loads
+    for (uint32_t t = tid; t < a.ntab; t += kBlock) {
+        tab_tile0[t] = a.desc[t].tile0;
+        tab_stile0[t] = a.desc[t].stile0;
+    }
     phase_stamp(hdr, n_stamp);
     __syncthreads();
+    auto owner = [&](const uint32_t* tab, uint32_t tile) -> uint32_t {    // last t with tab[t] <= tile
+        uint32_t lo = 0, hi = a.ntab;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (tab[mid] <= tile) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
 
     // ---------------------------------------------------------------- sample: coarse histogram per tensor
     if (a.nstiles) {
@@ -118,7 +136,7 @@ k_topk_multi(MultiArgs a) {
             if (t == 0xFFFFFFFFu || st >= d.stile0 + d.nstiles) {
                 if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));
                 __syncthreads();
-                t = find_tensor<SampleSpace>(a.desc, a.T, st);
+                t = a.ntab ? owner(tab_stile0, st) : find_tensor<SampleSpace>(a.desc, a.T, st);
                 d = a.desc[t];
             }
             const uint32_t ngroups = (d.n + 3u) >> 2;
@@ -174,7 +192,7 @@ k_topk_multi(MultiArgs a) {
             if (cur == 0xFFFFFFFFu || tile >= d.tile0 + d.ntiles) {
                 if (open) flush_hist(sm, a.bhist + (size_t)cur * kHistBins, 2048);
                 open = false;
-                cur = find_tensor(a.desc, a.T, tile);
+                cur = a.ntab ? owner(tab_tile0, tile) : find_tensor(a.desc, a.T, tile);
                 d = a.desc[cur];
                 if (d.kind != kKindSmall) {
                     // bracket of this tensor from its sample histogram: tau = lower edge of the bin of
