@@ -169,3 +169,50 @@ def test_rejects_misaligned_and_null_buffers():
         args[key] = bad
         assert plan.compress_ptr(**args) == api.GC_E_INVALID
     torch.cuda.synchronize()
+
+
+def test_maximum_size_properties():
+    """The largest plan the ABI accepts (2^31 - 1 elements, 8.6 GB per buffer): far beyond what
+    the CPU oracle can rank in a test, so the result is checked through the properties that
+    define it -- exactly k pairs, ascending indices, values are bit copies of a = g + r, every
+    sent magnitude key >= every unsent one with ties going to the lower index, residual = a with
+    +0 at the sent indices -- all evaluated with plain torch ops on the device."""
+    n = (1 << 31) - 1
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * (1 << 30):
+        pytest.skip("needs about 70 GB of device memory")
+    plan = api.Plan([n], 1e-4, device=0)
+    k = plan.tensor_k()[0]
+    assert k == oracle.k_from_density(n, 1e-4) and plan.total_n == n
+    gen = torch.Generator(device="cuda").manual_seed(2024)
+    g = torch.empty(n, device="cuda")
+    chunk = 1 << 28
+    for lo in range(0, n, chunk):
+        g[lo:lo + chunk].normal_(0.0, 1.0, generator=gen)
+    r = torch.zeros(n, device="cuda")
+    ws = plan.alloc_workspace()
+    idx, val, cnt = plan.alloc_outputs()
+    for step in range(2):
+        a = g + r                                           # what the fold computes (one rounded add)
+        plan.compress(g, r, idx, val, cnt, ws)
+        st, det = plan.last_status(ws)
+        assert st == api.GC_OK, (st, det)
+        assert cnt.cpu().tolist()[:2] == [k, k]
+        i64 = idx[:k].to(torch.int64) & 0xFFFFFFFF
+        assert bool((i64[1:] > i64[:-1]).all()) and int(i64[-1]) < n
+        assert torch.equal(val[:k].view(torch.int32), a[i64].view(torch.int32))
+        sent = torch.zeros(n, dtype=torch.bool, device="cuda")
+        sent[i64] = True
+        assert bool((r[i64].view(torch.int32) == 0).all())                  # +0.0 exactly
+        assert torch.equal(r[~sent].view(torch.int32), a[~sent].view(torch.int32))
+        key = a.view(torch.int32) & 0x7FFFFFFF
+        t_key = int(key[i64].min())
+        unsent_max = int(key[~sent].max())
+        assert unsent_max <= t_key
+        if unsent_max == t_key:                             # ties at the threshold: lower indices were taken
+            tie = key == t_key
+            last_sent_tie = int(torch.nonzero(tie & sent).max())
+            first_unsent_tie = int(torch.nonzero(tie & ~sent).min())
+            assert last_sent_tie < first_unsent_tie
+        del a, sent, key
+    torch.cuda.empty_cache()
