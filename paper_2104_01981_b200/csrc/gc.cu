@@ -11,6 +11,7 @@
 #include "gc_multi.cuh"
 #include "gc_threshold.cuh"
 #include "gc_thr_single.cuh"
+#include "gc_thr_multi.cuh"
 #include "gc_decode.cuh"
 
 using namespace gc;
@@ -28,6 +29,7 @@ struct gc_plan_s {
     TensorDesc* d_desc = nullptr;
     uint32_t* d_small = nullptr;            // ids of the small tensors (device), n_small entries
     std::vector<uint32_t> small_ids;
+    std::vector<uint32_t> reg_ids;          // tensors with elements that are not small (device copy follows the small ids)
     uint32_t nstiles = 0, ngroups = 0;
     uint32_t cand_cap = 0, cand_cap_alloc = 0;
     uint32_t n_sampled = 0;                 // tensors with a sample
@@ -49,6 +51,9 @@ struct gc_plan_s {
     int grid_thr_single_max = 0;
     uint32_t thr_grid = 0, thr_maxt = 0, thr_pool = 0, thr_rounds = 0;    // one-tensor threshold kernel (0 = no)
     size_t thr_smem = 0;
+    int grid_thr_multi_max = 0;
+    uint32_t thrm_grid = 0, thrm_per = 0, thrm_pool = 0, thrm_ntab = 0;   // many-tensor threshold kernel (0 = no)
+    size_t thrm_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
     uint32_t multi_ntab = 0;
     uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0;       // 0 = plan does not qualify
@@ -150,6 +155,7 @@ void finish_layout(gc_plan_s* p) {
     uint64_t stile0 = 0, group0 = 0, ccap_total = 0;
     p->n_sampled = 0;
     p->small_ids.clear();
+    p->reg_ids.clear();
     for (uint32_t t = 0; t < p->T; ++t) {
         TensorDesc& d = p->desc[t];
         d.kind = kKindRegular; d.pad = 0;
@@ -169,6 +175,7 @@ void finish_layout(gc_plan_s* p) {
                 m = (nsg - 1) * 4 + std::min<uint64_t>(4, d.n - last_first);
             }
             d.srank = (uint32_t)k_rule(m, p->density);
+            if (d.n > 0 && d.n < kSmallMax && p->T >= 2) d.kind = kKindSmall;    // one CTA finishes it (many-tensor kernel)
         }
         uint64_t nst = 0;
         if (d.sstride) {
@@ -180,6 +187,7 @@ void finish_layout(gc_plan_s* p) {
         d.stile0 = (uint32_t)stile0; d.nstiles = (uint32_t)nst;
         d.group0 = (uint32_t)group0; d.ngroups = (d.ntiles + kWarps - 1) / kWarps;
         if (d.kind == kKindSmall && d.n > 0) p->small_ids.push_back(t);
+        if (d.kind != kKindSmall && d.n > 0) p->reg_ids.push_back(t);
         stile0 += nst; group0 += d.ngroups; ccap_total += ccap;
     }
     p->nstiles = (uint32_t)stile0;
@@ -191,8 +199,8 @@ void finish_layout(gc_plan_s* p) {
         // one-tensor threshold plans keep a hit list: about k hits are expected (the sample says so),
         // up to the capacity factor are sent; the rest is slack for up to 1024 CTA regions
         ccap_total = 0;
-        if (p->T == 1 && p->desc[0].n > 0)
-            ccap_total = std::min<uint64_t>(0x7FFFFFFFull, (uint64_t)(2.5 * (double)p->desc[0].cap) + (1u << 20));
+        if (p->T >= 1 && p->total_cap > 0)
+            ccap_total = std::min<uint64_t>(0x7FFFFFFFull, (uint64_t)(1.25 * (double)p->total_cap) + (1u << 20));
     }
     if (p->cand_cap_alloc == 0) p->cand_cap_alloc = (uint32_t)ccap_total;   // fixed at plan creation
     p->cand_cap = (uint32_t)std::min<uint64_t>(ccap_total, p->cand_cap_alloc);
@@ -210,7 +218,7 @@ void finish_layout(gc_plan_s* p) {
     p->off_fine = p->control_bytes;
     p->control_bytes = align_up(p->off_fine + (T == 1 ? sizeof(uint32_t) * (size_t)kFineBins : 0), 256);
     // many-tensor kernel: sample and band histogram per tensor, short-list lengths
-    const size_t multi_hist = (T >= 2 && p->mode == GC_TOPK) ? sizeof(uint32_t) * (size_t)kHistBins * T : 0;
+    const size_t multi_hist = T >= 2 ? sizeof(uint32_t) * (size_t)kHistBins * T : 0;
     p->off_shist = p->control_bytes;
     p->off_bhist = align_up(p->off_shist + multi_hist, 256);
     p->off_midn = align_up(p->off_bhist + multi_hist, 256);
@@ -268,6 +276,35 @@ void plan_thr_single(gc_plan_s* p) {
     p->thr_smem = (size_t)maxt * (2 * kWarps + 2) * sizeof(uint32_t);
 }
 
+// Decides whether a threshold plan can use the many-tensor kernel and with which geometry.
+void plan_thr_multi(gc_plan_s* p) {
+    p->thrm_grid = 0;
+    if (p->mode != GC_THRESHOLD || p->T < 2 || p->grid_thr_multi_max <= 0 || p->ntiles == 0) return;
+    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_thr_multi_max, p->ntiles);
+    const uint32_t per = (p->ntiles + G - 1) / G;
+    if (per > kMultiMaxPer) return;
+    // one CTA ranks a whole tensor's kept sample keys: keep that bounded
+    for (uint32_t t : p->reg_ids)
+        if (p->desc[t].nstiles > 128 || p->desc[t].sstride == 0) return;
+    const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
+    // expected hits of the busiest CTA: about k per tensor, spread over its tiles
+    double worst = 0.0;
+    uint32_t t = 0;
+    for (uint32_t b = 0; b < G; ++b) {
+        double e = 0.0;
+        for (uint32_t tile = b * per; tile < std::min<uint32_t>(p->ntiles, (b + 1) * per); ++tile) {
+            while (t + 1 < p->T && (p->desc[t].ntiles == 0 || tile >= p->desc[t].tile0 + p->desc[t].ntiles)) ++t;
+            const TensorDesc& d = p->desc[t];
+            if (d.kind != kKindSmall && d.ntiles) e += std::min<double>(kTile, (double)d.k / (double)d.ntiles);
+        }
+        worst = std::max(worst, e);
+    }
+    if ((double)pool < 2.0 * worst + 512.0) return;
+    p->thrm_grid = G; p->thrm_per = per; p->thrm_pool = pool;
+    p->thrm_ntab = p->T <= kMultiMaxTab ? p->T : 0u;
+    p->thrm_smem = (size_t)per * kMultiRowBytes + 2 * sizeof(uint32_t) * (size_t)p->thrm_ntab;
+}
+
 // Decides whether the plan can use the many-tensor kernel and with which geometry.
 void plan_multi(gc_plan_s* p) {
     p->multi_grid = 0;
@@ -309,6 +346,9 @@ int upload_table(gc_plan_s* p) {
                                cudaMemcpyHostToDevice);
     if (e == cudaSuccess && !p->small_ids.empty())
         e = cudaMemcpy(p->d_small, p->small_ids.data(), sizeof(uint32_t) * p->small_ids.size(),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !p->reg_ids.empty())
+        e = cudaMemcpy(p->d_small + p->T, p->reg_ids.data(), sizeof(uint32_t) * p->reg_ids.size(),
                        cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { p->last_cuda_error = (int)e; (void)cudaGetLastError(); return GC_E_CUDA; }
     return GC_OK;
@@ -383,7 +423,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     if (e == cudaSuccess && n_tensors > 0) {
         e = cudaMalloc(reinterpret_cast<void**>(&p->d_desc), sizeof(TensorDesc) * (size_t)n_tensors);
         if (e == cudaSuccess)
-            e = cudaMalloc(reinterpret_cast<void**>(&p->d_small), sizeof(uint32_t) * (size_t)n_tensors);
+            e = cudaMalloc(reinterpret_cast<void**>(&p->d_small), sizeof(uint32_t) * 2 * (size_t)n_tensors);
         if (e == cudaSuccess) e = upload_table(p) == GC_OK ? cudaSuccess : cudaErrorUnknown;
     }
     if (e != cudaSuccess) {
@@ -423,6 +463,17 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
                 (void)cudaGetLastError();
         }
         plan_thr_single(p);
+        p->grid_thr_multi_max = 0;
+        if (coop) {
+            int nb = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_threshold_multi, kBlock,
+                                                              kMultiMaxPer * kMultiRowBytes + 8 * kMultiMaxTab) ==
+                    cudaSuccess && nb >= 1)
+                p->grid_thr_multi_max = p->sm_count * nb;
+            else
+                (void)cudaGetLastError();
+        }
+        plan_thr_multi(p);
         p->grid_multi_max = 0;
         if (coop) {
             int nb = 0;
@@ -550,6 +601,26 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         Timed tm(p, s, GC_K_FUSED);
         GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_threshold_single, dim3(p->thr_grid), dim3(kBlock),
                                                args, p->thr_smem, s));
+        return GC_OK;
+    }
+    if (p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thrm_grid > 0) {
+        // several tensors: sample, exact thresholds, fold + hits and emission in one cooperative launch
+        ThrMultiArgs ta;
+        ta.desc = p->d_desc; ta.T = p->T; ta.ntiles = nt; ta.nstiles = p->nstiles;
+        ta.per = p->thrm_per; ta.pool_cap = p->thrm_pool; ta.ntab = p->thrm_ntab;
+        ta.small_ids = p->d_small; ta.n_small = (uint32_t)p->small_ids.size();
+        ta.reg_ids = p->d_small + p->T; ta.n_reg = (uint32_t)p->reg_ids.size();
+        ta.g = grad; ta.r = residual; ta.out_idx = out_idx; ta.out_val = out_val; ta.out_count = out_count;
+        ta.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+        ta.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
+        ta.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
+        ta.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+        ta.tsel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+        ta.ws = ws;
+        void* args[] = {&ta};
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_threshold_multi, dim3(p->thrm_grid), dim3(kBlock),
+                                               args, p->thrm_smem, s));
         return GC_OK;
     }
     if (p->mode == GC_THRESHOLD) {

@@ -10,7 +10,8 @@ namespace gc {
 // look-back exchange, so output slots are index-ordered and a truncated tensor keeps exactly
 // its first `cap` hits.  tau of tensor t = ssel[t].T, or `tau_fixed` when ssel is null.
 // FOLD: a = g + r is computed here (and stored); otherwise r already holds a.
-template <bool FOLD>
+// SKIP_SMALL: tensors of kind "small" were finished elsewhere and are left alone.
+template <bool FOLD, bool SKIP_SMALL = false>
 static __device__ void threshold_emit_body(const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
                                            const float* __restrict__ g, float* __restrict__ r,
                                            uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
@@ -35,6 +36,7 @@ static __device__ void threshold_emit_body(const TensorDesc* __restrict__ desc, 
         if (tile >= ntiles) break;
         const uint32_t t = find_tensor(desc, T, tile);
         const TensorDesc d = desc[t];
+        if (SKIP_SMALL && d.kind == kKindSmall) continue;
         const uint32_t tau = ssel != nullptr ? ssel[t].T : tau_fixed;
         const TileGeom tg = tile_geom(d, tile - d.tile0);
         Tile tl;

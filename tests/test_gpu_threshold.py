@@ -129,3 +129,22 @@ def test_threshold_one_tensor_mild_truncation_and_two_valued_input():
     g[torch.rand(n, generator=torch.Generator().manual_seed(3)) < 0.1] = -3.0
     check_threshold([n], 0.5, [g, g])
     check_threshold([n], 0.05, [g])
+
+
+def test_threshold_many_tensors_hit_list_overflow_and_truncation():
+    """Several tensors in one plan (the fused many-tensor kernel).  In the large ones the sample
+    only sees tiny values, so nearly every element is a hit: the hit list overflows, the
+    look-back pass takes over (leaving the single-tile tensors, which are already done, alone),
+    and the capacity cuts every large tensor to a prefix."""
+    sizes = [70_001, 5, 300_000, 1000, 64, 131_073, 4092, 4093, 0, 9000]
+    n = sum(sizes)
+    g = randn(n, 77)
+    off = 0
+    for sz in sizes:
+        if sz > 65536:                      # stride 64 applies (smaller tensors are sampled in full)
+            loc = torch.arange(sz)
+            g[off:off + sz][((loc >> 2) % 64) == 0] *= 1e-3
+        off += sz
+    check_threshold(sizes, 0.01, [g, g], expect_truncated=True)
+    # the same plan on ordinary data: no overflow, mild or no truncation
+    check_threshold(sizes, 0.01, [randn(n, 78 + s) for s in range(3)], cap_factor=1.0)
