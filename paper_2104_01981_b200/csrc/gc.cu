@@ -133,7 +133,7 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
     const uint64_t n = d.n;
     d.sstride = 0; d.srank = 0;
     *ccap = n;
-    if (n < kSmallMax) { d.kind = kKindSmall; *ccap = 0; return; }   // one CTA does the whole tensor
+    if (d.ntiles <= 1) { d.kind = kKindSmall; *ccap = 0; return; }   // fits one tile: one CTA does the whole tensor
     uint64_t target = std::min<uint64_t>(target_max, std::max<uint64_t>(n / 128, std::min<uint64_t>(8192, n / 2)));
     uint64_t stride = std::max<uint64_t>(1, n / target);
     uint64_t groups = (n + 3) / 4;
@@ -175,7 +175,7 @@ void finish_layout(gc_plan_s* p) {
                 m = (nsg - 1) * 4 + std::min<uint64_t>(4, d.n - last_first);
             }
             d.srank = (uint32_t)k_rule(m, p->density);
-            if (d.n > 0 && d.n < kSmallMax && p->T >= 2) d.kind = kKindSmall;    // one CTA finishes it (many-tensor kernel)
+            if (d.n > 0 && d.ntiles == 1 && p->T >= 2) d.kind = kKindSmall;    // one CTA finishes it (many-tensor kernel)
         }
         uint64_t nst = 0;
         if (d.sstride) {
@@ -695,6 +695,8 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         ma.pool_cap = std::min<uint32_t>(p->multi_pool, p->cand_cap / p->multi_grid);     // each CTA's share
         ma.pool_smem_words = (p->multi_pool + 31) / 32; ma.ntab = p->multi_ntab;
         ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();
+        ma.reg_ids = p->d_small + p->T; ma.n_reg = (uint32_t)p->reg_ids.size();
+        ma.brk = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
         ma.g = grad; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
         ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
         ma.mid = reinterpret_cast<uint2*>(wb + p->off_mmid);

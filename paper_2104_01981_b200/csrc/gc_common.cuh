@@ -49,8 +49,8 @@ struct TensorDesc {          // one per tensor, immutable, plan-owned device mem
     uint32_t pad;
 };
 constexpr uint32_t kKindRegular = 0u, kKindSmall = 1u;
-constexpr uint32_t kSmallMax = kTile - 3;     // tensors below this many elements are "small": whatever
-                                              // their offset, they lie inside one tile
+constexpr uint32_t kSmallMax = kTile - 3;     // tensors below this many elements always lie inside one tile,
+                                              // whatever their offset; "small" = fits one tile
 static_assert(sizeof(TensorDesc) == 64, "tensor table entry is 64 bytes");
 
 struct TensorSel {           // one per tensor, in the workspace, rewritten every call

@@ -2,15 +2,17 @@
 //
 // The scheme of the one-tensor kernel, applied per tensor: sample -> bracket [tau, tau_hi) and a
 // guess tau_z of the threshold -> fold + candidates + band histogram -> band bin of the k-th
-// key -> short list ranked by every CTA that needs it -> index-ordered emission; three grid
+// key -> short list ranked by every CTA that needs it -> index-ordered emission; four grid
 // barriers.  What differs:
 //   * CTA b owns a contiguous run of tiles, so it sees one to a few tensors ("segments") and
 //     keeps one small record per segment in shared memory;
 //   * all histograms and short lists exist once per tensor in global memory; a CTA only looks
 //     at those of its own segments;
-//   * the sample is a coarse histogram only (top 11 key bits), so tau and tau_hi are bin edges:
-//     up to twice the candidates of an exact bracket, which is still a few per mille of the
-//     tensor; tau_z is interpolated inside its bin (it is only a guess);
+//   * the sample is a coarse histogram (top 11 key bits) per tensor plus the kept sampled keys;
+//     after the first barrier ONE CTA per tensor computes the bracket (the kept keys give tau a
+//     second radix level; tau_hi is a bin edge; tau_z is interpolated inside its bin -- it is
+//     only a guess) and publishes it, so the fold pass of the many CTAs that share a tensor
+//     only reads three words per segment;
 //   * the slot of a segment's first entry = what the tensor's earlier tiles send: the sum of
 //     their published counts + the sent short-list entries that lie before the segment;
 //   * tensors that fit one tile ("small") are finished by one CTA each between the arrival at
@@ -37,6 +39,9 @@ struct MultiArgs {
     uint32_t ntab;                   // T if the tile tables fit in shared memory, else 0
     const uint32_t* small_ids;
     uint32_t n_small;
+    const uint32_t* reg_ids;         // the tensors that are not small (and not empty)
+    uint32_t n_reg;
+    TensorSel* brk;                  // [T] bracket of every such tensor: .prefix = tau, .krem = tau_z, .T = shift
     const float* g;
     float* r;
     uint32_t* out_idx;
@@ -179,6 +184,72 @@ k_topk_multi(MultiArgs a) {
     if (!grid_wait(hdr, passed, &sm.ok)) return;
     phase_stamp(hdr, n_stamp);
 
+    // ---------------------------------------------------------------- bracket per tensor, one CTA each
+    // tau = the srank-th largest sampled key (22 bits when the kept keys allow the second radix
+    // level, else the lower edge of its coarse bin), tau_hi = upper edge of the bin of the key
+    // that stays below the expected rank by the same margin, tau_z inside the bin of the
+    // expected rank itself; published as (tau, tau_z, shift of the band histogram).
+    for (uint32_t q = b; q < a.n_reg; q += G) {
+        const uint32_t cur = a.reg_ids[q];
+        const TensorDesc d = a.desc[cur];
+        uint32_t tau = 0, tau_z = 0;
+        int shift = 0;
+        {
+            uint32_t tau_hi = 0x80000000u;
+            if (d.sstride != 0u) {
+                const uint32_t ngroups = (d.n + 3u) >> 2;
+                const float msamp = 4.0f * (float)((ngroups + d.sstride - 1) / d.sstride);
+                const float ks = (float)d.k * msamp / (float)d.n;
+                const float hi = floorf(ks - 6.0f * sqrtf(ks) - 8.0f);
+                // (a sample too small for that margin: the largest sampled key bounds the band instead)
+                const uint32_t want[3] = {d.srank, hi >= 1.0f ? (uint32_t)hi : 1u, max(1u, (uint32_t)ceilf(ks))};
+                Picked pk[3];
+                block_select_multi<(1 << level_bits(0)), 3>(sm, a.shist + (size_t)cur * kHistBins, want, pk);
+                if (pk[0].ok) tau = pk[0].bin << level_shift(0);
+                if (pk[0].ok && d.nstiles <= kRefineTiles) {
+                    // second radix level of the lower bracket over the kept sample keys:
+                    // tau gets 22 significant bits
+                    const uint4* sk = a.skeys + (size_t)d.stile0 * kBlock;
+                    const uint32_t nk = d.nstiles * kBlock, bin0 = pk[0].bin;
+                    for (uint32_t q0 = tid; q0 < nk; q0 += 4 * kBlock) {
+                        uint4 kv[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            kv[u] = q0 + u * kBlock < nk ? ld_cg(sk + q0 + u * kBlock)
+                                                         : make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint32_t kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if ((kk[e] >> level_shift(0)) == bin0)
+                                    atomicAdd(&sm.hist[(kk[e] >> (level_shift(0) - 11)) & 2047u], 1u);
+                        }
+                    }
+                    __syncthreads();
+                    uint32_t bin1, above1;
+                    const bool ok1 = block_select<2048, true>(sm, sm.hist, d.srank - pk[0].above, bin1, above1);
+                    for (int i2 = tid; i2 < 2048; i2 += kBlock) sm.hist[i2] = 0u;
+                    __syncthreads();
+                    if (ok1) tau |= bin1 << (level_shift(0) - 11);
+                }
+                if (pk[1].ok) tau_hi = (pk[1].bin + 1u) << level_shift(0);
+                if (pk[2].ok) {
+                    const float pos = ((float)(want[2] - pk[2].above) - 0.5f) / (float)pk[2].count;   // from the top of the bin
+                    tau_z = (pk[2].bin << level_shift(0)) +
+                            (uint32_t)((1.0f - pos) * (float)((1u << level_shift(0)) - 1u));
+                }
+            }
+            if (tau_z < tau) tau_z = tau;
+            if (tau_hi <= tau) tau_hi = 0x80000000u;
+            shift = 0;
+            while (((tau_hi - tau) >> shift) > 2046u) ++shift;
+        }
+        if (tid == 0) { a.brk[cur].prefix = tau; a.brk[cur].krem = tau_z; a.brk[cur].T = (uint32_t)shift; }
+    }
+    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    phase_stamp(hdr, n_stamp);
+
     // ---------------------------------------------------------------- fold + candidates, segment by segment
     uint32_t nseg = 0;
     {
@@ -195,60 +266,10 @@ k_topk_multi(MultiArgs a) {
                 cur = a.ntab ? owner(tab_tile0, tile) : find_tensor(a.desc, a.T, tile);
                 d = a.desc[cur];
                 if (d.kind != kKindSmall) {
-                    // bracket of this tensor from its sample histogram: tau = lower edge of the bin of
-                    // the srank-th largest sampled key, tau_hi = upper edge of the bin of the one that
-                    // stays below the expected rank by the same margin, tau_z inside the bin of the
-                    // expected rank itself
-                    uint32_t tau_hi = 0x80000000u;
-                    tau = 0; tau_z = 0;
-                    if (d.sstride != 0u) {
-                        const uint32_t ngroups = (d.n + 3u) >> 2;
-                        const float msamp = 4.0f * (float)((ngroups + d.sstride - 1) / d.sstride);
-                        const float ks = (float)d.k * msamp / (float)d.n;
-                        const float hi = floorf(ks - 6.0f * sqrtf(ks) - 8.0f);
-                        // (a sample too small for that margin: the largest sampled key bounds the band instead)
-                        const uint32_t want[3] = {d.srank, hi >= 1.0f ? (uint32_t)hi : 1u, max(1u, (uint32_t)ceilf(ks))};
-                        Picked pk[3];
-                        block_select_multi<(1 << level_bits(0)), 3>(sm, a.shist + (size_t)cur * kHistBins, want, pk);
-                        if (pk[0].ok) tau = pk[0].bin << level_shift(0);
-                        if (pk[0].ok && d.nstiles <= kRefineTiles) {
-                            // second radix level of the lower bracket over the kept sample keys:
-                            // tau gets 22 significant bits (sm.hist is free between segments)
-                            const uint4* sk = a.skeys + (size_t)d.stile0 * kBlock;
-                            const uint32_t nk = d.nstiles * kBlock, bin0 = pk[0].bin;
-                            for (uint32_t q0 = tid; q0 < nk; q0 += 4 * kBlock) {
-                                uint4 kv[4];
-#pragma unroll
-                                for (int u = 0; u < 4; ++u)
-                                    kv[u] = q0 + u * kBlock < nk ? ld_cg(sk + q0 + u * kBlock)
-                                                                 : make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    const uint32_t kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e)
-                                        if ((kk[e] >> level_shift(0)) == bin0)
-                                            atomicAdd(&sm.hist[(kk[e] >> (level_shift(0) - 11)) & 2047u], 1u);
-                                }
-                            }
-                            __syncthreads();
-                            uint32_t bin1, above1;
-                            const bool ok1 = block_select<2048, true>(sm, sm.hist, d.srank - pk[0].above, bin1, above1);
-                            for (int i2 = tid; i2 < 2048; i2 += kBlock) sm.hist[i2] = 0u;
-                            __syncthreads();
-                            if (ok1) tau |= bin1 << (level_shift(0) - 11);
-                        }
-                        if (pk[1].ok) tau_hi = (pk[1].bin + 1u) << level_shift(0);
-                        if (pk[2].ok) {
-                            const float pos = ((float)(want[2] - pk[2].above) - 0.5f) / (float)pk[2].count;   // from the top of the bin
-                            tau_z = (pk[2].bin << level_shift(0)) +
-                                    (uint32_t)((1.0f - pos) * (float)((1u << level_shift(0)) - 1u));
-                        }
-                    }
-                    if (tau_z < tau) tau_z = tau;
-                    if (tau_hi <= tau) tau_hi = 0x80000000u;
-                    shift = 0;
-                    while (((tau_hi - tau) >> shift) > 2046u) ++shift;
+                    // bracket of this tensor, published by the CTA that computed it
+                    tau = ld_cg(&a.brk[cur].prefix);
+                    tau_z = ld_cg(&a.brk[cur].krem);
+                    shift = (int)ld_cg(&a.brk[cur].T);
                     if (tid == 0) {
                         uint32_t* s = seg + (size_t)nseg * kSegWords;
                         const TileGeom tg0 = tile_geom(d, tile - d.tile0);
