@@ -171,7 +171,8 @@ int gc_compress(gc_plan_t *plan, const float *grad, float *residual,
  *              by the caller -- this call does not reset the status word
  * With count = NULL every list must be exactly as gc_compress wrote it in top-k mode (total_cap
  * pairs, ascending index): the dense buffer is then built tile by tile in shared memory and
- * written once.  With count arrays the sets are applied one launch per worker instead.
+ * written once; so are one-tensor plans with count arrays (the list's length is its count).
+ * Many-tensor plans with count arrays are applied one launch per worker instead.
  * An index >= total_n (or a list that is not ascending) is skipped and GC_E_INVALID is recorded
  * in the device status.
  * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_CUDA.  Asynchronous.

@@ -794,11 +794,16 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
     const int nbuf = W <= 2 ? 2 : 1;      // few workers per tile: overlap the tile's way out with the next tile
-    if (count == nullptr && W > 0 && p->total_cap > 0 && p->path != GC_PATH_EXACT && p->grid_decode[nbuf - 1] > 0) {
-        // every list holds exactly total_cap pairs in ascending index: tiled decode, dense buffer
+    if ((count == nullptr || p->T == 1) && W > 0 && p->total_cap > 0 && p->path != GC_PATH_EXACT &&
+        p->grid_decode[nbuf - 1] > 0) {
+        // every list is one run of pairs in ascending index (total_cap of them, or - one-tensor plans
+        // with count arrays - as many as the list's first count says): tiled decode, dense buffer
         // written once (and not read at all when it is cleared first)
         DecodeLists ls;
-        for (uint32_t w = 0; w < 64; ++w) { ls.idx[w] = idx[w < W ? w : 0]; ls.val[w] = val[w < W ? w : 0]; }
+        for (uint32_t w = 0; w < 64; ++w) {
+            ls.idx[w] = idx[w < W ? w : 0]; ls.val[w] = val[w < W ? w : 0];
+            ls.len[w] = count != nullptr ? count[w < W ? w : 0] : nullptr;
+        }
         const uint32_t ntl = (uint32_t)((p->total_n + kDecTile - 1) / kDecTile);
         const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[nbuf - 1]);
         const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;

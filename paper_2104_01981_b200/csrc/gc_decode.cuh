@@ -23,6 +23,7 @@ constexpr size_t kDecTileBytes = kDecTile * sizeof(float);
 struct DecodeLists {
     const uint32_t* idx[64];
     const float* val[64];
+    const uint32_t* len[64];     // device: number of valid pairs of the list (its first word), or null = `cnt`
 };
 
 // Starts the copy of one finished tile to global memory and returns at once; the tile buffer
@@ -69,17 +70,18 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     // nbuf tile buffers: with two, one fills while the other drains (pays off when there are few
     // workers per tile; with many workers more resident CTAs are worth more than the overlap)
     extern __shared__ __align__(128) float s_tiles[];
-    __shared__ uint32_t s_cur[64];
+    __shared__ uint32_t s_cur[64], s_len[64];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
     const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
     const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
     if (t0 >= t1) return;
 
-    // where each worker's list enters this CTA's run of tiles
+    // length of each worker's list, and where it enters this CTA's run of tiles
     for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
-        const uint32_t c = warp_lower_bound(ls.idx[w], cnt, t0 * (uint32_t)kDecTile, lane);
-        if (lane == 0) s_cur[w] = c;
+        const uint32_t len = ls.len[w] != nullptr ? min(__ldg(ls.len[w]), cnt) : cnt;
+        const uint32_t c = warp_lower_bound(ls.idx[w], len, t0 * (uint32_t)kDecTile, lane);
+        if (lane == 0) { s_cur[w] = c; s_len[w] = len; }
     }
     // E consecutive threads serve one worker; passes of Wp workers cover W > 256 / E
     int Wp = 1;
@@ -89,6 +91,7 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     const int sub = tid % E;
     const bool live = my_w < W;
     __syncthreads();
+    const uint32_t my_len = live ? s_len[my_w] : 0u;
 
     for (uint32_t tl = t0; tl < t1; ++tl) {
         float* const s_tile = s_tiles + (nbuf == 2 ? ((tl - t0) & 1u) : 0u) * kDecTile;
@@ -121,7 +124,7 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         for (int rd = 0; rd < kDecRounds; ++rd) {
             const uint32_t p = c0 + (uint32_t)(rd * E + sub);
             ix[rd] = 0xFFFFFFFFu; v[rd] = 0.f;
-            if (live && p < cnt) { ix[rd] = __ldg(ls.idx[my_w] + p); v[rd] = __ldg(ls.val[my_w] + p); }
+            if (live && p < my_len) { ix[rd] = __ldg(ls.idx[my_w] + p); v[rd] = __ldg(ls.val[my_w] + p); }
         }
 #pragma unroll
         for (int rd = 0; rd < kDecRounds; ++rd) nin += ix[rd] < hi;       // sorted lists: the ins are a prefix
@@ -145,12 +148,13 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         } else {
             for (uint32_t q = 0; q < W; ++q) {
                 uint32_t c = s_cur[q];
+                const uint32_t qlen = s_len[q];
                 __syncthreads();
                 while (true) {
                     const uint32_t pp = c + (uint32_t)tid;
                     uint32_t ix2 = 0xFFFFFFFFu;
                     float v2 = 0.f;
-                    if (pp < cnt) { ix2 = __ldg(ls.idx[q] + pp); v2 = __ldg(ls.val[q] + pp); }
+                    if (pp < qlen) { ix2 = __ldg(ls.idx[q] + pp); v2 = __ldg(ls.val[q] + pp); }
                     const bool in2 = ix2 < hi;
                     if (in2) {
                         if (ix2 >= lo) s_tile[ix2 - lo] = __fadd_rn(s_tile[ix2 - lo], v2);
@@ -172,7 +176,7 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         }
         __syncthreads();
     }
-    if (t1 == ntl && tid < (int)W && s_cur[tid] < cnt)
+    if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
         record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
     if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }

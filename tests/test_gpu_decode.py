@@ -179,3 +179,32 @@ def test_config4_eight_resnet_workers_decode():
                                workers[0].ws)
     want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
     assert np.array_equal(to_np_u32(out), bits(want))
+
+
+@pytest.mark.parametrize("W", [1, 3, 8])
+def test_one_tensor_lists_with_counts_use_their_length(W):
+    """Threshold-mode lists of a one-tensor plan: the slots hold `cap` pairs but only the first
+    count[0] are valid; whatever lies behind them (here: junk indices) must not be applied."""
+    n = 3_000_001
+    plan = api.Plan([n], 0.001, mode=api.GC_THRESHOLD, device=0)
+    cap = plan.tensor_cap()[0]
+    ws = plan.alloc_workspace()
+    pairs, d_idx, d_val, d_cnt = [], [], [], []
+    for w in range(W):
+        m = [cap, cap // 2 + 17 * w, 0, 1][(w + 1) % 4] if W > 1 else cap // 3
+        idx, val = synth.sparse_set([n], [m], seed=40 + w)
+        pairs.append((idx, val))
+        full_idx = np.full(cap, 0xFFFFFFFF, np.uint32); full_idx[:m] = idx
+        full_idx[m:] = np.arange(cap - m, dtype=np.uint32)[::-1] * 3 % n          # junk, not even ascending
+        full_val = np.full(cap, 1e30, np.float32); full_val[:m] = val
+        d_idx.append(torch.from_numpy(full_idx.view(np.int32)).cuda())
+        d_val.append(torch.from_numpy(full_val).cuda())
+        d_cnt.append(torch.tensor([m, m], dtype=torch.int32, device="cuda"))
+    out = torch.full((n,), 2.0, device="cuda")
+    for zero_first in (True, False):
+        before = out.cpu().numpy().copy()
+        plan.decompress_accumulate(d_idx, d_val, d_cnt, out, zero_first, ws)
+        want = oracle.decode_accumulate(pairs, before, zero_first)
+        assert np.array_equal(to_np_u32(out), bits(want)), (W, zero_first)
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_OK
