@@ -148,3 +148,22 @@ def test_threshold_many_tensors_hit_list_overflow_and_truncation():
     check_threshold(sizes, 0.01, [g, g], expect_truncated=True)
     # the same plan on ordinary data: no overflow, mild or no truncation
     check_threshold(sizes, 0.01, [randn(n, 78 + s) for s in range(3)], cap_factor=1.0)
+
+
+@pytest.mark.parametrize("seed", list(range(6)))
+def test_threshold_random_plans_match_the_oracle(seed):
+    """Seeded random plans for the threshold variant (sizes around the tile boundaries, empty
+    tensors, misaligned offsets, several densities, strides and capacity factors)."""
+    rng = np.random.default_rng(2000 + seed)
+    T = int(rng.integers(1, 30))
+    menu = [0, 1, 2, 5, 64, 1000, 4092, 4093, 4096, 4097, 8193, 16_384, 65_536, 65_537, 131_072, 300_007, 1_048_577]
+    sizes = [int(menu[int(rng.integers(0, len(menu)))]) for _ in range(T)]
+    if sum(sizes) == 0:
+        sizes[0] = 4097
+    density = float(rng.choice([1e-4, 1e-3, 0.01, 0.07]))
+    stride = int(rng.choice([0, 1, 7, 64]))
+    cap_factor = float(rng.choice([0.0, 1.0, 1.5, 3.0]))
+    n = sum(sizes)
+    scales = torch.cat([torch.full((s,), float(10.0 ** rng.integers(-2, 2))) for s in sizes])
+    grads = [randn(n, 6000 + 10 * seed + s) * scales for s in range(2)]
+    check_threshold(sizes, density, grads, stride=stride, cap_factor=cap_factor)

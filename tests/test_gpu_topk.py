@@ -216,3 +216,22 @@ def test_maximum_size_properties():
             assert last_sent_tie < first_unsent_tie
         del a, sent, key
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("seed", list(range(10)))
+def test_random_plans_match_the_oracle(seed):
+    """Seeded random plans: tensor counts, sizes around the tile and small-tensor boundaries,
+    empty tensors, misaligned offsets, densities from one in a million to one half, values on
+    very different scales per tensor.  Three error-feedback steps each, bit-exact."""
+    rng = np.random.default_rng(1000 + seed)
+    T = int(rng.integers(1, 40))
+    menu = [0, 1, 2, 3, 5, 63, 64, 1000, 4091, 4092, 4093, 4095, 4096, 4097, 8191, 8192, 8193, 12_289,
+            16_384, 50_001, 131_072, 300_007, 1_048_577]
+    sizes = [int(menu[int(rng.integers(0, len(menu)))]) for _ in range(T)]
+    if sum(sizes) == 0:
+        sizes[0] = 4097
+    density = float(rng.choice([1e-6, 1e-4, 1e-3, 0.01, 0.07, 0.5]))
+    n = sum(sizes)
+    scales = torch.cat([torch.full((s,), float(10.0 ** rng.integers(-3, 3))) for s in sizes])
+    grads = [randn(n, 5000 + 10 * seed + s) * scales for s in range(3)]
+    check_topk_against_oracle(sizes, density, grads)
