@@ -259,6 +259,26 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
         barrier()
         halves.append(e0.elapsed_time(e1) / args.steps)
     args.ms_compress, args.ms_decode = halves
+    # ---- timed region 1e: decode with momentum SGD fused behind it (top-k lists only)
+    args.ms_apply = None
+    if not thr:
+        param = torch.zeros(n, device=dev)
+        vel = torch.zeros(n, device=dev)
+
+        def apply_only(i: int):
+            plan.decompress_apply_momentum([o[0] for o in outs], [o[1] for o in outs], None, param, vel,
+                                           0.01, 0.9, 1.0 / W, ws, stream)
+
+        for i in range(3):
+            apply_only(i)
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            apply_only(i)
+        e1.record(stream)
+        barrier()
+        args.ms_apply = e0.elapsed_time(e1) / args.steps
+        del param, vel
 
     # ---- timed region 2: end to end through the host-buffer entry point
     if args.no_e2e:
@@ -359,6 +379,11 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     line["hbm_frac_of_8TBs"]["compress_ms_per_step"] = args.ms_compress
     line["hbm_frac_of_8TBs"]["decode_only"] = db / NOMINAL_HBM / (args.ms_decode * 1e-3)
     line["hbm_frac_of_8TBs"]["decode_ms_per_step"] = args.ms_decode
+    if getattr(args, "ms_apply", None):
+        ab = 16 * n + 8 * k * W                    # read and write parameter and velocity, read the pairs
+        line["fused_decode_momentum"] = {"ms_per_call": args.ms_apply, "bytes": ab,
+                                         "GB_per_s": ab / (args.ms_apply * 1e-3) / 1e9,
+                                         "frac_of_measured_peak": ab / (args.ms_apply * 1e-3) / 1e9 / peak}
     print(json.dumps(line))
 
 

@@ -193,6 +193,29 @@ int gc_last_status(gc_plan_t *plan, const void *workspace, void *stream,
                    int32_t *status, uint64_t *detail);
 
 /*
+ * gc_decompress_apply_momentum -- the decode with the optimizer fused behind it: the summed
+ * gradient is never written out.  For every element i:
+ *     s_i  = sum over workers w = 0..W-1, in that order, of the values sent for i (+0 if none)
+ *     v_i' = fl(fl(momentum * v_i) + fl(scale * s_i))
+ *     p_i' = fl(p_i - fl(lr * v_i'))
+ * (momentum SGD in its accumulate-then-step form; scale = 1 for a sum, 1/W for a mean; every
+ * operation rounded once, no fused multiply-add).  No counterpart in the source paper; it is
+ * the fusion a data-parallel step performs right after aggregation, and it replaces 24 bytes
+ * per element of traffic (write the sum, read it again with p and v, write p and v) by 16.
+ *   idx, val, count  as for gc_decompress_accumulate; count arrays only for one-tensor plans
+ *                    (GC_E_UNSUPPORTED otherwise)
+ *   param, velocity  device, fp32[total_n], 16-byte aligned, updated in place
+ *   workspace        device; only its status word is written (out-of-range or unordered
+ *                    index -> GC_E_INVALID recorded, the entry is skipped)
+ * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_UNSUPPORTED, GC_E_CUDA.
+ * Asynchronous.
+ */
+int gc_decompress_apply_momentum(gc_plan_t *plan, uint32_t W, const uint32_t *const *idx,
+                                 const float *const *val, const uint32_t *const *count,
+                                 float *param, float *velocity, float lr, float momentum, float scale,
+                                 void *workspace, void *stream);
+
+/*
  * gc_compress_host -- gc_compress for a gradient that lives in HOST memory, with the
  * compressed pairs returned to HOST memory (what a worker would hand to its network stack).
  * Enqueues, on the stream: copy host_grad -> grad_staging, gc_compress, copy the pairs

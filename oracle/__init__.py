@@ -134,3 +134,17 @@ def decode_accumulate(pairs: List[Tuple[np.ndarray, np.ndarray]], out: np.ndarra
     if rc:
         raise ValueError(f"oracle_decode_accumulate failed: {rc}")
     return out
+
+
+def decode_apply_momentum(pairs: List[Tuple[np.ndarray, np.ndarray]], param: np.ndarray, vel: np.ndarray,
+                          lr: float, momentum: float, scale: float) -> None:
+    """The decode followed by momentum SGD, in place on float32 ``param`` and ``vel``:
+    s = worker-ordered sum of the sparse sets (+0 where nothing was sent),
+    v' = fl(fl(momentum v) + fl(scale s)), p' = fl(p - fl(lr v')): one rounding per operation.
+    Written as the plain definition: the dense sum first, then three elementwise numpy steps."""
+    assert param.dtype == np.float32 and vel.dtype == np.float32
+    f = np.float32
+    s = decode_accumulate(pairs, np.empty(param.size, np.float32), True)
+    vn = ((f(momentum) * vel).astype(f) + (f(scale) * s).astype(f)).astype(f)
+    param[:] = (param - (f(lr) * vn).astype(f)).astype(f)
+    vel[:] = vn

@@ -63,6 +63,9 @@ def lib() -> ctypes.CDLL:
         L.gc_decompress_accumulate.argtypes = [vp, u32, vp, vp, vp, vp, i32, vp, vp]
         L.gc_last_status.restype = i32
         L.gc_last_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(u64)]
+        L.gc_decompress_apply_momentum.restype = i32
+        L.gc_decompress_apply_momentum.argtypes = [vp, u32, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
+                                                   ctypes.c_float, vp, vp]
         L.gc_compress_host.restype = i32
         L.gc_compress_host.argtypes = [vp] * 11
         L.gc_profile_enable.restype = i32
@@ -222,6 +225,23 @@ class Plan:
                                             _ptr(workspace), _stream_handle(stream))
         if rc < 0:
             raise GcError("gc_decompress_accumulate", rc)
+        return rc
+
+    # --- gc_decompress_apply_momentum
+    def decompress_apply_momentum(self, idx: Sequence[torch.Tensor], val: Sequence[torch.Tensor],
+                                  count: Optional[Sequence[torch.Tensor]], param: torch.Tensor,
+                                  velocity: torch.Tensor, lr: float, momentum: float, scale: float,
+                                  workspace: torch.Tensor, stream=None) -> int:
+        W = len(idx)
+        ip = (ctypes.c_void_p * max(W, 1))(*[t.data_ptr() for t in idx])
+        vp = (ctypes.c_void_p * max(W, 1))(*[t.data_ptr() for t in val])
+        cp = None
+        if count is not None:
+            cp = (ctypes.c_void_p * max(W, 1))(*[t.data_ptr() for t in count])
+        rc = lib().gc_decompress_apply_momentum(self._h, W, ip, vp, cp, _ptr(param), _ptr(velocity), lr, momentum,
+                                                scale, _ptr(workspace), _stream_handle(stream))
+        if rc < 0:
+            raise GcError("gc_decompress_apply_momentum", rc)
         return rc
 
     # --- gc_last_status (synchronises the stream)

@@ -488,12 +488,12 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     {
-        cudaError_t ed = cudaFuncSetAttribute(k_decode_tiles, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t ed = cudaFuncSetAttribute(k_decode_tiles<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)(2 * kDecTileBytes));
         for (int nbuf = 1; nbuf <= 2; ++nbuf) {
             int nb = 0;
             if (ed == cudaSuccess)
-                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_tiles, kDecBlock,
+                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_tiles<false>, kDecBlock,
                                                                    nbuf * kDecTileBytes);
             if (ed != cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
             p->grid_decode[nbuf - 1] = p->sm_count * nb;     // 0: fall back to one launch per worker
@@ -808,9 +808,10 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[nbuf - 1]);
         const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;
         Timed tm(p, s, GC_K_DECODE_TILES);
-        k_decode_tiles<<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap,
-                                                                     (uint32_t)p->total_n, dense_out,
-                                                                     zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr);
+        k_decode_tiles<false><<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap,
+                                                                            (uint32_t)p->total_n, dense_out,
+                                                                            zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr,
+                                                                            ApplyArgs{});
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
@@ -826,6 +827,42 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         k_scatter_add<<<grid, 256, 0, s>>>(p->d_desc, p->T, cap, (uint32_t)p->total_n, idx[w], val[w],
                                            count ? count[w] : nullptr, dense_out, ws.hdr);
     }
+    GC_CUDA(p, cudaGetLastError());
+    return GC_OK;
+}
+
+int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const* idx, const float* const* val,
+                                 const uint32_t* const* count, float* param, float* velocity, float lr,
+                                 float momentum, float scale, void* workspace, void* stream) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (W > GC_MAX_WORKERS) return GC_E_TOO_LARGE;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (p->total_n == 0) return GC_OK;
+    if (param == nullptr || velocity == nullptr || workspace == nullptr) return GC_E_INVALID;
+    if (W > 0 && (idx == nullptr || val == nullptr)) return GC_E_INVALID;
+    for (uint32_t w = 0; w < W; ++w) {
+        if (idx[w] == nullptr || val[w] == nullptr) return GC_E_INVALID;
+        if (count != nullptr && count[w] == nullptr) return GC_E_INVALID;
+    }
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(param) & 15u) ||
+        (reinterpret_cast<uintptr_t>(velocity) & 15u))
+        return GC_E_INVALID;
+    if (count != nullptr && p->T != 1) return GC_E_UNSUPPORTED;       // lists with gaps between tensors
+    if (p->grid_decode[0] <= 0) return GC_E_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    WsView ws = view(p, workspace);
+    DecodeLists ls;
+    for (uint32_t w = 0; w < 64; ++w) {
+        const uint32_t q = w < W ? w : 0;
+        ls.idx[w] = W ? idx[q] : nullptr; ls.val[w] = W ? val[q] : nullptr;
+        ls.len[w] = (W && count != nullptr) ? count[q] : nullptr;
+    }
+    const uint32_t ntl = (uint32_t)((p->total_n + kDecTile - 1) / kDecTile);
+    const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[0]);
+    ApplyArgs ap{param, velocity, lr, momentum, scale};
+    Timed tm(p, s, GC_K_DECODE_TILES);
+    k_decode_tiles<true><<<grid, kDecBlock, kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n,
+                                                                nullptr, 1, 0, 1, ws.hdr, ap);
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
 }

@@ -64,9 +64,19 @@ __device__ __forceinline__ uint32_t warp_lower_bound(const uint32_t* __restrict_
     return lo;
 }
 
+// Optimizer fused behind the decode (APPLY): the summed tile never goes to memory; it is scaled
+// and fed to momentum SGD, v' = mu v + scale * sum, p' = p - lr v', on the parameter and velocity
+// tiles read from and written back to global memory.
+struct ApplyArgs {
+    float* param;
+    float* vel;
+    float lr, mu, scale;
+};
+
+template <bool APPLY>
 static __global__ void __launch_bounds__(kDecBlock)
 k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float* __restrict__ out,
-               int zero_first, int use_bulk, int nbuf, WsHeader* hdr) {
+               int zero_first, int use_bulk, int nbuf, WsHeader* hdr, ApplyArgs ap) {
     // nbuf tile buffers: with two, one fills while the other drains (pays off when there are few
     // workers per tile; with many workers more resident CTAs are worth more than the overlap)
     extern __shared__ __align__(128) float s_tiles[];
@@ -168,6 +178,34 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
             }
         }
         __syncthreads();
+        if (APPLY) {
+            // the sum stays on chip: parameter and velocity tiles stream through registers
+            if (full) {
+#pragma unroll
+                for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q) {
+                    const uint32_t e4 = (uint32_t)(q * kDecBlock + tid);
+                    const float4 gs = *reinterpret_cast<const float4*>(s_tile + e4 * 4);
+                    float4 vv = __ldcs(reinterpret_cast<const float4*>(ap.vel + lo) + e4);
+                    float4 pp = __ldcs(reinterpret_cast<const float4*>(ap.param + lo) + e4);
+                    vv.x = __fadd_rn(__fmul_rn(ap.mu, vv.x), __fmul_rn(ap.scale, gs.x));
+                    vv.y = __fadd_rn(__fmul_rn(ap.mu, vv.y), __fmul_rn(ap.scale, gs.y));
+                    vv.z = __fadd_rn(__fmul_rn(ap.mu, vv.z), __fmul_rn(ap.scale, gs.z));
+                    vv.w = __fadd_rn(__fmul_rn(ap.mu, vv.w), __fmul_rn(ap.scale, gs.w));
+                    pp.x = __fsub_rn(pp.x, __fmul_rn(ap.lr, vv.x)); pp.y = __fsub_rn(pp.y, __fmul_rn(ap.lr, vv.y));
+                    pp.z = __fsub_rn(pp.z, __fmul_rn(ap.lr, vv.z)); pp.w = __fsub_rn(pp.w, __fmul_rn(ap.lr, vv.w));
+                    __stcs(reinterpret_cast<float4*>(ap.vel + lo) + e4, vv);
+                    __stcs(reinterpret_cast<float4*>(ap.param + lo) + e4, pp);
+                }
+            } else {
+                for (uint32_t q = tid; q < hi - lo; q += kDecBlock) {
+                    const float vn = __fadd_rn(__fmul_rn(ap.mu, ap.vel[lo + q]), __fmul_rn(ap.scale, s_tile[q]));
+                    ap.vel[lo + q] = vn;
+                    ap.param[lo + q] = __fsub_rn(ap.param[lo + q], __fmul_rn(ap.lr, vn));
+                }
+            }
+            __syncthreads();
+            continue;
+        }
         // the tile leaves shared memory
         if (full && use_bulk) {
             if (tid == 0) bulk_store_tile(out + lo, s_tile, (uint32_t)(kDecTile * sizeof(float)));

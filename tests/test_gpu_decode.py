@@ -208,3 +208,44 @@ def test_one_tensor_lists_with_counts_use_their_length(W):
         assert np.array_equal(to_np_u32(out), bits(want)), (W, zero_first)
     st, _ = plan.last_status(ws)
     assert st == api.GC_OK
+
+
+@pytest.mark.parametrize("W", [0, 1, 3, 16])
+@pytest.mark.parametrize("sizes,density", [([100_003], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02)])
+def test_decode_apply_momentum_matches_oracle_bitwise(W, sizes, density):
+    """The decode with momentum SGD fused behind it: parameter and velocity after three steps."""
+    plan = api.Plan(sizes, density, device=0)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    gen = torch.Generator().manual_seed(7)
+    p = torch.randn(n, generator=gen); v = torch.randn(n, generator=gen) * 0.1
+    d_p, d_v = p.cuda(), v.cuda()
+    h_p, h_v = p.numpy().copy(), v.numpy().copy()
+    for step in range(3):
+        pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=60 + step, share_every=2) if W else ([], [], [])
+        plan.decompress_apply_momentum(d_idx, d_val, None, d_p, d_v, 0.05, 0.9, 1.0 / max(W, 1), ws)
+        oracle.decode_apply_momentum(pairs, h_p, h_v, 0.05, 0.9, 1.0 / max(W, 1))
+        assert np.array_equal(to_np_u32(d_v), bits(h_v)), (W, step)
+        assert np.array_equal(to_np_u32(d_p), bits(h_p)), (W, step)
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_OK
+
+
+def test_decode_apply_momentum_full_size_matches_the_unfused_pair():
+    """110M-element workload, W = 1: the fused call gives the same bits as decode into a dense
+    buffer followed by the same momentum step written with torch ops that round once each."""
+    w = synth.workload(2)
+    plan = api.Plan(w.sizes, w.density, device=0)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    pairs, d_idx, d_val = synthetic_sets(plan, w.sizes, 1, seed=13)
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    p = torch.randn(n, device="cuda", generator=gen); v = torch.randn(n, device="cuda", generator=gen)
+    p2, v2 = p.clone(), v.clone()
+    plan.decompress_apply_momentum(d_idx, d_val, None, p, v, 0.01, 0.9, 1.0, ws)
+    dense = torch.empty(n, device="cuda")
+    plan.decompress_accumulate(d_idx, d_val, None, dense, True, ws)
+    v2 = torch.mul(v2, 0.9) + torch.mul(dense, 1.0)          # separate kernels: no contraction into an fma
+    p2 = p2 - torch.mul(v2, 0.01)
+    assert torch.equal(v.view(torch.int32), v2.view(torch.int32))
+    assert torch.equal(p.view(torch.int32), p2.view(torch.int32))

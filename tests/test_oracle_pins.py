@@ -345,3 +345,34 @@ def test_sample_definition():
     assert oracle.sample_count(10, 2) == 6             # group 0 (4) + group 2 (2 of 4)
     assert oracle.sample_count(1 << 20, 64) == (1 << 20) // 64
     assert oracle.effective_stride(65536, 64) == 1 and oracle.effective_stride(65537, 64) == 64
+
+
+def test_decode_apply_momentum_hand_values_and_torch_sgd():
+    """Fused decode + momentum SGD: hand values (dyadic, exact), the untouched elements still
+    take their momentum step, and many steps agree with torch.optim.SGD on the dense sum."""
+    import torch
+    p = np.array([1.0, 2.0, 3.0, 4.0], np.float32)
+    v = np.array([0.5, 0.0, -1.0, 2.0], np.float32)
+    pairs = [(np.array([1, 3], np.uint32), np.array([4.0, -2.0], np.float32)),
+             (np.array([3], np.uint32), np.array([6.0], np.float32))]
+    oracle.decode_apply_momentum(pairs, p, v, lr=0.25, momentum=0.5, scale=0.5)
+    # s = [0, 4, 0, 4]; v' = 0.5 v + 0.5 s = [0.25, 2, -0.5, 3]; p' = p - 0.25 v'
+    assert v.tolist() == [0.25, 2.0, -0.5, 3.0]
+    assert p.tolist() == [0.9375, 1.5, 3.125, 3.25]
+    rng = np.random.default_rng(3)
+    n, W = 500, 3
+    p = rng.standard_normal(n).astype(np.float32); v = np.zeros(n, np.float32)
+    tp = torch.nn.Parameter(torch.from_numpy(p.copy()))
+    opt = torch.optim.SGD([tp], lr=0.1, momentum=0.9)
+    for step in range(20):
+        pairs = []
+        dense = np.zeros(n, np.float32)
+        for w in range(W):
+            idx = np.sort(rng.choice(n, size=40, replace=False)).astype(np.uint32)
+            val = rng.standard_normal(40).astype(np.float32)
+            pairs.append((idx, val))
+            dense[idx] = (dense[idx] + val).astype(np.float32)
+        oracle.decode_apply_momentum(pairs, p, v, lr=0.1, momentum=0.9, scale=1.0)
+        tp.grad = torch.from_numpy(dense.copy())
+        opt.step()
+    assert np.allclose(p, tp.detach().numpy(), rtol=1e-5, atol=1e-6)
