@@ -47,9 +47,9 @@ def measured_peak_gbs():
         return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def min_bytes(n: int, k: int, W: int):
-    """Algorithmic bytes of one step: compress 12n + 8k per worker, decode 4n + 8*W*k."""
-    compress = (12 * n + 8 * k) * W
+def min_bytes(n: int, k: int, W: int, grad_bytes: int = 4):
+    """Algorithmic bytes of one step: compress (grad_bytes + 8) n + 8k per worker, decode 4n + 8*W*k."""
+    compress = ((grad_bytes + 8) * n + 8 * k) * W
     decode = 4 * n + 8 * k * W
     return compress, decode
 
@@ -186,6 +186,10 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     # cycled; each is far larger than the 126 MB L2, so no explicit flush is needed
     sets = max(1, min(args.input_sets, int(24e9 // (4 * n * W)) or 1))
     grads = [[synth.gradient(w, wk + 100 * rank, s, device=dev) for s in range(sets)] for wk in range(W)]
+    bf16 = args.grad_dtype == "bf16"
+    if bf16:                                 # the gradient arrives as bfloat16 (gc_compress_bf16)
+        grads = [[g.to(torch.bfloat16) for g in gs] for gs in grads]
+    do_compress = plan.compress_bf16 if bf16 else plan.compress
     resid = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(W)]
     outs = [plan.alloc_outputs() for _ in range(W)]
     ws = plan.alloc_workspace()
@@ -196,7 +200,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
 
     def step(i: int):
         for wk in range(W):
-            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
+            do_compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
                           ws, stream)
         plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], cnts, dense, True, ws, stream)
 
@@ -243,7 +247,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     # ---- timed regions 1c/1d: the two halves on their own (no per-kernel events)
     def compress_only(i: int):
         for wk in range(W):
-            plan.compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
+            do_compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
                           ws, stream)
 
     def decode_only(i: int):
@@ -281,7 +285,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
         del param, vel
 
     # ---- timed region 2: end to end through the host-buffer entry point
-    if args.no_e2e:
+    if args.no_e2e or args.grad_dtype == "bf16":
         e2e_steps, ms_e2e = 0, float("nan")
         return _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e, e2e_steps,
                        per_kernel, launches, clocks, counters)
@@ -321,7 +325,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     from paper_2104_01981_b200 import api
     grad_bytes_step = 4.0 * n * W * world
     value = whole_job_value(n, W, world, args.steps, ms_plain)
-    cb, db = min_bytes(n, k, W)
+    cb, db = min_bytes(n, k, W, 2 if args.grad_dtype == "bf16" else 4)
     t_step = ms_plain * 1e-3 / args.steps
     peak, peak_src = measured_peak_gbs()
 
@@ -350,7 +354,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_plain / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "mode": args.mode, "elements": n, "k": k, "density": w.density, "workers": W,
+        "config": {"workload": w.name, "mode": args.mode, "grad_dtype": args.grad_dtype, "elements": n, "k": k, "density": w.density, "workers": W,
                    "tensors": len(w.sizes), "input_sets": sets,
                    "l2": "inputs larger than L2 (no flush): each gradient and residual is %d MB" % (4 * n >> 20)},
         "elements_per_s": n * W * world * args.steps / (ms_plain * 1e-3),
@@ -527,6 +531,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end region")
     ap.add_argument("--input-sets", type=int, default=N_INPUT_SETS,
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")
+    ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"],
+                    help="storage type of the gradient (bf16: gc_compress_bf16, 10n + 8k bytes per compress; no e2e leg)")
     ap.add_argument("--workload", default="gc", choices=["gc", "ecrm"],
                     help="gc: gradient compression (the headline line); ecrm: erasure-coded embedding-table rows")
     ap.add_argument("--ecrm-rows", type=int, default=8 * 1024 * 1024, help="rows of the embedding-table shard")

@@ -155,6 +155,18 @@ int gc_compress(gc_plan_t *plan, const float *grad, float *residual,
                 void *workspace, void *stream);
 
 /*
+ * gc_compress_bf16 -- gc_compress for a gradient stored as bfloat16 (total_n 16-bit values, 16-byte
+ * aligned, same flat layout).  Every value is widened exactly (16 zero bits appended) and then
+ * treated as the fp32 gradient of gc_compress: a = fl32(g + r), same selection, same outputs,
+ * fp32 residual.  Reads 2 instead of 4 bytes per element of g: 10n + 8k bytes per call.
+ * No counterpart in the source paper.  Top-k mode with the default route only
+ * (GC_E_UNSUPPORTED otherwise, and for plans the two fused top-k kernels do not take).
+ */
+int gc_compress_bf16(gc_plan_t *plan, const void *grad_bf16, float *residual,
+                     uint32_t *out_idx, float *out_val, uint32_t *out_count,
+                     void *workspace, void *stream);
+
+/*
  * gc_decompress_accumulate -- decode W sparse sets and sum them into a dense buffer
  * (problem statement: "decode and sum the sparse contributions of W simulated workers into
  * one dense buffer"; a sum, not a mean).  For every flat index the additions happen in

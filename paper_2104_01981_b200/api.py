@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.gc_plan_query.argtypes = [vp, i32, u32, ctypes.POINTER(u64)]
         L.gc_compress.restype = i32
         L.gc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.gc_compress_bf16.restype = i32
+        L.gc_compress_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         L.gc_decompress_accumulate.restype = i32
         L.gc_decompress_accumulate.argtypes = [vp, u32, vp, vp, vp, vp, i32, vp, vp]
         L.gc_last_status.restype = i32
@@ -172,6 +174,17 @@ class Plan:
                                _ptr(out_count), _ptr(workspace), _stream_handle(stream))
         if rc < 0:
             raise GcError("gc_compress", rc)
+        return rc
+
+    def compress_bf16(self, grad_bf16: torch.Tensor, residual: torch.Tensor, out_idx: torch.Tensor,
+                      out_val: torch.Tensor, out_count: Optional[torch.Tensor], workspace: torch.Tensor,
+                      stream=None) -> int:
+        """``compress`` for a gradient stored as torch.bfloat16."""
+        assert grad_bf16.dtype == torch.bfloat16
+        rc = lib().gc_compress_bf16(self._h, _ptr(grad_bf16), _ptr(residual), _ptr(out_idx), _ptr(out_val),
+                                    _ptr(out_count), _ptr(workspace), _stream_handle(stream))
+        if rc < 0:
+            raise GcError("gc_compress_bf16", rc)
         return rc
 
     def compress_ptr(self, grad: int, residual: int, out_idx: int, out_val: int, out_count: Optional[int],

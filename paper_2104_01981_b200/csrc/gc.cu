@@ -72,7 +72,7 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr size_t kSingleMidCap = 8192;       // short list of k_topk_single (candidates in the band bin of the threshold)
+constexpr size_t kSingleMidCap = 65536;      // short list of k_topk_single (candidates in the band bin of the threshold)
 constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tensor
 constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
 constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
@@ -446,7 +446,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_single_max = 0;
         if (coop) {
             int nb = 0;       // sized for the largest chunk-record block the kernel may be given
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single, kBlock, kSingleMaxT * kSingleRowBytes + kSinglePoolMax / 8) ==
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_single<GradF32>, kBlock, kSingleMaxT * kSingleRowBytes + kSinglePoolMax / 8) ==
                     cudaSuccess && nb >= 1)
                 p->grid_single_max = p->sm_count * nb;
         }
@@ -477,7 +477,7 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_multi_max = 0;
         if (coop) {
             int nb = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi, kBlock,
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi<GradF32>, kBlock,
                                                               kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8 + 8 * kMultiMaxTab) ==
                     cudaSuccess && nb >= 1)
                 p->grid_multi_max = p->sm_count * nb;
@@ -554,10 +554,14 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
     }
 }
 
-int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_idx, float* out_val,
-                uint32_t* out_count, void* workspace, void* stream) {
+static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* residual, uint32_t* out_idx,
+                         float* out_val, uint32_t* out_count, void* workspace, void* stream) {
+    const float* grad = static_cast<const float*>(grad_any);       // only dereferenced as such when !bf16
     if (p == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    // a bf16 gradient is read by the two fused top-k kernels only
+    if (bf16 && !(p->mode == GC_TOPK && p->path == GC_PATH_AUTO && (p->single_grid > 0 || p->multi_grid > 0)))
+        return GC_E_UNSUPPORTED;
     if (p->total_n == 0) return GC_OK;
     if (grad == nullptr || residual == nullptr || out_idx == nullptr || out_val == nullptr ||
         workspace == nullptr)
@@ -673,7 +677,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         sa.d = p->desc[0]; sa.desc = p->d_desc; sa.ntiles = nt; sa.maxt = p->single_maxt;
         sa.pool_cap = std::min<uint32_t>(p->single_pool, p->cand_cap);
         sa.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
-        sa.g = grad; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;
+        sa.g = grad_any; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;
         sa.hist5 = reinterpret_cast<uint32_t*>(wb + p->off_hist5);
         sa.srank_hi = p->single_srank_hi; sa.srank_mid = p->single_srank_mid; sa.mid_cap = (uint32_t)kSingleMidCap;
         sa.mid = reinterpret_cast<uint2*>(wb + p->off_mid);
@@ -683,8 +687,8 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         sa.ws = ws; sa.gws = gws;
         void* args[] = {&sa};
         Timed tm(p, s, GC_K_FUSED);
-        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_single, dim3(p->single_grid), dim3(kBlock),
-                                               args, p->single_smem, s));
+        const void* kfn = bf16 ? (const void*)k_topk_single<GradBF16> : (const void*)k_topk_single<GradF32>;
+        GC_CUDA(p, cudaLaunchCooperativeKernel(kfn, dim3(p->single_grid), dim3(kBlock), args, p->single_smem, s));
         return GC_OK;
     }
     if (p->path == GC_PATH_AUTO && p->multi_grid > 0) {
@@ -697,7 +701,7 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();
         ma.reg_ids = p->d_small + p->T; ma.n_reg = (uint32_t)p->reg_ids.size();
         ma.brk = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
-        ma.g = grad; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
+        ma.g = grad_any; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
         ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
         ma.mid = reinterpret_cast<uint2*>(wb + p->off_mmid);
         ma.mid_n = reinterpret_cast<uint32_t*>(wb + p->off_midn);
@@ -708,8 +712,8 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
         ma.ws = ws; ma.gws = gws;
         void* args[] = {&ma};
         Timed tm(p, s, GC_K_FUSED);
-        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_multi, dim3(p->multi_grid), dim3(kBlock),
-                                               args, p->multi_smem, s));
+        const void* kfn = bf16 ? (const void*)k_topk_multi<GradBF16> : (const void*)k_topk_multi<GradF32>;
+        GC_CUDA(p, cudaLaunchCooperativeKernel(kfn, dim3(p->multi_grid), dim3(kBlock), args, p->multi_smem, s));
         return GC_OK;
     }
     if (p->path == GC_PATH_AUTO && p->grid_fused > 0) {
@@ -775,6 +779,16 @@ int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_
     }
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
+}
+
+int gc_compress(gc_plan_t* p, const float* grad, float* residual, uint32_t* out_idx, float* out_val,
+                uint32_t* out_count, void* workspace, void* stream) {
+    return compress_impl(p, grad, false, residual, out_idx, out_val, out_count, workspace, stream);
+}
+
+int gc_compress_bf16(gc_plan_t* p, const void* grad_bf16, float* residual, uint32_t* out_idx, float* out_val,
+                     uint32_t* out_count, void* workspace, void* stream) {
+    return compress_impl(p, grad_bf16, true, residual, out_idx, out_val, out_count, workspace, stream);
 }
 
 int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* idx,

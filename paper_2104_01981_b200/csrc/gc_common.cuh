@@ -116,6 +116,33 @@ __device__ __forceinline__ uint2 ld_cg(const uint2* p) { return __ldcg(p); }
 __device__ __forceinline__ uint4 ld_cg(const uint4* p) { return __ldcg(p); }
 __device__ __forceinline__ unsigned long long ld_cg(const unsigned long long* p) { return __ldcg(p); }
 
+// How the gradient is stored.  The kernels that read g are templates on one of these; the
+// arithmetic is fp32 either way (a bf16 value is an fp32 value with 16 zero bits appended).
+struct GradF32 {
+    static __device__ __forceinline__ float ld1(const void* g, uint32_t i) {
+        return __ldg(reinterpret_cast<const float*>(g) + i);
+    }
+    static __device__ __forceinline__ float4 ld4(const void* g, uint32_t i) {          // i a multiple of 4
+        return __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g) + i));
+    }
+    static __device__ __forceinline__ const void* at(const void* g, uint32_t i) {
+        return reinterpret_cast<const float*>(g) + i;
+    }
+};
+struct GradBF16 {
+    static __device__ __forceinline__ float ld1(const void* g, uint32_t i) {
+        return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(g) + i) << 16);
+    }
+    static __device__ __forceinline__ float4 ld4(const void* g, uint32_t i) {          // i a multiple of 4
+        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(g) + i));
+        return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+    }
+    static __device__ __forceinline__ const void* at(const void* g, uint32_t i) {
+        return reinterpret_cast<const unsigned short*>(g) + i;
+    }
+};
+
 constexpr int kEmitStage = 64;               // candidates of one warp chunk staged in shared memory
 
 // Static shared memory of every streaming kernel (one instance per CTA, reused by all phases).

@@ -60,14 +60,15 @@ __device__ __forceinline__ uint32_t cand_slot(const TileCands& tc, uint32_t j) {
 // levels (shared memory, __syncthreads only) and the ordered emission, so hundreds of tiny
 // tensors cost one memory round trip each, no global atomics, no completion counters and no
 // grid barriers.
+template <typename GL = GradF32>
 static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const TensorDesc& d, uint32_t t, uint32_t T,
-                                         const float* __restrict__ g, float* __restrict__ r,
+                                         const void* __restrict__ g, float* __restrict__ r,
                                          uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
                                          uint32_t* __restrict__ out_count) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const TileGeom tg = tile_geom(d, 0u);
     Tile tl;
-    load_tile<true>(g, r, tg, warp, lane, tl);           // r = a = g + r; sent entries get +0 below
+    load_tile<true, GL>(g, r, tg, warp, lane, tl);           // r = a = g + r; sent entries get +0 below
     uint32_t prefix = 0, krem = d.k;
 #pragma unroll 1
     for (int level = 0; level < kLevels; ++level) {

@@ -19,8 +19,8 @@ struct Tile {
 // stored to r; otherwise a is read from r.  Interior vectors use 128-bit accesses; vectors
 // that straddle the tensor's first or last element fall back to guarded scalar accesses.
 // r is read at L2 (it may have been written by another CTA earlier in the same launch).
-template <bool FOLD>
-__device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __restrict__ r,
+template <bool FOLD, typename GL = GradF32>
+__device__ __forceinline__ void load_tile(const void* __restrict__ g, float* __restrict__ r,
                                           const TileGeom& tg, int warp, int lane, Tile& t) {
     t.valid = 0;
     float4 gv[kVpt], rv[kVpt];
@@ -31,7 +31,7 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __
         full[j] = (f0 >= tg.lo) && (f0 + 4 <= tg.hi);
         if (full[j]) {
             rv[j] = ld_cg(reinterpret_cast<const float4*>(r + f0));
-            if (FOLD) gv[j] = __ldg(reinterpret_cast<const float4*>(g + f0));
+            if (FOLD) gv[j] = GL::ld4(g, f0);
         }
     }
 #pragma unroll
@@ -54,7 +54,7 @@ __device__ __forceinline__ void load_tile(const float* __restrict__ g, float* __
                 float v = 0.0f;
                 if (f >= tg.lo && f < tg.hi) {
                     v = ld_cg(r + f);
-                    if (FOLD) { v = __fadd_rn(__ldg(g + f), v); r[f] = v; }
+                    if (FOLD) { v = __fadd_rn(GL::ld1(g, f), v); r[f] = v; }
                     t.valid |= 1u << (4 * j + e);
                 }
                 t.a[j][e] = v;

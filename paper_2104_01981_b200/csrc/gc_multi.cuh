@@ -42,7 +42,7 @@ struct MultiArgs {
     const uint32_t* reg_ids;         // the tensors that are not small (and not empty)
     uint32_t n_reg;
     TensorSel* brk;                  // [T] bracket of every such tensor: .prefix = tau, .krem = tau_z, .T = shift
-    const float* g;
+    const void* g;                   // fp32 or bf16, see the kernel's template argument
     float* r;
     uint32_t* out_idx;
     float* out_val;
@@ -92,6 +92,7 @@ __device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* 
     return *s_ok != 0;
 }
 
+template <typename GL>
 static __global__ void __launch_bounds__(kBlock, 4)
 k_topk_multi(MultiArgs a) {
     __shared__ BlockSmem sm;
@@ -156,7 +157,7 @@ k_topk_multi(MultiArgs a) {
                 for (int e = 0; e < 4; ++e) {
                     const bool v = i0 + e < d.n;
                     const uint32_t f = d.off + (v ? i0 + e : 0u);
-                    gv[e] = v ? __ldg(a.g + f) : 0.f;
+                    gv[e] = v ? GL::ld1(a.g, f) : 0.f;
                     rv[e] = v ? ld_cg(a.r + f) : 0.f;
                 }
 #pragma unroll
@@ -177,7 +178,7 @@ k_topk_multi(MultiArgs a) {
     for (uint32_t q = G - 1u - b; q < a.n_small; q += G) {
         const uint32_t t = a.small_ids[q];
         const TensorDesc d = a.desc[t];
-        small_tensor_body(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
+        small_tensor_body<GL>(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
     }
     __syncthreads();
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
@@ -291,7 +292,7 @@ k_topk_multi(MultiArgs a) {
                 float4 gv[kVpt], rv[kVpt];
 #pragma unroll
                 for (int j = 0; j < kVpt; ++j) {
-                    gv[j] = __ldg(reinterpret_cast<const float4*>(a.g + tg.base + my_off + j * 128));
+                    gv[j] = GL::ld4(a.g, tg.base + my_off + j * 128);
                     rv[j] = ld_cg(reinterpret_cast<const float4*>(a.r + tg.base + my_off + j * 128));
                 }
 #pragma unroll
@@ -308,7 +309,7 @@ k_topk_multi(MultiArgs a) {
                         const uint32_t f = tg.base + my_off + j * 128 + e;
                         float v = 0.0f;
                         if (f >= tg.lo && f < tg.hi) {
-                            v = __fadd_rn(__ldg(a.g + f), ld_cg(a.r + f));
+                            v = __fadd_rn(GL::ld1(a.g, f), ld_cg(a.r + f));
                             valid |= 1u << (4 * j + e);
                         }
                         av[j][e] = v;

@@ -52,7 +52,7 @@ struct SingleArgs {
     uint32_t srank_hi;               // sample rank of the upper bracket (at least 1)
     uint32_t srank_mid;              // sample rank that estimates the threshold itself
     uint32_t mid_cap;                // capacity of the short list
-    const float* g;
+    const void* g;                   // fp32 or bf16, see the kernel's template argument
     float* r;
     uint32_t* out_idx;
     float* out_val;
@@ -164,6 +164,7 @@ __device__ bool short_list_select(BlockSmem& sm, const uint2 (&e)[kMidRegs], con
     return ok;
 }
 
+template <typename GL>
 static __global__ void __launch_bounds__(kBlock, 4)
 k_topk_single(SingleArgs a) {
     __shared__ BlockSmem sm;
@@ -215,7 +216,7 @@ k_topk_single(SingleArgs a) {
             for (int e = 0; e < 4; ++e) {
                 const bool v = in && i0 + e < d.n;
                 const uint32_t f = d.off + (v ? i0 + e : 0u);
-                gv[e] = v ? __ldg(a.g + f) : 0.f;
+                gv[e] = v ? GL::ld1(a.g, f) : 0.f;
                 rv[e] = v ? ld_cg(a.r + f) : 0.f;
                 sok |= (uint32_t)v << (4 * q + e);
             }
@@ -237,7 +238,7 @@ k_topk_single(SingleArgs a) {
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
                 if (pb + j * 128 + 4 <= d.off + d.n) {
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.g + pb + j * 128));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(GL::at(a.g, pb + j * 128)));
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.r + pb + j * 128));
                 }
             }
@@ -301,7 +302,7 @@ k_topk_single(SingleArgs a) {
             float4 gv[kVpt], rv[kVpt];
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
-                gv[j] = __ldg(reinterpret_cast<const float4*>(a.g + tg.base + my_off + j * 128));
+                gv[j] = GL::ld4(a.g, tg.base + my_off + j * 128);
                 rv[j] = ld_cg(reinterpret_cast<const float4*>(a.r + tg.base + my_off + j * 128));
             }
 #pragma unroll
@@ -318,7 +319,7 @@ k_topk_single(SingleArgs a) {
                     const uint32_t f = tg.base + my_off + j * 128 + e;
                     float v = 0.0f;
                     if (f >= tg.lo && f < tg.hi) {
-                        v = __fadd_rn(__ldg(a.g + f), ld_cg(a.r + f));
+                        v = __fadd_rn(GL::ld1(a.g, f), ld_cg(a.r + f));
                         valid |= 1u << (4 * j + e);
                     }
                     av[j][e] = v;

@@ -235,3 +235,40 @@ def test_random_plans_match_the_oracle(seed):
     scales = torch.cat([torch.full((s,), float(10.0 ** rng.integers(-3, 3))) for s in sizes])
     grads = [randn(n, 5000 + 10 * seed + s) * scales for s in range(3)]
     check_topk_against_oracle(sizes, density, grads)
+
+
+@pytest.mark.parametrize("sizes,density", [([3_000_001], 0.01), ([70_001], 0.001),
+                                           ([300_000, 5, 1_500_001, 131_072, 64, 131_071, 4093, 0, 2_000_003], 0.001),
+                                           ([5, 3, 1000, 7], 0.3)])
+def test_bf16_gradient_matches_the_oracle_on_the_widened_values(sizes, density):
+    """gc_compress_bf16: the gradient arrives as bfloat16, is widened exactly and folded into the
+    fp32 residual; indices, values and residual must be the oracle's on the widened gradient."""
+    plan = api.Plan(sizes, density, device=0)
+    n, ks = plan.total_n, plan.tensor_k()
+    wk = GpuWorker(plan)
+    r_cpu = np.zeros(n, np.float32)
+    for step in range(3):
+        g16 = (randn(n, 8000 + step) * 0.37).to(torch.bfloat16)
+        pad = torch.zeros(8, dtype=torch.bfloat16)
+        d_g = torch.cat([g16, pad]).cuda()[:n]
+        plan.compress_bf16(d_g, wk.residual, wk.idx, wk.val, wk.count, wk.ws)
+        oi, ov = oracle.topk_compress_tensors(sizes, ks, g16.float().numpy(), r_cpu)
+        tot = plan.total_cap
+        assert np.array_equal(to_np_u32(wk.idx[:tot]), oi), step
+        assert np.array_equal(to_np_u32(wk.val[:tot]), bits(ov)), step
+        assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r_cpu)), step
+        st, det = plan.last_status(wk.ws)
+        assert st == api.GC_OK, (st, det)
+
+
+def test_bf16_gradient_is_refused_where_no_kernel_reads_it():
+    plan = api.Plan([100_000], 0.01, device=0)
+    plan.set_option(api.GC_OPT_PATH, api.GC_PATH_EXACT)
+    wk = GpuWorker(plan)
+    g = torch.zeros(100_000, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(api.GcError):
+        plan.compress_bf16(g, wk.residual, wk.idx, wk.val, wk.count, wk.ws)
+    thr = api.Plan([100_000], 0.01, mode=api.GC_THRESHOLD, device=0)
+    wt = GpuWorker(thr)
+    with pytest.raises(api.GcError):
+        thr.compress_bf16(g, wt.residual, wt.idx, wt.val, wt.count, wt.ws)
