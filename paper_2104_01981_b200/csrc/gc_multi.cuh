@@ -93,7 +93,8 @@ __device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* 
 }
 
 template <typename GL>
-static __global__ void __launch_bounds__(kBlock, 4)
+// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
+static __global__ void __launch_bounds__(kBlock, 3)
 k_topk_multi(MultiArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used, s_cnt;

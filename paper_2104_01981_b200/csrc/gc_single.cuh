@@ -164,8 +164,10 @@ __device__ bool short_list_select(BlockSmem& sm, const uint2 (&e)[kMidRegs], con
     return ok;
 }
 
+// Three CTAs per SM (80 registers, no spills): measured 15 us faster on the 110M-element workload
+// than four CTAs at 64 registers with spills, and than two.
 template <typename GL>
-static __global__ void __launch_bounds__(kBlock, 4)
+static __global__ void __launch_bounds__(kBlock, 3)
 k_topk_single(SingleArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used;

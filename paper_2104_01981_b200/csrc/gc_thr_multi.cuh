@@ -132,7 +132,8 @@ static __device__ __noinline__ void small_threshold_body(BlockSmem& sm, const Te
     __syncthreads();
 }
 
-static __global__ void __launch_bounds__(kBlock, 4)
+// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
+static __global__ void __launch_bounds__(kBlock, 3)
 k_threshold_multi(ThrMultiArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used, s_cnt;

@@ -45,7 +45,8 @@ struct ThrSingleArgs {
     WsView ws;
 };
 
-static __global__ void __launch_bounds__(kBlock, 4)
+// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
+static __global__ void __launch_bounds__(kBlock, 3)
 k_threshold_single(ThrSingleArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used;
