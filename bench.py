@@ -340,7 +340,11 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
     # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
-    ncu_traffic = {("c3_bert_base_110m_student_t", "compress_fused"): 1390.4e6}.get((w.name, dom))
+    ncu_traffic, ncu_src = {
+        ("c3_bert_base_110m_student_t", "topk", "compress_fused"): (1361.5e6, "profiles/k_topk_single_c3_bert110m.md"),
+        ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): (1407.5e6, "profiles/k_threshold_single_c3_bert110m.md"),
+        ("c2_resnet50_layerwise", "topk", "compress_fused"): (322.1e6, "profiles/k_topk_multi_c2_resnet50.md"),
+    }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None, (None, None))
 
     # CPU baseline: the oracle on a bounded sample of the same workload
     cpu = None
@@ -365,7 +369,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
         "kernels": breakdown,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic, "peak_source": peak_src,
-                     "traffic_source": "profiles/k_topk_single_c3_bert110m.md" if ncu_traffic else None,
+                     "traffic_source": ncu_src,
                      "algorithmic_bytes_per_launch": alg_bytes.get(dom)},
         "cpu_baseline": cpu,
         "e2e": None if not e2e_steps else {"value": grad_bytes_step * e2e_steps / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
