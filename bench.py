@@ -519,6 +519,95 @@ def run_ecrm(args, rank: int, world: int, local_rank: int):
 
 
 
+# --------------------------------------------------------------------------- multi-GPU aggregation
+def run_exchange(args, w: synth.Workload, rank: int, world: int, local_rank: int):
+    """Third workload (`--workload exchange`): every rank is ONE worker.  A step = compress this
+    rank's gradient into its exchange block, one NCCL all-gather of the blocks, decode of the
+    `world` gathered lists in rank order.  At one GPU the group has one rank (the collective is
+    a local copy inside NCCL).  Prints its own JSON line."""
+    from paper_2104_01981_b200 import api, exchange
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    api.lib()
+    mode = api.GC_THRESHOLD if args.mode == "threshold" else api.GC_TOPK
+    plan = api.Plan(w.sizes, w.density, mode=mode, device=local_rank)
+    n, k = plan.total_n, plan.total_cap
+    stream = torch.cuda.current_stream()
+    ex = exchange.PairExchange.for_plan(plan)
+    sets = max(1, min(args.input_sets, int(24e9 // (4 * n)) or 1))
+    grads = [synth.gradient(w, 100 * rank, s, device=dev) for s in range(sets)]
+    resid = torch.zeros(n, dtype=torch.float32, device=dev)
+    ws = plan.alloc_workspace()
+    dense = torch.empty(n, dtype=torch.float32, device=dev)
+    oi, ov, oc = ex.outputs()
+    thr = mode == api.GC_THRESHOLD
+
+    def do_compress(i):
+        plan.compress(grads[i % sets], resid, oi, ov, oc if thr else None, ws, stream)
+
+    def do_gather(i):
+        ex.all_gather()
+
+    def do_decode(i):
+        ex.decode(plan, dense, True, ws, stream)
+
+    def step(i):
+        do_compress(i); do_gather(i); do_decode(i)
+
+    def barrier():
+        torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            fn(args.warmup + i)
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    for i in range(args.warmup):
+        step(i)
+    launches0 = plan.launches()
+    sampler = ClockSampler(local_rank, os.path.join("/tmp", f"gc_bench_clocks_{os.getpid()}.csv")) \
+        if rank == 0 else None
+    ms = timed(step)
+    launches = plan.launches() - launches0
+    legs = [timed(do_compress), timed(do_gather), timed(do_decode)]
+    clocks = sampler.stop() if sampler else None
+    st, det = plan.last_status(ws)
+    if st not in (api.GC_OK, api.GC_W_TRUNCATED):
+        raise RuntimeError(f"device status {st} (detail {det}) after the timed region")
+    ms, *legs = reduce_max_over_ranks([ms] + legs, world, dev)
+    if rank != 0:
+        return
+    peak, peak_src = measured_peak_gbs()
+    t_step = ms * 1e-3 / args.steps
+    wire = ex.bytes_on_wire_per_rank()
+    line = {
+        "metric": METRIC, "value": whole_job_value(n, 1, world, args.steps, ms), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name + "_exchange", "mode": args.mode, "elements": n, "k": k, "density": w.density,
+                   "workers": world, "workers_per_rank": 1, "tensors": len(w.sizes), "input_sets": sets,
+                   "collective": "all_gather_into_tensor (NCCL) of one fixed-size block per rank",
+                   "l2": f"inputs larger than L2 (no flush): each gradient and residual is {4 * n / 1e6:.0f} MB"},
+        "legs_ms_per_step": {"compress": legs[0] / args.steps, "all_gather": legs[1] / args.steps,
+                             "decode": legs[2] / args.steps},
+        "exchange": {"block_bytes": 4 * ex.layout.words, "bytes_received_per_rank": wire,
+                     "all_gather_GB_per_s_per_rank": (wire / (legs[1] * 1e-3 / args.steps) / 1e9) if wire else None},
+        "roofline": {"bound": "hbm", "kernel": "step (compress + decode of `world` lists)",
+                     "achieved": (12.0 * n + 8.0 * k + 4.0 * n + 8.0 * k * world) / t_step / 1e9, "peak": peak,
+                     "unit": "GB/s", "frac": (12.0 * n + 8.0 * k + 4.0 * n + 8.0 * k * world) / t_step / 1e9 / peak,
+                     "traffic": None, "peak_source": peak_src},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": launches, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -537,8 +626,9 @@ def main():
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of the gradient (bf16: gc_compress_bf16, 10n + 8k bytes per compress; no e2e leg)")
-    ap.add_argument("--workload", default="gc", choices=["gc", "ecrm"],
-                    help="gc: gradient compression (the headline line); ecrm: erasure-coded embedding-table rows")
+    ap.add_argument("--workload", default="gc", choices=["gc", "ecrm", "exchange"],
+                    help="gc: gradient compression (the headline line); ecrm: erasure-coded embedding-table rows; "
+                         "exchange: one worker per rank, NCCL all-gather of the pairs, decode of all ranks' lists")
     ap.add_argument("--ecrm-rows", type=int, default=8 * 1024 * 1024, help="rows of the embedding-table shard")
     ap.add_argument("--ecrm-batch", type=int, default=1024 * 1024, help="distinct rows one batch updates")
     args = ap.parse_args()
@@ -550,15 +640,22 @@ def main():
     if args.impl == "reference":
         run_reference(args, w, rank)
         return
+    group = world > 1 or args.workload == "exchange"
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    elif group:                                  # a one-rank group, so that the collective itself runs
+        rdv = os.path.join(tempfile.mkdtemp(prefix="gc_bench_"), "rendezvous")
+        torch.distributed.init_process_group("nccl", init_method=f"file://{rdv}", rank=0, world_size=1,
+                                             device_id=torch.device(f"cuda:{local_rank}"))
     try:
         if args.workload == "ecrm":
             run_ecrm(args, rank, world, local_rank)
+        elif args.workload == "exchange":
+            run_exchange(args, w, rank, world, local_rank)
         else:
             run_gpu(args, w, rank, world, local_rank)
     finally:
-        if world > 1:
+        if group:
             torch.distributed.destroy_process_group()
 
 
