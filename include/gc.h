@@ -111,11 +111,21 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                (1000 = default; small values make the candidate set too small
  *                                and so exercise the safety net -- a testing aid)
  *   GC_OPT_CANDIDATE_CAPACITY    lowers the candidate-list capacity (testing aid for overflow)
+ *   GC_OPT_DECODE_ROUTE          which tiled decode kernel gc_decompress_accumulate and
+ *                                gc_decompress_apply_momentum take: GC_DECODE_AUTO (default) picks
+ *                                by the expected number of pairs per worker and 8192-element tile --
+ *                                GC_DECODE_NARROW pre-loads 4 x (256 / W) pairs per worker in
+ *                                registers, GC_DECODE_WIDE keeps up to 4096 / W pairs per worker in
+ *                                shared-memory rings (many workers, dense lists).  Same result.
  * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
  */
 #define GC_OPT_PATH                  0
 #define GC_OPT_SAMPLE_RANK_PERMILLE  1
 #define GC_OPT_CANDIDATE_CAPACITY    2
+#define GC_OPT_DECODE_ROUTE          3
+#define GC_DECODE_AUTO   0
+#define GC_DECODE_NARROW 1
+#define GC_DECODE_WIDE   2
 #define GC_PATH_AUTO   0
 #define GC_PATH_EXACT  1
 #define GC_PATH_STAGED 2

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "gc_single.cuh"
@@ -34,12 +35,15 @@ struct gc_plan_s {
     uint32_t cand_cap = 0, cand_cap_alloc = 0;
     uint32_t n_sampled = 0;                 // tensors with a sample
     int path = 0;                           // GC_PATH_AUTO or GC_PATH_EXACT
+    int decode_route = 0;                   // GC_DECODE_AUTO, GC_DECODE_NARROW or GC_DECODE_WIDE
     uint32_t rank_permille = 1000;          // scales the sample rank (testing aid)
     // workspace layout (byte offsets)
     size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
            control_bytes = 0, off_tinfo = 0, off_cidx = 0, ws_bytes = 0;
     int sm_count = 0;
     int grid_thr = 0, grid_decode[2] = {0, 0};
+    bool wide_ok = false;                         // k_decode_wide may use up to 64 KB of dynamic shared memory
+    std::vector<std::pair<size_t, int>> wide_occ[2];      // (shared-memory bytes -> CTAs per SM), plain / with optimizer
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
     int grid_fused = 0;                     // CTAs of the cooperative launch (0 = not available)
     // single-tensor shared-memory-pool kernel
@@ -366,6 +370,46 @@ int blocks_per_sm(K kernel, int threads) {
 
 }  // namespace
 
+// Which decode kernel a call takes.  The narrow kernel pre-loads 4 x (256 / W) entries per worker
+// and tile in registers; lists that are expected to hold more per tile than that (many workers,
+// or dense lists) go to the wide kernel, which keeps `win` entries per worker in shared memory.
+struct DecodeRoute {
+    bool wide = false;
+    uint32_t win = 0;
+    size_t smem = 0;
+    int grid = 0;
+};
+template <bool APPLY>
+static DecodeRoute decode_route(gc_plan_t* p, uint32_t W) {
+    DecodeRoute r;
+    if (!p->wide_ok || W == 0 || p->total_n == 0) return r;
+    const uint64_t avg = (p->total_cap * (uint64_t)kDecTile + p->total_n - 1) / p->total_n;     // per worker and tile
+    const uint64_t need = avg + avg / 2 + 16;
+    uint32_t Wp = 1;
+    while (Wp < W && Wp < 64) Wp <<= 1;
+    const uint64_t narrow_window = (uint64_t)kDecRounds * (kDecBlock / Wp);
+    // measured: the narrow kernel wins as long as most tiles fit its window
+    r.wide = p->decode_route == GC_DECODE_AUTO ? avg + avg / 4 > narrow_window : p->decode_route == GC_DECODE_WIDE;
+    if (!r.wide) return r;
+    uint32_t win = 32;
+    while (win < need && win < 1024) win <<= 1;
+    while ((uint64_t)W * win > kDecWideEntries && win > 32) win >>= 1;
+    r.win = win;
+    r.smem = kDecTileBytes + 8 * (size_t)W * win;
+    int nb = -1;
+    for (auto& e : p->wide_occ[APPLY ? 1 : 0]) if (e.first == r.smem) nb = e.second;
+    if (nb < 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_wide<APPLY>, kDecBlock, r.smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            nb = 0;
+        }
+        p->wide_occ[APPLY ? 1 : 0].emplace_back(r.smem, nb);
+    }
+    r.grid = p->sm_count * nb;
+    if (r.grid <= 0) r.wide = false;
+    return r;
+}
+
 extern "C" {
 
 uint32_t gc_version(void) { return 1u; }
@@ -499,6 +543,11 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
             p->grid_decode[nbuf - 1] = p->sm_count * nb;     // 0: fall back to one launch per worker
         }
     }
+    p->wide_ok = cudaFuncSetAttribute(k_decode_wide<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess &&
+                 cudaFuncSetAttribute(k_decode_wide<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess;
+    (void)cudaGetLastError();
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
     p->grid_chist = p->sm_count * blocks_per_sm(k_cand_hist<1>, kBlock);
     p->grid_ccompact = p->sm_count * blocks_per_sm(k_cand_compact<true>, kBlock);
@@ -523,6 +572,10 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
         case GC_OPT_CANDIDATE_CAPACITY:
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
             p->cand_cap = (uint32_t)value;
+            return GC_OK;
+        case GC_OPT_DECODE_ROUTE:
+            if (value != GC_DECODE_AUTO && value != GC_DECODE_NARROW && value != GC_DECODE_WIDE) return GC_E_INVALID;
+            p->decode_route = (int)value;
             return GC_OK;
         default:
             return GC_E_INVALID;
@@ -822,6 +875,14 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[nbuf - 1]);
         const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;
         Timed tm(p, s, GC_K_DECODE_TILES);
+        const DecodeRoute rt = decode_route<false>(p, W);
+        if (rt.wide) {
+            k_decode_wide<false><<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
+                ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, dense_out, zero_first ? 1 : 0, use_bulk, rt.win,
+                ws.hdr, ApplyArgs{});
+            GC_CUDA(p, cudaGetLastError());
+            return GC_OK;
+        }
         k_decode_tiles<false><<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap,
                                                                             (uint32_t)p->total_n, dense_out,
                                                                             zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr,
@@ -875,6 +936,13 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
     const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[0]);
     ApplyArgs ap{param, velocity, lr, momentum, scale};
     Timed tm(p, s, GC_K_DECODE_TILES);
+    const DecodeRoute rt = decode_route<true>(p, W);
+    if (rt.wide) {
+        k_decode_wide<true><<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
+            ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, nullptr, 1, 0, rt.win, ws.hdr, ap);
+        GC_CUDA(p, cudaGetLastError());
+        return GC_OK;
+    }
     k_decode_tiles<true><<<grid, kDecBlock, kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n,
                                                                 nullptr, 1, 0, 1, ws.hdr, ap);
     GC_CUDA(p, cudaGetLastError());

@@ -18,6 +18,7 @@ namespace gc {
 constexpr int kDecTile = 8192;               // floats per CTA tile
 constexpr int kDecBlock = 256;
 constexpr int kDecRounds = 4;                // entries a thread pre-loads per tile
+constexpr size_t kDecWideEntries = 4096;     // ring entries (8 bytes each) the wide kernel keeps in shared memory, all workers together
 constexpr size_t kDecTileBytes = kDecTile * sizeof(float);
 
 struct DecodeLists {
@@ -73,6 +74,52 @@ struct ApplyArgs {
     float lr, mu, scale;
 };
 
+// The optimizer step on one finished tile: the sum stays on chip, parameter and velocity tiles
+// stream through registers.
+__device__ __forceinline__ void apply_tile(const ApplyArgs& ap, const float* s_tile, uint32_t lo, uint32_t hi,
+                                           bool full, int tid) {
+    if (full) {
+#pragma unroll
+        for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q) {
+            const uint32_t e4 = (uint32_t)(q * kDecBlock + tid);
+            const float4 gs = *reinterpret_cast<const float4*>(s_tile + e4 * 4);
+            float4 vv = __ldcs(reinterpret_cast<const float4*>(ap.vel + lo) + e4);
+            float4 pp = __ldcs(reinterpret_cast<const float4*>(ap.param + lo) + e4);
+            vv.x = __fadd_rn(__fmul_rn(ap.mu, vv.x), __fmul_rn(ap.scale, gs.x));
+            vv.y = __fadd_rn(__fmul_rn(ap.mu, vv.y), __fmul_rn(ap.scale, gs.y));
+            vv.z = __fadd_rn(__fmul_rn(ap.mu, vv.z), __fmul_rn(ap.scale, gs.z));
+            vv.w = __fadd_rn(__fmul_rn(ap.mu, vv.w), __fmul_rn(ap.scale, gs.w));
+            pp.x = __fsub_rn(pp.x, __fmul_rn(ap.lr, vv.x)); pp.y = __fsub_rn(pp.y, __fmul_rn(ap.lr, vv.y));
+            pp.z = __fsub_rn(pp.z, __fmul_rn(ap.lr, vv.z)); pp.w = __fsub_rn(pp.w, __fmul_rn(ap.lr, vv.w));
+            __stcs(reinterpret_cast<float4*>(ap.vel + lo) + e4, vv);
+            __stcs(reinterpret_cast<float4*>(ap.param + lo) + e4, pp);
+        }
+    } else {
+        for (uint32_t q = tid; q < hi - lo; q += kDecBlock) {
+            const float vn = __fadd_rn(__fmul_rn(ap.mu, ap.vel[lo + q]), __fmul_rn(ap.scale, s_tile[q]));
+            ap.vel[lo + q] = vn;
+            ap.param[lo + q] = __fsub_rn(ap.param[lo + q], __fmul_rn(ap.lr, vn));
+        }
+    }
+}
+
+// Clears the tile, or loads it from the dense buffer when the sum continues what is there.
+__device__ __forceinline__ void stage_tile(float* s_tile, const float* out, uint32_t lo, uint32_t hi, bool full,
+                                           int zero_first, int use_bulk, int tid) {
+    if (zero_first) {
+#pragma unroll
+        for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q)
+            *reinterpret_cast<float4*>(s_tile + (q * kDecBlock + tid) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else if (full && use_bulk) {
+#pragma unroll
+        for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q)
+            *reinterpret_cast<float4*>(s_tile + (q * kDecBlock + tid) * 4) =
+                *reinterpret_cast<const float4*>(out + lo + (q * kDecBlock + tid) * 4);
+    } else {
+        for (uint32_t q = tid; q < (uint32_t)kDecTile; q += kDecBlock) s_tile[q] = (lo + q < hi) ? out[lo + q] : 0.f;
+    }
+}
+
 template <bool APPLY>
 static __global__ void __launch_bounds__(kDecBlock)
 k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float* __restrict__ out,
@@ -112,19 +159,7 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         const uint32_t lo = tl * (uint32_t)kDecTile;
         const uint32_t hi = min(total_n, lo + (uint32_t)kDecTile);
         const bool full = hi - lo == (uint32_t)kDecTile;
-        // stage the tile
-        if (zero_first) {
-#pragma unroll
-            for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q)
-                *reinterpret_cast<float4*>(s_tile + (q * kDecBlock + tid) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        } else if (full && use_bulk) {
-#pragma unroll
-            for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q)
-                *reinterpret_cast<float4*>(s_tile + (q * kDecBlock + tid) * 4) =
-                    *reinterpret_cast<const float4*>(out + lo + (q * kDecBlock + tid) * 4);
-        } else {
-            for (uint32_t q = tid; q < (uint32_t)kDecTile; q += kDecBlock) s_tile[q] = (lo + q < hi) ? out[lo + q] : 0.f;
-        }
+        stage_tile(s_tile, out, lo, hi, full, zero_first, use_bulk, tid);
         // pre-load the next kDecRounds * E entries of every worker
         const uint32_t c0 = live ? s_cur[my_w] : 0u;
         uint32_t ix[kDecRounds];
@@ -179,30 +214,7 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         }
         __syncthreads();
         if (APPLY) {
-            // the sum stays on chip: parameter and velocity tiles stream through registers
-            if (full) {
-#pragma unroll
-                for (int q = 0; q < kDecTile / (4 * kDecBlock); ++q) {
-                    const uint32_t e4 = (uint32_t)(q * kDecBlock + tid);
-                    const float4 gs = *reinterpret_cast<const float4*>(s_tile + e4 * 4);
-                    float4 vv = __ldcs(reinterpret_cast<const float4*>(ap.vel + lo) + e4);
-                    float4 pp = __ldcs(reinterpret_cast<const float4*>(ap.param + lo) + e4);
-                    vv.x = __fadd_rn(__fmul_rn(ap.mu, vv.x), __fmul_rn(ap.scale, gs.x));
-                    vv.y = __fadd_rn(__fmul_rn(ap.mu, vv.y), __fmul_rn(ap.scale, gs.y));
-                    vv.z = __fadd_rn(__fmul_rn(ap.mu, vv.z), __fmul_rn(ap.scale, gs.z));
-                    vv.w = __fadd_rn(__fmul_rn(ap.mu, vv.w), __fmul_rn(ap.scale, gs.w));
-                    pp.x = __fsub_rn(pp.x, __fmul_rn(ap.lr, vv.x)); pp.y = __fsub_rn(pp.y, __fmul_rn(ap.lr, vv.y));
-                    pp.z = __fsub_rn(pp.z, __fmul_rn(ap.lr, vv.z)); pp.w = __fsub_rn(pp.w, __fmul_rn(ap.lr, vv.w));
-                    __stcs(reinterpret_cast<float4*>(ap.vel + lo) + e4, vv);
-                    __stcs(reinterpret_cast<float4*>(ap.param + lo) + e4, pp);
-                }
-            } else {
-                for (uint32_t q = tid; q < hi - lo; q += kDecBlock) {
-                    const float vn = __fadd_rn(__fmul_rn(ap.mu, ap.vel[lo + q]), __fmul_rn(ap.scale, s_tile[q]));
-                    ap.vel[lo + q] = vn;
-                    ap.param[lo + q] = __fsub_rn(ap.param[lo + q], __fmul_rn(ap.lr, vn));
-                }
-            }
+            apply_tile(ap, s_tile, lo, hi, full, tid);
             __syncthreads();
             continue;
         }
@@ -217,6 +229,131 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
         record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
     if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// 4-byte asynchronous copy global -> shared, and the wait for all such copies of this thread.
+__device__ __forceinline__ void cp_async_4(void* sdst, const void* gsrc) {
+    const uint32_t sa = (uint32_t)__cvta_generic_to_shared(sdst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sa), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Decode for many workers or dense lists.  Every worker's next `win` entries sit in a ring in
+// shared memory that is topped up with asynchronous copies as entries are consumed, so every
+// list entry is fetched once and the fetch for the next tile overlaps with this tile's way out.
+// The workers are applied one after the other, each by the whole CTA (one ring entry per
+// thread), so a worker's share of a tile may be as large as the ring whatever the number of
+// workers, and the block-wide count that separates two workers also yields how far the cursor
+// moves.  If some worker has more than `win` entries in the tile, the pass ends at the smallest
+// index up to which every worker's ring is complete and the rest of the tile takes another
+// pass.  One tile buffer; `win` is a power of two.
+template <bool APPLY>
+static __global__ void __launch_bounds__(kDecBlock)
+k_decode_wide(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float* __restrict__ out,
+              int zero_first, int use_bulk, uint32_t win, WsHeader* hdr, ApplyArgs ap) {
+    extern __shared__ __align__(128) float s_tiles[];
+    float* const s_tile = s_tiles;
+    uint32_t* const rg_idx = reinterpret_cast<uint32_t*>(s_tiles + kDecTile);      // [W][win]
+    float* const rg_val = reinterpret_cast<float*>(rg_idx + W * win);              // [W][win]
+    __shared__ uint32_t s_cur[64], s_len[64], s_adv[64], s_bound;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
+    const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
+    if (t0 >= t1) return;
+    const uint32_t mask = win - 1u;
+    // E consecutive threads top up one worker's ring
+    int Wp = 1;
+    while (Wp < (int)W && Wp < 64) Wp <<= 1;
+    const int E = kDecBlock / Wp;
+    const uint32_t my_w = (uint32_t)(tid / E);
+    const int sub = tid % E;
+
+    for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
+        const uint32_t len = ls.len[w] != nullptr ? min(__ldg(ls.len[w]), cnt) : cnt;
+        const uint32_t c = warp_lower_bound(ls.idx[w], len, t0 * (uint32_t)kDecTile, lane);
+        if (lane == 0) { s_cur[w] = c; s_len[w] = len; s_adv[w] = 0u; }
+    }
+    __syncthreads();
+    // list positions [from, to) of worker my_w go to their ring slots
+    auto top_up = [&](uint32_t from, uint32_t to) {
+        for (uint32_t p = from + (uint32_t)sub; p < to; p += (uint32_t)E) {
+            cp_async_4(rg_idx + my_w * win + (p & mask), ls.idx[my_w] + p);
+            cp_async_4(rg_val + my_w * win + (p & mask), ls.val[my_w] + p);
+        }
+    };
+    if (my_w < W) top_up(s_cur[my_w], min(s_len[my_w], s_cur[my_w] + win));
+
+    for (uint32_t tl = t0; tl < t1; ++tl) {
+        const uint32_t lo = tl * (uint32_t)kDecTile;
+        const uint32_t hi = min(total_n, lo + (uint32_t)kDecTile);
+        const bool full = hi - lo == (uint32_t)kDecTile;
+        if (use_bulk && !APPLY && tid == 0) bulk_wait_read<0>();     // the previous tile has left the buffer
+        cp_async_wait_all();
+        if (tid == 0) s_bound = hi;
+        __syncthreads();                                 // rings complete, cursors settled, buffer free
+        stage_tile(s_tile, out, lo, hi, full, zero_first, use_bulk, tid);
+        uint32_t sub_lo = lo;
+        while (true) {
+            // a worker whose ring is full and ends inside the tile may have more entries there
+            if ((uint32_t)tid < W) {
+                const uint32_t cur = s_cur[tid];
+                if (s_len[tid] - cur >= win) {
+                    const uint32_t last = rg_idx[tid * win + ((cur + win - 1u) & mask)];
+                    if (last < hi) atomicMin(&s_bound, last + 1u);
+                }
+            }
+            __syncthreads();                             // (also: the staged tile is visible)
+            uint32_t bound = s_bound;
+            if (bound <= sub_lo) {                       // no progress: a list is not ascending
+                if (tid == 0) record_status(hdr, -1 /*GC_E_INVALID*/, sub_lo);
+                bound = hi;
+            }
+            for (uint32_t q = 0; q < W; ++q) {           // worker order
+                const uint32_t cur = s_cur[q];
+                const uint32_t avail = min(s_len[q] - cur, win);
+                uint32_t adv = 0;
+                for (uint32_t i0 = 0; i0 < win; i0 += kDecBlock) {
+                    const uint32_t i = i0 + (uint32_t)tid;
+                    const uint32_t slot = q * win + ((cur + i) & mask);
+                    const uint32_t ix = i < avail ? rg_idx[slot] : 0xFFFFFFFFu;
+                    const bool in = ix < bound;
+                    if (in) {
+                        if (ix >= sub_lo) s_tile[ix - lo] = __fadd_rn(s_tile[ix - lo], rg_val[slot]);
+                        else record_status(hdr, -1 /*GC_E_INVALID*/, ix);      // behind the cursor: skipped
+                    }
+                    const uint32_t c = (uint32_t)__syncthreads_count(in ? 1 : 0);   // next worker may start
+                    adv += c;
+                    if (c < (uint32_t)kDecBlock) break;                          // ascending: nothing more below the bound
+                }
+                if (tid == 0) { s_cur[q] = cur + adv; s_adv[q] = adv; }
+            }
+            if (tid == 0) s_bound = hi;
+            __syncthreads();                             // cursors moved
+            if (my_w < W) {                              // the consumed slots are topped up
+                const uint32_t cur = s_cur[my_w], len = s_len[my_w];
+                top_up(min(len, cur - s_adv[my_w] + win), min(len, cur + win));
+            }
+            if (bound >= hi) break;
+            cp_async_wait_all();
+            __syncthreads();
+            sub_lo = bound;
+        }
+        if (APPLY) {
+            apply_tile(ap, s_tile, lo, hi, full, tid);
+            continue;                                    // (the barrier at the top of the loop orders the reuse)
+        }
+        if (full && use_bulk) {
+            if (tid == 0) bulk_store_tile(out + lo, s_tile, (uint32_t)(kDecTile * sizeof(float)));
+        } else {
+            for (uint32_t q = tid; q < hi - lo; q += kDecBlock) out[lo + q] = s_tile[q];
+        }
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
+        record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
+    if (use_bulk && !APPLY && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 }  // namespace gc

@@ -16,6 +16,16 @@ def _built():
     api.lib()
 
 
+ROUTES = {"auto": api.GC_DECODE_AUTO, "narrow": api.GC_DECODE_NARROW, "wide": api.GC_DECODE_WIDE}
+
+
+def routed_plan(route, *args, **kwargs):
+    """A plan whose tiled decode is pinned to one of its two kernels (or left to choose)."""
+    plan = api.Plan(*args, **kwargs)
+    plan.set_option(api.GC_OPT_DECODE_ROUTE, ROUTES[route])
+    return plan
+
+
 def run_workers(sizes, density, W, seed, steps=1, dist_scale=None):
     """W workers compress `steps` times on GPU; returns plan, workers, last gradients (cpu)."""
     plan = api.Plan(sizes, density, device=0)
@@ -50,8 +60,9 @@ def synthetic_sets(plan, sizes, W, seed, share_every=0):
 @pytest.mark.parametrize("W", [1, 2, 8])
 @pytest.mark.parametrize("sizes,density", [([100_000], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02),
                                            ([40_000], 0.5)])
-def test_decode_matches_oracle_bitwise(W, sizes, density):
-    plan = api.Plan(sizes, density, device=0)
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_decode_matches_oracle_bitwise(W, sizes, density, route):
+    plan = routed_plan(route, sizes, density, device=0)
     ws = plan.alloc_workspace()
     pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=3, share_every=2)
     n = plan.total_n
@@ -74,11 +85,12 @@ def test_decode_matches_oracle_bitwise(W, sizes, density):
 
 
 @pytest.mark.parametrize("W", [3, 16, 33, 64])
-def test_decode_many_workers_and_unaligned_output(W):
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_decode_many_workers_and_unaligned_output(W, route):
     """Worker counts that are not powers of two, more than 32 workers, duplicate indices across
     workers, and a dense buffer that is only 4-byte aligned (no bulk copies)."""
     sizes = [70_001, 9, 20_000]
-    plan = api.Plan(sizes, 0.03, device=0)
+    plan = routed_plan(route, sizes, 0.03, device=0)
     ws = plan.alloc_workspace()
     n = plan.total_n
     pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=5, share_every=3)
@@ -91,6 +103,34 @@ def test_decode_many_workers_and_unaligned_output(W):
             want = oracle.decode_accumulate(pairs, before, zero_first)
             assert np.array_equal(to_np_u32(out), bits(want)), (W, shift, zero_first)
         assert backing[shift + n:].eq(3.0).all() and backing[:shift].eq(3.0).all()
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_OK
+
+
+@pytest.mark.parametrize("W,density", [(16, 0.01), (32, 0.01), (64, 0.004), (8, 0.04)])
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_decode_many_workers_at_one_percent(W, density, route):
+    """Sixteen and more workers at 1 % density (the all-gathered lists of as many ranks): a
+    worker's share of a tile exceeds four entries per thread, so the wider pre-load is taken;
+    plain decode in both modes and the fused momentum step."""
+    sizes = [1_000_003]
+    plan = routed_plan(route, sizes, density, device=0)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=17, share_every=5)
+    out = torch.full((n,), 2.0, device="cuda")
+    for zero_first in (True, False):
+        before = out.cpu().numpy().copy()
+        plan.decompress_accumulate(d_idx, d_val, None, out, zero_first, ws)
+        want = oracle.decode_accumulate(pairs, before, zero_first)
+        assert np.array_equal(to_np_u32(out), bits(want)), (W, zero_first)
+    gen = torch.Generator().manual_seed(3)
+    p = torch.randn(n, generator=gen); v = torch.randn(n, generator=gen) * 0.1
+    d_p, d_v = p.cuda(), v.cuda()
+    h_p, h_v = p.numpy().copy(), v.numpy().copy()
+    plan.decompress_apply_momentum(d_idx, d_val, None, d_p, d_v, 0.05, 0.9, 1.0 / W, ws)
+    oracle.decode_apply_momentum(pairs, h_p, h_v, 0.05, 0.9, 1.0 / W)
+    assert np.array_equal(to_np_u32(d_v), bits(h_v)) and np.array_equal(to_np_u32(d_p), bits(h_p))
     st, _ = plan.last_status(ws)
     assert st == api.GC_OK
 
@@ -126,8 +166,9 @@ def test_density_one_reproduces_the_dense_sum():
         assert not w.residual.any()
 
 
-def test_worker_order_is_observable_and_fixed():
-    plan = api.Plan([8], 1.0, device=0)
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_worker_order_is_observable_and_fixed(route):
+    plan = routed_plan(route, [8], 1.0, device=0)
     ws = plan.alloc_workspace()
     idx = torch.arange(8, dtype=torch.int32, device="cuda")
     a = torch.full((8,), 1e8, device="cuda")
@@ -139,8 +180,9 @@ def test_worker_order_is_observable_and_fixed():
     assert out.tolist() == [1.0] * 8
 
 
-def test_out_of_range_index_is_skipped_and_reported():
-    plan = api.Plan([100], 0.04, device=0)          # k = 4
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_out_of_range_index_is_skipped_and_reported(route):
+    plan = routed_plan(route, [100], 0.04, device=0)          # k = 4
     ws = plan.alloc_workspace()
     idx = torch.tensor([1, 50, 99, 100], dtype=torch.int32, device="cuda")
     val = torch.ones(4, device="cuda")
@@ -156,6 +198,24 @@ def test_out_of_range_index_is_skipped_and_reported():
     st, det = plan.last_status(ws)
     assert st == api.GC_E_INVALID and det == 3
     assert out.sum().item() == 3.0
+
+
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_list_that_is_not_ascending_is_reported_and_stays_in_bounds(route):
+    """A list whose indices step backwards across a tile boundary: the call ends, writes only
+    inside the dense buffer and leaves GC_E_INVALID in the status word."""
+    plan = routed_plan(route, [20_000], 0.0002, device=0)          # k = 4
+    assert plan.total_cap == 4
+    ws = plan.alloc_workspace()
+    idx = torch.tensor([9000, 5, 9001, 9002], dtype=torch.int32, device="cuda")
+    val = torch.ones(4, device="cuda")
+    backing = torch.full((20_000 + 64,), 7.0, device="cuda")
+    out = backing[32:32 + 20_000]
+    plan.decompress_accumulate([idx], [val], None, out, True, ws)
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_E_INVALID
+    assert backing[:32].eq(7.0).all() and backing[32 + 20_000:].eq(7.0).all()
+    assert 0.0 <= out.sum().item() <= 4.0
 
 
 def test_config4_eight_resnet_workers_decode():
@@ -182,11 +242,12 @@ def test_config4_eight_resnet_workers_decode():
 
 
 @pytest.mark.parametrize("W", [1, 3, 8])
-def test_one_tensor_lists_with_counts_use_their_length(W):
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_one_tensor_lists_with_counts_use_their_length(W, route):
     """Threshold-mode lists of a one-tensor plan: the slots hold `cap` pairs but only the first
     count[0] are valid; whatever lies behind them (here: junk indices) must not be applied."""
     n = 3_000_001
-    plan = api.Plan([n], 0.001, mode=api.GC_THRESHOLD, device=0)
+    plan = routed_plan(route, [n], 0.001, mode=api.GC_THRESHOLD, device=0)
     cap = plan.tensor_cap()[0]
     ws = plan.alloc_workspace()
     pairs, d_idx, d_val, d_cnt = [], [], [], []
@@ -212,9 +273,10 @@ def test_one_tensor_lists_with_counts_use_their_length(W):
 
 @pytest.mark.parametrize("W", [0, 1, 3, 16])
 @pytest.mark.parametrize("sizes,density", [([100_003], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02)])
-def test_decode_apply_momentum_matches_oracle_bitwise(W, sizes, density):
+@pytest.mark.parametrize("route", list(ROUTES))
+def test_decode_apply_momentum_matches_oracle_bitwise(W, sizes, density, route):
     """The decode with momentum SGD fused behind it: parameter and velocity after three steps."""
-    plan = api.Plan(sizes, density, device=0)
+    plan = routed_plan(route, sizes, density, device=0)
     ws = plan.alloc_workspace()
     n = plan.total_n
     gen = torch.Generator().manual_seed(7)
