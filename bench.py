@@ -349,9 +349,9 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     # CPU baseline: the oracle on a bounded sample of the same workload
     cpu = None
     if not args.no_cpu_baseline:
-        sn, sk, times = oracle_sample_run(w, min(n, 1 << 24), 2, 1)
+        sn, sk, times = oracle_sample_run(w, min(n, 1 << 26), 8, 1)           # about 10 s of CPU work
         cpu = {"value": 4.0 * sn * len(times) / sum(times) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"first {sn} elements of the workload gradient, k={sk}, 2 steps after 1 warm-up, "
+               "sample": f"first {sn} elements of the workload gradient, k={sk}, 8 steps after 1 warm-up, "
                          f"compress + decode, single thread"}
 
     line = {
