@@ -608,6 +608,56 @@ def run_exchange(args, w: synth.Workload, rank: int, world: int, local_rank: int
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- decode sweep
+def run_decode_sweep(args, w: synth.Workload, rank: int, world: int, local_rank: int):
+    """Fourth workload (`--workload decode`): gc_decompress_accumulate alone on W seeded sparse sets
+    shaped like the workload's top-k output (a flat tensor of the workload's size and density), for
+    every W in --decode-workers and each of the two tiled decode kernels.  Prints its own JSON line."""
+    from paper_2104_01981_b200 import api
+    if rank != 0:
+        return
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    api.lib()
+    n = w.total_n
+    plan = api.Plan([n], w.density, device=local_rank)
+    k = plan.total_cap
+    ws = plan.alloc_workspace()
+    dense = torch.empty(n, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    peak, peak_src = measured_peak_gbs()
+    Ws = [int(x) for x in args.decode_workers.split(",")]
+    idx, val = [], []
+    for wk in range(max(Ws)):
+        i, v = synth.sparse_set([n], [k], 4000 + wk)
+        idx.append(torch.from_numpy(i.view(np.int32)).to(dev)); val.append(torch.from_numpy(v).to(dev))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    routes = {"auto": api.GC_DECODE_AUTO, "narrow": api.GC_DECODE_NARROW, "wide": api.GC_DECODE_WIDE}
+    rows = []
+    for W in Ws:
+        row = {"workers": W, "bytes": 4 * n + 8 * k * W}
+        for name, code in routes.items():
+            plan.set_option(api.GC_OPT_DECODE_ROUTE, code)
+            for _ in range(max(args.warmup, 3)):
+                plan.decompress_accumulate(idx[:W], val[:W], None, dense, True, ws, stream)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(args.steps):
+                plan.decompress_accumulate(idx[:W], val[:W], None, dense, True, ws, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / args.steps * 1e3
+            row[name + "_us"] = us
+            row[name + "_frac_of_measured_peak"] = row["bytes"] / us / 1e3 / peak
+        rows.append(row)
+    st, det = plan.last_status(ws)
+    if st != api.GC_OK:
+        raise RuntimeError(f"device status {st} (detail {det})")
+    print(json.dumps({"workload": w.name + "_decode_sweep", "elements": n, "pairs_per_worker": k, "density": w.density,
+                      "steps": args.steps, "peak_GB_per_s": peak, "peak_source": peak_src, "rows": rows,
+                      "l2": "dense buffer larger than L2 (no flush)"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -626,9 +676,11 @@ def main():
                     help="distinct gradients per worker cycled through (1 keeps profiler captures small)")
     ap.add_argument("--grad-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of the gradient (bf16: gc_compress_bf16, 10n + 8k bytes per compress; no e2e leg)")
-    ap.add_argument("--workload", default="gc", choices=["gc", "ecrm", "exchange"],
+    ap.add_argument("--decode-workers", default="1,2,4,8,16,32", help="worker counts of --workload decode")
+    ap.add_argument("--workload", default="gc", choices=["gc", "ecrm", "exchange", "decode"],
                     help="gc: gradient compression (the headline line); ecrm: erasure-coded embedding-table rows; "
-                         "exchange: one worker per rank, NCCL all-gather of the pairs, decode of all ranks' lists")
+                         "exchange: one worker per rank, NCCL all-gather of the pairs, decode of all ranks' lists; "
+                         "decode: the decode alone for several worker counts and both tiled kernels")
     ap.add_argument("--ecrm-rows", type=int, default=8 * 1024 * 1024, help="rows of the embedding-table shard")
     ap.add_argument("--ecrm-batch", type=int, default=1024 * 1024, help="distinct rows one batch updates")
     args = ap.parse_args()
@@ -652,6 +704,8 @@ def main():
             run_ecrm(args, rank, world, local_rank)
         elif args.workload == "exchange":
             run_exchange(args, w, rank, world, local_rank)
+        elif args.workload == "decode":
+            run_decode_sweep(args, w, rank, world, local_rank)
         else:
             run_gpu(args, w, rank, world, local_rank)
     finally:
