@@ -649,6 +649,19 @@ def run_decode_sweep(args, w: synth.Workload, rank: int, world: int, local_rank:
             us = e0.elapsed_time(e1) / args.steps * 1e3
             row[name + "_us"] = us
             row[name + "_frac_of_measured_peak"] = row["bytes"] / us / 1e3 / peak
+        # no fixed order among the workers (within 1e-6 relative of the fixed-order sum up to 16 workers)
+        plan.set_option(api.GC_OPT_DECODE_ROUTE, api.GC_DECODE_AUTO)
+        plan.set_option(api.GC_OPT_DECODE_ORDER, api.GC_ORDER_ANY)
+        for _ in range(max(args.warmup, 3)):
+            plan.decompress_accumulate(idx[:W], val[:W], None, dense, True, ws, stream)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            plan.decompress_accumulate(idx[:W], val[:W], None, dense, True, ws, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        row["any_order_us"] = e0.elapsed_time(e1) / args.steps * 1e3
+        plan.set_option(api.GC_OPT_DECODE_ORDER, api.GC_ORDER_FIXED)
         rows.append(row)
     st, det = plan.last_status(ws)
     if st != api.GC_OK:

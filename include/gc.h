@@ -117,6 +117,15 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                GC_DECODE_NARROW pre-loads 4 x (256 / W) pairs per worker in
  *                                registers, GC_DECODE_WIDE keeps up to 4096 / W pairs per worker in
  *                                shared-memory rings (many workers, dense lists).  Same result.
+ *   GC_OPT_DECODE_ORDER          GC_ORDER_FIXED (default): every element's contributions are added in
+ *                                worker order 0..W-1, so the result is bit-reproducible.
+ *                                GC_ORDER_ANY: the contributions of an element that several workers
+ *                                hit are added in an order that may change from run to run (shared-
+ *                                memory atomics; faster for 16 and more workers); each result lies
+ *                                within (hits - 1) x 2^-24 x sum |values| of the fixed-order one and
+ *                                equals it where one worker hits.  Applies to the tiled decode of
+ *                                both decode calls; lists with counts of many-tensor plans keep
+ *                                their fixed-order route.
  * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
  */
 #define GC_OPT_PATH                  0
@@ -126,6 +135,9 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
 #define GC_DECODE_AUTO   0
 #define GC_DECODE_NARROW 1
 #define GC_DECODE_WIDE   2
+#define GC_OPT_DECODE_ORDER          4
+#define GC_ORDER_FIXED   0
+#define GC_ORDER_ANY     1
 #define GC_PATH_AUTO   0
 #define GC_PATH_EXACT  1
 #define GC_PATH_STAGED 2

@@ -26,6 +26,8 @@ GC_K_COUNT = 16
  GC_Q_KERNEL_LAUNCHES, GC_Q_CANDIDATE_CAPACITY) = range(13)
 GC_OPT_PATH, GC_OPT_SAMPLE_RANK_PERMILLE, GC_OPT_CANDIDATE_CAPACITY, GC_OPT_DECODE_ROUTE = 0, 1, 2, 3
 GC_DECODE_AUTO, GC_DECODE_NARROW, GC_DECODE_WIDE = 0, 1, 2
+GC_OPT_DECODE_ORDER = 4
+GC_ORDER_FIXED, GC_ORDER_ANY = 0, 1
 GC_PATH_AUTO, GC_PATH_EXACT, GC_PATH_STAGED = 0, 1, 2
 
 _ERR = {GC_E_INVALID: "GC_E_INVALID", GC_E_UNSUPPORTED: "GC_E_UNSUPPORTED", GC_E_CUDA: "GC_E_CUDA",

@@ -36,6 +36,7 @@ struct gc_plan_s {
     uint32_t n_sampled = 0;                 // tensors with a sample
     int path = 0;                           // GC_PATH_AUTO or GC_PATH_EXACT
     int decode_route = 0;                   // GC_DECODE_AUTO, GC_DECODE_NARROW or GC_DECODE_WIDE
+    int decode_order = 0;                   // GC_ORDER_FIXED or GC_ORDER_ANY
     uint32_t rank_permille = 1000;          // scales the sample rank (testing aid)
     // workspace layout (byte offsets)
     size_t off_sel = 0, off_ssel = 0, off_gsel = 0, off_hist = 0, off_state = 0, off_gstate = 0,
@@ -375,6 +376,7 @@ int blocks_per_sm(K kernel, int threads) {
 // or dense lists) go to the wide kernel, which keeps `win` entries per worker in shared memory.
 struct DecodeRoute {
     bool wide = false;
+    bool any = false;           // (with wide) the kernel that adds without a fixed worker order
     uint32_t win = 0;
     size_t smem = 0;
     int grid = 0;
@@ -389,7 +391,9 @@ static DecodeRoute decode_route(gc_plan_t* p, uint32_t W) {
     while (Wp < W && Wp < 64) Wp <<= 1;
     const uint64_t narrow_window = (uint64_t)kDecRounds * (kDecBlock / Wp);
     // measured: the narrow kernel wins as long as most tiles fit its window
-    r.wide = p->decode_route == GC_DECODE_AUTO ? avg + avg / 4 > narrow_window : p->decode_route == GC_DECODE_WIDE;
+    r.any = p->decode_order == GC_ORDER_ANY;
+    r.wide = r.any || (p->decode_route == GC_DECODE_AUTO ? avg + avg / 4 > narrow_window
+                                                          : p->decode_route == GC_DECODE_WIDE);
     if (!r.wide) return r;
     uint32_t win = 32;
     while (win < need && win < 1024) win <<= 1;
@@ -397,13 +401,17 @@ static DecodeRoute decode_route(gc_plan_t* p, uint32_t W) {
     r.win = win;
     r.smem = kDecTileBytes + 8 * (size_t)W * win;
     int nb = -1;
-    for (auto& e : p->wide_occ[APPLY ? 1 : 0]) if (e.first == r.smem) nb = e.second;
+    const size_t key = r.smem + (r.any ? 1 : 0);          // (shared-memory sizes are multiples of 256)
+    for (auto& e : p->wide_occ[APPLY ? 1 : 0]) if (e.first == key) nb = e.second;
     if (nb < 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_wide<APPLY>, kDecBlock, r.smem) != cudaSuccess) {
+        const cudaError_t eo = r.any
+            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_any<APPLY>, kDecBlock, r.smem)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_wide<APPLY>, kDecBlock, r.smem);
+        if (eo != cudaSuccess) {
             (void)cudaGetLastError();
             nb = 0;
         }
-        p->wide_occ[APPLY ? 1 : 0].emplace_back(r.smem, nb);
+        p->wide_occ[APPLY ? 1 : 0].emplace_back(key, nb);
     }
     r.grid = p->sm_count * nb;
     if (r.grid <= 0) r.wide = false;
@@ -546,6 +554,10 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     p->wide_ok = cudaFuncSetAttribute(k_decode_wide<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess &&
                  cudaFuncSetAttribute(k_decode_wide<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess &&
+                 cudaFuncSetAttribute(k_decode_any<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess &&
+                 cudaFuncSetAttribute(k_decode_any<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess;
     (void)cudaGetLastError();
     p->grid_sample = p->sm_count * blocks_per_sm(k_hist<0, SRC_SAMPLE>, kBlock);
@@ -572,6 +584,10 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
         case GC_OPT_CANDIDATE_CAPACITY:
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
             p->cand_cap = (uint32_t)value;
+            return GC_OK;
+        case GC_OPT_DECODE_ORDER:
+            if (value != GC_ORDER_FIXED && value != GC_ORDER_ANY) return GC_E_INVALID;
+            p->decode_order = (int)value;
             return GC_OK;
         case GC_OPT_DECODE_ROUTE:
             if (value != GC_DECODE_AUTO && value != GC_DECODE_NARROW && value != GC_DECODE_WIDE) return GC_E_INVALID;
@@ -877,7 +893,8 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         Timed tm(p, s, GC_K_DECODE_TILES);
         const DecodeRoute rt = decode_route<false>(p, W);
         if (rt.wide) {
-            k_decode_wide<false><<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
+            auto kw = rt.any ? k_decode_any<false> : k_decode_wide<false>;
+            kw<<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
                 ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, dense_out, zero_first ? 1 : 0, use_bulk, rt.win,
                 ws.hdr, ApplyArgs{});
             GC_CUDA(p, cudaGetLastError());
@@ -938,7 +955,8 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
     Timed tm(p, s, GC_K_DECODE_TILES);
     const DecodeRoute rt = decode_route<true>(p, W);
     if (rt.wide) {
-        k_decode_wide<true><<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
+        auto kw = rt.any ? k_decode_any<true> : k_decode_wide<true>;
+        kw<<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
             ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, nullptr, 1, 0, rt.win, ws.hdr, ap);
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;

@@ -356,4 +356,115 @@ k_decode_wide(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float*
     if (use_bulk && !APPLY && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
+// Decode without a fixed order among the workers (GC_OPT_DECODE_ORDER = GC_ORDER_ANY): the rings
+// of k_decode_wide, but all entries of a pass are added at once with shared-memory atomics, so
+// a tile costs a constant number of block-wide steps whatever W is.  The sum of an element that
+// several workers hit is then rounded in an order that may change from run to run: every result
+// is within (hits - 1) x 2^-24 x sum |values| of the fixed-order one, and equal to it for
+// elements hit once.
+template <bool APPLY>
+static __global__ void __launch_bounds__(kDecBlock)
+k_decode_any(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float* __restrict__ out,
+             int zero_first, int use_bulk, uint32_t win, WsHeader* hdr, ApplyArgs ap) {
+    extern __shared__ __align__(128) float s_tiles[];
+    float* const s_tile = s_tiles;
+    uint32_t* const rg_idx = reinterpret_cast<uint32_t*>(s_tiles + kDecTile);      // [W][win]
+    float* const rg_val = reinterpret_cast<float*>(rg_idx + W * win);              // [W][win]
+    __shared__ uint32_t s_cur[64], s_len[64], s_adv[64], s_bound;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
+    const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
+    if (t0 >= t1) return;
+    const uint32_t mask = win - 1u;
+    // E consecutive threads serve one worker: they top up its ring and add its entries
+    int Wp = 1;
+    while (Wp < (int)W && Wp < 64) Wp <<= 1;
+    const int E = kDecBlock / Wp;
+    const uint32_t my_w = (uint32_t)(tid / E);
+    const int sub = tid % E;
+
+    for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
+        const uint32_t len = ls.len[w] != nullptr ? min(__ldg(ls.len[w]), cnt) : cnt;
+        const uint32_t c = warp_lower_bound(ls.idx[w], len, t0 * (uint32_t)kDecTile, lane);
+        if (lane == 0) { s_cur[w] = c; s_len[w] = len; s_adv[w] = 0u; }
+    }
+    __syncthreads();
+    auto top_up = [&](uint32_t from, uint32_t to) {      // list positions [from, to) of worker my_w go to their ring slots
+        for (uint32_t p = from + (uint32_t)sub; p < to; p += (uint32_t)E) {
+            cp_async_4(rg_idx + my_w * win + (p & mask), ls.idx[my_w] + p);
+            cp_async_4(rg_val + my_w * win + (p & mask), ls.val[my_w] + p);
+        }
+    };
+    if (my_w < W) top_up(s_cur[my_w], min(s_len[my_w], s_cur[my_w] + win));
+
+    for (uint32_t tl = t0; tl < t1; ++tl) {
+        const uint32_t lo = tl * (uint32_t)kDecTile;
+        const uint32_t hi = min(total_n, lo + (uint32_t)kDecTile);
+        const bool full = hi - lo == (uint32_t)kDecTile;
+        if (use_bulk && !APPLY && tid == 0) bulk_wait_read<0>();     // the previous tile has left the buffer
+        cp_async_wait_all();
+        if (tid == 0) s_bound = hi;
+        __syncthreads();                                 // rings complete, cursors settled, buffer free
+        stage_tile(s_tile, out, lo, hi, full, zero_first, use_bulk, tid);
+        uint32_t sub_lo = lo;
+        while (true) {
+            if ((uint32_t)tid < W) {                     // a full ring that ends inside the tile may hide more entries
+                const uint32_t cur = s_cur[tid];
+                s_adv[tid] = 0u;
+                if (s_len[tid] - cur >= win) {
+                    const uint32_t last = rg_idx[tid * win + ((cur + win - 1u) & mask)];
+                    if (last < hi) atomicMin(&s_bound, last + 1u);
+                }
+            }
+            __syncthreads();                             // (also: the staged tile is visible)
+            uint32_t bound = s_bound;
+            if (bound <= sub_lo) {                       // no progress: a list is not ascending
+                if (tid == 0) record_status(hdr, -1 /*GC_E_INVALID*/, sub_lo);
+                bound = hi;
+            }
+            if (my_w < W) {
+                const uint32_t cur = s_cur[my_w];
+                const uint32_t avail = min(s_len[my_w] - cur, win);
+                uint32_t below = 0;
+                for (uint32_t i = (uint32_t)sub; i < avail; i += (uint32_t)E) {
+                    const uint32_t slot = my_w * win + ((cur + i) & mask);
+                    const uint32_t ix = rg_idx[slot];
+                    if (ix >= bound) break;                                      // ascending: the rest lies above
+                    ++below;
+                    if (ix < sub_lo) { record_status(hdr, -1 /*GC_E_INVALID*/, ix); continue; }   // behind the cursor: skipped
+                    atomicAdd(&s_tile[ix - lo], rg_val[slot]);
+                }
+                if (below) atomicAdd(&s_adv[my_w], below);
+            }
+            __syncthreads();                             // the tile is complete up to the bound
+            if ((uint32_t)tid < W) s_cur[tid] += s_adv[tid];
+            if (tid == 0) s_bound = hi;
+            __syncthreads();                             // cursors moved
+            if (my_w < W) {                              // the consumed slots are topped up
+                const uint32_t nc = s_cur[my_w], len = s_len[my_w];
+                top_up(min(len, nc - s_adv[my_w] + win), min(len, nc + win));
+            }
+            if (bound >= hi) break;
+            cp_async_wait_all();
+            __syncthreads();
+            sub_lo = bound;
+        }
+        if (APPLY) {
+            apply_tile(ap, s_tile, lo, hi, full, tid);
+            continue;                                    // (the barrier at the top of the loop orders the reuse)
+        }
+        if (full && use_bulk) {
+            if (tid == 0) bulk_store_tile(out + lo, s_tile, (uint32_t)(kDecTile * sizeof(float)));
+        } else {
+            for (uint32_t q = tid; q < hi - lo; q += kDecBlock) out[lo + q] = s_tile[q];
+        }
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
+        record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
+    if (use_bulk && !APPLY && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 }  // namespace gc

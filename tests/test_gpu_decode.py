@@ -343,3 +343,40 @@ def test_random_plans_and_worker_counts_match_the_oracle(seed):
     assert np.array_equal(to_np_u32(d_p), bits(p0)) and np.array_equal(to_np_u32(d_v), bits(v0))
     st, det = plan.last_status(ws)
     assert st == api.GC_OK, (st, det)
+
+
+@pytest.mark.parametrize("W,density,share", [(1, 0.01, 0), (4, 0.02, 2), (16, 0.01, 0), (16, 0.01, 4), (8, 0.3, 0)])
+def test_any_order_decode_stays_within_the_rounding_bound(W, density, share):
+    """GC_ORDER_ANY: elements hit by one worker equal the fixed-order result bit for bit; the
+    others lie within (hits - 1) x 2^-24 x sum |values| of it, which is below the 1e-6 relative
+    bound for up to 16 workers.  Plain decode, accumulate mode and the fused momentum step."""
+    sizes = [300_007, 8193]
+    plan = api.Plan(sizes, density, device=0)
+    plan.set_option(api.GC_OPT_DECODE_ORDER, api.GC_ORDER_ANY)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    pairs, d_idx, d_val = synthetic_sets(plan, sizes, W, seed=31, share_every=share)
+    hits = np.zeros(n, np.int64)
+    mag = np.zeros(n, np.float64)
+    for i, v in pairs:
+        np.add.at(hits, i, 1)
+        np.add.at(mag, i, np.abs(v.astype(np.float64)))
+    out = torch.full((n,), 0.5, device="cuda")
+    for zero_first in (True, False):
+        before = out.cpu().numpy().copy()
+        plan.decompress_accumulate(d_idx, d_val, None, out, zero_first, ws)
+        want = oracle.decode_accumulate(pairs, before.copy(), zero_first)
+        got = out.cpu().numpy()
+        lone = hits <= (1 if zero_first else 0)
+        assert np.array_equal(got[lone].view(np.uint32), want[lone].view(np.uint32))
+        bound = 1e-6 * (mag + np.abs(before.astype(np.float64)) * (0 if zero_first else 1))
+        assert np.all(np.abs(got.astype(np.float64) - want.astype(np.float64)) <= bound + 1e-30), (W, zero_first)
+    p0 = np.random.default_rng(5).standard_normal(n).astype(np.float32)
+    v0 = (p0 * np.float32(0.1)).astype(np.float32)
+    d_p, d_v = torch.from_numpy(p0.copy()).cuda(), torch.from_numpy(v0.copy()).cuda()
+    plan.decompress_apply_momentum(d_idx, d_val, None, d_p, d_v, 0.05, 0.9, 1.0, ws)
+    oracle.decode_apply_momentum(pairs, p0, v0, 0.05, 0.9, 1.0)
+    assert np.all(np.abs(d_v.cpu().numpy().astype(np.float64) - v0) <= 1e-6 * (mag + np.abs(v0)) + 1e-30)
+    assert np.all(np.abs(d_p.cpu().numpy().astype(np.float64) - p0) <= 1e-6 * (mag + np.abs(p0) + np.abs(v0)) + 1e-30)
+    st, det = plan.last_status(ws)
+    assert st == api.GC_OK, (st, det)
