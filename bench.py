@@ -225,7 +225,6 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     e1.record(stream)
     barrier()
     ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None
     per_kernel = plan.profile_read()
     launches = plan.launches() - launches0
     plan.profile_enable(0)
@@ -243,6 +242,7 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     e1.record(stream)
     barrier()
     ms_plain = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None          # sampled across both timed loops
 
     # ---- timed regions 1c/1d: the two halves on their own (no per-kernel events)
     def compress_only(i: int):
