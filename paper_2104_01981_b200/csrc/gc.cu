@@ -50,6 +50,7 @@ struct gc_plan_s {
     // single-tensor shared-memory-pool kernel
     int grid_single_max = 0;                // resident CTAs (0 = not available)
     uint32_t single_grid = 0, single_maxt = 0, single_pool = 0;   // 0 = plan does not qualify
+    RowMap single_rows = {};
     size_t single_smem = 0;
     size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0;
     uint32_t single_srank_hi = 0, single_srank_mid = 0;
@@ -81,6 +82,9 @@ constexpr size_t kSingleMidCap = 65536;      // short list of k_topk_single (can
 constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tensor
 constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
 constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
+// Share of the oldest CTA of an SM above (and of the youngest below) the middle one's: measured
+// best between 6 and 10 % on the 110M-element workload.
+constexpr double kSingleSkew = 0.08;
 constexpr size_t kSingleRowBytes = (2 * kWarps + 3) * sizeof(uint32_t);   // shared memory per owned tile
 constexpr uint32_t kMultiMaxTab = 1024;      // tensors whose tile tables k_topk_multi keeps in shared memory
 constexpr size_t kMultiMaxPer = 160;         // most tiles one CTA of k_topk_multi may own
@@ -245,8 +249,28 @@ void plan_single(gc_plan_s* p) {
     const TensorDesc& d = p->desc[0];
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
-    const uint32_t maxt = (d.ntiles + G - 1) / G;
+    uint32_t maxt = (d.ntiles + G - 1) / G;
+    // shares of the tensor: equal, or - when the launch fills every SM three CTAs deep - in the
+    // proportion in which the oldest, middle and youngest CTA of an SM advance
+    RowMap rm;
+    rm.G = G; rm.gA = G; rm.n0 = rm.n1 = rm.n2 = maxt; rm.s1 = rm.s2 = maxt * G;
+    if (G == 3u * (uint32_t)p->sm_count && d.ntiles >= 12u * G) {
+        const uint32_t gA = (uint32_t)p->sm_count;
+        const uint32_t total = (d.ntiles + gA - 1) / gA;             // rows of the three classes together
+        const uint32_t n1 = maxt;
+        const uint32_t dd = std::max<uint32_t>(1u, (uint32_t)((double)d.ntiles / G * kSingleSkew + 0.5));
+        const uint32_t n0 = n1 + dd;
+        if (total > n0 + n1 && total - n0 - n1 <= n1) {
+            rm.gA = gA; rm.n0 = n0; rm.n1 = n1; rm.n2 = total - n0 - n1;
+            rm.s1 = rm.n2 * G; rm.s2 = rm.s1 + (rm.n1 - rm.n2) * 2u * gA;
+            maxt = n0;
+        }
+    }
     if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
+    if (d.ntiles >= (1u << 20)) return;                              // (the row arithmetic divides by multiplication)
+    rm.mG = (uint32_t)((1ull << 32) / rm.G) + 1u;
+    rm.m2A = (uint32_t)((1ull << 32) / (2u * rm.gA)) + 1u;
+    rm.mA = (uint32_t)((1ull << 32) / rm.gA) + 1u;
     // region per CTA; one bit per slot has to fit in shared memory beside the chunk records
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
     const size_t rec_bytes = (size_t)maxt * kSingleRowBytes + sizeof(uint32_t) * ((pool + 31) / 32);
@@ -261,6 +285,7 @@ void plan_single(gc_plan_s* p) {
     p->single_srank_hi = hi >= 1.0 ? (uint32_t)hi : 1u;    // small sample: the largest sampled key bounds the band
     p->single_srank_mid = (uint32_t)std::max(1.0, std::ceil(ks));
     p->single_grid = G; p->single_maxt = maxt; p->single_pool = pool; p->single_smem = rec_bytes;
+    p->single_rows = rm;
 }
 
 // Decides whether a threshold plan can use the one-tensor kernel and with which geometry.
@@ -743,7 +768,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     if (p->path == GC_PATH_AUTO && p->single_grid > 0) {
         // one large tensor: candidates stay in shared memory
         SingleArgs sa;
-        sa.d = p->desc[0]; sa.desc = p->d_desc; sa.ntiles = nt; sa.maxt = p->single_maxt;
+        sa.d = p->desc[0]; sa.desc = p->d_desc; sa.ntiles = nt; sa.maxt = p->single_maxt; sa.rows = p->single_rows;
         sa.pool_cap = std::min<uint32_t>(p->single_pool, p->cand_cap);
         sa.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
         sa.g = grad_any; sa.r = residual; sa.out_idx = out_idx; sa.out_val = out_val; sa.out_count = out_count;

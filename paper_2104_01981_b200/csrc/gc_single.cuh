@@ -45,10 +45,36 @@ __device__ __forceinline__ uint32_t fine_slot(uint32_t bin) { return (bin * 4050
 constexpr uint32_t kMidRegs = 4;                       // short-list entries a thread keeps in registers
 constexpr uint32_t kMidFast = kMidRegs * kBlock;       // short lists up to this size are read once
 
+// Rows of tiles.  A column is one CTA's share of the tensor: row i of column c is one tile, and
+// the tiles are numbered row by row.  The three CTAs that share an SM do not advance at the same
+// speed (the oldest one gets the most issue slots: with equal shares the first finished its fold
+// pass at 182 us, the third at 209 us on the 110M-element workload), so the columns come in
+// three classes of gA each with n0 >= n1 >= n2 rows, and every CTA takes a column of the class
+// that matches its age on its SM.  Row i is G wide below n2, 2 gA wide below n1, gA wide below
+// n0.  Plans that do not fill the GPU three CTAs deep use one class (gA = G, n0 = n1 = n2).
+struct RowMap {
+    uint32_t G, gA, n0, n1, n2;
+    uint32_t s1, s2;                 // first tile of row n2 and of row n1
+    uint32_t mG, m2A, mA;            // floor(2^32 / d) + 1 for d = G, 2 gA, gA: t / d = mulhi(t, m) for t < 2^20
+    __device__ __forceinline__ uint32_t rows_of(uint32_t c) const { return c < gA ? n0 : c < 2u * gA ? n1 : n2; }
+    __device__ __forceinline__ uint32_t tile_of(uint32_t i, uint32_t c) const {
+        return i < n2 ? i * G + c : i < n1 ? s1 + (i - n2) * 2u * gA + c : s2 + (i - n1) * gA + c;
+    }
+    __device__ __forceinline__ void locate(uint32_t t, uint32_t& row, uint32_t& col) const {
+        if (t < s1) { row = __umulhi(t, mG); col = t - row * G; }
+        else if (t < s2) { const uint32_t q = __umulhi(t - s1, m2A); row = n2 + q; col = t - s1 - q * 2u * gA; }
+        else { const uint32_t q = __umulhi(t - s2, mA); row = n1 + q; col = t - s2 - q * gA; }
+    }
+    __device__ __forceinline__ uint32_t row_of(uint32_t t) const {
+        return t < s1 ? __umulhi(t, mG) : t < s2 ? n2 + __umulhi(t - s1, m2A) : n1 + __umulhi(t - s2, mA);
+    }
+};
+
 struct SingleArgs {
     TensorDesc d;                    // the tensor (by value)
     const TensorDesc* desc;          // device table (for the redo phases)
     uint32_t ntiles, maxt, pool_cap; // tiles, max tiles per CTA, pool slots per CTA
+    RowMap rows;                     // which tile is row i of column c
     uint32_t srank_hi;               // sample rank of the upper bracket (at least 1)
     uint32_t srank_mid;              // sample rank that estimates the threshold itself
     uint32_t mid_cap;                // capacity of the short list
@@ -60,7 +86,7 @@ struct SingleArgs {
     uint2* cand;                     // [gridDim.x * pool_cap] candidate list, one region per CTA
     uint2* mid;                      // [mid_cap] candidates inside the band bin of the threshold
     uint32_t* hist5;                 // [0] coarse sample histogram, [2] band histogram,
-                                     // [3][0] short-list length (all zeroed)
+                                     // [3][0] short-list length, [4] CTAs per SM and per age class (all zeroed)
     uint32_t* fine;                  // [kFineBins] fine sample histogram (zeroed)
     uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
     uint32_t* seg_tot;               // [maxt][ceil(G/32)] the same summed over each run of 32 CTAs of a row (zeroed)
@@ -188,12 +214,21 @@ k_topk_single(SingleArgs a) {
     const TensorDesc& d = a.d;
     WsHeader* hdr = a.ws.hdr;
     uint32_t passed = 0, n_stamp = 0;
-    const uint32_t n_own = b < a.ntiles ? (a.ntiles - b + G - 1) / G : 0u;
+    const RowMap& rm = a.rows;
+    __shared__ uint32_t s_age[2];
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
-    for (uint32_t i = tid; i < n_own * kWarps; i += kBlock) rec2[i] = 0u;
-    for (uint32_t i = tid; i < n_own; i += kBlock) row_mid[i] = 0u;
-    const uint32_t nseg = (G + 31u) / 32u, myseg = b / 32u;
-    if (tid == 0) s_used = 0u;
+    for (uint32_t i = tid; i < a.maxt * kWarps; i += kBlock) rec2[i] = 0u;
+    for (uint32_t i = tid; i < a.maxt; i += kBlock) row_mid[i] = 0u;
+    const uint32_t nseg = (G + 31u) / 32u;
+    // This CTA's age among the CTAs of its SM = its arrival number at the SM's counter, taken
+    // first thing (the answer is only looked at once the sample loads are under way).
+    uint32_t my_age = 0;
+    if (tid == 0) {
+        s_used = 0u;
+        uint32_t smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        my_age = atomicAdd(a.hist5 + 4 * kHistBins + (smid & 1023u), 1u);
+    }
     phase_stamp(hdr, n_stamp);
 
     // ---------------------------------------------------------------- sample
@@ -202,6 +237,7 @@ k_topk_single(SingleArgs a) {
     // into global memory; few samples share a fine bin).  tau = the srank-th largest sampled
     // key cut to 16 bits; tau_hi = upper edge of the 16-bit cell of the srank_hi-th largest.
     uint32_t tau = 0, tau_hi = 0x80000000u, tau_z = 0;
+    uint32_t col = b, n_own = 0, myseg = 0;      // set after the first barrier
     {
         const uint32_t ngroups = (d.n + 3u) >> 2;
         const uint32_t nsg = (ngroups + d.sstride - 1) / d.sstride;
@@ -225,6 +261,11 @@ k_topk_single(SingleArgs a) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) skey[q][e] = key_of(__fadd_rn(gv[e], rv[e]));
         }
+        if (tid == 0) {
+            uint32_t smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            s_age[0] = my_age; s_age[1] = smid;
+        }
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kMaxOwn; ++q)
@@ -235,7 +276,7 @@ k_topk_single(SingleArgs a) {
                     atomicAdd(a.fine + fine_slot(skey[q][e] >> kFineShift), 1u);
                 }
         // the first own tile is asked into L2 while the sample is being settled
-        if (n_own) {
+        if (b < a.ntiles) {
             const uint32_t pb = (d.off & ~3u) + b * (uint32_t)kTile + warp * kWarpChunk + lane * 4;
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
@@ -248,6 +289,18 @@ k_topk_single(SingleArgs a) {
         flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr, n_stamp);
+        {   // Columns go to the CTAs by age, oldest first: column = age x gA + SM number.  That is
+            // a one-to-one assignment only if SMs 0..gA-1 hold three CTAs each; every CTA checks
+            // the same counters (all CTAs have registered by now) and otherwise keeps column b.
+            const uint32_t* const per_sm = a.hist5 + 4 * kHistBins;
+            const bool fits = (uint32_t)tid >= rm.gA || ld_cg(per_sm + tid) == 3u;
+            const bool none_beyond = (uint32_t)tid < rm.gA || tid >= 1024 || ld_cg(per_sm + tid) == 0u;
+            const bool aged = rm.gA * 3u == G && rm.gA <= (uint32_t)kBlock && __syncthreads_and(fits && none_beyond);
+            col = aged ? min(s_age[0], 2u) * rm.gA + s_age[1] : b;
+            n_own = rm.rows_of(col);
+            while (n_own > 0u && rm.tile_of(n_own - 1u, col) >= a.ntiles) --n_own;
+            myseg = col / 32u;
+        }
         // both brackets from one read of the coarse histogram, then the kFineBits finer bits of
         // each from the 2^kFineBits fine bins under its coarse bin (one warp per bracket)
         const uint32_t want[3] = {d.srank, a.srank_hi, a.srank_mid};
@@ -295,7 +348,7 @@ k_topk_single(SingleArgs a) {
     const uint32_t my_off = warp * kWarpChunk + lane * 4;
     bool block_overflow = false;
     for (uint32_t i = 0; i < n_own; ++i) {
-        const uint32_t tile = b + i * G;
+        const uint32_t tile = rm.tile_of(i, col);
         const TileGeom tg = tile_geom(d, tile);
         const bool interior = tg.lo == tg.base && tg.hi == tg.base + (uint32_t)kTile;
         float av[kVpt][4];
@@ -430,7 +483,7 @@ k_topk_single(SingleArgs a) {
             const uint32_t bin = min(((pr.y & kKeyMask) - tau) >> shift, 2047u);
             if (bin > A) {
                 const uint32_t rel = pr.x - base0;
-                atomicAdd(&rec2[((rel >> 12) / G) * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
+                atomicAdd(&rec2[rm.row_of(rel >> 12) * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
             } else if (bin == A) {
                 const uint32_t slot = atomicAdd(a.hist5 + 3 * kHistBins, 1u);
                 if (slot < a.mid_cap) a.mid[slot] = pr;
@@ -455,7 +508,7 @@ k_topk_single(SingleArgs a) {
             uint32_t tot = 0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) tot += rec2[i * kWarps + w];
-            a.tile_cnt[b + i * G] = tot;
+            a.tile_cnt[rm.tile_of(i, col)] = tot;
             atomicAdd(a.seg_tot + (size_t)i * nseg + myseg, tot);
         }
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
@@ -478,7 +531,7 @@ k_topk_single(SingleArgs a) {
             for (int u = 0; u < 2; ++u) {
                 const uint32_t i = i0 + u, q = myseg * 32u + (uint32_t)lane;
                 sv[u] = (i < n_own && (uint32_t)lane < nseg) ? ld_cg(a.seg_tot + (size_t)i * nseg + lane) : 0u;
-                tv[u] = (i < n_own && q < b) ? ld_cg(a.tile_cnt + (size_t)i * G + q) : 0u;
+                tv[u] = (i < n_own && q < col) ? ld_cg(a.tile_cnt + rm.tile_of(i, q)) : 0u;
             }
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
@@ -535,10 +588,12 @@ k_topk_single(SingleArgs a) {
             };
             auto below = [&](const uint2& pr) {
                 if (!sent_key(pr)) return;
-                const uint32_t rel = pr.x - base0, t = rel >> 12, row = t / G, owner = t - row * G;
-                const uint32_t first = row + (owner < b ? 0u : 1u);
+                const uint32_t rel = pr.x - base0;
+                uint32_t row, owner;
+                rm.locate(rel >> 12, row, owner);
+                const uint32_t first = row + (owner < col ? 0u : 1u);
                 if (first < n_own) atomicAdd(&row_mid[first], 1u);
-                if (owner == b) atomicAdd(&rec2[row * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
+                if (owner == col) atomicAdd(&rec2[row * kWarps + ((rel >> 9) & (kWarps - 1u))], 1u);
             };
 #pragma unroll
             for (uint32_t u = 0; u < kMidRegs; ++u)
@@ -607,7 +662,7 @@ k_topk_single(SingleArgs a) {
                     }
                     if (!zeroed) a.r[pr[u].x] = 0.0f;
                     const uint32_t rel = pr[u].x - base0;
-                    const uint32_t c = ((rel >> 12) / G) * kWarps + ((rel >> 9) & (kWarps - 1u));
+                    const uint32_t c = rm.row_of(rel >> 12) * kWarps + ((rel >> 9) & (kWarps - 1u));
                     const uint32_t s = rec[c] >> 10;                   // first list position of the chunk
                     uint32_t before;
                     if ((s >> 5) == (i >> 5)) {

@@ -97,6 +97,26 @@ def test_config5_gpt2_medium_full_size_two_workers():
         torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("n,density,quantised", [(24_000_001, 0.01, True), (21_823_500, 0.003, False),
+                                                (47_999_999, 0.01, False)])
+def test_one_tensor_with_unequal_shares_per_cta(n, density, quantised):
+    """Tensors of twelve and more rows of tiles per CTA column: the one-tensor kernel gives the
+    three CTAs of an SM unequal numbers of rows (the last rows are only partly filled).  Three
+    error-feedback steps, one of them with values quantised to 1/8 (thousands of ties at the
+    threshold); also the safety-net routes on the same geometry."""
+    gen = torch.Generator(device="cuda").manual_seed(n % 1000)
+    grads = []
+    for s in range(3):
+        g = torch.randn(n, device="cuda", generator=gen)
+        if quantised and s == 1:
+            g = torch.round(g * 8) / 8
+        grads.append(g)
+    check_topk_against_oracle([n], density, grads)
+    if quantised:
+        check_topk_against_oracle([n], density, grads[:2], options={api.GC_OPT_SAMPLE_RANK_PERMILLE: 30})
+        check_topk_against_oracle([n], density, grads[:1], options={api.GC_OPT_CANDIDATE_CAPACITY: 100})
+
+
 PATHS = {
     "auto": {},
     "exact": {api.GC_OPT_PATH: api.GC_PATH_EXACT},
