@@ -3,8 +3,10 @@
 //
 // Same idea as the general candidate path (sample -> fold + candidates -> select on the
 // candidates -> index-ordered emission, exact multi-pass redo as the safety net), specialised:
-//   * CTA b owns tiles b, b + G, b + 2G, ... (G = grid size): every CTA sees every region of
-//     the tensor, so candidate counts stay balanced even when magnitudes differ between layers;
+//   * a CTA owns one column of a row map over the tiles (in the simplest case tiles c, c + G,
+//     c + 2G, ... for column c; see RowMap for the unequal shares of large tensors): every CTA
+//     sees every region of the tensor, so candidate counts stay balanced even when magnitudes
+//     differ between layers;
 //   * a CTA appends the candidates of its own tiles to a private, contiguous region of the
 //     candidate list (L2-resident) and keeps the per-chunk records in shared memory.  (Holding
 //     the candidates themselves in shared memory was measured slower: the large carve-out
@@ -25,7 +27,7 @@
 //     shared memory);
 //   * every histogram is flushed to global memory and, after the grid barrier, EVERY CTA scans
 //     it and derives the same result -- no completion counters, no designated CTA;
-//   * output slots come from per-row totals: row i is the i-th tile of every CTA.
+//   * output slots come from per-row totals: row i holds the i-th tile of every column.
 // Nothing here is probabilistic in its result: the counts decide, and whenever the bracket
 // misses (or a list overflows) the exact multi-pass kernels redo the tensor.
 #pragma once
