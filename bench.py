@@ -341,7 +341,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
     # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
     ncu_traffic, ncu_src = {
-        ("c3_bert_base_110m_student_t", "topk", "compress_fused"): (1361.5e6, "profiles/k_topk_single_c3_bert110m.md"),
+        ("c3_bert_base_110m_student_t", "topk", "compress_fused"): (1374.4e6, "profiles/k_topk_single_c3_bert110m.md"),
         ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): (1407.5e6, "profiles/k_threshold_single_c3_bert110m.md"),
         ("c2_resnet50_layerwise", "topk", "compress_fused"): (322.1e6, "profiles/k_topk_multi_c2_resnet50.md"),
     }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None, (None, None))
