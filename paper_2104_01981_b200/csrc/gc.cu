@@ -52,7 +52,7 @@ struct gc_plan_s {
     uint32_t single_grid = 0, single_maxt = 0, single_pool = 0;   // 0 = plan does not qualify
     RowMap single_rows = {};
     size_t single_smem = 0;
-    size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0;
+    size_t off_hist5 = 0, off_rowseg = 0, off_mid = 0, off_fine = 0, off_age = 0;
     uint32_t single_srank_hi = 0, single_srank_mid = 0;
     int grid_thr_single_max = 0;
     uint32_t thr_grid = 0, thr_maxt = 0, thr_pool = 0, thr_rounds = 0;    // one-tensor threshold kernel (0 = no)
@@ -226,6 +226,8 @@ void finish_layout(gc_plan_s* p) {
     p->control_bytes = align_up(p->off_rowseg + (T == 1 ? sizeof(uint32_t) * kSingleMaxT * 20 : 0), 256);
     p->off_fine = p->control_bytes;
     p->control_bytes = align_up(p->off_fine + (T == 1 ? sizeof(uint32_t) * (size_t)kFineBins : 0), 256);
+    p->off_age = p->control_bytes;                                   // CTAs arrived per SM (one-tensor kernels)
+    p->control_bytes = align_up(p->off_age + (T == 1 ? sizeof(uint32_t) * 1024 : 0), 256);
     // many-tensor kernel: sample and band histogram per tensor, short-list lengths
     const size_t multi_hist = T >= 2 ? sizeof(uint32_t) * (size_t)kHistBins * T : 0;
     p->off_shist = p->control_bytes;
@@ -242,6 +244,31 @@ void finish_layout(gc_plan_s* p) {
 }
 
 
+// Shares of a one-tensor plan's CTAs: equal, or - when the launch fills every SM three CTAs deep
+// and every column has at least twelve rows - in the proportion in which the oldest, middle and
+// youngest CTA of an SM advance.  `maxt` comes in as the rows of an equal share and goes out as
+// the rows of the largest one.
+static RowMap make_row_map(const gc_plan_s* p, uint32_t ntiles, uint32_t G, uint32_t& maxt, double skew) {
+    RowMap rm;
+    rm.G = G; rm.gA = G; rm.n0 = rm.n1 = rm.n2 = maxt; rm.s1 = rm.s2 = maxt * G;
+    if (skew > 0.0 && G == 3u * (uint32_t)p->sm_count && ntiles >= 12u * G) {
+        const uint32_t gA = (uint32_t)p->sm_count;
+        const uint32_t total = (ntiles + gA - 1) / gA;               // rows of the three classes together
+        const uint32_t n1 = maxt;
+        const uint32_t dd = std::max<uint32_t>(1u, (uint32_t)((double)ntiles / G * skew + 0.5));
+        const uint32_t n0 = n1 + dd;
+        if (total > n0 + n1 && total - n0 - n1 <= n1) {
+            rm.gA = gA; rm.n0 = n0; rm.n1 = n1; rm.n2 = total - n0 - n1;
+            rm.s1 = rm.n2 * G; rm.s2 = rm.s1 + (rm.n1 - rm.n2) * 2u * gA;
+            maxt = n0;
+        }
+    }
+    rm.mG = (uint32_t)((1ull << 32) / rm.G) + 1u;
+    rm.m2A = (uint32_t)((1ull << 32) / (2u * rm.gA)) + 1u;
+    rm.mA = (uint32_t)((1ull << 32) / rm.gA) + 1u;
+    return rm;
+}
+
 // Decides whether the plan can use the single-tensor kernel and with which geometry.
 void plan_single(gc_plan_s* p) {
     p->single_grid = 0;
@@ -250,27 +277,9 @@ void plan_single(gc_plan_s* p) {
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
     uint32_t maxt = (d.ntiles + G - 1) / G;
-    // shares of the tensor: equal, or - when the launch fills every SM three CTAs deep - in the
-    // proportion in which the oldest, middle and youngest CTA of an SM advance
-    RowMap rm;
-    rm.G = G; rm.gA = G; rm.n0 = rm.n1 = rm.n2 = maxt; rm.s1 = rm.s2 = maxt * G;
-    if (G == 3u * (uint32_t)p->sm_count && d.ntiles >= 12u * G) {
-        const uint32_t gA = (uint32_t)p->sm_count;
-        const uint32_t total = (d.ntiles + gA - 1) / gA;             // rows of the three classes together
-        const uint32_t n1 = maxt;
-        const uint32_t dd = std::max<uint32_t>(1u, (uint32_t)((double)d.ntiles / G * kSingleSkew + 0.5));
-        const uint32_t n0 = n1 + dd;
-        if (total > n0 + n1 && total - n0 - n1 <= n1) {
-            rm.gA = gA; rm.n0 = n0; rm.n1 = n1; rm.n2 = total - n0 - n1;
-            rm.s1 = rm.n2 * G; rm.s2 = rm.s1 + (rm.n1 - rm.n2) * 2u * gA;
-            maxt = n0;
-        }
-    }
+    const RowMap rm = make_row_map(p, d.ntiles, G, maxt, kSingleSkew);
     if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
     if (d.ntiles >= (1u << 20)) return;                              // (the row arithmetic divides by multiplication)
-    rm.mG = (uint32_t)((1ull << 32) / rm.G) + 1u;
-    rm.m2A = (uint32_t)((1ull << 32) / (2u * rm.gA)) + 1u;
-    rm.mA = (uint32_t)((1ull << 32) / rm.gA) + 1u;
     // region per CTA; one bit per slot has to fit in shared memory beside the chunk records
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
     const size_t rec_bytes = (size_t)maxt * kSingleRowBytes + sizeof(uint32_t) * ((pool + 31) / 32);
@@ -295,7 +304,8 @@ void plan_thr_single(gc_plan_s* p) {
     const TensorDesc& d = p->desc[0];
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_thr_single_max, d.ntiles);
-    const uint32_t maxt = (d.ntiles + G - 1) / G;
+    const uint32_t maxt = (d.ntiles + G - 1) / G;     // equal shares (unequal ones as in the top-k kernel: 268.5 us
+                                                      // against 262.5 us on the 110M-element workload)
     if (maxt > kSingleMaxT || G > 640) return;
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
     if ((double)pool < 1.25 * (double)d.k / (double)G + 256.0) return;
@@ -776,6 +786,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         sa.srank_hi = p->single_srank_hi; sa.srank_mid = p->single_srank_mid; sa.mid_cap = (uint32_t)kSingleMidCap;
         sa.mid = reinterpret_cast<uint2*>(wb + p->off_mid);
         sa.fine = reinterpret_cast<uint32_t*>(wb + p->off_fine);
+        sa.age = reinterpret_cast<uint32_t*>(wb + p->off_age);
         sa.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
         sa.seg_tot = reinterpret_cast<uint32_t*>(wb + p->off_rowseg);
         sa.ws = ws; sa.gws = gws;

@@ -72,6 +72,24 @@ struct RowMap {
     }
 };
 
+// This CTA's arrival number on its SM (0 = it got there first) and the SM's number; the counters
+// are zeroed before the launch.
+__device__ __forceinline__ uint32_t note_age(uint32_t* per_sm, uint32_t& smid) {
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    return atomicAdd(per_sm + (smid & 1023u), 1u);
+}
+// Column of this CTA once every CTA has called note_age (after a grid barrier): by age, oldest
+// first, column = age x gA + SM number.  That is a one-to-one assignment only if SMs 0..gA-1
+// hold three CTAs each; every CTA checks the same counters and otherwise keeps column b.
+// Called by the whole CTA (contains a block-wide vote).
+__device__ __forceinline__ uint32_t aged_column(const RowMap& rm, const uint32_t* per_sm, uint32_t age, uint32_t smid,
+                                                uint32_t G, uint32_t b, int tid) {
+    const bool fits = (uint32_t)tid >= rm.gA || ld_cg(per_sm + tid) == 3u;
+    const bool none_beyond = (uint32_t)tid < rm.gA || tid >= 1024 || ld_cg(per_sm + tid) == 0u;
+    const bool aged = __syncthreads_and(fits && none_beyond) && rm.gA * 3u == G && rm.gA <= (uint32_t)kBlock;
+    return aged ? min(age, 2u) * rm.gA + smid : b;
+}
+
 struct SingleArgs {
     TensorDesc d;                    // the tensor (by value)
     const TensorDesc* desc;          // device table (for the redo phases)
@@ -88,7 +106,8 @@ struct SingleArgs {
     uint2* cand;                     // [gridDim.x * pool_cap] candidate list, one region per CTA
     uint2* mid;                      // [mid_cap] candidates inside the band bin of the threshold
     uint32_t* hist5;                 // [0] coarse sample histogram, [2] band histogram,
-                                     // [3][0] short-list length, [4] CTAs per SM and per age class (all zeroed)
+                                     // [3][0] short-list length (all zeroed)
+    uint32_t* age;                   // [1024] CTAs that have arrived on every SM (zeroed)
     uint32_t* fine;                  // [kFineBins] fine sample histogram (zeroed)
     uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
     uint32_t* seg_tot;               // [maxt][ceil(G/32)] the same summed over each run of 32 CTAs of a row (zeroed)
@@ -224,12 +243,10 @@ k_topk_single(SingleArgs a) {
     const uint32_t nseg = (G + 31u) / 32u;
     // This CTA's age among the CTAs of its SM = its arrival number at the SM's counter, taken
     // first thing (the answer is only looked at once the sample loads are under way).
-    uint32_t my_age = 0;
+    uint32_t my_age = 0, my_sm = 0;
     if (tid == 0) {
         s_used = 0u;
-        uint32_t smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        my_age = atomicAdd(a.hist5 + 4 * kHistBins + (smid & 1023u), 1u);
+        my_age = note_age(a.age, my_sm);
     }
     phase_stamp(hdr, n_stamp);
 
@@ -263,11 +280,7 @@ k_topk_single(SingleArgs a) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) skey[q][e] = key_of(__fadd_rn(gv[e], rv[e]));
         }
-        if (tid == 0) {
-            uint32_t smid;
-            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-            s_age[0] = my_age; s_age[1] = smid;
-        }
+        if (tid == 0) { s_age[0] = my_age; s_age[1] = my_sm; }
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kMaxOwn; ++q)
@@ -291,14 +304,8 @@ k_topk_single(SingleArgs a) {
         flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr, n_stamp);
-        {   // Columns go to the CTAs by age, oldest first: column = age x gA + SM number.  That is
-            // a one-to-one assignment only if SMs 0..gA-1 hold three CTAs each; every CTA checks
-            // the same counters (all CTAs have registered by now) and otherwise keeps column b.
-            const uint32_t* const per_sm = a.hist5 + 4 * kHistBins;
-            const bool fits = (uint32_t)tid >= rm.gA || ld_cg(per_sm + tid) == 3u;
-            const bool none_beyond = (uint32_t)tid < rm.gA || tid >= 1024 || ld_cg(per_sm + tid) == 0u;
-            const bool aged = rm.gA * 3u == G && rm.gA <= (uint32_t)kBlock && __syncthreads_and(fits && none_beyond);
-            col = aged ? min(s_age[0], 2u) * rm.gA + s_age[1] : b;
+        {
+            col = aged_column(rm, a.age, s_age[0], s_age[1], G, b, tid);
             n_own = rm.rows_of(col);
             while (n_own > 0u && rm.tile_of(n_own - 1u, col) >= a.ntiles) --n_own;
             myseg = col / 32u;
