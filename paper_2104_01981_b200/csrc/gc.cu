@@ -62,7 +62,7 @@ struct gc_plan_s {
     size_t thrm_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
     uint32_t multi_ntab = 0;
-    uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0;       // 0 = plan does not qualify
+    uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0, multi_full = 0;       // 0 = plan does not qualify
     size_t multi_smem = 0;
     size_t off_shist = 0, off_bhist = 0, off_midn = 0, off_mmid = 0, off_skeys = 0;
     uint32_t n_empty = 0;                   // tensors without elements
@@ -363,18 +363,34 @@ void plan_multi(gc_plan_s* p) {
         const uint64_t groups = ((uint64_t)d.n + 3) / 4, nsg = (groups + d.sstride - 1) / d.sstride;
         per_tile[t] = std::min<double>(kTile, 2.0 * (double)kTile * (double)d.srank / (4.0 * (double)nsg));
     }
+    // runs: `per` tiles for the first two thirds of a full grid, the rest spread over the last third
+    // (the youngest CTAs of their SMs, which advance the slowest); every CTA `per` tiles otherwise
+    uint32_t full_ctas = G;
+    if (G == (uint32_t)p->grid_multi_max && per >= 8) {
+        const uint32_t fc = (uint32_t)((uint64_t)G * 2u / 3u);
+        if ((uint64_t)fc * per < p->ntiles) full_ctas = fc;
+    }
+    auto run_of = [&](uint32_t b, uint32_t& f, uint32_t& l) {
+        if (b < full_ctas) { f = std::min<uint32_t>(p->ntiles, b * per); l = std::min<uint32_t>(p->ntiles, f + per); return; }
+        const uint32_t s0 = std::min<uint32_t>(p->ntiles, full_ctas * per), rest = p->ntiles - s0, nb = G - full_ctas;
+        f = s0 + (uint32_t)(((uint64_t)(b - full_ctas) * rest) / nb);
+        l = s0 + (uint32_t)(((uint64_t)(b - full_ctas + 1) * rest) / nb);
+    };
     double worst = 0.0;
     uint32_t t = 0;
     for (uint32_t b = 0; b < G; ++b) {
         double e = 0.0;
-        for (uint32_t tile = b * per; tile < std::min<uint32_t>(p->ntiles, (b + 1) * per); ++tile) {
+        uint32_t f, l;
+        run_of(b, f, l);
+        if (l - f > per) return;
+        for (uint32_t tile = f; tile < l; ++tile) {
             while (t + 1 < p->T && (p->desc[t].ntiles == 0 || tile >= p->desc[t].tile0 + p->desc[t].ntiles)) ++t;
             e += per_tile[t];
         }
         worst = std::max(worst, e);
     }
     if ((double)pool < 1.5 * worst + 512.0) return;
-    p->multi_grid = G; p->multi_per = per; p->multi_pool = pool;
+    p->multi_grid = G; p->multi_per = per; p->multi_pool = pool; p->multi_full = full_ctas;
     p->multi_ntab = p->T <= kMultiMaxTab ? p->T : 0u;
     p->multi_smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32) +
                     2 * sizeof(uint32_t) * (size_t)p->multi_ntab;
@@ -800,7 +816,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         // many tensors: one cooperative launch, three grid barriers
         MultiArgs ma;
         ma.desc = p->d_desc; ma.T = p->T; ma.ntiles = nt; ma.nstiles = p->nstiles;
-        ma.per = p->multi_per;
+        ma.per = p->multi_per; ma.full_ctas = p->multi_full;
         ma.pool_cap = std::min<uint32_t>(p->multi_pool, p->cand_cap / p->multi_grid);     // each CTA's share
         ma.pool_smem_words = (p->multi_pool + 31) / 32; ma.ntab = p->multi_ntab;
         ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();

@@ -33,7 +33,8 @@ constexpr uint32_t kRefineTiles = 32;            // samples of up to this many s
 struct MultiArgs {
     const TensorDesc* desc;
     uint32_t T, ntiles, nstiles;
-    uint32_t per;                    // tiles per CTA (contiguous run)
+    uint32_t per;                    // tiles per CTA (contiguous run), at most
+    uint32_t full_ctas;              // CTAs 0 .. full_ctas - 1 take `per` tiles each, the others share the rest evenly
     uint32_t pool_cap;               // candidate slots per CTA
     uint32_t pool_smem_words;        // words of shared memory reserved for one bit per candidate slot
     uint32_t ntab;                   // T if the tile tables fit in shared memory, else 0
@@ -111,7 +112,16 @@ k_topk_multi(MultiArgs a) {
     const uint32_t G = gridDim.x, b = blockIdx.x;
     WsHeader* hdr = a.ws.hdr;
     uint32_t passed = 0, n_stamp = 0;
-    const uint32_t first = min(a.ntiles, b * a.per), last = min(a.ntiles, first + a.per);
+    // The CTAs launched last are the youngest on their SMs and advance the slowest (see RowMap in
+    // the one-tensor kernel), so whatever the full runs leave over is spread evenly over them.
+    uint32_t first, last;
+    if (b < a.full_ctas) {
+        first = min(a.ntiles, b * a.per); last = min(a.ntiles, first + a.per);
+    } else {
+        const uint32_t s0 = min(a.ntiles, a.full_ctas * a.per), rest = a.ntiles - s0, nb = G - a.full_ctas;
+        first = s0 + (uint32_t)(((unsigned long long)(b - a.full_ctas) * rest) / nb);
+        last = s0 + (uint32_t)(((unsigned long long)(b - a.full_ctas + 1u) * rest) / nb);
+    }
     const uint32_t ntl = last - first;                                         // own tiles
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     for (uint32_t i = tid; i < ntl * kWarps; i += kBlock) { rec[i] = 0u; rec2[i] = 0u; }
