@@ -83,8 +83,10 @@ constexpr uint64_t kSampleMax = 131072;       // most sampled elements per tenso
 constexpr uint64_t kSampleMaxSingle = 262144;   // ... when the plan holds one tensor (the sample is read in one step)
 constexpr uint32_t kSinglePoolMax = 16384;   // most candidates one CTA of k_topk_single may hold
 // Share of the oldest CTA of an SM above (and of the youngest below) the middle one's: measured
-// best between 6 and 10 % on the 110M-element workload.
-constexpr double kSingleSkew = 0.08;
+// best between 6 and 10 % on the 110M-element workload at 1 % density.  At 0.1 % density the
+// fold loop has fewer candidates to handle, competes less for issue slots, and 4 % did better
+// than 8 % (with 8 % the oldest CTAs of the 355M-element workload finished last).
+constexpr double kSingleSkew = 0.08, kSingleSkewSparse = 0.04;
 constexpr size_t kSingleRowBytes = (2 * kWarps + 3) * sizeof(uint32_t);   // shared memory per owned tile
 constexpr uint32_t kMultiMaxTab = 1024;      // tensors whose tile tables k_topk_multi keeps in shared memory
 constexpr size_t kMultiMaxPer = 160;         // most tiles one CTA of k_topk_multi may own
@@ -277,7 +279,7 @@ void plan_single(gc_plan_s* p) {
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
     const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
     uint32_t maxt = (d.ntiles + G - 1) / G;
-    const RowMap rm = make_row_map(p, d.ntiles, G, maxt, kSingleSkew);
+    const RowMap rm = make_row_map(p, d.ntiles, G, maxt, p->density >= 0.005 ? kSingleSkew : kSingleSkewSparse);
     if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
     if (d.ntiles >= (1u << 20)) return;                              // (the row arithmetic divides by multiplication)
     // region per CTA; one bit per slot has to fit in shared memory beside the chunk records
