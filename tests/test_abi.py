@@ -89,6 +89,20 @@ def test_empty_and_zero_sized_tensors(lib):
         p.query(api.GC_Q_TENSOR_K, 3)
 
 
+def test_plan_options_accept_their_values_and_reject_others(lib):
+    p = api.Plan([1000], 0.01, device=-1)
+    for opt, good, bad in [(api.GC_OPT_PATH, (api.GC_PATH_AUTO, api.GC_PATH_EXACT, api.GC_PATH_STAGED), 3),
+                           (api.GC_OPT_DECODE_ROUTE, (api.GC_DECODE_AUTO, api.GC_DECODE_NARROW, api.GC_DECODE_WIDE), 3),
+                           (api.GC_OPT_DECODE_ORDER, (api.GC_ORDER_FIXED, api.GC_ORDER_ANY), 2)]:
+        for v in good:
+            p.set_option(opt, v)
+        with pytest.raises(api.GcError) as e:
+            p.set_option(opt, bad)
+        assert e.value.code == api.GC_E_INVALID
+    with pytest.raises(api.GcError):
+        p.set_option(99, 0)
+
+
 def test_host_only_plan_refuses_compute(lib):
     p = api.Plan([16], 0.5, device=-1)
     assert p.compress_ptr(16, 16, 16, 16, None, 256, 0) == api.GC_E_UNSUPPORTED
