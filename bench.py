@@ -295,12 +295,14 @@ def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
         host_g[j].copy_(grads[0][j % sets])
     host_idx = torch.empty(max(k, 1), dtype=torch.int32).pin_memory()
     host_val = torch.empty(max(k, 1), dtype=torch.float32).pin_memory()
-    staging = torch.empty(n, dtype=torch.float32, device=dev)
+    staging = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2)]      # alternated: the next copy
+    call = [0]                                                                         # overlaps this compress
 
     def e2e_step(i: int):
         for wk in range(W):
-            plan.compress_host(host_g[i % 2], staging, resid[wk], outs[wk][0], outs[wk][1], None,
+            plan.compress_host(host_g[i % 2], staging[call[0] % 2], resid[wk], outs[wk][0], outs[wk][1], None,
                                host_idx, host_val, ws, stream)
+            call[0] += 1
         plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], None, dense, True, ws, stream)
 
     for i in range(2):
@@ -375,8 +377,8 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
         "e2e": None if not e2e_steps else {"value": grad_bytes_step * e2e_steps / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": 4 * n * W, "d2h_bytes_per_step": 8 * k * W,
                 "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps,
-                "what": "gc_compress_host: pinned host gradient -> device, compress, pairs -> pinned host; "
-                        "decode stays on the device"},
+                "what": "gc_compress_host: pinned host gradient -> device (two staging buffers alternate, the copy "
+                        "runs on the plan's copy stream), compress, pairs -> pinned host; decode stays on the device"},
         "fused_phase_us_last_step": [round(x, 2) for x in args.phase_us],
         "gpu_launches": launches,
         "path_counters": {"candidates_last_step": counters[0], "candidate_overflow": counters[1],

@@ -252,9 +252,15 @@ int gc_decompress_apply_momentum(gc_plan_t *plan, uint32_t W, const uint32_t *co
 /*
  * gc_compress_host -- gc_compress for a gradient that lives in HOST memory, with the
  * compressed pairs returned to HOST memory (what a worker would hand to its network stack).
- * Enqueues, on the stream: copy host_grad -> grad_staging, gc_compress, copy the pairs
- * device -> host.  No counterpart in the source paper; it exists so that end-to-end
- * throughput including both PCIe copies can be measured through this ABI.
+ * Enqueues: copy host_grad -> grad_staging, gc_compress, copy the pairs device -> host.  The
+ * compress and the copy of the pairs run on the caller's stream.  The host -> device copy runs
+ * on a stream owned by the plan and is ordered after the last compress that read the same
+ * grad_staging buffer, so a caller that alternates two staging buffers (and two host buffers)
+ * gets the next gradient's copy under way while the current one is compressed and its pairs
+ * travel back.  (While gc_profile_enable is on, the copy stays on the caller's stream.)
+ * host_grad must not change before the caller's stream has passed this call.  No counterpart in
+ * the source paper; it exists so that end-to-end throughput including both PCIe copies can be
+ * measured through this ABI.
  *
  *   host_grad     host (pinned for a truly asynchronous copy), fp32[total_n]
  *   grad_staging  device, fp32[total_n], 16-byte aligned; overwritten

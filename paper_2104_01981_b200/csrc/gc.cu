@@ -69,6 +69,12 @@ struct gc_plan_s {
     unsigned long long launches = 0;
     int last_cuda_error = 0;
     // optional per-kernel event timing
+    // gc_compress_host: the host -> device copy runs on a stream of the plan's own, so that it
+    // overlaps with the previous call's compress and device -> host copy
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied = nullptr;
+    struct StagingUse { const void* ptr; cudaEvent_t done; };      // last compress that read a staging buffer
+    std::vector<StagingUse> staging;
     struct Rec { cudaEvent_t a, b; int id; };
     std::vector<Rec> recs;
     size_t recs_used = 0;
@@ -1042,13 +1048,39 @@ int gc_compress_host(gc_plan_t* p, const float* host_grad, float* grad_staging, 
     if (host_grad == nullptr || grad_staging == nullptr || host_idx == nullptr || host_val == nullptr)
         return GC_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    {
+    gc_plan_s::StagingUse* use = nullptr;
+    if (!p->recs.empty()) {
+        // per-kernel timing is on: everything on the caller's stream, bracketed by its events
         Timed tm(p, s, GC_K_COPY);
         GC_CUDA(p, cudaMemcpyAsync(grad_staging, host_grad, sizeof(float) * (size_t)p->total_n,
                                    cudaMemcpyHostToDevice, s));
+    } else {
+        if (p->copy_stream == nullptr) {
+            GC_CUDA(p, cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
+            GC_CUDA(p, cudaEventCreateWithFlags(&p->ev_copied, cudaEventDisableTiming));
+        }
+        for (auto& u : p->staging) if (u.ptr == grad_staging) use = &u;
+        if (use == nullptr) {
+            // first call with this staging buffer: whatever the caller's stream still does with it comes first
+            if (p->staging.size() >= 8) {                // (callers rotate two or three buffers)
+                for (auto& u : p->staging) cudaEventDestroy(u.done);
+                p->staging.clear();
+            }
+            gc_plan_s::StagingUse u{grad_staging, nullptr};
+            GC_CUDA(p, cudaEventCreateWithFlags(&u.done, cudaEventDisableTiming));
+            p->staging.push_back(u);
+            use = &p->staging.back();
+            GC_CUDA(p, cudaEventRecord(use->done, s));
+        }
+        GC_CUDA(p, cudaStreamWaitEvent(p->copy_stream, use->done, 0));      // the compress that last read the buffer
+        GC_CUDA(p, cudaMemcpyAsync(grad_staging, host_grad, sizeof(float) * (size_t)p->total_n,
+                                   cudaMemcpyHostToDevice, p->copy_stream));
+        GC_CUDA(p, cudaEventRecord(p->ev_copied, p->copy_stream));
+        GC_CUDA(p, cudaStreamWaitEvent(s, p->ev_copied, 0));
     }
     int rc = gc_compress(p, grad_staging, residual, out_idx, out_val, out_count, workspace, stream);
     if (rc < 0) return rc;
+    if (use != nullptr) GC_CUDA(p, cudaEventRecord(use->done, s));          // the staging buffer may be refilled
     {
         Timed tm(p, s, GC_K_COPY);
         GC_CUDA(p, cudaMemcpyAsync(host_idx, out_idx, sizeof(uint32_t) * (size_t)p->total_cap,
@@ -1151,6 +1183,9 @@ int gc_destroy(gc_plan_t* p) {
     if (p == nullptr) return GC_OK;
     int rc = GC_OK;
     for (auto& r : p->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto& u : p->staging) cudaEventDestroy(u.done);
+    if (p->ev_copied) cudaEventDestroy(p->ev_copied);
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     if (p->d_small) { (void)cudaSetDevice(p->device); (void)cudaFree(p->d_small); }
     if (p->d_desc) {
         (void)cudaSetDevice(p->device);

@@ -292,3 +292,37 @@ def test_bf16_gradient_is_refused_where_no_kernel_reads_it():
     wt = GpuWorker(thr)
     with pytest.raises(api.GcError):
         thr.compress_bf16(g, wt.residual, wt.idx, wt.val, wt.count, wt.ws)
+
+
+@pytest.mark.parametrize("sizes", [[3_000_001], [300_000, 5, 1_500_001, 64, 131_071]])
+def test_host_buffer_entry_point_with_alternating_staging_buffers(sizes):
+    """gc_compress_host: pinned host gradient in, pairs back in pinned host memory.  Five
+    error-feedback steps are enqueued back to back with two staging buffers and two host gradient
+    buffers alternating (the copy of the next gradient overlaps the current compress); every
+    step's pairs and the final residual must equal the oracle's, and so must a run with the
+    per-kernel timing on (copy on the caller's stream)."""
+    density = 0.01
+    plan = api.Plan(sizes, density, device=0)
+    n, ks = plan.total_n, plan.tensor_k()
+    for profiled in (False, True):
+        plan.profile_enable(256 if profiled else 0)
+        ws = plan.alloc_workspace()
+        idx, val, cnt = plan.alloc_outputs()
+        resid = torch.zeros(n, device="cuda")
+        staging = [torch.empty(n, device="cuda") for _ in range(2)]
+        steps = 5
+        host_g = [torch.randn(n, generator=torch.Generator().manual_seed(90 + s)).pin_memory() for s in range(steps)]
+        host_idx = [torch.empty(plan.total_cap, dtype=torch.int32).pin_memory() for _ in range(steps)]
+        host_val = [torch.empty(plan.total_cap, dtype=torch.float32).pin_memory() for _ in range(steps)]
+        for s in range(steps):
+            plan.compress_host(host_g[s], staging[s % 2], resid, idx, val, None, host_idx[s], host_val[s], ws)
+        torch.cuda.synchronize()
+        r_cpu = np.zeros(n, np.float32)
+        for s in range(steps):
+            oi, ov = oracle.topk_compress_tensors(sizes, ks, host_g[s].numpy(), r_cpu)
+            assert np.array_equal(host_idx[s].numpy().view(np.uint32), oi), (profiled, s)
+            assert np.array_equal(host_val[s].numpy().view(np.uint32), ov.view(np.uint32)), (profiled, s)
+        assert np.array_equal(resid.cpu().numpy().view(np.uint32), r_cpu.view(np.uint32)), profiled
+        st, det = plan.last_status(ws)
+        assert st == api.GC_OK, (st, det)
+    plan.profile_enable(0)
