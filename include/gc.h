@@ -25,6 +25,9 @@
  *     workspace; the plan owns only its own small host and device tables.
  *   - gc_compress and gc_decompress_accumulate enqueue work on the given stream and return
  *     without synchronising.  No call allocates device memory except gc_plan.
+ *   - A plan is bound to one device.  Every call that touches the device (compress, decode,
+ *     gc_last_*, gc_compress_host) must be made while that device is the current one and
+ *     returns GC_E_INVALID otherwise; gc_plan leaves the caller's current device as it was.
  *   - Return value: 0 = GC_OK, negative = error, positive = warning.  Conditions detected on
  *     the device (truncation in threshold mode, an internal wait that ran out) are written
  *     to a status word at the head of the workspace; read it with gc_last_status.
@@ -109,7 +112,8 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                GC_PATH_EXACT: multi-pass kernels only
  *   GC_OPT_SAMPLE_RANK_PERMILLE  scales the sample rank that sets the candidate threshold
  *                                (1000 = default; small values make the candidate set too small
- *                                and so exercise the safety net -- a testing aid)
+ *                                and so exercise the safety net -- a testing aid).  The workspace
+ *                                size reported at plan creation stays sufficient.
  *   GC_OPT_CANDIDATE_CAPACITY    lowers the candidate-list capacity (testing aid for overflow)
  *   GC_OPT_DECODE_ROUTE          which tiled decode kernel gc_decompress_accumulate and
  *                                gc_decompress_apply_momentum take: GC_DECODE_AUTO (default) picks
@@ -310,15 +314,17 @@ const char *gc_kernel_name(int kernel_id);
  * cudaMalloc can fail, and would in any case stall every stream of the device while it
  * runs), or a latency-bound loop that may not touch the allocator.  Such callers cannot use
  * gc_plan, which allocates its tensor table.  Here the scratch the kernels need (histograms,
- * tile words, selection record; about 26 KB) is a fixed array inside the library image, so
+ * tile words, selection record; 41,728 bytes, about 41 KB) is a fixed array inside the library image, so
  * every GPU that loads libgc carries it until the process exits.
  *
  *   grad, residual  device, fp32[n], 16-byte aligned; residual is in/out exactly as in gc_compress
  *   n               elements, at most GC_NOALLOC_MAX_N; larger -> GC_E_TOO_LARGE (use gc_plan)
  *   k               entries to keep, k <= n (k > n -> GC_E_INVALID); same selection rule,
- *                   same output order and same residual rule as gc_compress in top-k mode
- *   out_idx/out_val device, uint32/fp32[k]
+ *                   same output order and same residual rule as gc_compress in top-k mode.
+ *                   k = 0 sends nothing and still folds: the residual becomes g + r
+ *   out_idx/out_val device, uint32/fp32[k] (may be NULL when k = 0)
  *   device_status   device int32 or NULL: receives GC_OK or GC_E_TIMEOUT when the work is done
+ *                   (on every path that returns GC_OK, n = 0 and k = 0 included)
  *   stream          cudaStream_t; the call is asynchronous
  * The current device is used.  The first call on each device resolves the device address of
  * the array (cudaGetSymbolAddress) and sizes its grids; make that first call outside any

@@ -33,6 +33,7 @@ struct gc_plan_s {
     std::vector<uint32_t> reg_ids;          // tensors with elements that are not small (device copy follows the small ids)
     uint32_t nstiles = 0, ngroups = 0;
     uint32_t cand_cap = 0, cand_cap_alloc = 0;
+    uint32_t skeys_tiles_alloc = 0;         // sample tiles the kept-keys section is sized for (fixed at plan creation)
     uint32_t n_sampled = 0;                 // tensors with a sample
     int path = 0;                           // GC_PATH_AUTO or GC_PATH_EXACT
     int decode_route = 0;                   // GC_DECODE_AUTO, GC_DECODE_NARROW or GC_DECODE_WIDE
@@ -116,6 +117,14 @@ inline uint64_t k_rule(uint64_t n, double density) {
         }                                                             \
     } while (0)
 
+// A plan's tables, grids and streams belong to one device: a compute call made while another
+// device is current would launch there with this plan's device pointers.
+inline bool on_plan_device(const gc_plan_s* p) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    return cur == p->device;
+}
+
 // Brackets one enqueued operation with events when timing is on; always counts the launch.
 struct Timed {
     gc_plan_s* p; cudaStream_t s; gc_plan_s::Rec* r = nullptr;
@@ -146,15 +155,17 @@ WsView view(const gc_plan_s* p, void* ws) {
 // sits six standard deviations of the sampling noise above the expected rank density*m, so a
 // candidate set smaller than k is a < 1e-8 event for well-mixed data (and only costs a redo).
 void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64_t* ccap, uint64_t target_max,
-                   double coarse_factor) {
+                   double coarse_factor, uint64_t* nsg_if_sampled) {
     const uint64_t n = d.n;
     d.sstride = 0; d.srank = 0;
     *ccap = n;
+    *nsg_if_sampled = 0;
     if (d.ntiles <= 1) { d.kind = kKindSmall; *ccap = 0; return; }   // fits one tile: one CTA does the whole tensor
     uint64_t target = std::min<uint64_t>(target_max, std::max<uint64_t>(n / 128, std::min<uint64_t>(8192, n / 2)));
     uint64_t stride = std::max<uint64_t>(1, n / target);
     uint64_t groups = (n + 3) / 4;
     uint64_t nsg = (groups + stride - 1) / stride;
+    *nsg_if_sampled = nsg;             // (whether it is sampled depends on the rank option; its sample size does not)
     double m = 4.0 * (double)nsg;
     double ks = density * m;
     double rank = std::ceil(ks + 6.0 * std::sqrt(ks) + 8.0) * (double)rank_permille / 1000.0;
@@ -169,7 +180,7 @@ void sample_params(TensorDesc& d, double density, uint32_t rank_permille, uint64
 
 // Fills the derived fields of the tensor table and the workspace layout.
 void finish_layout(gc_plan_s* p) {
-    uint64_t stile0 = 0, group0 = 0, ccap_total = 0;
+    uint64_t stile0 = 0, group0 = 0, ccap_total = 0, stiles_worst = 0;
     p->n_sampled = 0;
     p->small_ids.clear();
     p->reg_ids.clear();
@@ -179,8 +190,10 @@ void finish_layout(gc_plan_s* p) {
         uint64_t ccap = d.n;
         if (p->mode == GC_TOPK) {
             // (many tensors: the bracket is a histogram bin edge, up to twice the candidates)
+            uint64_t nsg_w = 0;
             sample_params(d, p->density, p->rank_permille, &ccap, p->T == 1 ? kSampleMaxSingle : kSampleMax,
-                          p->T == 1 ? 1.0 : 2.0);
+                          p->T == 1 ? 1.0 : 2.0, &nsg_w);
+            stiles_worst += (nsg_w + (uint64_t)kSampleTile - 1) / (uint64_t)kSampleTile;
         } else {
             // threshold mode: the sample is part of the definition -- one 4-element group out of
             // `stride`, rank k_s = min(m, max(1, ceil(density * m))) over its m elements
@@ -209,6 +222,9 @@ void finish_layout(gc_plan_s* p) {
     }
     p->nstiles = (uint32_t)stile0;
     p->ngroups = (uint32_t)group0;
+    // kept sample keys: room for every tensor that GC_OPT_SAMPLE_RANK_PERMILLE could turn into a
+    // sampled one, fixed at plan creation so that the workspace never grows afterwards
+    if (p->skeys_tiles_alloc == 0) p->skeys_tiles_alloc = (uint32_t)std::max<uint64_t>(stile0, stiles_worst);
     // every warp of the fold pass may strand part of a slab; CTAs never outnumber tiles
     ccap_total += (uint64_t)std::min<uint32_t>(p->ntiles, 1024u) * kWarps * kSlab;
     if (ccap_total > 0x7FFFFFFFull) ccap_total = 0x7FFFFFFFull;
@@ -248,7 +264,8 @@ void finish_layout(gc_plan_s* p) {
     p->off_mmid = align_up(p->off_mid + (T == 1 ? sizeof(uint2) * (size_t)kSingleMidCap : 0), 256);
     p->off_skeys = align_up(p->off_mmid + (multi_hist ? sizeof(uint2) * (size_t)kMultiMidCap * T : 0), 256);
     const bool keep_keys = multi_hist != 0 || (T == 1 && p->mode == GC_THRESHOLD);
-    p->ws_bytes = align_up(p->off_skeys + (keep_keys ? sizeof(uint4) * (size_t)kBlock * p->nstiles : 0), 256);
+    p->ws_bytes = align_up(p->off_skeys + (keep_keys ? sizeof(uint4) * (size_t)kBlock *
+                                                       std::max(p->nstiles, p->skeys_tiles_alloc) : 0), 256);
 }
 
 
@@ -529,6 +546,12 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         *out = p;
         return GC_OK;
     }
+    int caller_device = -1;
+    if (cudaGetDevice(&caller_device) != cudaSuccess) { (void)cudaGetLastError(); caller_device = -1; }
+    struct RestoreDevice {           // the caller's current device is left as it was found
+        int dev;
+        ~RestoreDevice() { if (dev >= 0) (void)cudaSetDevice(dev); }
+    } restore_device{caller_device};
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess && n_tensors > 0) {
@@ -635,8 +658,9 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
             return GC_OK;
         case GC_OPT_SAMPLE_RANK_PERMILLE:
             if (value < 1 || value > 100000) return GC_E_INVALID;
+            if (p->device >= 0 && !on_plan_device(p)) return GC_E_INVALID;      // (the table is uploaded again)
             p->rank_permille = (uint32_t)value;
-            finish_layout(p);                          // workspace size stays as planned
+            finish_layout(p);                          // workspace size stays as planned (see skeys_tiles_alloc)
             plan_single(p);
             plan_multi(p);
             return upload_table(p);
@@ -687,6 +711,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     const float* grad = static_cast<const float*>(grad_any);       // only dereferenced as such when !bf16
     if (p == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     // a bf16 gradient is read by the two fused top-k kernels only
     if (bf16 && !(p->mode == GC_TOPK && p->path == GC_PATH_AUTO && (p->single_grid > 0 || p->multi_grid > 0)))
         return GC_E_UNSUPPORTED;
@@ -926,6 +951,7 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
     if (p == nullptr) return GC_E_INVALID;
     if (W > GC_MAX_WORKERS) return GC_E_TOO_LARGE;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     if (p->total_n == 0) return GC_OK;
     if (dense_out == nullptr || workspace == nullptr) return GC_E_INVALID;
     if (W > 0 && (idx == nullptr || val == nullptr)) return GC_E_INVALID;
@@ -989,6 +1015,7 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
     if (p == nullptr) return GC_E_INVALID;
     if (W > GC_MAX_WORKERS) return GC_E_TOO_LARGE;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     if (p->total_n == 0) return GC_OK;
     if (param == nullptr || velocity == nullptr || workspace == nullptr) return GC_E_INVALID;
     if (W > 0 && (idx == nullptr || val == nullptr)) return GC_E_INVALID;
@@ -1030,6 +1057,7 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
 int gc_last_status(gc_plan_t* p, const void* workspace, void* stream, int32_t* status, uint64_t* detail) {
     if (p == nullptr || workspace == nullptr || status == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     WsHeader h;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
@@ -1044,6 +1072,7 @@ int gc_compress_host(gc_plan_t* p, const float* host_grad, float* grad_staging, 
                      float* host_val, void* workspace, void* stream) {
     if (p == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     if (p->total_n == 0) return GC_OK;
     if (host_grad == nullptr || grad_staging == nullptr || host_idx == nullptr || host_val == nullptr)
         return GC_E_INVALID;
@@ -1152,6 +1181,7 @@ const char* gc_kernel_name(int id) {
 int gc_last_counters(gc_plan_t* p, const void* workspace, void* stream, uint32_t counters[3]) {
     if (p == nullptr || workspace == nullptr || counters == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     WsHeader h;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));
@@ -1163,6 +1193,7 @@ int gc_last_counters(gc_plan_t* p, const void* workspace, void* stream, uint32_t
 int gc_last_phase_times(gc_plan_t* p, const void* workspace, void* stream, uint64_t ns[20], uint32_t* n_phases) {
     if (p == nullptr || workspace == nullptr || ns == nullptr || n_phases == nullptr) return GC_E_INVALID;
     if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
     WsHeader h;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     GC_CUDA(p, cudaMemcpyAsync(&h, workspace, sizeof(WsHeader), cudaMemcpyDeviceToHost, s));

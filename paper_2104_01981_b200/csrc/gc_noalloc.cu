@@ -22,7 +22,9 @@ constexpr size_t kScratchBytes = kOffDesc + 256;
 static_assert(kOffSel + sizeof(TensorSel) <= kOffHist, "selection record fits before the histogram");
 static_assert(kOffState % 256 == 0 && kOffDesc % 256 == 0, "aligned sections");
 
-// The scratch itself.  Every GPU that loads this library carries these ~26 KB until the
+static_assert(kScratchBytes == 41728, "the documented size of the fixed scratch (about 41 KB) follows this layout");
+
+// The scratch itself.  Every GPU that loads this library carries these 41,728 bytes until the
 // process exits.  In host code this name is only a handle for cudaGetSymbolAddress; it is not
 // a device address and must never be handed to a kernel directly.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
@@ -55,6 +57,15 @@ __global__ void k_noalloc_finish(const unsigned char* scratch, int32_t* status_o
     if (status_out != nullptr) *status_out = reinterpret_cast<const WsHeader*>(scratch)->status;
 }
 
+// k = 0: nothing is sent, but the gradient still has to reach the error-feedback residual
+// (r' = g + r, one rounding), exactly as the top-k rule leaves every unsent entry.
+__global__ void __launch_bounds__(256) k_noalloc_fold_only(const float* __restrict__ g, float* __restrict__ r,
+                                                           uint32_t n, int32_t* status_out) {
+    const uint32_t nth = gridDim.x * blockDim.x;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nth) r[i] = __fadd_rn(g[i], r[i]);
+    if (status_out != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *status_out = GC_OK;
+}
+
 }  // namespace
 
 extern "C" int gc_compress_noalloc(const float* grad, float* residual, uint32_t n, uint32_t k,
@@ -62,10 +73,20 @@ extern "C" int gc_compress_noalloc(const float* grad, float* residual, uint32_t 
                                    void* stream) {
     if (n > kMaxN) return GC_E_TOO_LARGE;        // beyond the fixed scratch: use gc_plan + gc_compress
     if (k > n) return GC_E_INVALID;
-    if (n == 0 || k == 0) return GC_OK;
-    if (grad == nullptr || residual == nullptr || out_idx == nullptr || out_val == nullptr) return GC_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n > 0 && (grad == nullptr || residual == nullptr)) return GC_E_INVALID;
+    if (k > 0 && (out_idx == nullptr || out_val == nullptr)) return GC_E_INVALID;
     if ((reinterpret_cast<uintptr_t>(grad) & 15u) || (reinterpret_cast<uintptr_t>(residual) & 15u))
         return GC_E_INVALID;
+    if (k == 0) {
+        // nothing to select (and the scratch is not needed): fold only, or just report success
+        if (n > 0 || device_status != nullptr) {
+            const uint32_t blocks = n == 0 ? 1u : (n + 1023u) / 1024u;
+            k_noalloc_fold_only<<<(int)(blocks < 1184u ? blocks : 1184u), 256, 0, s>>>(grad, residual, n, device_status);
+            if (cudaGetLastError() != cudaSuccess) return GC_E_CUDA;
+        }
+        return GC_OK;
+    }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         (void)cudaGetLastError();
@@ -105,7 +126,6 @@ extern "C" int gc_compress_noalloc(const float* grad, float* residual, uint32_t 
     const uint32_t nt = (n + kTile - 1) / kTile;
     const int gh = (int)(nt < (uint32_t)pd.grid_hist ? nt : (uint32_t)pd.grid_hist);
     const int gcp = (int)(nt < (uint32_t)pd.grid_compact ? nt : (uint32_t)pd.grid_compact);
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     k_noalloc_init<<<8, 256, 0, s>>>(sc, n, k, nt);
     k_hist<0, SRC_FOLD><<<gh, kBlock, 0, s>>>(desc, 1u, nt, grad, residual, ws);
     k_hist<1, SRC_RESID><<<gh, kBlock, 0, s>>>(desc, 1u, nt, nullptr, residual, ws);

@@ -52,10 +52,11 @@ class GpuWorker:
         return st, det
 
 
-def check_topk_against_oracle(sizes: Sequence[int], density: float, grads: List[torch.Tensor],
+def check_topk_against_oracle(sizes: Sequence[int], density: float, grads,
                               r0: Optional[torch.Tensor] = None, device: int = 0, options=None,
                               expect_counters=None):
-    """Runs len(grads) consecutive steps of one worker on GPU and oracle; asserts bitwise
+    """Runs one step per gradient in `grads` (a list, or any iterable that yields them one at a
+    time) of one worker on GPU and oracle; asserts bitwise
     equality of indices, values, counts and residual after every step.  Returns the plan
     worker (for decode tests) and the oracle's last (idx, val)."""
     plan = api.Plan(sizes, density, device=device)
@@ -78,6 +79,7 @@ def check_topk_against_oracle(sizes: Sequence[int], density: float, grads: List[
         if expect_counters is not None:
             expect_counters(plan.last_counters(w.ws))
         g_cpu = g.cpu().numpy()
+        del g_dev
         oi, ov = oracle.topk_compress_tensors(list(sizes), ks, g_cpu, r_cpu)
         tot = sum(ks)
         gi = to_np_u32(w.idx[:tot])

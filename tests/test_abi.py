@@ -103,6 +103,20 @@ def test_plan_options_accept_their_values_and_reject_others(lib):
         p.set_option(99, 0)
 
 
+def test_workspace_size_survives_the_sample_rank_option(lib):
+    """At densities near 1 a tensor's default sample rank reaches its sample size and the tensor is
+    left unsampled; a smaller rank option samples it after all.  The workspace size reported at
+    plan creation must already cover the sample keys kept then."""
+    for sizes, density in (([300_000, 5, 1_500_001, 131_072], 0.9), ([300_000, 70_000], 0.99),
+                           ([2_000_000], 0.95), ([300_000, 5, 1_500_001], 0.01)):
+        p = api.Plan(sizes, density, device=-1)
+        before = p.query(api.GC_Q_WORKSPACE_BYTES)
+        for permille in (30, 500, 1000, 5000):
+            p.set_option(api.GC_OPT_SAMPLE_RANK_PERMILLE, permille)
+            assert p.query(api.GC_Q_WORKSPACE_BYTES) <= before, (sizes, density, permille)
+        p.destroy()
+
+
 def test_host_only_plan_refuses_compute(lib):
     p = api.Plan([16], 0.5, device=-1)
     assert p.compress_ptr(16, 16, 16, 16, None, 256, 0) == api.GC_E_UNSUPPORTED

@@ -91,7 +91,8 @@ def test_threshold_config4_resnet_workers_and_decode():
     T, n = len(w.sizes), plan.total_n
     caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
     strides = [plan.query(api.GC_Q_TENSOR_STRIDE, t) for t in range(T)]
-    workers, pairs = [GpuWorker(plan) for _ in range(3)], []
+    assert w.workers == 8
+    workers, pairs = [GpuWorker(plan) for _ in range(w.workers)], []
     for i, wk in enumerate(workers):
         g = synth.gradient(w, i, 0, device="cuda")
         wk.step(g)
@@ -111,6 +112,26 @@ def test_threshold_config4_resnet_workers_and_decode():
     out = torch.empty(n, device="cuda")
     plan.decompress_accumulate([x.idx for x in workers], [x.val for x in workers], [x.count for x in workers],
                                out, True, workers[0].ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
+
+
+@pytest.mark.parametrize("config_id", [2, 4], ids=["bert_110m", "gpt2_medium_355m"])
+def test_threshold_full_size_one_tensor_workloads(config_id):
+    """One full-size step of the threshold variant on the 110M- and the 355M-element workload (the
+    one-tensor kernel at the sizes the benchmark quotes it on), then the decode of that list by
+    its count against the oracle."""
+    w = synth.workload(config_id)
+    g = synth.gradient(w, 0, 0, device="cuda")
+    plan, wk = check_threshold(w.sizes, w.density, [g.cpu()])
+    del g
+    n = plan.total_n
+    m = int(wk.count[0].item())
+    pairs = [(to_np_u32(wk.idx[:m]), wk.val[:m].cpu().numpy())]
+    wk.residual = None
+    torch.cuda.empty_cache()
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([wk.idx], [wk.val], [wk.count], out, True, wk.ws)
     want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
     assert np.array_equal(to_np_u32(out), bits(want))
 

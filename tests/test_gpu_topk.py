@@ -77,24 +77,74 @@ def test_config1_three_steps_error_feedback():
     check_topk_against_oracle(w.sizes, w.density, grads)
 
 
-def test_config2_resnet50_layerwise():
+class LazyGrads:
+    """The gradients of one worker, generated step by step (one full-size buffer alive at a time)."""
+
+    def __init__(self, w, worker, steps):
+        self.w, self.worker, self.steps = w, worker, steps
+
+    def __iter__(self):
+        for s in range(self.steps):
+            yield synth.gradient(self.w, self.worker, s, device="cuda")
+
+
+def test_config2_resnet50_layerwise_ten_steps():
     w = synth.workload(1)
-    grads = [synth.gradient(w, 0, s, device="cuda") for s in range(4)]
-    check_topk_against_oracle(w.sizes, w.density, grads)
+    assert w.steps == 10
+    seen = []
+    check_topk_against_oracle(w.sizes, w.density, LazyGrads(w, 0, w.steps), expect_counters=seen.append)
+    assert all(c[1] == 0 for c in seen), seen            # no candidate-list overflow on the workload itself
 
 
-def test_config3_bert_full_size():
+def test_config3_bert_full_size_ten_steps():
+    """All ten error-feedback steps at full size: the unsent entries pile up under the threshold
+    from step to step, which is what strains the sampled bracket."""
     w = synth.workload(2)
-    grads = [synth.gradient(w, 0, s, device="cuda") for s in range(2)]
-    check_topk_against_oracle(w.sizes, w.density, grads)
+    assert w.steps == 10
+    seen = []
+    check_topk_against_oracle(w.sizes, w.density, LazyGrads(w, 0, w.steps), expect_counters=seen.append)
+    assert all(c[1] == 0 and c[2] == 0 for c in seen), seen     # the safety net stayed idle
 
 
-def test_config5_gpt2_medium_full_size_two_workers():
+def test_config5_gpt2_medium_two_workers_five_steps():
     w = synth.workload(4)
+    assert w.steps == 5
     for worker in (0, 15):
-        grads = [synth.gradient(w, worker, 0, device="cuda")]
-        check_topk_against_oracle(w.sizes, w.density, grads)
+        check_topk_against_oracle(w.sizes, w.density, LazyGrads(w, worker, w.steps))
         torch.cuda.empty_cache()
+
+
+def test_config5_gpt2_medium_sixteen_workers_compress_then_decode():
+    """All 16 workers of the 355M-element workload, one step each: every worker's pairs and residual
+    against the oracle, then ONE decode call over the 16 lists the CUDA compress produced against
+    the oracle's sequential aggregation of the oracle's own lists."""
+    w = synth.workload(4)
+    assert w.workers == 16
+    plan = api.Plan(w.sizes, w.density, device=0)
+    ks, n, cap = plan.tensor_k(), plan.total_n, plan.total_cap
+    wk = GpuWorker(plan)
+    lists, pairs = [], []
+    g = torch.empty(n, device="cuda")
+    for worker in range(w.workers):
+        synth.gradient(w, worker, 0, device="cuda", out=g)
+        wk.residual.zero_()
+        wk.step(g)
+        wk.check_status()
+        r_cpu = np.zeros(n, np.float32)
+        oi, ov = oracle.topk_compress_tensors(w.sizes, ks, g.cpu().numpy(), r_cpu)
+        assert np.array_equal(to_np_u32(wk.idx[:cap]), oi), worker
+        assert np.array_equal(to_np_u32(wk.val[:cap]), bits(ov)), worker
+        assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r_cpu)), worker
+        lists.append((wk.idx[:cap].clone(), wk.val[:cap].clone()))
+        pairs.append((oi, ov))
+    del g
+    wk.residual = None
+    torch.cuda.empty_cache()
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([x[0] for x in lists], [x[1] for x in lists], None, out, True, wk.ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
+    wk.check_status()
 
 
 @pytest.mark.parametrize("n,density,quantised", [(24_000_001, 0.01, True), (21_823_500, 0.003, False),
