@@ -100,13 +100,16 @@ class ClockSampler:
         return out
 
 
-# --------------------------------------------------------------------------- reference arm
-def oracle_sample_run(w: synth.Workload, sample_n: int, steps: int, warmup: int):
-    """Times the CPU oracle on the first `sample_n` elements of the workload's gradient
-    (same density, one worker, compress + decode per step)."""
+# --------------------------------------------------------------------------- CPU oracle legs
+CPU_SAMPLE_ELEMENTS = 1 << 26        # one sample size for `cpu_baseline` and for `--impl reference`
+
+
+def oracle_sample_inputs(w: synth.Workload, sample_n: int, n_grads: int = 2, worker: int = 0):
+    """(sizes, ks, gradients) of the bounded sample the CPU oracle is timed on: the first `sample_n`
+    elements of the workload's flat gradient (layer-wise workloads: whole tensors up to that)."""
     import oracle
     oracle.build()
-    sizes = [sample_n] if len(w.sizes) == 1 else None
+    sizes = [min(sample_n, w.total_n)] if len(w.sizes) == 1 else None
     if sizes is None:                       # layer-wise workloads: keep whole tensors up to sample_n
         sizes, acc = [], 0
         for s in w.sizes:
@@ -115,9 +118,18 @@ def oracle_sample_run(w: synth.Workload, sample_n: int, steps: int, warmup: int)
             sizes.append(s); acc += s
     n = sum(sizes)
     ks = [oracle.k_from_density(s, w.density) for s in sizes]
+    grads = [synth.gradient(w, worker, s, device="cpu")[:n].numpy().copy() for s in range(n_grads)]
+    return sizes, ks, grads
+
+
+def oracle_sample_run(w: synth.Workload, sample_n: int, steps: int, warmup: int, inputs=None):
+    """Times the CPU oracle, one thread, on the sample (same density, one worker, compress + decode
+    per step).  Returns (elements, k, seconds per timed step)."""
+    import oracle
+    sizes, ks, grads = inputs or oracle_sample_inputs(w, sample_n)
+    n = sum(sizes)
     r = np.zeros(n, np.float32)
     out = np.empty(n, np.float32)
-    grads = [synth.gradient(w, 0, s, device="cpu")[:n].numpy().copy() for s in range(2)]
     times = []
     for it in range(warmup + steps):
         g = grads[it % len(grads)]
@@ -130,20 +142,84 @@ def oracle_sample_run(w: synth.Workload, sample_n: int, steps: int, warmup: int)
     return n, sum(ks), times
 
 
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_threads_run(w: synth.Workload, sample_n: int, steps: int, warmup: int, max_threads: int = 32,
+                       inputs=None):
+    """The same oracle step on one thread per simulated worker, all at once: every thread owns one
+    worker's sample (its own gradient window, residual and dense buffer) and calls the oracle as it
+    stands; the library calls run outside the interpreter lock.  Returns (threads, elements per
+    thread, wall seconds of the timed steps)."""
+    import threading
+    import oracle
+    sizes, ks, grads = inputs or oracle_sample_inputs(w, sample_n, n_grads=2)
+    n = sum(sizes)
+    threads = max(1, min(host_cores(), max_threads))
+    try:
+        import psutil
+        room = int(psutil.virtual_memory().available * 0.5 // (8 * 4 * n))     # g, r, out + the oracle's index arrays
+        threads = max(1, min(threads, room))
+    except Exception:
+        pass
+    state = [(np.zeros(n, np.float32), np.empty(n, np.float32)) for _ in range(threads)]
+    gate = threading.Barrier(threads + 1)
+
+    def body(t: int):
+        r, out = state[t]
+        for it in range(warmup + steps):
+            if it == warmup:
+                gate.wait()
+            g = grads[(it + t) % len(grads)]
+            idx, val = oracle.topk_compress_tensors(sizes, ks, g, r)
+            oracle.decode_accumulate([(idx, val)], out, True)
+        gate.wait()
+
+    th = [threading.Thread(target=body, args=(t,)) for t in range(threads)]
+    for x in th:
+        x.start()
+    gate.wait()
+    t0 = time.perf_counter()
+    gate.wait()
+    dt = time.perf_counter() - t0
+    for x in th:
+        x.join()
+    return threads, n, dt
+
+
+def cpu_baseline(w: synth.Workload, steps: int = 8, warmup: int = 1, with_threads: bool = True):
+    """The `cpu_baseline` object: the oracle on one thread, and on one thread per worker."""
+    inputs = oracle_sample_inputs(w, CPU_SAMPLE_ELEMENTS)
+    sn, sk, times = oracle_sample_run(w, CPU_SAMPLE_ELEMENTS, steps, warmup, inputs)
+    cpu = {"value": 4.0 * sn * len(times) / sum(times) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "cores_available": host_cores(),
+           "sample": f"first {sn} elements of the workload gradient, k={sk}, {len(times)} steps after {warmup} "
+                     f"warm-up, compress + decode, single thread"}
+    if with_threads:
+        nth, tn, dt = oracle_threads_run(w, CPU_SAMPLE_ELEMENTS, 3, 1, inputs=inputs)
+        cpu["multi_thread"] = {"value": 4.0 * tn * nth * 3 / dt / 1e9, "unit": UNIT, "cores": nth,
+                               "sample": f"{nth} threads (one per simulated worker, each on its own {tn}-element "
+                                         f"sample, residual and dense buffer), 3 steps after 1 warm-up"}
+    return cpu
+
+
 def run_reference(args, w: synth.Workload, rank: int):
     if rank != 0:
         return
-    sample_n = min(w.total_n, 1 << 22)
-    n, k, times = oracle_sample_run(w, sample_n, args.steps, args.warmup)
+    n, k, times = oracle_sample_run(w, CPU_SAMPLE_ELEMENTS, args.steps, args.warmup)
     t = sum(times)
     value = 4.0 * n * len(times) / t / 1e9
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": w.name, "elements": w.total_n, "density": w.density,
-                                         "workers": 1},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "data": "synthetic", "config": {"workload": w.name, "mode": "topk", "grad_dtype": "f32", "elements": w.total_n,
+                                         "density": w.density, "workers": w.workers, "tensors": len(w.sizes)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "cores_available": host_cores(),
                          "sample": f"first {n} elements of the workload gradient per step, k={k}, "
                                    f"compress + decode, single thread"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -169,166 +245,257 @@ def whole_job_value(n: int, workers: int, world: int, steps: int, ms: float) -> 
     return 4.0 * n * workers * world * steps / (ms * 1e-3) / 1e9
 
 
+def profile_traffic(name: str):
+    """DRAM bytes of one launch as an ncu capture measured them: the `dram_bytes_per_launch = N` line
+    of the summary under profiles/ (None when the summary or the line is missing)."""
+    import re
+    path = os.path.join(ROOT, "profiles", name)
+    try:
+        m = re.search(r"^dram_bytes_per_launch\s*=\s*(\d+)", open(path).read(), re.M)
+        return (float(m.group(1)), "profiles/" + name) if m else (None, None)
+    except OSError:
+        return None, None
+
+
 # --------------------------------------------------------------------------- GPU arm
+class Rig:
+    """Buffers of one (workload, mode) on one GPU and the calls of one step."""
+
+    def __init__(self, api, w: synth.Workload, mode_name: str, dev: str, device_index: int, input_sets: int,
+                 seed_worker0: int = 0, grad_dtype: str = "f32", path: str = "auto"):
+        self.api, self.w = api, w
+        self.mode = api.GC_THRESHOLD if mode_name == "threshold" else api.GC_TOPK
+        self.plan = api.Plan(w.sizes, w.density, mode=self.mode, device=device_index)
+        if path != "auto":
+            self.plan.set_option(api.GC_OPT_PATH, {"exact": api.GC_PATH_EXACT, "staged": api.GC_PATH_STAGED}[path])
+        self.n, self.k, self.W = self.plan.total_n, self.plan.total_cap, w.workers
+        n, W = self.n, self.W
+        self.stream = torch.cuda.current_stream()
+        # inputs resident in HBM before the timed region: `sets` gradients per worker slot, cycled;
+        # each is far larger than the 126 MB L2 (or, for the small workloads, the set of buffers a
+        # step touches is), so no explicit flush is needed
+        self.sets = max(1, min(input_sets, int(24e9 // (4 * n * W)) or 1))
+        self.grads = [[synth.gradient(w, wk + seed_worker0, s, device=dev) for s in range(self.sets)]
+                      for wk in range(W)]
+        self.bf16 = grad_dtype == "bf16"
+        if self.bf16:                            # the gradient arrives as bfloat16 (gc_compress_bf16)
+            self.grads = [[g.to(torch.bfloat16) for g in gs] for gs in self.grads]
+        self.do_compress = self.plan.compress_bf16 if self.bf16 else self.plan.compress
+        self.resid = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(W)]
+        self.outs = [self.plan.alloc_outputs() for _ in range(W)]
+        self.ws = self.plan.alloc_workspace()
+        self.dense = torch.empty(n, dtype=torch.float32, device=dev)
+        self.thr = self.mode == api.GC_THRESHOLD          # threshold mode: variable counts travel with the pairs
+        self.cnts = [o[2] for o in self.outs] if self.thr else None
+        self.idx, self.val = [o[0] for o in self.outs], [o[1] for o in self.outs]
+        # several workers: one gc_compress_workers call per step (own workspace per worker; the
+        # library shares launches among them where the plan allows it, else it loops itself)
+        self.workers_call = W > 1 and not self.bf16
+        self.wss = [self.ws] + [self.plan.alloc_workspace() for _ in range(W - 1)] if self.workers_call else None
+
+    def compress_only(self, i: int):
+        if self.workers_call:
+            self.plan.compress_workers([gs[i % self.sets] for gs in self.grads], self.resid, self.idx, self.val,
+                                       self.cnts, self.wss, self.stream)
+            return
+        self.compress_separate(i)
+
+    def compress_separate(self, i: int):
+        for wk in range(self.W):
+            o = self.outs[wk]
+            self.do_compress(self.grads[wk][i % self.sets], self.resid[wk], o[0], o[1], o[2] if self.thr else None,
+                             self.ws, self.stream)
+
+    def decode_only(self, i: int):
+        self.plan.decompress_accumulate(self.idx, self.val, self.cnts, self.dense, True, self.ws, self.stream)
+
+    def step(self, i: int):
+        self.compress_only(i)
+        self.decode_only(i)
+
+    def check(self):
+        worst = self.api.GC_OK
+        for ws in (self.wss or [self.ws]):
+            st, det = self.plan.last_status(ws)
+            if st not in (self.api.GC_OK, self.api.GC_W_TRUNCATED):
+                raise RuntimeError(f"device status {st} (detail {det}) after the timed region")
+            worst = max(worst, st)
+        return worst
+
+
+class Timer:
+    """K-step loops timed with CUDA events on the launching stream, a barrier and a synchronize on
+    both sides of every loop, the slowest rank's time per loop.  A loop is repeated until about
+    `min_total_ms` of device time have passed (so that clock samples land under load); the
+    reported time is the median loop."""
+
+    def __init__(self, stream, world: int, dev, min_total_ms: float = 1000.0):
+        self.stream, self.world, self.dev, self.min_total_ms = stream, world, dev, min_total_ms
+        self.e0, self.e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def barrier(self):
+        if self.world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def one_loop(self, fn, steps: int, first: int = 0) -> float:
+        self.barrier()
+        self.e0.record(self.stream)
+        for i in range(steps):
+            fn(first + i)
+        self.e1.record(self.stream)
+        self.barrier()
+        return reduce_max_over_ranks([self.e0.elapsed_time(self.e1)], self.world, self.dev)[0]
+
+    def loops(self, fn, steps: int, first: int = 0, max_loops: int = 400, min_loops: int = 3):
+        """Returns the per-loop times (ms), every rank the same list."""
+        t = [self.one_loop(fn, steps, first)]
+        want = int(min(max_loops, max(min_loops, -(-self.min_total_ms // max(t[0], 1e-3)))))
+        while len(t) < want:
+            t.append(self.one_loop(fn, steps, first))
+        return t
+
+
+def spread(times, steps):
+    """(median, min, max) of the loop times, per step."""
+    return statistics.median(times) / steps, min(times) / steps, max(times) / steps
+
+
 def run_gpu(args, w: synth.Workload, rank: int, world: int, local_rank: int):
     from paper_2104_01981_b200 import api
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     api.lib()                                    # no fallback: raises when libgc.so is missing
-    mode = api.GC_THRESHOLD if args.mode == "threshold" else api.GC_TOPK
-    plan = api.Plan(w.sizes, w.density, mode=mode, device=local_rank)
-    if args.path != "auto":
-        plan.set_option(api.GC_OPT_PATH, {"exact": api.GC_PATH_EXACT, "staged": api.GC_PATH_STAGED}[args.path])
-    n, k, W = plan.total_n, plan.total_cap, w.workers
-    stream = torch.cuda.current_stream()
-
-    # inputs resident in HBM before the timed region: N_INPUT_SETS gradients per worker slot,
-    # cycled; each is far larger than the 126 MB L2, so no explicit flush is needed
-    sets = max(1, min(args.input_sets, int(24e9 // (4 * n * W)) or 1))
-    grads = [[synth.gradient(w, wk + 100 * rank, s, device=dev) for s in range(sets)] for wk in range(W)]
-    bf16 = args.grad_dtype == "bf16"
-    if bf16:                                 # the gradient arrives as bfloat16 (gc_compress_bf16)
-        grads = [[g.to(torch.bfloat16) for g in gs] for gs in grads]
-    do_compress = plan.compress_bf16 if bf16 else plan.compress
-    resid = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(W)]
-    outs = [plan.alloc_outputs() for _ in range(W)]
-    ws = plan.alloc_workspace()
-    dense = torch.empty(n, dtype=torch.float32, device=dev)
-
-    thr = mode == api.GC_THRESHOLD          # threshold mode: variable counts travel with the pairs
-    cnts = [o[2] for o in outs] if thr else None
-
-    def step(i: int):
-        for wk in range(W):
-            do_compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
-                          ws, stream)
-        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], cnts, dense, True, ws, stream)
-
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
+    rig = Rig(api, w, args.mode, dev, local_rank, args.input_sets, 100 * rank, args.grad_dtype, args.path)
+    plan, n, k, W, sets, stream = rig.plan, rig.n, rig.k, rig.W, rig.sets, rig.stream
+    tm = Timer(stream, world, dev, args.min_loop_ms)
+    res = {}
 
     for i in range(args.warmup):
-        step(i)
-    barrier()
-    # ---- timed region 1: device-resident inputs, per-kernel events on
-    launches0 = plan.launches()
-    plan.profile_enable(args.steps * (8 * W + 8))
-    sampler = ClockSampler(local_rank, os.path.join("/tmp", f"gc_bench_clocks_{os.getpid()}.csv")) \
+        rig.step(i)
+    tm.barrier()
+    sampler = ClockSampler(local_rank, os.path.join(tempfile.gettempdir(), f"gc_bench_clocks_{os.getpid()}.csv")) \
         if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
-    e1.record(stream)
-    barrier()
-    ms = e0.elapsed_time(e1)
-    per_kernel = plan.profile_read()
-    launches = plan.launches() - launches0
+    # ---- timed region 1: device-resident inputs, K steps per loop (the headline value)
+    launches0 = plan.launches()
+    res["plain"] = tm.loops(rig.step, args.steps, args.warmup)
+    res["launches_per_loop"] = (plan.launches() - launches0) // len(res["plain"])
+    # ---- timed region 1b: the same loop once more with per-kernel events on (the kernel table)
+    plan.profile_enable(args.steps * (8 * W + 8))
+    res["with_events"] = tm.one_loop(rig.step, args.steps, args.warmup)
+    res["per_kernel"] = plan.profile_read()
     plan.profile_enable(0)
-    st, det = plan.last_status(ws)
-    if st not in (api.GC_OK, api.GC_W_TRUNCATED):
-        raise RuntimeError(f"device status {st} (detail {det}) after the timed region")
-    counters = plan.last_counters(ws)
-    args.phase_us = plan.last_phase_times(ws)
-
-    # ---- timed region 1b: same loop without the per-kernel events (the headline value)
-    barrier()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
-    e1.record(stream)
-    barrier()
-    ms_plain = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None          # sampled across both timed loops
-
-    # ---- timed regions 1c/1d: the two halves on their own (no per-kernel events)
-    def compress_only(i: int):
-        for wk in range(W):
-            do_compress(grads[wk][i % sets], resid[wk], outs[wk][0], outs[wk][1], outs[wk][2] if thr else None,
-                          ws, stream)
-
-    def decode_only(i: int):
-        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], cnts, dense, True, ws, stream)
-
-    halves = []
-    for fn in (compress_only, decode_only):
-        barrier()
-        e0.record(stream)
-        for i in range(args.steps):
-            fn(args.warmup + i)
-        e1.record(stream)
-        barrier()
-        halves.append(e0.elapsed_time(e1) / args.steps)
-    args.ms_compress, args.ms_decode = halves
+    rig.check()
+    res["counters"] = plan.last_counters(rig.ws)
+    res["phase_us"] = plan.last_phase_times(rig.ws)
+    # ---- timed regions 1c/1d: the two halves on their own
+    res["compress"] = tm.loops(rig.compress_only, args.steps, args.warmup)
+    res["decode"] = tm.loops(rig.decode_only, args.steps, args.warmup)
+    res["clocks"] = sampler.stop() if sampler else None          # sampled across the loops above
     # ---- timed region 1e: decode with momentum SGD fused behind it (top-k lists only)
-    args.ms_apply = None
-    if not thr:
+    res["apply"] = None
+    if not rig.thr:
         param = torch.zeros(n, device=dev)
         vel = torch.zeros(n, device=dev)
 
         def apply_only(i: int):
-            plan.decompress_apply_momentum([o[0] for o in outs], [o[1] for o in outs], None, param, vel,
-                                           0.01, 0.9, 1.0 / W, ws, stream)
+            plan.decompress_apply_momentum(rig.idx, rig.val, None, param, vel, 0.01, 0.9, 1.0 / W, rig.ws, stream)
 
         for i in range(3):
             apply_only(i)
-        barrier()
-        e0.record(stream)
-        for i in range(args.steps):
-            apply_only(i)
-        e1.record(stream)
-        barrier()
-        args.ms_apply = e0.elapsed_time(e1) / args.steps
+        res["apply"] = tm.one_loop(apply_only, args.steps) / args.steps
         del param, vel
 
     # ---- timed region 2: end to end through the host-buffer entry point
-    if args.no_e2e or args.grad_dtype == "bf16":
-        e2e_steps, ms_e2e = 0, float("nan")
-        return _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e, e2e_steps,
-                       per_kernel, launches, clocks, counters)
-    e2e_steps = max(3, min(args.steps, 10))
-    host_g = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(2)]
-    for j in range(2):
-        host_g[j].copy_(grads[0][j % sets])
-    host_idx = torch.empty(max(k, 1), dtype=torch.int32).pin_memory()
-    host_val = torch.empty(max(k, 1), dtype=torch.float32).pin_memory()
-    staging = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2)]      # alternated: the next copy
-    call = [0]                                                                         # overlaps this compress
+    res["e2e_steps"], res["e2e"] = 0, float("nan")
+    if not (args.no_e2e or args.grad_dtype == "bf16" or rig.thr):
+        e2e_steps = max(3, min(args.steps, 10))
+        host_g = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(2)]
+        for j in range(2):
+            host_g[j].copy_(rig.grads[0][j % sets])
+        host_idx = torch.empty(max(k, 1), dtype=torch.int32).pin_memory()
+        host_val = torch.empty(max(k, 1), dtype=torch.float32).pin_memory()
+        staging = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(2)]      # alternated: the next copy
+        call = [0]                                                                         # overlaps this compress
 
-    def e2e_step(i: int):
-        for wk in range(W):
-            plan.compress_host(host_g[i % 2], staging[call[0] % 2], resid[wk], outs[wk][0], outs[wk][1], None,
-                               host_idx, host_val, ws, stream)
-            call[0] += 1
-        plan.decompress_accumulate([o[0] for o in outs], [o[1] for o in outs], None, dense, True, ws, stream)
+        def e2e_step(i: int):
+            for wk in range(W):
+                plan.compress_host(host_g[i % 2], staging[call[0] % 2], rig.resid[wk], rig.outs[wk][0], rig.outs[wk][1],
+                                   None, host_idx, host_val, rig.ws, stream)
+                call[0] += 1
+            plan.decompress_accumulate(rig.idx, rig.val, None, rig.dense, True, rig.ws, stream)
 
-    for i in range(2):
-        e2e_step(i)
-    barrier()
-    e0.record(stream)
-    for i in range(e2e_steps):
-        e2e_step(i)
-    e1.record(stream)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    return _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e, e2e_steps,
-                   per_kernel, launches, clocks, counters)
+        for i in range(2):
+            e2e_step(i)
+        res["e2e"] = tm.one_loop(e2e_step, e2e_steps)
+        res["e2e_steps"] = e2e_steps
+        del host_g, staging
+    # ---- the other workloads, each timed the same way with fewer steps (rank 0 only: replicas)
+    others = {}
+    if args.configs == "all" and rank == 0 and args.grad_dtype == "f32" and args.path == "auto":
+        del rig.grads, rig.resid, rig.dense
+        torch.cuda.empty_cache()
+        peak, _ = measured_peak_gbs()
+        for cfg, mode in ((0, "topk"), (1, "topk"), (3, "topk"), (3, "threshold"), (4, "topk")):
+            if cfg == w.config_id and mode == args.mode:
+                continue
+            others[f"c{cfg + 1}_{mode}"] = bench_other(api, cfg, mode, dev, local_rank, peak, args)
+    _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others)
 
 
-def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e, e2e_steps,
-            per_kernel, launches, clocks, counters):
-    ms, ms_plain, ms_e2e = reduce_max_over_ranks([ms, ms_plain, ms_e2e], world, dev)
+def bench_other(api, cfg: int, mode: str, dev: str, device_index: int, peak: float, args):
+    """One of the other workloads: compress per worker, decode and whole step by CUDA events."""
+    w = synth.workload(cfg)
+    rig = Rig(api, w, mode, dev, device_index, args.input_sets)
+    n, k, W = rig.n, rig.k, rig.W
+    tm = Timer(rig.stream, 1, dev, min_total_ms=300.0)
+    steps = max(3, min(args.steps, int(200.0 / max(0.02, 12.0 * n * W / 5e9))))      # about 0.2 s per loop
+    for i in range(3):
+        rig.step(i)
+    t_step, t_lo, t_hi = spread(tm.loops(rig.step, steps, 3), steps)
+    t_c = spread(tm.loops(rig.compress_only, steps, 3), steps)[0]
+    t_d = spread(tm.loops(rig.decode_only, steps, 3), steps)[0]
+    t_sep = spread(tm.loops(rig.compress_separate, steps, 3), steps)[0] if rig.workers_call else None
+    st = rig.check()
+    counters = rig.plan.last_counters(rig.ws)
+    sent = k
+    if rig.thr:                                   # pairs actually sent by the last step (the lists are not full)
+        T = len(w.sizes)
+        sent = int(sum(int(c[:T].sum().item()) for c in rig.cnts) / W)
+    cb, db = 12.0 * n + 8.0 * sent, 4.0 * n + 8.0 * sent * W
+    out = {
+        "workload": w.name, "mode": mode, "elements": n, "workers": W, "tensors": len(w.sizes), "steps_per_loop": steps,
+        "pairs_per_worker": sent, "capacity_per_worker": k,
+        "compress_us_per_worker": 1e3 * t_c / W, "decode_us": 1e3 * t_d, "ms_per_step": t_step,
+        "compress_call": "gc_compress_workers (one call per step)" if rig.workers_call else "gc_compress",
+        "compress_us_per_worker_separate_calls": None if t_sep is None else 1e3 * t_sep / W,
+        "ms_per_step_min_max": [t_lo, t_hi],
+        "gradient_GB_per_s": 4.0 * n * W / (t_step * 1e-3) / 1e9,
+        "compress_frac_of_8TBs": cb / NOMINAL_HBM / (t_c / W * 1e-3),
+        "compress_frac_of_measured": cb / (peak * 1e9) / (t_c / W * 1e-3),
+        "decode_frac_of_8TBs": db / NOMINAL_HBM / (t_d * 1e-3),
+        "decode_frac_of_measured": db / (peak * 1e9) / (t_d * 1e-3),
+        "path_counters": {"candidates_last_step": counters[0], "candidate_overflow": counters[1],
+                          "tensors_redone": counters[2], "status": st},
+        "input_sets": rig.sets,
+    }
+    del rig
+    torch.cuda.empty_cache()
+    return out
+
+
+def _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others):
     if rank != 0:
         return
-
-    from paper_2104_01981_b200 import api
+    per_kernel, counters, clocks = res["per_kernel"], res["counters"], res["clocks"]
+    ms_step, ms_lo, ms_hi = spread(res["plain"], args.steps)
+    ms_compress = spread(res["compress"], args.steps)[0]
+    ms_decode = spread(res["decode"], args.steps)[0]
+    e2e_steps, ms_e2e = res["e2e_steps"], res["e2e"]
     grad_bytes_step = 4.0 * n * W * world
-    value = whole_job_value(n, W, world, args.steps, ms_plain)
+    value = whole_job_value(n, W, world, 1, ms_step)
     cb, db = min_bytes(n, k, W, 2 if args.grad_dtype == "bf16" else 4)
-    t_step = ms_plain * 1e-3 / args.steps
+    t_step = ms_step * 1e-3
     peak, peak_src = measured_peak_gbs()
 
     # dominant kernel: largest share of the per-kernel event time
@@ -341,33 +508,35 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
                  "threshold_emit": 12.0 * n + 4.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
-    # DRAM bytes of one launch of the dominant kernel from an ncu capture (profiles/), where one exists
-    ncu_traffic, ncu_src = {
-        ("c3_bert_base_110m_student_t", "topk", "compress_fused"): (1374.4e6, "profiles/k_topk_single_c3_bert110m.md"),
-        ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): (1407.5e6, "profiles/k_threshold_single_c3_bert110m.md"),
-        ("c2_resnet50_layerwise", "topk", "compress_fused"): (322.1e6, "profiles/k_topk_multi_c2_resnet50.md"),
-    }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None, (None, None))
+    # DRAM bytes of one launch of the dominant kernel as ncu measured them (read from the summary)
+    prof = {("c3_bert_base_110m_student_t", "topk", "compress_fused"): "k_topk_single_c3_bert110m.md",
+            ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): "k_threshold_single_c3_bert110m.md",
+            ("c2_resnet50_layerwise", "topk", "compress_fused"): "k_topk_multi_c2_resnet50.md",
+            }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None)
+    ncu_traffic, ncu_src = profile_traffic(prof) if prof else (None, None)
 
     # CPU baseline: the oracle on a bounded sample of the same workload
-    cpu = None
-    if not args.no_cpu_baseline:
-        sn, sk, times = oracle_sample_run(w, min(n, 1 << 26), 8, 1)           # about 10 s of CPU work
-        cpu = {"value": 4.0 * sn * len(times) / sum(times) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"first {sn} elements of the workload gradient, k={sk}, 8 steps after 1 warm-up, "
-                         f"compress + decode, single thread"}
+    cpu = None if args.no_cpu_baseline else cpu_baseline(w)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_plain / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "mode": args.mode, "grad_dtype": args.grad_dtype, "elements": n, "k": k, "density": w.density, "workers": W,
                    "tensors": len(w.sizes), "input_sets": sets,
                    "l2": "inputs larger than L2 (no flush): each gradient and residual is %d MB" % (4 * n >> 20)},
-        "elements_per_s": n * W * world * args.steps / (ms_plain * 1e-3),
+        "timing": {"what": "the K-step loop (barrier + synchronize on both sides, CUDA events on the launching stream) "
+                           "is repeated until about one second of device time has passed; ms_per_step is the median loop",
+                   "loops": len(res["plain"]), "ms_per_step_min": ms_lo, "ms_per_step_max": ms_hi,
+                   "timed_region_ms_per_loop": ms_step * args.steps},
+        "elements_per_s": n * W * world / t_step,
         "hbm_frac_of_8TBs": {"step": (cb + db) / NOMINAL_HBM / t_step,
                              "min_bytes_compress": cb, "min_bytes_decode": db,
-                             "compress_only": None},
-        "ms_per_step_with_kernel_events": ms / args.steps,
+                             "compress_only": cb / NOMINAL_HBM / (ms_compress * 1e-3),
+                             "compress_ms_per_step": ms_compress,
+                             "decode_only": db / NOMINAL_HBM / (ms_decode * 1e-3),
+                             "decode_ms_per_step": ms_decode},
+        "ms_per_step_with_kernel_events": res["with_events"] / args.steps,
         "kernels": breakdown,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic, "peak_source": peak_src,
@@ -379,21 +548,19 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, ms, ms_plain, ms_e2e
                 "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps,
                 "what": "gc_compress_host: pinned host gradient -> device (two staging buffers alternate, the copy "
                         "runs on the plan's copy stream), compress, pairs -> pinned host; decode stays on the device"},
-        "fused_phase_us_last_step": [round(x, 2) for x in args.phase_us],
-        "gpu_launches": launches,
+        "fused_phase_us_last_step": [round(x, 2) for x in res["phase_us"]],
+        "gpu_launches": res["launches_per_loop"],
         "path_counters": {"candidates_last_step": counters[0], "candidate_overflow": counters[1],
                           "tensors_redone": counters[2], "k": k},
         "clocks": clocks,
     }
-    line["hbm_frac_of_8TBs"]["compress_only"] = cb / NOMINAL_HBM / (args.ms_compress * 1e-3)
-    line["hbm_frac_of_8TBs"]["compress_ms_per_step"] = args.ms_compress
-    line["hbm_frac_of_8TBs"]["decode_only"] = db / NOMINAL_HBM / (args.ms_decode * 1e-3)
-    line["hbm_frac_of_8TBs"]["decode_ms_per_step"] = args.ms_decode
-    if getattr(args, "ms_apply", None):
+    if res.get("apply"):
         ab = 16 * n + 8 * k * W                    # read and write parameter and velocity, read the pairs
-        line["fused_decode_momentum"] = {"ms_per_call": args.ms_apply, "bytes": ab,
-                                         "GB_per_s": ab / (args.ms_apply * 1e-3) / 1e9,
-                                         "frac_of_measured_peak": ab / (args.ms_apply * 1e-3) / 1e9 / peak}
+        line["fused_decode_momentum"] = {"ms_per_call": res["apply"], "bytes": ab,
+                                         "GB_per_s": ab / (res["apply"] * 1e-3) / 1e9,
+                                         "frac_of_measured_peak": ab / (res["apply"] * 1e-3) / 1e9 / peak}
+    if others:
+        line["configs"] = others
     print(json.dumps(line))
 
 
@@ -676,11 +843,16 @@ def run_decode_sweep(args, w: synth.Workload, rank: int, world: int, local_rank:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, help="workload 0..4 (default 2: 110M BERT-base shape)")
     ap.add_argument("--impl", default="gc", choices=["gc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--configs", default="all", choices=["all", "none"],
+                    help="all: after the headline workload, time the other four workloads (and the threshold variant "
+                         "of the 8-worker one) and report them under `configs`; none: headline only")
+    ap.add_argument("--min-loop-ms", type=float, default=1000.0,
+                    help="repeat every K-step loop until this much device time has passed (median loop reported)")
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "exact"],
                     help="auto: one-pass candidate path in one cooperative launch (default); staged: the "
                          "same phases as separate launches; exact: multi-pass kernels only")

@@ -129,7 +129,7 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                within (hits - 1) x 2^-24 x sum |values| of the fixed-order one and
  *                                equals it where one worker hits.  Applies to the tiled decode of
  *                                both decode calls; lists with counts of many-tensor plans keep
- *                                their fixed-order route.
+ *                                their fixed-order kernel.
  * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
  */
 #define GC_OPT_PATH                  0
@@ -193,6 +193,30 @@ int gc_compress_bf16(gc_plan_t *plan, const void *grad_bf16, float *residual,
                      void *workspace, void *stream);
 
 /*
+ * gc_compress_workers -- gc_compress for W simulated workers of one plan in one go: worker w
+ * folds residuals[w] into grads[w], writes its pairs to out_idx[w] / out_val[w] (and its counts
+ * to out_count[w]) and uses workspaces[w]; every result is exactly what W separate gc_compress
+ * calls would give.  No counterpart in the source paper: the problem statement only says that
+ * the 8-worker workload runs its workers on one GPU, and this call is how that is done without
+ * paying a kernel's cold phases once per worker.  For top-k plans of several tensors on the
+ * default route the workers share cooperative launches: the resident CTAs are dealt out evenly
+ * among up to 12 workers per launch, each group of CTAs runs the many-tensor kernel on its own
+ * worker and synchronises only with itself.  Every other plan (one tensor, threshold mode,
+ * GC_PATH_EXACT / GC_PATH_STAGED) is served by W consecutive gc_compress calls.
+ *
+ *   W            1..GC_MAX_WORKERS (0 does nothing)
+ *   grads, residuals, out_idx, out_val, workspaces
+ *                host arrays of W device pointers, each as in gc_compress; no two workers may
+ *                share a residual, an output array or a workspace (GC_E_INVALID): the workers'
+ *                kernels run at the same time
+ *   out_count    host array of W device pointers, or NULL for none
+ * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_CUDA.  Asynchronous.
+ */
+int gc_compress_workers(gc_plan_t *plan, uint32_t W, const float *const *grads, float *const *residuals,
+                        uint32_t *const *out_idx, float *const *out_val, uint32_t *const *out_count,
+                        void *const *workspaces, void *stream);
+
+/*
  * gc_decompress_accumulate -- decode W sparse sets and sum them into a dense buffer
  * (problem statement: "decode and sum the sparse contributions of W simulated workers into
  * one dense buffer"; a sum, not a mean).  For every flat index the additions happen in
@@ -210,7 +234,11 @@ int gc_compress_bf16(gc_plan_t *plan, const void *grad_bf16, float *residual,
  * With count = NULL every list must be exactly as gc_compress wrote it in top-k mode (total_cap
  * pairs, ascending index): the dense buffer is then built tile by tile in shared memory and
  * written once; so are one-tensor plans with count arrays (the list's length is its count).
- * Many-tensor plans with count arrays are applied one launch per worker instead.
+ * Plans of several tensors with count arrays take the same tile loop cut at the tensor
+ * boundaries: tensor t's live pairs are slots [out offset of t, + count[t]) of the list, the
+ * slots up to its capacity are ignored (GC_OPT_DECODE_ROUTE and GC_OPT_DECODE_ORDER do not
+ * apply to such lists: one kernel, fixed worker order).  A live pair whose index lies outside
+ * its tensor is skipped and GC_E_INVALID is recorded.
  * An index >= total_n (or a list that is not ascending) is skipped and GC_E_INVALID is recorded
  * in the device status.
  * Errors: GC_E_INVALID, GC_E_TOO_LARGE (W > GC_MAX_WORKERS), GC_E_CUDA.  Asynchronous.
@@ -240,8 +268,7 @@ int gc_last_status(gc_plan_t *plan, const void *workspace, void *stream,
  * operation rounded once, no fused multiply-add).  No counterpart in the source paper; it is
  * the fusion a data-parallel step performs right after aggregation, and it replaces 24 bytes
  * per element of traffic (write the sum, read it again with p and v, write p and v) by 16.
- *   idx, val, count  as for gc_decompress_accumulate; count arrays only for one-tensor plans
- *                    (GC_E_UNSUPPORTED otherwise)
+ *   idx, val, count  as for gc_decompress_accumulate
  *   param, velocity  device, fp32[total_n], 16-byte aligned, updated in place
  *   workspace        device; only its status word is written (out-of-range or unordered
  *                    index -> GC_E_INVALID recorded, the entry is skipped)

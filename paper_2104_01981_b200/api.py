@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.gc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
         L.gc_compress_bf16.restype = i32
         L.gc_compress_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.gc_compress_workers.restype = i32
+        L.gc_compress_workers.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp]
         L.gc_decompress_accumulate.restype = i32
         L.gc_decompress_accumulate.argtypes = [vp, u32, vp, vp, vp, vp, i32, vp, vp]
         L.gc_last_status.restype = i32
@@ -177,6 +179,21 @@ class Plan:
                                _ptr(out_count), _ptr(workspace), _stream_handle(stream))
         if rc < 0:
             raise GcError("gc_compress", rc)
+        return rc
+
+    # --- gc_compress_workers
+    def compress_workers(self, grads: Sequence[torch.Tensor], residuals: Sequence[torch.Tensor],
+                         out_idx: Sequence[torch.Tensor], out_val: Sequence[torch.Tensor],
+                         out_count: Optional[Sequence[torch.Tensor]], workspaces: Sequence[torch.Tensor],
+                         stream=None) -> int:
+        """All workers of one step in one call (one workspace, residual and output set per worker)."""
+        W = len(grads)
+        arr = lambda ts: (ctypes.c_void_p * max(W, 1))(*[t.data_ptr() for t in ts])
+        rc = lib().gc_compress_workers(self._h, W, arr(grads), arr(residuals), arr(out_idx), arr(out_val),
+                                       arr(out_count) if out_count is not None else None, arr(workspaces),
+                                       _stream_handle(stream))
+        if rc < 0:
+            raise GcError("gc_compress_workers", rc)
         return rc
 
     def compress_bf16(self, grad_bf16: torch.Tensor, residual: torch.Tensor, out_idx: torch.Tensor,

@@ -17,6 +17,8 @@
 
 using namespace gc;
 
+struct MultiGeom { uint32_t G = 0, per = 0, pool = 0, full = 0, ntab = 0; size_t smem = 0; };   // see multi_geometry
+
 struct gc_plan_s {
     int device = 0;
     int mode = GC_TOPK;
@@ -28,8 +30,10 @@ struct gc_plan_s {
     uint32_t ntiles = 0;
     std::vector<TensorDesc> desc;
     TensorDesc* d_desc = nullptr;
+    uint32_t* d_dectile = nullptr;          // plans of several tensors: tensor that holds the first element of each decode tile
     uint32_t* d_small = nullptr;            // ids of the small tensors (device), n_small entries
     std::vector<uint32_t> small_ids;
+    uint32_t n_tiny = 0;                    // the first n_tiny of them are tiny (see tiny_tensor_warp)
     std::vector<uint32_t> reg_ids;          // tensors with elements that are not small (device copy follows the small ids)
     uint32_t nstiles = 0, ngroups = 0;
     uint32_t cand_cap = 0, cand_cap_alloc = 0;
@@ -44,6 +48,7 @@ struct gc_plan_s {
            control_bytes = 0, off_tinfo = 0, off_cidx = 0, ws_bytes = 0;
     int sm_count = 0;
     int grid_thr = 0, grid_decode[2] = {0, 0};
+    int grid_decode_seg[2] = {0, 0}, grid_decode_seg_apply = 0;    // k_decode_segments: one / two tile buffers; with optimizer
     bool wide_ok = false;                         // k_decode_wide may use up to 64 KB of dynamic shared memory
     std::vector<std::pair<size_t, int>> wide_occ[2];      // (shared-memory bytes -> CTAs per SM), plain / with optimizer
     int grid_hist = 0, grid_compact = 0, grid_fold = 0, grid_sample = 0, grid_chist = 0, grid_ccompact = 0;
@@ -62,6 +67,9 @@ struct gc_plan_s {
     uint32_t thrm_grid = 0, thrm_per = 0, thrm_pool = 0, thrm_ntab = 0;   // many-tensor threshold kernel (0 = no)
     size_t thrm_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
+    size_t multi_smem_max = 0;              // dynamic shared memory that occupancy figure was taken with
+    uint32_t wk_W = 0, wk_batch = 0;        // gc_compress_workers: workers per launch chosen for the last W seen
+    MultiGeom wk_geom;
     uint32_t multi_ntab = 0;
     uint32_t multi_grid = 0, multi_per = 0, multi_pool = 0, multi_full = 0;       // 0 = plan does not qualify
     size_t multi_smem = 0;
@@ -222,6 +230,12 @@ void finish_layout(gc_plan_s* p) {
     }
     p->nstiles = (uint32_t)stile0;
     p->ngroups = (uint32_t)group0;
+    // tiny tensors (one warp each in the many-tensor top-k kernel) first in the list of small ones
+    {
+        auto tiny = [&](uint32_t t) { return p->mode == GC_TOPK && is_tiny(p->desc[t].n, p->desc[t].k); };
+        std::stable_partition(p->small_ids.begin(), p->small_ids.end(), tiny);
+        p->n_tiny = (uint32_t)std::count_if(p->small_ids.begin(), p->small_ids.end(), tiny);
+    }
     // kept sample keys: room for every tensor that GC_OPT_SAMPLE_RANK_PERMILLE could turn into a
     // sampled one, fixed at plan creation so that the workspace never grows afterwards
     if (p->skeys_tiles_alloc == 0) p->skeys_tiles_alloc = (uint32_t)std::max<uint64_t>(stile0, stiles_worst);
@@ -370,13 +384,17 @@ void plan_thr_multi(gc_plan_s* p) {
     p->thrm_smem = (size_t)per * kMultiRowBytes + 2 * sizeof(uint32_t) * (size_t)p->thrm_ntab;
 }
 
-// Decides whether the plan can use the many-tensor kernel and with which geometry.
-void plan_multi(gc_plan_s* p) {
-    p->multi_grid = 0;
-    if (p->mode != GC_TOPK || p->T < 2 || p->grid_multi_max <= 0 || p->ntiles == 0) return;
-    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_multi_max, p->ntiles);
+// Geometry of the many-tensor kernel when G CTAs share one worker's tiles: MultiGeom.
+
+// Decides whether G CTAs can run the many-tensor kernel on this plan (G = 0 in the result: no).
+// `age_skew`: the CTA index follows the CTAs' age on their SMs (a launch that fills the device
+// with this plan alone), so the leftover tiles go to the youngest third.
+MultiGeom multi_geometry(const gc_plan_s* p, uint32_t G, bool age_skew) {
+    MultiGeom mg;
+    if (p->mode != GC_TOPK || p->T < 2 || G == 0 || p->ntiles == 0) return mg;
+    G = std::min<uint32_t>(G, p->ntiles);
     const uint32_t per = (p->ntiles + G - 1) / G;
-    if (per > kMultiMaxPer) return;
+    if (per > kMultiMaxPer) return mg;
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
     // expected candidates of the busiest CTA (bracket rank over sample size, times two for the
     // bin edge), with head-room
@@ -391,7 +409,7 @@ void plan_multi(gc_plan_s* p) {
     // runs: `per` tiles for the first two thirds of a full grid, the rest spread over the last third
     // (the youngest CTAs of their SMs, which advance the slowest); every CTA `per` tiles otherwise
     uint32_t full_ctas = G;
-    if (G == (uint32_t)p->grid_multi_max && per >= 8) {
+    if (age_skew && per >= 8) {
         const uint32_t fc = (uint32_t)((uint64_t)G * 2u / 3u);
         if ((uint64_t)fc * per < p->ntiles) full_ctas = fc;
     }
@@ -407,18 +425,28 @@ void plan_multi(gc_plan_s* p) {
         double e = 0.0;
         uint32_t f, l;
         run_of(b, f, l);
-        if (l - f > per) return;
+        if (l - f > per) return mg;
         for (uint32_t tile = f; tile < l; ++tile) {
             while (t + 1 < p->T && (p->desc[t].ntiles == 0 || tile >= p->desc[t].tile0 + p->desc[t].ntiles)) ++t;
             e += per_tile[t];
         }
         worst = std::max(worst, e);
     }
-    if ((double)pool < 1.5 * worst + 512.0) return;
-    p->multi_grid = G; p->multi_per = per; p->multi_pool = pool; p->multi_full = full_ctas;
-    p->multi_ntab = p->T <= kMultiMaxTab ? p->T : 0u;
-    p->multi_smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32) +
-                    2 * sizeof(uint32_t) * (size_t)p->multi_ntab;
+    if ((double)pool < 1.5 * worst + 512.0) return mg;
+    mg.G = G; mg.per = per; mg.pool = pool; mg.full = full_ctas;
+    mg.ntab = p->T <= kMultiMaxTab ? p->T : 0u;
+    mg.smem = (size_t)per * kMultiRowBytes + sizeof(uint32_t) * ((pool + 31) / 32) + 2 * sizeof(uint32_t) * (size_t)mg.ntab;
+    return mg;
+}
+
+// Decides whether the plan can use the many-tensor kernel and with which geometry.
+void plan_multi(gc_plan_s* p) {
+    p->multi_grid = 0;
+    if (p->grid_multi_max <= 0) return;
+    const MultiGeom mg = multi_geometry(p, (uint32_t)p->grid_multi_max, p->ntiles >= (uint32_t)p->grid_multi_max);
+    if (mg.G == 0) return;
+    p->multi_grid = mg.G; p->multi_per = mg.per; p->multi_pool = mg.pool; p->multi_full = mg.full;
+    p->multi_ntab = mg.ntab; p->multi_smem = mg.smem;
 }
 
 int upload_table(gc_plan_s* p) {
@@ -559,11 +587,25 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         if (e == cudaSuccess)
             e = cudaMalloc(reinterpret_cast<void**>(&p->d_small), sizeof(uint32_t) * 2 * (size_t)n_tensors);
         if (e == cudaSuccess) e = upload_table(p) == GC_OK ? cudaSuccess : cudaErrorUnknown;
+        if (e == cudaSuccess && n_tensors > 1 && p->total_n > 0) {
+            const uint32_t ntl = (uint32_t)((p->total_n + kDecTile - 1) / kDecTile);
+            std::vector<uint32_t> tt(ntl);
+            uint32_t t = 0;
+            for (uint32_t tl = 0; tl < ntl; ++tl) {
+                const uint64_t e0 = (uint64_t)tl * kDecTile;
+                while (t + 1 < n_tensors && (p->desc[t].n == 0 || e0 >= (uint64_t)p->desc[t].off + p->desc[t].n)) ++t;
+                tt[tl] = t;
+            }
+            e = cudaMalloc(reinterpret_cast<void**>(&p->d_dectile), sizeof(uint32_t) * (size_t)ntl);
+            if (e == cudaSuccess)
+                e = cudaMemcpy(p->d_dectile, tt.data(), sizeof(uint32_t) * (size_t)ntl, cudaMemcpyHostToDevice);
+        }
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         if (p->d_desc) cudaFree(p->d_desc);
         if (p->d_small) cudaFree(p->d_small);
+        if (p->d_dectile) cudaFree(p->d_dectile);
         delete p;
         return GC_E_CUDA;
     }
@@ -611,10 +653,13 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_multi_max = 0;
         if (coop) {
             int nb = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi<GradF32>, kBlock,
-                                                              kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8 + 8 * kMultiMaxTab) ==
-                    cudaSuccess && nb >= 1)
-                p->grid_multi_max = p->sm_count * nb;
+            p->multi_smem_max = kMultiMaxPer * kMultiRowBytes + kSinglePoolMax / 8 + 8 * kMultiMaxTab;
+            int nbw = 0;          // (the several-workers form of the kernel must be as resident as the kernel itself)
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_topk_multi<GradF32>, kBlock, p->multi_smem_max) ==
+                    cudaSuccess && nb >= 1 &&
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nbw, k_topk_workers<GradF32>, kBlock, p->multi_smem_max) ==
+                    cudaSuccess && nbw >= 1)
+                p->grid_multi_max = p->sm_count * std::min(nb, nbw);
             else
                 (void)cudaGetLastError();
         }
@@ -632,6 +677,23 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
             if (ed != cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
             p->grid_decode[nbuf - 1] = p->sm_count * nb;     // 0: fall back to one launch per worker
         }
+    }
+    {
+        // lists with per-tensor counts (plans of several tensors): the segment-walking tile kernel
+        cudaError_t ed = cudaFuncSetAttribute(k_decode_segments<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)(2 * kDecTileBytes));
+        for (int nbuf = 1; nbuf <= 2; ++nbuf) {
+            int nb = 0;
+            if (ed == cudaSuccess)
+                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_segments<false>, kDecBlock,
+                                                                   nbuf * kDecTileBytes);
+            if (ed != cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
+            p->grid_decode_seg[nbuf - 1] = p->sm_count * nb;
+        }
+        int nb = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_segments<true>, kDecBlock, kDecTileBytes) !=
+                cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
+        p->grid_decode_seg_apply = p->sm_count * nb;
     }
     p->wide_ok = cudaFuncSetAttribute(k_decode_wide<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)(kDecTileBytes + 8 * kDecWideEntries)) == cudaSuccess &&
@@ -660,6 +722,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
             if (value < 1 || value > 100000) return GC_E_INVALID;
             if (p->device >= 0 && !on_plan_device(p)) return GC_E_INVALID;      // (the table is uploaded again)
             p->rank_permille = (uint32_t)value;
+            p->wk_W = 0;
             finish_layout(p);                          // workspace size stays as planned (see skeys_tiles_alloc)
             plan_single(p);
             plan_multi(p);
@@ -667,6 +730,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
         case GC_OPT_CANDIDATE_CAPACITY:
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
             p->cand_cap = (uint32_t)value;
+            p->wk_W = 0;
             return GC_OK;
         case GC_OPT_DECODE_ORDER:
             if (value != GC_ORDER_FIXED && value != GC_ORDER_ANY) return GC_E_INVALID;
@@ -704,6 +768,34 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
         case GC_Q_TENSOR_STRIDE: *value = d.stride; return GC_OK;
         default: return GC_E_INVALID;
     }
+}
+
+// Argument block of the many-tensor kernel for one worker's buffers and a given geometry.
+static MultiArgs multi_args(const gc_plan_s* p, const MultiGeom& mg, const void* grad, float* residual,
+                            uint32_t* out_idx, float* out_val, uint32_t* out_count, void* workspace) {
+    char* wb = static_cast<char*>(workspace);
+    WsView ws = view(p, workspace);
+    WsView gws = ws;                 // redo of failed tensors: own records, gated by the main ones
+    gws.sel = reinterpret_cast<TensorSel*>(wb + p->off_gsel);
+    gws.gate = ws.sel;
+    MultiArgs ma;
+    ma.desc = p->d_desc; ma.T = p->T; ma.ntiles = p->ntiles; ma.nstiles = p->nstiles;
+    ma.per = mg.per; ma.full_ctas = mg.full;
+    ma.pool_cap = std::min<uint32_t>(mg.pool, p->cand_cap / mg.G);     // each CTA's share
+    ma.pool_smem_words = (mg.pool + 31) / 32; ma.ntab = mg.ntab;
+    ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size(); ma.n_tiny = p->n_tiny;
+    ma.reg_ids = p->d_small + p->T; ma.n_reg = (uint32_t)p->reg_ids.size();
+    ma.brk = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+    ma.g = grad; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
+    ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+    ma.mid = reinterpret_cast<uint2*>(wb + p->off_mmid);
+    ma.mid_n = reinterpret_cast<uint32_t*>(wb + p->off_midn);
+    ma.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
+    ma.bhist = reinterpret_cast<uint32_t*>(wb + p->off_bhist);
+    ma.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+    ma.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
+    ma.ws = ws; ma.gws = gws;
+    return ma;
 }
 
 static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* residual, uint32_t* out_idx,
@@ -846,24 +938,11 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         return GC_OK;
     }
     if (p->path == GC_PATH_AUTO && p->multi_grid > 0) {
-        // many tensors: one cooperative launch, three grid barriers
-        MultiArgs ma;
-        ma.desc = p->d_desc; ma.T = p->T; ma.ntiles = nt; ma.nstiles = p->nstiles;
-        ma.per = p->multi_per; ma.full_ctas = p->multi_full;
-        ma.pool_cap = std::min<uint32_t>(p->multi_pool, p->cand_cap / p->multi_grid);     // each CTA's share
-        ma.pool_smem_words = (p->multi_pool + 31) / 32; ma.ntab = p->multi_ntab;
-        ma.small_ids = p->d_small; ma.n_small = (uint32_t)p->small_ids.size();
-        ma.reg_ids = p->d_small + p->T; ma.n_reg = (uint32_t)p->reg_ids.size();
-        ma.brk = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
-        ma.g = grad_any; ma.r = residual; ma.out_idx = out_idx; ma.out_val = out_val; ma.out_count = out_count;
-        ma.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
-        ma.mid = reinterpret_cast<uint2*>(wb + p->off_mmid);
-        ma.mid_n = reinterpret_cast<uint32_t*>(wb + p->off_midn);
-        ma.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
-        ma.bhist = reinterpret_cast<uint32_t*>(wb + p->off_bhist);
-        ma.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
-        ma.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
-        ma.ws = ws; ma.gws = gws;
+        // many tensors: one cooperative launch, four grid barriers
+        MultiGeom mg;
+        mg.G = p->multi_grid; mg.per = p->multi_per; mg.pool = p->multi_pool; mg.full = p->multi_full;
+        mg.ntab = p->multi_ntab; mg.smem = p->multi_smem;
+        MultiArgs ma = multi_args(p, mg, grad_any, residual, out_idx, out_val, out_count, workspace);
         void* args[] = {&ma};
         Timed tm(p, s, GC_K_FUSED);
         const void* kfn = bf16 ? (const void*)k_topk_multi<GradBF16> : (const void*)k_topk_multi<GradF32>;
@@ -945,6 +1024,88 @@ int gc_compress_bf16(gc_plan_t* p, const void* grad_bf16, float* residual, uint3
     return compress_impl(p, grad_bf16, true, residual, out_idx, out_val, out_count, workspace, stream);
 }
 
+int gc_compress_workers(gc_plan_t* p, uint32_t W, const float* const* grads, float* const* residuals,
+                        uint32_t* const* out_idx, float* const* out_val, uint32_t* const* out_count,
+                        void* const* workspaces, void* stream) {
+    if (p == nullptr) return GC_E_INVALID;
+    if (W > GC_MAX_WORKERS) return GC_E_TOO_LARGE;
+    if (p->device < 0) return GC_E_UNSUPPORTED;
+    if (!on_plan_device(p)) return GC_E_INVALID;
+    if (W == 0 || p->total_n == 0) return GC_OK;
+    if (grads == nullptr || residuals == nullptr || out_idx == nullptr || out_val == nullptr || workspaces == nullptr)
+        return GC_E_INVALID;
+    for (uint32_t w = 0; w < W; ++w) {
+        if (grads[w] == nullptr || residuals[w] == nullptr || out_idx[w] == nullptr || out_val[w] == nullptr ||
+            workspaces[w] == nullptr || (out_count != nullptr && out_count[w] == nullptr))
+            return GC_E_INVALID;
+        if ((reinterpret_cast<uintptr_t>(grads[w]) & 15u) || (reinterpret_cast<uintptr_t>(residuals[w]) & 15u) ||
+            (reinterpret_cast<uintptr_t>(workspaces[w]) & 255u) || (reinterpret_cast<uintptr_t>(out_idx[w]) & 3u) ||
+            (reinterpret_cast<uintptr_t>(out_val[w]) & 3u))
+            return GC_E_INVALID;
+        for (uint32_t v = 0; v < w; ++v)         // the calls run at the same time: nothing may be shared
+            if (workspaces[v] == workspaces[w] || residuals[v] == residuals[w] || out_idx[v] == out_idx[w] ||
+                out_val[v] == out_val[w])
+                return GC_E_INVALID;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // how many workers one launch takes: the resident CTAs are dealt out evenly, and a worker's
+    // share must still satisfy the kernel's limits (tiles and candidates per CTA)
+    uint32_t batch = 0;
+    MultiGeom mg;
+    if (p->mode == GC_TOPK && p->path == GC_PATH_AUTO && p->multi_grid > 0 && W >= 2) {
+        if (p->wk_W != W) {                      // (kept for the next call; options that change the layout reset it)
+            p->wk_W = W; p->wk_batch = 0;
+            for (uint32_t wb = std::min<uint32_t>(W, kWorkersPerLaunch); wb >= 2 && p->wk_batch == 0; --wb) {
+                const MultiGeom g2 = multi_geometry(p, (uint32_t)p->grid_multi_max / wb, false);
+                if (g2.G > 0 && g2.smem <= p->multi_smem_max) { p->wk_batch = wb; p->wk_geom = g2; }
+            }
+        }
+        batch = p->wk_batch; mg = p->wk_geom;
+    }
+    if (batch == 0) {                            // no shared launch for this plan: one call per worker
+        for (uint32_t w = 0; w < W; ++w) {
+            const int rc = compress_impl(p, grads[w], false, residuals[w], out_idx[w], out_val[w],
+                                         out_count ? out_count[w] : nullptr, workspaces[w], stream);
+            if (rc < 0) return rc;
+        }
+        return GC_OK;
+    }
+    for (uint32_t w0 = 0; w0 < W; w0 += batch) {
+        const uint32_t wn = std::min<uint32_t>(batch, W - w0);
+        if (wn == 1) {                           // a lone leftover worker takes the whole device
+            const int rc = compress_impl(p, grads[w0], false, residuals[w0], out_idx[w0], out_val[w0],
+                                         out_count ? out_count[w0] : nullptr, workspaces[w0], stream);
+            if (rc < 0) return rc;
+            continue;
+        }
+        ClearMany cm;
+        WorkersArgs wa;
+        wa.W = wn; wa.G = mg.G;
+        for (uint32_t i = 0; i < wn; ++i) {
+            const uint32_t w = w0 + i;
+            cm.p[i] = reinterpret_cast<uint4*>(workspaces[w]);
+            wa.per[i] = multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w],
+                                   out_count ? out_count[w] : nullptr, workspaces[w]);
+            if (out_count != nullptr && p->n_empty > 0) {
+                Timed tm(p, s, GC_K_CLEAR_CTRL);
+                GC_CUDA(p, cudaMemsetAsync(out_count[w], 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
+            }
+        }
+        for (uint32_t i = wn; i < kWorkersPerLaunch; ++i) { cm.p[i] = nullptr; wa.per[i] = wa.per[0]; }
+        {
+            Timed tm(p, s, GC_K_CLEAR_CTRL);
+            const size_t n16 = p->control_bytes / 16;
+            const unsigned gx = (unsigned)std::min<size_t>((n16 + kBlock - 1) / kBlock, (size_t)p->sm_count * 8 / wn + 1);
+            k_clear_many<<<dim3(gx, wn), kBlock, 0, s>>>(cm, n16);
+        }
+        void* args[] = {&wa};
+        Timed tm(p, s, GC_K_FUSED);
+        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_workers<GradF32>, dim3(mg.G * wn), dim3(kBlock),
+                                               args, mg.smem, s));
+    }
+    return GC_OK;
+}
+
 int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* idx,
                              const float* const* val, const uint32_t* const* count,
                              float* dense_out, int zero_first, void* workspace, void* stream) {
@@ -993,6 +1154,24 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
+    if (count != nullptr && p->T > 1 && W > 0 && p->total_cap > 0 && p->path != GC_PATH_EXACT &&
+        p->grid_decode_seg[nbuf - 1] > 0 && p->d_dectile != nullptr) {
+        // lists with per-tensor counts: ascending inside a tensor, unused slots between tensors --
+        // the same tile loop, cut at the tensor boundaries
+        DecodeLists ls;
+        for (uint32_t w = 0; w < 64; ++w) {
+            ls.idx[w] = idx[w < W ? w : 0]; ls.val[w] = val[w < W ? w : 0]; ls.len[w] = count[w < W ? w : 0];
+        }
+        const uint32_t ntl = (uint32_t)((p->total_n + kDecTile - 1) / kDecTile);
+        const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode_seg[nbuf - 1]);
+        const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;
+        Timed tm(p, s, GC_K_DECODE_TILES);
+        k_decode_segments<false><<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(
+            ls, W, p->d_desc, p->T, p->d_dectile, (uint32_t)p->total_n, dense_out, zero_first ? 1 : 0, use_bulk, nbuf,
+            ws.hdr, ApplyArgs{});
+        GC_CUDA(p, cudaGetLastError());
+        return GC_OK;
+    }
     if (zero_first) {
         Timed tm(p, s, GC_K_DECODE_CLEAR);
         GC_CUDA(p, cudaMemsetAsync(dense_out, 0, sizeof(float) * (size_t)p->total_n, s));
@@ -1026,8 +1205,9 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(param) & 15u) ||
         (reinterpret_cast<uintptr_t>(velocity) & 15u))
         return GC_E_INVALID;
-    if (count != nullptr && p->T != 1) return GC_E_UNSUPPORTED;       // lists with gaps between tensors
-    if (p->grid_decode[0] <= 0) return GC_E_UNSUPPORTED;
+    const bool segmented = count != nullptr && p->T != 1;              // lists with unused slots between tensors
+    if ((segmented ? p->grid_decode_seg_apply : p->grid_decode[0]) <= 0) return GC_E_UNSUPPORTED;
+    if (segmented && p->d_dectile == nullptr) return GC_E_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
     DecodeLists ls;
@@ -1040,6 +1220,13 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
     const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[0]);
     ApplyArgs ap{param, velocity, lr, momentum, scale};
     Timed tm(p, s, GC_K_DECODE_TILES);
+    if (segmented && W > 0) {
+        k_decode_segments<true><<<(int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode_seg_apply), kDecBlock,
+                                  kDecTileBytes, s>>>(ls, W, p->d_desc, p->T, p->d_dectile, (uint32_t)p->total_n,
+                                                      nullptr, 1, 0, 1, ws.hdr, ap);
+        GC_CUDA(p, cudaGetLastError());
+        return GC_OK;
+    }
     const DecodeRoute rt = decode_route<true>(p, W);
     if (rt.wide) {
         auto kw = rt.any ? k_decode_any<true> : k_decode_wide<true>;
@@ -1213,15 +1400,19 @@ int gc_last_cuda_error(const gc_plan_t* p) { return p ? p->last_cuda_error : 0; 
 int gc_destroy(gc_plan_t* p) {
     if (p == nullptr) return GC_OK;
     int rc = GC_OK;
+    int caller_device = -1;
+    if (p->device >= 0) {                           // the device memory is freed with the plan's device current;
+        if (cudaGetDevice(&caller_device) != cudaSuccess) { (void)cudaGetLastError(); caller_device = -1; }
+        (void)cudaSetDevice(p->device);             // the caller's device is put back below
+    }
     for (auto& r : p->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto& u : p->staging) cudaEventDestroy(u.done);
     if (p->ev_copied) cudaEventDestroy(p->ev_copied);
     if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
-    if (p->d_small) { (void)cudaSetDevice(p->device); (void)cudaFree(p->d_small); }
-    if (p->d_desc) {
-        (void)cudaSetDevice(p->device);
-        if (cudaFree(p->d_desc) != cudaSuccess) { (void)cudaGetLastError(); rc = GC_E_CUDA; }
-    }
+    if (p->d_small) (void)cudaFree(p->d_small);
+    if (p->d_dectile) (void)cudaFree(p->d_dectile);
+    if (p->d_desc && cudaFree(p->d_desc) != cudaSuccess) { (void)cudaGetLastError(); rc = GC_E_CUDA; }
+    if (caller_device >= 0) (void)cudaSetDevice(caller_device);
     delete p;
     return rc;
 }

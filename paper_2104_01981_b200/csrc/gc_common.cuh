@@ -246,6 +246,26 @@ __device__ __forceinline__ void warp_rank(const uint32_t (&c)[kVpt], int lane,
     total = run;
 }
 
+// Where the top-k kernels look for their sample (the sample only steers the candidate bracket;
+// no result depends on it).  Sample group number sg -> 4-element group of the tensor: runs of
+// eight consecutive groups, i.e. one 128-byte line, every 8 x sstride groups.  The same number
+// of samples as one group every `sstride`, but an eighth of the scattered DRAM accesses -- the
+// sample phase is bound by how many scattered reads per second the memory serves (about 24 G/s
+// measured here), not by anything on the SM.  (The threshold variant's sample is part of its
+// definition and stays one group every `stride`.)
+__device__ __forceinline__ uint64_t sample_group(uint64_t sg, uint32_t sstride) {
+    return (sg >> 3) * (8ull * sstride) + (sg & 7ull);
+}
+
+// One count per lane into a shared-memory histogram, aggregated over the warp first: lanes that
+// hit the same bin elect one of them to add their number (keys of one tensor crowd into a
+// handful of coarse bins, and 32 atomics on one shared-memory word are served one after the
+// other).  bin = 0xFFFFFFFF: this lane has nothing to count.  All 32 lanes must call.
+__device__ __forceinline__ void hist_add_warp(uint32_t* hist, uint32_t bin, int lane) {
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, bin);
+    if (bin != 0xFFFFFFFFu && (__ffs(peers) - 1) == lane) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+}
+
 // ----------------------------------------------------------------------------- ordered tiles
 // Tile descriptors: bits 63..62 = flag (0 none, 1 aggregate of this tile, 2 inclusive prefix
 // up to and including this tile), bits 61..0 = value.  Flag and value travel in one 64-bit
@@ -314,8 +334,8 @@ __device__ __forceinline__ unsigned long long lookback(unsigned long long* state
 // Phase time stamp by CTA 0 (diagnostic).  The running index lives in a register of the caller
 // so that the stamp is two stores and no load: a load here would sit on CTA 0's path to the
 // next grid barrier, and every other CTA waits for that one.
-__device__ __forceinline__ void phase_stamp(WsHeader* hdr, uint32_t& n) {
-    if (blockIdx.x == 0 && threadIdx.x == 0 && n < 20u) {
+__device__ __forceinline__ void phase_stamp(WsHeader* hdr, uint32_t& n, uint32_t b) {
+    if (b == 0 && threadIdx.x == 0 && n < 20u) {
         unsigned long long ts;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
         hdr->stamp[n] = ts;
@@ -323,6 +343,8 @@ __device__ __forceinline__ void phase_stamp(WsHeader* hdr, uint32_t& n) {
     }
     ++n;
 }
+
+__device__ __forceinline__ void phase_stamp(WsHeader* hdr, uint32_t& n) { phase_stamp(hdr, n, blockIdx.x); }
 
 __device__ __forceinline__ void exit_stamp(WsHeader* hdr) {
     if (threadIdx.x == 0) {
@@ -333,15 +355,17 @@ __device__ __forceinline__ void exit_stamp(WsHeader* hdr) {
 }
 
 // ----------------------------------------------------------------------------- grid barrier
-// Barrier across all CTAs of a cooperative launch (all of them are resident).  The counter
-// only grows: the b-th barrier waits for b * gridDim.x arrivals.  The wait is bounded; if it
-// runs out the abort flag is raised, GC_E_TIMEOUT is recorded and every CTA leaves.
-__device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+// Barrier across the G CTAs that share one workspace header: all CTAs of a cooperative launch,
+// or one of several independent groups inside it (all CTAs of the launch are resident either
+// way).  The counter only grows: the b-th barrier waits for b * G arrivals.  The wait is
+// bounded; if it runs out the abort flag is raised, GC_E_TIMEOUT is recorded and every CTA of
+// the group leaves.
+__device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, int* s_ok, uint32_t G) {
     __syncthreads();
     if (threadIdx.x == 0) {
         int ok = 1;
         __threadfence();
-        const uint32_t target = (passed + 1u) * gridDim.x;
+        const uint32_t target = (passed + 1u) * G;
         atomicAdd(&hdr->barrier, 1u);
         uint32_t spins = 0;
         while (ld_cg(&hdr->barrier) < target) {
@@ -358,6 +382,9 @@ __device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, in
     __syncthreads();
     ++passed;
     return *s_ok != 0;
+}
+__device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+    return grid_barrier(hdr, passed, s_ok, gridDim.x);
 }
 
 }  // namespace gc

@@ -231,6 +231,149 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
+// Tiled decode of lists that carry per-tensor counts (threshold mode, plans of several tensors):
+// worker w's pairs of tensor t sit in slots [out_off_t, out_off_t + count_w[t]) and the slots up
+// to the tensor's capacity are unused, so a list is ascending only inside a tensor.  The tile
+// loop of k_decode_tiles is kept (staged tile, workers applied in order, one bulk copy out); a
+// tile is cut into segments at the tensor boundaries that fall inside it, and whenever the CTA
+// moves on to the next tensor every worker's cursor jumps to that tensor's first slot and its
+// end becomes that tensor's count.  Tiles inside one tensor (nearly all of them) cost what they
+// cost in k_decode_tiles; a boundary costs one more round trip for the counts.
+template <bool APPLY>
+static __global__ void __launch_bounds__(kDecBlock)
+k_decode_segments(DecodeLists ls, uint32_t W, const TensorDesc* __restrict__ desc, uint32_t T,
+                  const uint32_t* __restrict__ tile_tensor, uint32_t total_n, float* __restrict__ out, int zero_first, int use_bulk, int nbuf, WsHeader* hdr, ApplyArgs ap) {
+    extern __shared__ __align__(128) float s_tiles[];
+    __shared__ uint32_t s_cur[64], s_len[64];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
+    const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
+    const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
+    if (t0 >= t1) return;
+
+    // the tensor that holds the first element of this CTA's run (a table the plan made: one load
+    // instead of a binary search over the tensor table in front of every CTA's first tile)
+    uint32_t ct = __ldg(tile_tensor + t0);
+    uint32_t d_end = __ldg(&desc[ct].off) + __ldg(&desc[ct].n);       // one past the tensor's last element
+    uint32_t d_out = __ldg(&desc[ct].out_off), d_cap = __ldg(&desc[ct].cap);
+    for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
+        const uint32_t m = min(__ldg(ls.len[w] + ct), d_cap);
+        const uint32_t c = warp_lower_bound(ls.idx[w] + d_out, m, t0 * (uint32_t)kDecTile, lane);
+        if (lane == 0) { s_cur[w] = d_out + c; s_len[w] = d_out + m; }
+    }
+    int Wp = 1;
+    while (Wp < (int)W && Wp < 64) Wp <<= 1;
+    const int E = kDecBlock / Wp;
+    const uint32_t my_w = (uint32_t)(tid / E);
+    const int sub = tid % E;
+    const bool live = my_w < W;
+    __syncthreads();
+
+    for (uint32_t tl = t0; tl < t1; ++tl) {
+        float* const s_tile = s_tiles + (nbuf == 2 ? ((tl - t0) & 1u) : 0u) * kDecTile;
+        if (use_bulk) {                                  // the copy that last used this buffer must have read it
+            if (tid == 0) { if (nbuf == 2) bulk_wait_read<1>(); else bulk_wait_read<0>(); }
+            __syncthreads();
+        }
+        const uint32_t lo = tl * (uint32_t)kDecTile;
+        const uint32_t hi = min(total_n, lo + (uint32_t)kDecTile);
+        const bool full = hi - lo == (uint32_t)kDecTile;
+        stage_tile(s_tile, out, lo, hi, full, zero_first, use_bulk, tid);
+        uint32_t seg_lo = lo;
+        while (true) {
+            const uint32_t seg_hi = min(hi, d_end);
+            const uint32_t my_len = live ? s_len[my_w] : 0u;
+            const uint32_t c0 = live ? s_cur[my_w] : 0u;
+            // the tensor ends inside this tile: the next tensor's table entry and this worker's count
+            // for it are fetched together with the list entries (one round trip for both)
+            const bool ends = d_end <= hi && ct + 1u < T;
+            uint32_t nn = 0, n_off = 0, n_out = 0, n_cap = 0, ncnt = 0;
+            if (ends) {
+                nn = __ldg(&desc[ct + 1u].n); n_off = __ldg(&desc[ct + 1u].off);
+                n_out = __ldg(&desc[ct + 1u].out_off); n_cap = __ldg(&desc[ct + 1u].cap);
+                if (tid < (int)W) ncnt = __ldg(ls.len[tid] + ct + 1u);
+            }
+            uint32_t ix[kDecRounds];
+            float v[kDecRounds];
+            uint32_t nin = 0;
+#pragma unroll
+            for (int rd = 0; rd < kDecRounds; ++rd) {
+                const uint32_t p = c0 + (uint32_t)(rd * E + sub);
+                ix[rd] = 0xFFFFFFFFu; v[rd] = 0.f;
+                if (live && p < my_len) { ix[rd] = __ldg(ls.idx[my_w] + p); v[rd] = __ldg(ls.val[my_w] + p); }
+            }
+#pragma unroll
+            for (int rd = 0; rd < kDecRounds; ++rd) nin += ix[rd] < seg_hi;
+            const bool maybe_more = (ix[kDecRounds - 1] < seg_hi) && sub == E - 1;
+            if (!__syncthreads_or(maybe_more ? 1 : 0)) {                  // (also: tile staged, cursors read)
+                for (uint32_t q = 0; q < W; ++q) {                         // apply in worker order
+                    if (my_w == q) {
+#pragma unroll
+                        for (int rd = 0; rd < kDecRounds; ++rd) {
+                            if (ix[rd] < seg_hi) {
+                                if (ix[rd] >= seg_lo) s_tile[ix[rd] - lo] = __fadd_rn(s_tile[ix[rd] - lo], v[rd]);
+                                else record_status(hdr, -1 /*GC_E_INVALID*/, c0);      // not ascending / outside its tensor
+                            }
+                        }
+                    }
+                    __syncthreads();
+                }
+                if (live && nin) atomicAdd(&s_cur[my_w], nin);
+            } else {
+                for (uint32_t q = 0; q < W; ++q) {
+                    uint32_t c = s_cur[q];
+                    const uint32_t qlen = s_len[q];
+                    __syncthreads();
+                    while (true) {
+                        const uint32_t pp = c + (uint32_t)tid;
+                        uint32_t ix2 = 0xFFFFFFFFu;
+                        float v2 = 0.f;
+                        if (pp < qlen) { ix2 = __ldg(ls.idx[q] + pp); v2 = __ldg(ls.val[q] + pp); }
+                        const bool in2 = ix2 < seg_hi;
+                        if (in2) {
+                            if (ix2 >= seg_lo) s_tile[ix2 - lo] = __fadd_rn(s_tile[ix2 - lo], v2);
+                            else record_status(hdr, -1 /*GC_E_INVALID*/, pp);
+                        }
+                        const int m = __syncthreads_count(in2 ? 1 : 0);
+                        c += (uint32_t)m;
+                        if (m != kDecBlock) break;
+                    }
+                    if (tid == 0) s_cur[q] = c;
+                }
+            }
+            __syncthreads();
+            if (seg_hi < d_end) break;                   // the tile ends inside the tensor
+            // the tensor ends here: whatever a list still holds for it points beyond its end
+            if (tid < (int)W && s_cur[tid] < s_len[tid]) record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);
+            ++ct;
+            while (ct < T && nn == 0u) {                  // (tensors without elements are stepped over)
+                if (++ct >= T) break;
+                nn = __ldg(&desc[ct].n); n_off = __ldg(&desc[ct].off);
+                n_out = __ldg(&desc[ct].out_off); n_cap = __ldg(&desc[ct].cap);
+                if (tid < (int)W) ncnt = __ldg(ls.len[tid] + ct);
+            }
+            if (ct >= T) { d_end = 0xFFFFFFFFu; break; }  // (only after the last element of the buffer)
+            d_end = n_off + nn; d_out = n_out; d_cap = n_cap;
+            if (tid < (int)W) { s_cur[tid] = d_out; s_len[tid] = d_out + min(ncnt, d_cap); }   // (own entries only)
+            __syncthreads();
+            if (seg_hi >= hi) break;                     // the tensor ended together with the tile
+            seg_lo = seg_hi;
+        }
+        if (APPLY) {
+            apply_tile(ap, s_tile, lo, hi, full, tid);
+            __syncthreads();
+            continue;
+        }
+        if (full && use_bulk) {
+            if (tid == 0) bulk_store_tile(out + lo, s_tile, (uint32_t)(kDecTile * sizeof(float)));
+        } else {
+            for (uint32_t q = tid; q < hi - lo; q += kDecBlock) out[lo + q] = s_tile[q];
+        }
+        __syncthreads();
+    }
+    if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 // 4-byte asynchronous copy global -> shared, and the wait for all such copies of this thread.
 __device__ __forceinline__ void cp_async_4(void* sdst, const void* gsrc) {
     const uint32_t sa = (uint32_t)__cvta_generic_to_shared(sdst);

@@ -83,7 +83,8 @@ static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const Tenso
                 const uint32_t key = key_of(tl.a[j][e]);
                 bool in = (tl.valid >> (4 * j + e)) & 1u;
                 if (level > 0) in = in && ((key >> (sh + bits)) == prefix);
-                if (in) atomicAdd(&sm.hist[(key >> sh) & ((1u << bits) - 1u)], 1u);
+                if (level == 0) hist_add_warp(sm.hist, in ? key >> sh : 0xFFFFFFFFu, lane);    // (crowded coarse bins)
+                else if (in) atomicAdd(&sm.hist[(key >> sh) & ((1u << bits) - 1u)], 1u);
             }
         }
         __syncthreads();
@@ -145,6 +146,92 @@ static __device__ __noinline__ void small_tensor_body(BlockSmem& sm, const Tenso
     }
     if (out_count != nullptr && tid == 0) { out_count[t] = d.k; out_count[T + t] = d.k; }
     __syncthreads();
+}
+
+// Exact top-k of one TINY tensor (at most kTinyMaxN elements, k at most kTinyMaxK) by ONE WARP:
+// no shared memory and no block-wide barrier, so the eight warps of a CTA finish eight such
+// tensors at once (layer-wise plans hold dozens of normalisation vectors of 64 to 512 elements
+// with k = 1).  The tensor is read once (all loads of a lane in flight together) and stays in
+// registers, 16 values per lane.  Pass 0 finds the largest key, ties to the lower index; every
+// further pass finds the largest entry that comes strictly after the previous winner in that
+// order (key descending, index ascending).  The k winners are then ranked by index for the output.
+constexpr uint32_t kTinyMaxN = 512, kTinyMaxK = 16;
+__host__ __device__ inline bool is_tiny(uint32_t n, uint32_t k) { return n > 0 && n <= kTinyMaxN && k <= kTinyMaxK; }
+
+__device__ __forceinline__ unsigned long long warp_max64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, d);
+        v = o > v ? o : v;
+    }
+    return v;
+}
+
+template <typename GL = GradF32>
+static __device__ __noinline__ void tiny_tensor_warp(const uint32_t off, const uint32_t n, const uint32_t k,
+                                                     const uint32_t out_off, uint32_t t, uint32_t T,
+                                                     const void* __restrict__ g, float* __restrict__ r,
+                                                     uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                                     uint32_t* __restrict__ out_count, int lane) {
+    constexpr int kU = (int)kTinyMaxN / 32;               // values per lane: element i sits in lane i % 32, slot i / 32
+    float gv[kU], rv[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const uint32_t i = (uint32_t)lane + 32u * u;
+        gv[u] = i < n ? GL::ld1(g, off + i) : 0.f;
+        rv[u] = i < n ? r[off + i] : 0.f;
+    }
+    // order of two entries as one 64-bit compare: key in the high word, ~index in the low one
+    // (a real entry is never 0: ~index > 0)
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const uint32_t i = (uint32_t)lane + 32u * u;
+        gv[u] = __fadd_rn(gv[u], rv[u]);                  // a = g + r
+        const unsigned long long o = ((unsigned long long)key_of(gv[u]) << 32) | (unsigned long long)(~i);
+        if (i < n && o > best) best = o;
+    }
+    unsigned long long win = warp_max64(best), mine = 0ull;    // lane j keeps winner j
+    if (lane == 0) mine = win;
+    for (uint32_t j = 1; j < k; ++j) {
+        best = 0ull;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const uint32_t i = (uint32_t)lane + 32u * u;
+            const unsigned long long o = ((unsigned long long)key_of(gv[u]) << 32) | (unsigned long long)(~i);
+            if (i < n && o < win && o > best) best = o;
+        }
+        win = warp_max64(best);
+        if ((uint32_t)lane == j) mine = win;
+    }
+    // rank of winner `lane` among the winners by index (the low words hold ~index: larger = lower index)
+    const uint32_t my_ni = (uint32_t)mine;
+    uint32_t rank = 0;
+    for (uint32_t j = 0; j < k; ++j) {
+        const uint32_t o = __shfl_sync(0xFFFFFFFFu, my_ni, (int)j);
+        rank += o > my_ni ? 1u : 0u;
+    }
+    // the pairs: the lane that holds winner j's value writes it at that winner's rank
+    uint32_t sent = 0;                                    // bit u: this lane's slot u is a winner
+    for (uint32_t j = 0; j < k; ++j) {
+        const uint32_t wi = ~__shfl_sync(0xFFFFFFFFu, my_ni, (int)j);
+        const uint32_t rk = __shfl_sync(0xFFFFFFFFu, rank, (int)j);
+        if ((wi & 31u) == (uint32_t)lane) {
+            float v = 0.f;
+#pragma unroll
+            for (int u = 0; u < kU; ++u) if ((uint32_t)u == (wi >> 5)) v = gv[u];
+            out_idx[out_off + rk] = off + wi;
+            out_val[out_off + rk] = v;                    // bit copy of a
+            sent |= 1u << (wi >> 5);
+        }
+    }
+    // the residual: a everywhere, +0 at the winners
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const uint32_t i = (uint32_t)lane + 32u * u;
+        if (i < n) r[off + i] = ((sent >> u) & 1u) ? 0.0f : gv[u];
+    }
+    if (out_count != nullptr && lane == 0) { out_count[t] = k; out_count[T + t] = k; }
 }
 
 // All small tensors of the plan, dealt out to the CTAs round-robin.
@@ -552,7 +639,7 @@ struct FusedArgs {
 // Phases are separated by grid barriers; every decision taken after a barrier reads values
 // that were final before it, so all CTAs take the same route.
 static __global__ void __launch_bounds__(kBlock, 4)
-k_compress_fused(FusedArgs a) {
+k_compress_fused(const __grid_constant__ FusedArgs a) {
     __shared__ BlockSmem sm;
     uint32_t passed = 0, n_stamp = 0;
     WsHeader* hdr = a.ws.hdr;

@@ -210,6 +210,14 @@ static __global__ void __launch_bounds__(kBlock) k_clear(uint4* __restrict__ p, 
     for (size_t i = (size_t)blockIdx.x * kBlock + threadIdx.x; i < n16; i += (size_t)gridDim.x * kBlock) p[i] = z;
 }
 
+// The same for several workspaces at once (blockIdx.y picks the workspace).
+struct ClearMany { uint4* p[12]; };
+static __global__ void __launch_bounds__(kBlock) k_clear_many(const __grid_constant__ ClearMany c, size_t n16) {
+    uint4* const p = c.p[blockIdx.y];
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t i = (size_t)blockIdx.x * kBlock + threadIdx.x; i < n16; i += (size_t)gridDim.x * kBlock) p[i] = z;
+}
+
 // ----------------------------------------------------------------------------- histogram pass
 // One radix-select level over all tensors.  CTAs take contiguous runs of tiles, keep a
 // shared-memory histogram while the tensor stays the same, flush it with global atomics when
@@ -223,14 +231,15 @@ constexpr int SRC_FOLD = 0, SRC_RESID = 1, SRC_SAMPLE = 2;
 
 template <int LEVEL, int SRC>
 __device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
-                          const float* __restrict__ g, float* __restrict__ r, const WsView& ws) {
+                          const float* __restrict__ g, float* __restrict__ r, const WsView& ws,
+                          uint32_t G, uint32_t b_in_group) {       // G CTAs share the work, this is CTA b of them
     using S = typename std::conditional<SRC == SRC_SAMPLE, SampleSpace, FullSpace>::type;
     constexpr int NB = 1 << level_bits(LEVEL);
     constexpr int SH = level_shift(LEVEL);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (nothing_to_redo(ws)) return;
-    const uint32_t per = (ntiles + gridDim.x - 1) / gridDim.x;
-    const uint32_t first = blockIdx.x * per;
+    const uint32_t per = (ntiles + G - 1) / G;
+    const uint32_t first = b_in_group * per;
     const uint32_t last = min(ntiles, first + per);
     if (first >= last) return;
     for (int b = tid; b < NB; b += kBlock) sm.hist[b] = 0u;
@@ -294,6 +303,12 @@ __device__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, ui
         ++tiles_here;
     }
     if (active && tiles_here) flush_and_select<LEVEL, false>(sm, ws, t, tiles_here, S::ntiles(d), S::rank(d));
+}
+
+template <int LEVEL, int SRC>
+__device__ __forceinline__ void hist_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T, uint32_t ntiles,
+                                          const float* __restrict__ g, float* __restrict__ r, const WsView& ws) {
+    hist_body<LEVEL, SRC>(sm, desc, T, ntiles, g, r, ws, gridDim.x, blockIdx.x);
 }
 
 template <int LEVEL, int SRC>

@@ -38,8 +38,8 @@ struct MultiArgs {
     uint32_t pool_cap;               // candidate slots per CTA
     uint32_t pool_smem_words;        // words of shared memory reserved for one bit per candidate slot
     uint32_t ntab;                   // T if the tile tables fit in shared memory, else 0
-    const uint32_t* small_ids;
-    uint32_t n_small;
+    const uint32_t* small_ids;       // the tensors that fit one tile, the tiny ones (one warp each) first
+    uint32_t n_small, n_tiny;
     const uint32_t* reg_ids;         // the tensors that are not small (and not empty)
     uint32_t n_reg;
     TensorSel* brk;                  // [T] bracket of every such tensor: .prefix = tau, .krem = tau_z, .T = shift
@@ -72,10 +72,10 @@ __device__ __forceinline__ void grid_arrive(WsHeader* hdr) {
     }
 }
 // second half of a barrier whose arrival was signalled with grid_arrive
-__device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+__device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* s_ok, uint32_t G) {
     if (threadIdx.x == 0) {
         int ok = 1;
-        const uint32_t target = (passed + 1u) * gridDim.x;
+        const uint32_t target = (passed + 1u) * G;
         uint32_t spins = 0;
         while (ld_cg(&hdr->barrier) < target) {
             if (++spins > kSpinLimit || ((spins & 15u) == 0u && ld_cg(&hdr->abort) != 0u)) { ok = 0; break; }
@@ -92,24 +92,24 @@ __device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* 
     ++passed;
     return *s_ok != 0;
 }
+__device__ __forceinline__ bool grid_wait(WsHeader* hdr, uint32_t& passed, int* s_ok) {
+    return grid_wait(hdr, passed, s_ok, gridDim.x);
+}
 
+// The whole compress of one worker by the G CTAs of one group (this CTA is number b of them);
+// the group's barriers count on the worker's own workspace header.
 template <typename GL>
-// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
-static __global__ void __launch_bounds__(kBlock, 3)
-k_topk_multi(MultiArgs a) {
-    __shared__ BlockSmem sm;
-    __shared__ uint32_t s_used, s_cnt;
-    extern __shared__ __align__(16) unsigned char s_dyn[];
+__device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32_t G, const uint32_t b, BlockSmem& sm,
+                                                uint32_t& s_used, uint32_t& s_cnt, unsigned char* s_dyn) {
     uint32_t* const rec = reinterpret_cast<uint32_t*>(s_dyn);                  // [per*kWarps] off<<10 | cnt
     uint32_t* const rec2 = rec + (size_t)a.per * kWarps;                       // [per*kWarps] counts, later slots
     uint32_t* const seg = rec2 + (size_t)a.per * kWarps;                       // [per][kSegWords]
     uint32_t* const sent_bits = seg + (size_t)a.per * kSegWords;               // [ceil(pool_cap / 32)]
     uint32_t* const tab_tile0 = sent_bits + (a.pool_smem_words);               // [ntab] first tile of every tensor
     uint32_t* const tab_stile0 = tab_tile0 + a.ntab;                           // [ntab] first sample tile
-    uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
+    uint2* const pool = a.cand + (size_t)b * a.pool_cap;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t G = gridDim.x, b = blockIdx.x;
     WsHeader* hdr = a.ws.hdr;
     uint32_t passed = 0, n_stamp = 0;
     // The CTAs launched last are the youngest on their SMs and advance the slowest (see RowMap in
@@ -132,7 +132,7 @@ k_topk_multi(MultiArgs a) {
         tab_tile0[t] = a.desc[t].tile0;
         tab_stile0[t] = a.desc[t].stile0;
     }
-    phase_stamp(hdr, n_stamp);
+    phase_stamp(hdr, n_stamp, b);
     __syncthreads();
     auto owner = [&](const uint32_t* tab, uint32_t tile) -> uint32_t {    // last t with tab[t] <= tile
         uint32_t lo = 0, hi = a.ntab;
@@ -149,52 +149,86 @@ k_topk_multi(MultiArgs a) {
         const uint32_t sfirst = min(a.nstiles, b * sper), slast = min(a.nstiles, sfirst + sper);
         uint32_t t = 0xFFFFFFFFu;
         TensorDesc d;
-        for (uint32_t st = sfirst; st < slast; ++st) {
+        for (uint32_t st = sfirst; st < slast;) {
             if (t == 0xFFFFFFFFu || st >= d.stile0 + d.nstiles) {
                 if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));
                 __syncthreads();
                 t = a.ntab ? owner(tab_stile0, st) : find_tensor<SampleSpace>(a.desc, a.T, st);
                 d = a.desc[t];
             }
+            // up to kSampleBatch sample tiles of this tensor at once: all their loads are in flight
+            // together, so a CTA that owns several sample tiles (a group of CTAs that serves one of
+            // several workers) pays one round trip for the batch instead of one per tile
+            constexpr uint32_t kSampleBatch = 4;
+            const uint32_t nb = min(kSampleBatch, min(slast, d.stile0 + d.nstiles) - st);
             const uint32_t ngroups = (d.n + 3u) >> 2;
             const uint32_t nsg = (ngroups + d.sstride - 1) / d.sstride;
-            const uint64_t sg = (uint64_t)(st - d.stile0) * kBlock + tid;
-            const uint64_t gi = sg * d.sstride;
-            uint32_t key[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};     // = not a sample
-            if (sg < nsg && gi < ngroups) {
-                const uint32_t i0 = (uint32_t)gi * 4u;
-                float gv[4], rv[4];
+            const bool vec_ok = (d.off & 3u) == 0u;           // the tensor's groups are 16-byte aligned in the flat buffers
+            float gv[kSampleBatch][4], rv[kSampleBatch][4];
+            uint32_t i0[kSampleBatch];
+            bool live[kSampleBatch];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const bool v = i0 + e < d.n;
-                    const uint32_t f = d.off + (v ? i0 + e : 0u);
-                    gv[e] = v ? GL::ld1(a.g, f) : 0.f;
-                    rv[e] = v ? ld_cg(a.r + f) : 0.f;
-                }
+            for (uint32_t u = 0; u < kSampleBatch; ++u) {
+                const uint64_t sg = (uint64_t)(st + u - d.stile0) * kBlock + tid;
+                const uint64_t gi = sample_group(sg, d.sstride);
+                live[u] = u < nb && sg < nsg && gi < ngroups;
+                i0[u] = live[u] ? (uint32_t)gi * 4u : 0u;
+                if (vec_ok && live[u] && i0[u] + 3u < d.n) {
+                    // the whole group in one 16-byte load each (a quarter of the load instructions and
+                    // of the sectors the L1 has to look up: the groups lie `sstride` x 16 bytes apart)
+                    const float4 g4 = GL::ld4(a.g, d.off + i0[u]);
+                    const float4 r4 = ld_cg(reinterpret_cast<const float4*>(a.r + d.off + i0[u]));
+                    gv[u][0] = g4.x; gv[u][1] = g4.y; gv[u][2] = g4.z; gv[u][3] = g4.w;
+                    rv[u][0] = r4.x; rv[u][1] = r4.y; rv[u][2] = r4.z; rv[u][3] = r4.w;
+                } else {
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (i0 + e < d.n) {
-                        key[e] = key_of(__fadd_rn(gv[e], rv[e]));
-                        atomicAdd(&sm.hist[key[e] >> level_shift(0)], 1u);
+                    for (int e = 0; e < 4; ++e) {
+                        const bool v = live[u] && i0[u] + e < d.n;
+                        const uint32_t f = d.off + (v ? i0[u] + e : 0u);
+                        gv[u][e] = v ? GL::ld1(a.g, f) : 0.f;
+                        rv[u][e] = v ? ld_cg(a.r + f) : 0.f;
                     }
+                }
             }
-            // the keys are kept: the fold pass ranks them a second time, and by then the residual
-            // they were computed from has been overwritten
-            if (d.nstiles <= kRefineTiles) a.skeys[(size_t)st * kBlock + tid] = make_uint4(key[0], key[1], key[2], key[3]);
+#pragma unroll
+            for (uint32_t u = 0; u < kSampleBatch; ++u) {
+                if (u < nb) {                             // (uniform over the CTA)
+                    uint32_t key[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};     // = not a sample
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (live[u] && i0[u] + e < d.n) key[e] = key_of(__fadd_rn(gv[u][e], rv[u][e]));
+                        hist_add_warp(sm.hist, key[e] == 0xFFFFFFFFu ? 0xFFFFFFFFu : key[e] >> level_shift(0), lane);
+                    }
+                    // the keys are kept: the fold pass ranks them a second time, and by then the residual
+                    // they were computed from has been overwritten
+                    if (d.nstiles <= kRefineTiles)
+                        a.skeys[(size_t)(st + u) * kBlock + tid] = make_uint4(key[0], key[1], key[2], key[3]);
+                }
+            }
+            st += nb;
         }
         if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));
     }
     grid_arrive(hdr);
     // small tensors need nothing from anyone: they fill the wait (CTAs from the top take them)
-    for (uint32_t q = G - 1u - b; q < a.n_small; q += G) {
+    for (uint32_t q8 = G - 1u - b; q8 * kWarps < a.n_tiny; q8 += G) {        // tiny ones: a warp each, eight at a time
+        const uint32_t q = q8 * kWarps + (uint32_t)warp;
+        if (q < a.n_tiny) {
+            const uint32_t t = a.small_ids[q];
+            const TensorDesc d = a.desc[t];
+            tiny_tensor_warp<GL>(d.off, d.n, d.k, d.out_off, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count, lane);
+        }
+    }
+    // (the other small ones start with the CTAs next to those that took the tiny ones)
+    for (uint32_t q = a.n_tiny + (2u * G - 1u - b - ((a.n_tiny + kWarps - 1u) / kWarps) % G) % G; q < a.n_small; q += G) {
         const uint32_t t = a.small_ids[q];
         const TensorDesc d = a.desc[t];
         small_tensor_body<GL>(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
     }
     __syncthreads();
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
-    if (!grid_wait(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_wait(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     // ---------------------------------------------------------------- bracket per tensor, one CTA each
     // tau = the srank-th largest sampled key (22 bits when the kept keys allow the second radix
@@ -259,8 +293,8 @@ k_topk_multi(MultiArgs a) {
         }
         if (tid == 0) { a.brk[cur].prefix = tau; a.brk[cur].krem = tau_z; a.brk[cur].T = (uint32_t)shift; }
     }
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     // ---------------------------------------------------------------- fold + candidates, segment by segment
     uint32_t nseg = 0;
@@ -402,8 +436,8 @@ k_topk_multi(MultiArgs a) {
         if (tid == 0) atomicAdd(&hdr->cand_total, min(s_used, a.pool_cap));
     }
     const uint32_t used = s_used;      // read linearly only when no chunk anywhere overflowed
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     // segment of a candidate: the last one that begins at or before its index
     auto seg_of = [&](uint32_t idx) -> uint32_t* {
@@ -465,8 +499,8 @@ k_topk_multi(MultiArgs a) {
             a.tile_cnt[first + i] = tot;
         }
     }
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     if (!overflowed) {
         if (nseg != 0u) {
@@ -545,7 +579,7 @@ k_topk_multi(MultiArgs a) {
             }
             __syncthreads();
         }
-        phase_stamp(hdr, n_stamp);
+        phase_stamp(hdr, n_stamp, b);
         // sent flags of the CTA's candidates in list order, one bit each
         auto sent_of = [&](const uint32_t* s, const uint2& pr) {
             const uint32_t key = pr.y & kKeyMask;
@@ -599,7 +633,7 @@ k_topk_multi(MultiArgs a) {
             }
         }
         __syncthreads();
-        phase_stamp(hdr, n_stamp);
+        phase_stamp(hdr, n_stamp, b);
         exit_stamp(hdr);
         if (ld_cg(&hdr->n_failed) == 0u) return;
     } else {
@@ -615,15 +649,55 @@ k_topk_multi(MultiArgs a) {
 
     // ---------------------------------------------------------------- exact redo (rare)
     // of the flagged tensors, or of all of them after an overflow: r holds a = g + r for them again
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
-    hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws);
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
+    hist_body<0, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws, G, b);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    hist_body<1, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws, G, b);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws, G, b);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
     compact_body(sm, a.desc, a.T, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
+}
+
+template <typename GL>
+// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
+static __global__ void __launch_bounds__(kBlock, 3)
+k_topk_multi(const __grid_constant__ MultiArgs a) {
+    __shared__ BlockSmem sm;
+    __shared__ uint32_t s_used, s_cnt;
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    topk_multi_body<GL>(a, gridDim.x, blockIdx.x, sm, s_used, s_cnt, s_dyn);
+}
+
+// Several workers' compress calls in ONE cooperative launch: the grid is cut into one group of
+// CTAs per worker (CTA x serves worker x mod W as number x / W of its group, so every worker's
+// CTAs are spread over all SMs), and each group runs the kernel above on its own gradient,
+// residual, outputs and workspace.  Nothing is shared between the groups, not even a barrier:
+// a group's phases wait only for that worker's CTAs, so while one worker's CTAs sit in a
+// barrier the SMs stream another worker's tiles.
+constexpr uint32_t kWorkersPerLaunch = 12;       // per-worker argument blocks travel as kernel parameters
+struct WorkersArgs {
+    uint32_t W, G;                               // workers in this launch, CTAs per worker
+    MultiArgs per[kWorkersPerLaunch];
+};
+static_assert(sizeof(WorkersArgs) <= 4000, "kernel parameters stay below 4 KB");
+
+template <typename GL>
+static __global__ void __launch_bounds__(kBlock, 3)
+k_topk_workers(const __grid_constant__ WorkersArgs wa) {
+    __shared__ BlockSmem sm;
+    __shared__ uint32_t s_used, s_cnt;
+    __shared__ MultiArgs s_args;                  // this CTA's worker (dynamic indexing of the parameters happens once)
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    const uint32_t w = blockIdx.x % wa.W, b = blockIdx.x / wa.W;
+    {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(&wa.per[w]);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&s_args);
+        for (uint32_t i = threadIdx.x; i < sizeof(MultiArgs) / 4; i += kBlock) dst[i] = src[i];
+    }
+    __syncthreads();
+    topk_multi_body<GL>(s_args, wa.G, b, sm, s_used, s_cnt, s_dyn);
 }
 
 }  // namespace gc

@@ -215,7 +215,7 @@ __device__ bool short_list_select(BlockSmem& sm, const uint2 (&e)[kMidRegs], con
 // than four CTAs at 64 registers with spills, and than two.
 template <typename GL>
 static __global__ void __launch_bounds__(kBlock, 3)
-k_topk_single(SingleArgs a) {
+k_topk_single(const __grid_constant__ SingleArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used;
     extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -265,7 +265,7 @@ k_topk_single(SingleArgs a) {
 #pragma unroll
         for (int q = 0; q < kMaxOwn; ++q) {
             const uint64_t sg = (uint64_t)q * G * kBlock + (uint64_t)b * kBlock + tid;
-            const uint64_t gi = sg * d.sstride;
+            const uint64_t gi = sample_group(sg, d.sstride);
             const bool in = sg < nsg && gi < ngroups;
             const uint32_t i0 = in ? (uint32_t)gi * 4u : 0u;
             float gv[4], rv[4];
@@ -285,11 +285,11 @@ k_topk_single(SingleArgs a) {
 #pragma unroll
         for (int q = 0; q < kMaxOwn; ++q)
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if ((sok >> (4 * q + e)) & 1u) {
-                    atomicAdd(&sm.hist[skey[q][e] >> level_shift(0)], 1u);
-                    atomicAdd(a.fine + fine_slot(skey[q][e] >> kFineShift), 1u);
-                }
+            for (int e = 0; e < 4; ++e) {
+                const bool okq = (sok >> (4 * q + e)) & 1u;
+                hist_add_warp(sm.hist, okq ? skey[q][e] >> level_shift(0) : 0xFFFFFFFFu, lane);
+                if (okq) atomicAdd(a.fine + fine_slot(skey[q][e] >> kFineShift), 1u);
+            }
         // the first own tile is asked into L2 while the sample is being settled
         if (b < a.ntiles) {
             const uint32_t pb = (d.off & ~3u) + b * (uint32_t)kTile + warp * kWarpChunk + lane * 4;

@@ -134,7 +134,7 @@ static __device__ __noinline__ void small_threshold_body(BlockSmem& sm, const Te
 
 // (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
 static __global__ void __launch_bounds__(kBlock, 3)
-k_threshold_multi(ThrMultiArgs a) {
+k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used, s_cnt;
     extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -200,11 +200,11 @@ k_threshold_multi(ThrMultiArgs a) {
                 }
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (i0 + e < d.n) {
-                        key[e] = key_of(__fadd_rn(gv[e], rv[e]));
-                        atomicAdd(&sm.hist[key[e] >> level_shift(0)], 1u);
-                    }
+                    if (i0 + e < d.n) key[e] = key_of(__fadd_rn(gv[e], rv[e]));
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)          // (all lanes: the coarse counts are aggregated over the warp)
+                hist_add_warp(sm.hist, key[e] == 0xFFFFFFFFu ? 0xFFFFFFFFu : key[e] >> level_shift(0), lane);
             a.skeys[(size_t)st * kBlock + tid] = make_uint4(key[0], key[1], key[2], key[3]);
         }
         if (t != 0xFFFFFFFFu) flush_hist(sm, a.shist + (size_t)t * kHistBins, 1 << level_bits(0));

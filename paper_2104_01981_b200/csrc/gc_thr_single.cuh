@@ -47,7 +47,7 @@ struct ThrSingleArgs {
 
 // (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
 static __global__ void __launch_bounds__(kBlock, 3)
-k_threshold_single(ThrSingleArgs a) {
+k_threshold_single(const __grid_constant__ ThrSingleArgs a) {
     __shared__ BlockSmem sm;
     __shared__ uint32_t s_used;
     extern __shared__ __align__(16) unsigned char s_dyn[];
@@ -74,13 +74,13 @@ k_threshold_single(ThrSingleArgs a) {
     const uint32_t nsg = (ngroups + d.sstride - 1) / d.sstride;
     for (uint32_t q = 0; q < a.sample_rounds; ++q) {
         const uint64_t sg = (uint64_t)q * G * kBlock + (uint64_t)b * kBlock + tid;
-        if (sg >= nsg) continue;
-        const uint64_t gi = sg * d.sstride;                 // < ngroups by the definition of nsg
-        const uint32_t i0 = (uint32_t)gi * 4u;
+        const bool mine = sg < nsg;                         // (every lane stays in the loop: the coarse counts are
+        const uint64_t gi = sg * d.sstride;                 //  aggregated over the warp)  gi < ngroups by the definition of nsg
+        const uint32_t i0 = mine ? (uint32_t)gi * 4u : 0u;
         float gv[4], rv[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const bool v = i0 + e < d.n;
+            const bool v = mine && i0 + e < d.n;
             const uint32_t f = d.off + (v ? i0 + e : 0u);
             gv[e] = v ? __ldg(a.g + f) : 0.f;
             rv[e] = v ? ld_cg(a.r + f) : 0.f;
@@ -89,13 +89,13 @@ k_threshold_single(ThrSingleArgs a) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             key[e] = 0xFFFFFFFFu;                           // = not a sample
-            if (i0 + e < d.n) {
+            if (mine && i0 + e < d.n) {
                 key[e] = key_of(__fadd_rn(gv[e], rv[e]));
-                atomicAdd(&sm.hist[key[e] >> level_shift(0)], 1u);
                 atomicAdd(a.fine + fine_slot(key[e] >> kFineShift), 1u);
             }
+            hist_add_warp(sm.hist, key[e] == 0xFFFFFFFFu ? 0xFFFFFFFFu : key[e] >> level_shift(0), lane);
         }
-        a.skeys[sg] = make_uint4(key[0], key[1], key[2], key[3]);
+        if (mine) a.skeys[sg] = make_uint4(key[0], key[1], key[2], key[3]);
     }
     flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
     if (!grid_barrier(hdr, passed, &sm.ok)) return;

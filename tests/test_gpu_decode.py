@@ -271,6 +271,88 @@ def test_one_tensor_lists_with_counts_use_their_length(W, route):
     assert st == api.GC_OK
 
 
+def lists_with_counts(plan, sizes, W, seed, fill):
+    """W threshold-mode lists of a many-tensor plan built from the input generator: worker w sends
+    m[w][t] <= cap[t] pairs of tensor t (from nothing to the full capacity), laid out at the tensor's
+    output offset; the unused slots behind them hold junk (indices that are not ascending and lie
+    in other tensors, huge values) that must never be applied.  Returns oracle pairs and device
+    idx / val / count tensors."""
+    rng = np.random.default_rng(seed)
+    caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
+    T, n, total_cap = len(sizes), plan.total_n, plan.total_cap
+    pairs, d_idx, d_val, d_cnt = [], [], [], []
+    for w in range(W):
+        m = []
+        for t in range(T):
+            mode = (w + t) % 4 if fill == "mixed" else fill
+            m.append(int({0: caps[t], 1: caps[t] // 2, 2: 0, 3: min(caps[t], 1), "full": caps[t]}[mode]))
+        idx, val = synth.sparse_set(sizes, m, seed + 31 * w, scale=10.0 ** (w % 4 - 2))
+        pairs.append((idx, val))
+        full_idx = ((rng.integers(0, max(n, 1), size=max(total_cap, 1))).astype(np.uint32))[:total_cap]
+        full_val = np.full(total_cap, 3e30, np.float32)
+        pos = 0
+        for t in range(T):
+            full_idx[offs[t]:offs[t] + m[t]] = idx[pos:pos + m[t]]
+            full_val[offs[t]:offs[t] + m[t]] = val[pos:pos + m[t]]
+            pos += m[t]
+        d_idx.append(torch.from_numpy(full_idx.view(np.int32)).cuda())
+        d_val.append(torch.from_numpy(full_val).cuda())
+        d_cnt.append(torch.tensor(m + [x + 5 for x in m], dtype=torch.int32, device="cuda"))    # [T + t] = hits: unused here
+    return pairs, d_idx, d_val, d_cnt
+
+
+@pytest.mark.parametrize("W", [1, 2, 3, 8, 17, 64])
+@pytest.mark.parametrize("sizes,density,fill", [
+    ([5, 3, 1000, 7, 8193, 64, 1, 0, 2, 70_001, 300_000, 0, 6, 131_073], 0.01, "mixed"),
+    ([0, 0, 40_000, 0, 8192, 8192, 16_384, 3, 0], 0.05, "mixed"),
+    ([300_007, 64, 64, 128, 2_000_001, 512, 512], 0.002, "full"),
+    ([20_000] * 40, 0.3, "mixed"),
+])
+def test_many_tensor_lists_with_counts_match_the_oracle(W, sizes, density, fill):
+    """Threshold-mode lists of plans with several tensors: every tensor's pairs start at its output
+    offset and only count[t] of its slots are live.  Plain decode in both modes and the fused
+    momentum step, bit for bit, through the tile kernel that walks the tensors' segments."""
+    plan = api.Plan(sizes, density, mode=api.GC_THRESHOLD, device=0, cap_factor=1.5)
+    ws = plan.alloc_workspace()
+    n = plan.total_n
+    pairs, d_idx, d_val, d_cnt = lists_with_counts(plan, sizes, W, seed=90 + W, fill=fill)
+    launches0 = plan.launches()
+    out = torch.full((n,), 2.0, device="cuda")
+    for zero_first in (True, False):
+        before = out.cpu().numpy().copy()
+        plan.decompress_accumulate(d_idx, d_val, d_cnt, out, zero_first, ws)
+        want = oracle.decode_accumulate(pairs, before, zero_first)
+        assert np.array_equal(to_np_u32(out), bits(want)), (W, zero_first)
+    assert plan.launches() - launches0 == 2            # one tile kernel per call, no per-worker launches
+    gen = torch.Generator().manual_seed(3)
+    p = torch.randn(n, generator=gen); v = torch.randn(n, generator=gen) * 0.1
+    d_p, d_v = p.cuda(), v.cuda()
+    h_p, h_v = p.numpy().copy(), v.numpy().copy()
+    plan.decompress_apply_momentum(d_idx, d_val, d_cnt, d_p, d_v, 0.05, 0.9, 1.0 / W, ws)
+    oracle.decode_apply_momentum(pairs, h_p, h_v, 0.05, 0.9, 1.0 / W)
+    assert np.array_equal(to_np_u32(d_v), bits(h_v)) and np.array_equal(to_np_u32(d_p), bits(h_p))
+    st, det = plan.last_status(ws)
+    assert st == api.GC_OK, (st, det)
+
+
+def test_many_tensor_lists_with_counts_report_an_index_outside_its_tensor():
+    """A live pair whose index lies beyond its tensor's last element is skipped and reported."""
+    sizes = [10_000, 10_000]
+    plan = api.Plan(sizes, 0.001, mode=api.GC_THRESHOLD, device=0)       # cap 20 per tensor
+    caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
+    ws = plan.alloc_workspace()
+    idx = torch.zeros(plan.total_cap, dtype=torch.int32, device="cuda")
+    val = torch.ones(plan.total_cap, device="cuda")
+    idx[offs[0]:offs[0] + 3] = torch.tensor([5, 9_000, 10_500], dtype=torch.int32)    # the third belongs to tensor 1
+    idx[offs[1]:offs[1] + 2] = torch.tensor([12_000, 19_999], dtype=torch.int32)
+    cnt = torch.tensor([3, 2, 3, 2], dtype=torch.int32, device="cuda")
+    out = torch.empty(plan.total_n, device="cuda")
+    plan.decompress_accumulate([idx], [val], [cnt], out, True, ws)
+    st, _ = plan.last_status(ws)
+    assert st == api.GC_E_INVALID
+    assert out.sum().item() == 4.0 and out[10_500].item() == 0.0
+
+
 @pytest.mark.parametrize("W", [0, 1, 3, 16])
 @pytest.mark.parametrize("sizes,density", [([100_003], 0.01), ([5, 3, 1000, 7, 8193, 64, 70001], 0.02)])
 @pytest.mark.parametrize("route", list(ROUTES))

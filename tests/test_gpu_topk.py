@@ -198,6 +198,103 @@ def test_every_route_gives_the_same_bits(path, sizes):
         assert all(c[1] == 1 for c in seen), seen
 
 
+def run_workers_call(sizes, density, W, steps, seed, options=None, grads_fn=None, with_counts=True):
+    """`steps` calls of gc_compress_workers for W workers; every worker's pairs, counts and residual
+    against the oracle after every step.  Returns plan, workers and the oracle's last pairs."""
+    plan = api.Plan(sizes, density, device=0)
+    for opt, value in (options or {}).items():
+        plan.set_option(opt, value)
+    ks, n, T = plan.tensor_k(), plan.total_n, len(sizes)
+    workers = [GpuWorker(plan) for _ in range(W)]
+    r_cpu = [np.zeros(n, np.float32) for _ in range(W)]
+    pairs = None
+    for step in range(steps):
+        if grads_fn is not None:
+            grads = [grads_fn(w, step) for w in range(W)]
+        else:
+            grads = [randn(n, seed + 100 * w + step, scale=10.0 ** (w % 3 - 1)).cuda() for w in range(W)]
+        for wk in workers:
+            wk.idx.fill_(-1); wk.val.fill_(float("nan")); wk.count.fill_(-1)
+        plan.compress_workers(grads, [wk.residual for wk in workers], [wk.idx for wk in workers],
+                              [wk.val for wk in workers], [wk.count for wk in workers] if with_counts else None,
+                              [wk.ws for wk in workers])
+        pairs = []
+        for w, wk in enumerate(workers):
+            wk.check_status()
+            oi, ov = oracle.topk_compress_tensors(list(sizes), ks, grads[w].cpu().numpy(), r_cpu[w])
+            tot = sum(ks)
+            assert np.array_equal(to_np_u32(wk.idx[:tot]), oi), (step, w)
+            assert np.array_equal(to_np_u32(wk.val[:tot]), bits(ov)), (step, w)
+            assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r_cpu[w])), (step, w)
+            if with_counts:
+                cnt = wk.count.cpu().numpy()
+                assert cnt[:T].tolist() == ks and cnt[T:2 * T].tolist() == ks, (step, w)
+            pairs.append((oi, ov))
+    return plan, workers, pairs
+
+
+@pytest.mark.parametrize("W", [1, 2, 3, 8, 13, 27])
+def test_workers_call_many_tensors_matches_the_oracle(W):
+    """gc_compress_workers on a plan of several tensors (ragged sizes, misaligned starts, an empty
+    tensor, single-tile tensors): the workers share cooperative launches -- from two to twelve per
+    launch, a lone leftover worker on its own -- and each must come out exactly as a call of its own."""
+    sizes = [300_000, 5, 1_500_001, 131_072, 64, 0, 131_071, 2_000_003, 4097, 1000]
+    plan, workers, _ = run_workers_call(sizes, 0.003, W, steps=3, seed=4000 + W)
+    seen = [plan.last_counters(wk.ws) for wk in workers]
+    assert all(c[1] == 0 and c[2] == 0 for c in seen), seen
+
+
+@pytest.mark.parametrize("options", [{api.GC_OPT_SAMPLE_RANK_PERMILLE: 30}, {api.GC_OPT_CANDIDATE_CAPACITY: 100},
+                                     {api.GC_OPT_PATH: api.GC_PATH_EXACT}, {api.GC_OPT_PATH: api.GC_PATH_STAGED}],
+                         ids=["starved", "overflow", "exact", "staged"])
+def test_workers_call_safety_net_and_other_routes(options):
+    """The redo routes inside the shared launch (brackets that miss, candidate regions that
+    overflow) run per group of CTAs; plans on the other routes take one call per worker."""
+    sizes = [300_000, 5, 1_500_001, 131_072, 64, 131_071, 2_000_003]
+    plan, workers, _ = run_workers_call(sizes, 0.01, 4, steps=2, seed=4100, options=options)
+    seen = [plan.last_counters(wk.ws) for wk in workers]
+    if api.GC_OPT_SAMPLE_RANK_PERMILLE in options:
+        assert all(c[2] >= 1 for c in seen), seen
+    if api.GC_OPT_CANDIDATE_CAPACITY in options:
+        assert all(c[1] == 1 for c in seen), seen
+
+
+def test_workers_call_one_tensor_plan_and_ties():
+    """One-tensor plans are served worker by worker; quantised values put thousands of ties at the
+    thresholds of a many-tensor plan."""
+    run_workers_call([3_000_001], 0.01, 3, steps=2, seed=4200, with_counts=False)
+    n = 300_000
+    run_workers_call([n, n, n], 0.01, 5, steps=2, seed=0,
+                     grads_fn=lambda w, s: synth.quantised_gradient(3 * n, 40 + 7 * w + s).cuda())
+
+
+def test_workers_call_rejects_shared_buffers():
+    plan = api.Plan([100_000, 50_000], 0.01, device=0)
+    a, b = GpuWorker(plan), GpuWorker(plan)
+    g = torch.zeros(plan.total_n, device="cuda")
+    with pytest.raises(api.GcError) as e:
+        plan.compress_workers([g, g], [a.residual, b.residual], [a.idx, b.idx], [a.val, b.val], None, [a.ws, a.ws])
+    assert e.value.code == api.GC_E_INVALID
+    with pytest.raises(api.GcError):
+        plan.compress_workers([g, g], [a.residual, a.residual], [a.idx, b.idx], [a.val, b.val], None, [a.ws, b.ws])
+    plan.compress_workers([], [], [], [], None, [])            # no workers: nothing happens
+    torch.cuda.synchronize()
+
+
+def test_config4_eight_resnet_workers_in_one_call_then_decode():
+    """The 8-worker ResNet-50 workload as one gc_compress_workers call per step (two steps, so the
+    error feedback of every worker is exercised), then the decode of the 8 lists."""
+    w = synth.workload(3)
+    assert w.workers == 8
+    plan, workers, pairs = run_workers_call(w.sizes, w.density, w.workers, steps=2, seed=0,
+                                            grads_fn=lambda wk, s: synth.gradient(w, wk, s, device="cuda"))
+    n = plan.total_n
+    out = torch.empty(n, device="cuda")
+    plan.decompress_accumulate([x.idx for x in workers], [x.val for x in workers], None, out, True, workers[0].ws)
+    want = oracle.decode_accumulate(pairs, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(out), bits(want))
+
+
 def test_candidate_path_needs_no_redo_in_error_feedback_steady_state():
     """Re-using a few gradients makes unsent entries pile up just below the threshold (a cliff in
     the magnitude distribution).  The sampled threshold is an exact order statistic, so the
