@@ -506,6 +506,10 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others):
     alg_bytes = {"fold_hist": 12.0 * n, "hist_refine": 4.0 * n, "compact": 4.0 * n + 8.0 * k,
                  "decode_clear": 4.0 * n, "decode_add": 8.0 * k, "fold_cand": 12.0 * n, "compress_fused": 12.0 * n + 8.0 * k,
                  "threshold_emit": 12.0 * n + 4.0 * k, "decode_tiles": 4.0 * n + 8.0 * k * W}
+    # a compress launch may serve several workers (gc_compress_workers): its bytes are theirs together
+    fused_per_step = per_kernel.get("compress_fused", (0.0, 0))[1] / args.steps
+    workers_per_launch = W / fused_per_step if fused_per_step else 1.0
+    alg_bytes["compress_fused"] *= workers_per_launch
     dom_ms = breakdown[dom]["ms_per_launch"]
     achieved = alg_bytes.get(dom, 12.0 * n) / (dom_ms * 1e-3) / 1e9
     # DRAM bytes of one launch of the dominant kernel as ncu measured them (read from the summary)
@@ -541,7 +545,8 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others):
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic, "peak_source": peak_src,
                      "traffic_source": ncu_src,
-                     "algorithmic_bytes_per_launch": alg_bytes.get(dom)},
+                     "algorithmic_bytes_per_launch": alg_bytes.get(dom),
+                     "workers_per_launch": workers_per_launch if dom == "compress_fused" else None},
         "cpu_baseline": cpu,
         "e2e": None if not e2e_steps else {"value": grad_bytes_step * e2e_steps / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": 4 * n * W, "d2h_bytes_per_step": 8 * k * W,

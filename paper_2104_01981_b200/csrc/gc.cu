@@ -67,7 +67,7 @@ struct gc_plan_s {
     uint32_t thrm_grid = 0, thrm_per = 0, thrm_pool = 0, thrm_ntab = 0;   // many-tensor threshold kernel (0 = no)
     size_t thrm_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
-    size_t multi_smem_max = 0;              // dynamic shared memory that occupancy figure was taken with
+    size_t multi_smem_max = 0, thrm_smem_max = 0;   // dynamic shared memory those occupancy figures were taken with
     uint32_t wk_W = 0, wk_batch = 0;        // gc_compress_workers: workers per launch chosen for the last W seen
     MultiGeom wk_geom;
     uint32_t multi_ntab = 0;
@@ -355,16 +355,16 @@ void plan_thr_single(gc_plan_s* p) {
     p->thr_smem = (size_t)maxt * (2 * kWarps + 2) * sizeof(uint32_t);
 }
 
-// Decides whether a threshold plan can use the many-tensor kernel and with which geometry.
-void plan_thr_multi(gc_plan_s* p) {
-    p->thrm_grid = 0;
-    if (p->mode != GC_THRESHOLD || p->T < 2 || p->grid_thr_multi_max <= 0 || p->ntiles == 0) return;
-    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_thr_multi_max, p->ntiles);
+// Geometry of the many-tensor threshold kernel when G CTAs share one worker's tiles (G = 0: no).
+MultiGeom thr_multi_geometry(const gc_plan_s* p, uint32_t G) {
+    MultiGeom mg;
+    if (p->mode != GC_THRESHOLD || p->T < 2 || G == 0 || p->ntiles == 0) return mg;
+    G = std::min<uint32_t>(G, p->ntiles);
     const uint32_t per = (p->ntiles + G - 1) / G;
-    if (per > kMultiMaxPer) return;
+    if (per > kMultiMaxPer) return mg;
     // one CTA ranks a whole tensor's kept sample keys: keep that bounded
     for (uint32_t t : p->reg_ids)
-        if (p->desc[t].nstiles > 128 || p->desc[t].sstride == 0) return;
+        if (p->desc[t].nstiles > 128 || p->desc[t].sstride == 0) return mg;
     const uint32_t pool = std::min<uint32_t>(p->cand_cap_alloc / G, kSinglePoolMax);
     // expected hits of the busiest CTA: about k per tensor, spread over its tiles
     double worst = 0.0;
@@ -378,10 +378,20 @@ void plan_thr_multi(gc_plan_s* p) {
         }
         worst = std::max(worst, e);
     }
-    if ((double)pool < 2.0 * worst + 512.0) return;
-    p->thrm_grid = G; p->thrm_per = per; p->thrm_pool = pool;
-    p->thrm_ntab = p->T <= kMultiMaxTab ? p->T : 0u;
-    p->thrm_smem = (size_t)per * kMultiRowBytes + 2 * sizeof(uint32_t) * (size_t)p->thrm_ntab;
+    if ((double)pool < 2.0 * worst + 512.0) return mg;
+    mg.G = G; mg.per = per; mg.pool = pool; mg.full = G;
+    mg.ntab = p->T <= kMultiMaxTab ? p->T : 0u;
+    mg.smem = (size_t)per * kMultiRowBytes + 2 * sizeof(uint32_t) * (size_t)mg.ntab;
+    return mg;
+}
+
+// Decides whether a threshold plan can use the many-tensor kernel and with which geometry.
+void plan_thr_multi(gc_plan_s* p) {
+    p->thrm_grid = 0;
+    if (p->grid_thr_multi_max <= 0) return;
+    const MultiGeom mg = thr_multi_geometry(p, (uint32_t)p->grid_thr_multi_max);
+    if (mg.G == 0) return;
+    p->thrm_grid = mg.G; p->thrm_per = mg.per; p->thrm_pool = mg.pool; p->thrm_ntab = mg.ntab; p->thrm_smem = mg.smem;
 }
 
 // Geometry of the many-tensor kernel when G CTAs share one worker's tiles: MultiGeom.
@@ -642,10 +652,13 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
         p->grid_thr_multi_max = 0;
         if (coop) {
             int nb = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_threshold_multi, kBlock,
-                                                              kMultiMaxPer * kMultiRowBytes + 8 * kMultiMaxTab) ==
-                    cudaSuccess && nb >= 1)
-                p->grid_thr_multi_max = p->sm_count * nb;
+            p->thrm_smem_max = kMultiMaxPer * kMultiRowBytes + 8 * kMultiMaxTab;
+            int nbw = 0;          // (the several-workers form of the kernel must be as resident as the kernel itself)
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_threshold_multi, kBlock, p->thrm_smem_max) ==
+                    cudaSuccess && nb >= 1 &&
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nbw, k_threshold_workers, kBlock, p->thrm_smem_max) ==
+                    cudaSuccess && nbw >= 1)
+                p->grid_thr_multi_max = p->sm_count * std::min(nb, nbw);
             else
                 (void)cudaGetLastError();
         }
@@ -798,6 +811,25 @@ static MultiArgs multi_args(const gc_plan_s* p, const MultiGeom& mg, const void*
     return ma;
 }
 
+// Argument block of the many-tensor threshold kernel for one worker's buffers and a given geometry.
+static ThrMultiArgs thr_multi_args(const gc_plan_s* p, const MultiGeom& mg, const float* grad, float* residual,
+                                   uint32_t* out_idx, float* out_val, uint32_t* out_count, void* workspace) {
+    char* wb = static_cast<char*>(workspace);
+    ThrMultiArgs ta;
+    ta.desc = p->d_desc; ta.T = p->T; ta.ntiles = p->ntiles; ta.nstiles = p->nstiles;
+    ta.per = mg.per; ta.pool_cap = mg.pool; ta.ntab = mg.ntab;
+    ta.small_ids = p->d_small; ta.n_small = (uint32_t)p->small_ids.size();
+    ta.reg_ids = p->d_small + p->T; ta.n_reg = (uint32_t)p->reg_ids.size();
+    ta.g = grad; ta.r = residual; ta.out_idx = out_idx; ta.out_val = out_val; ta.out_count = out_count;
+    ta.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
+    ta.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
+    ta.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
+    ta.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
+    ta.tsel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
+    ta.ws = view(p, workspace);
+    return ta;
+}
+
 static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* residual, uint32_t* out_idx,
                          float* out_val, uint32_t* out_count, void* workspace, void* stream) {
     const float* grad = static_cast<const float*>(grad_any);       // only dereferenced as such when !bf16
@@ -854,18 +886,9 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     }
     if (p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thrm_grid > 0) {
         // several tensors: sample, exact thresholds, fold + hits and emission in one cooperative launch
-        ThrMultiArgs ta;
-        ta.desc = p->d_desc; ta.T = p->T; ta.ntiles = nt; ta.nstiles = p->nstiles;
-        ta.per = p->thrm_per; ta.pool_cap = p->thrm_pool; ta.ntab = p->thrm_ntab;
-        ta.small_ids = p->d_small; ta.n_small = (uint32_t)p->small_ids.size();
-        ta.reg_ids = p->d_small + p->T; ta.n_reg = (uint32_t)p->reg_ids.size();
-        ta.g = grad; ta.r = residual; ta.out_idx = out_idx; ta.out_val = out_val; ta.out_count = out_count;
-        ta.cand = reinterpret_cast<uint2*>(wb + p->off_cidx);
-        ta.shist = reinterpret_cast<uint32_t*>(wb + p->off_shist);
-        ta.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
-        ta.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
-        ta.tsel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
-        ta.ws = ws;
+        MultiGeom mg;
+        mg.G = p->thrm_grid; mg.per = p->thrm_per; mg.pool = p->thrm_pool; mg.ntab = p->thrm_ntab; mg.smem = p->thrm_smem;
+        ThrMultiArgs ta = thr_multi_args(p, mg, grad, residual, out_idx, out_val, out_count, workspace);
         void* args[] = {&ta};
         Timed tm(p, s, GC_K_FUSED);
         GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_threshold_multi, dim3(p->thrm_grid), dim3(kBlock),
@@ -1052,12 +1075,17 @@ int gc_compress_workers(gc_plan_t* p, uint32_t W, const float* const* grads, flo
     // share must still satisfy the kernel's limits (tiles and candidates per CTA)
     uint32_t batch = 0;
     MultiGeom mg;
-    if (p->mode == GC_TOPK && p->path == GC_PATH_AUTO && p->multi_grid > 0 && W >= 2) {
+    const bool topk_multi = p->mode == GC_TOPK && p->path == GC_PATH_AUTO && p->multi_grid > 0;
+    const bool thr_multi = p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thrm_grid > 0;
+    if ((topk_multi || thr_multi) && W >= 2) {
         if (p->wk_W != W) {                      // (kept for the next call; options that change the layout reset it)
             p->wk_W = W; p->wk_batch = 0;
             for (uint32_t wb = std::min<uint32_t>(W, kWorkersPerLaunch); wb >= 2 && p->wk_batch == 0; --wb) {
-                const MultiGeom g2 = multi_geometry(p, (uint32_t)p->grid_multi_max / wb, false);
-                if (g2.G > 0 && g2.smem <= p->multi_smem_max) { p->wk_batch = wb; p->wk_geom = g2; }
+                const MultiGeom g2 = topk_multi ? multi_geometry(p, (uint32_t)p->grid_multi_max / wb, false)
+                                                : thr_multi_geometry(p, (uint32_t)p->grid_thr_multi_max / wb);
+                if (g2.G > 0 && g2.smem <= (topk_multi ? p->multi_smem_max : p->thrm_smem_max)) {
+                    p->wk_batch = wb; p->wk_geom = g2;
+                }
             }
         }
         batch = p->wk_batch; mg = p->wk_geom;
@@ -1080,28 +1108,33 @@ int gc_compress_workers(gc_plan_t* p, uint32_t W, const float* const* grads, flo
         }
         ClearMany cm;
         WorkersArgs wa;
-        wa.W = wn; wa.G = mg.G;
+        ThrWorkersArgs ta;
+        wa.W = ta.W = wn; wa.G = ta.G = mg.G;
         for (uint32_t i = 0; i < wn; ++i) {
             const uint32_t w = w0 + i;
             cm.p[i] = reinterpret_cast<uint4*>(workspaces[w]);
-            wa.per[i] = multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w],
-                                   out_count ? out_count[w] : nullptr, workspaces[w]);
-            if (out_count != nullptr && p->n_empty > 0) {
+            uint32_t* const oc = out_count ? out_count[w] : nullptr;
+            if (topk_multi) wa.per[i] = multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w]);
+            else ta.per[i] = thr_multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w]);
+            if (oc != nullptr && p->n_empty > 0) {
                 Timed tm(p, s, GC_K_CLEAR_CTRL);
-                GC_CUDA(p, cudaMemsetAsync(out_count[w], 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
+                GC_CUDA(p, cudaMemsetAsync(oc, 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
             }
         }
-        for (uint32_t i = wn; i < kWorkersPerLaunch; ++i) { cm.p[i] = nullptr; wa.per[i] = wa.per[0]; }
+        for (uint32_t i = wn; i < kWorkersPerLaunch; ++i) {
+            cm.p[i] = nullptr;
+            if (topk_multi) wa.per[i] = wa.per[0]; else ta.per[i] = ta.per[0];
+        }
         {
             Timed tm(p, s, GC_K_CLEAR_CTRL);
             const size_t n16 = p->control_bytes / 16;
             const unsigned gx = (unsigned)std::min<size_t>((n16 + kBlock - 1) / kBlock, (size_t)p->sm_count * 8 / wn + 1);
             k_clear_many<<<dim3(gx, wn), kBlock, 0, s>>>(cm, n16);
         }
-        void* args[] = {&wa};
+        void* args[] = {topk_multi ? (void*)&wa : (void*)&ta};
         Timed tm(p, s, GC_K_FUSED);
-        GC_CUDA(p, cudaLaunchCooperativeKernel((const void*)k_topk_workers<GradF32>, dim3(mg.G * wn), dim3(kBlock),
-                                               args, mg.smem, s));
+        GC_CUDA(p, cudaLaunchCooperativeKernel(topk_multi ? (const void*)k_topk_workers<GradF32> : (const void*)k_threshold_workers,
+                                               dim3(mg.G * wn), dim3(kBlock), args, mg.smem, s));
     }
     return GC_OK;
 }

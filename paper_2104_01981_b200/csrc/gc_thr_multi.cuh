@@ -132,21 +132,19 @@ static __device__ __noinline__ void small_threshold_body(BlockSmem& sm, const Te
     __syncthreads();
 }
 
-// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
-static __global__ void __launch_bounds__(kBlock, 3)
-k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
-    __shared__ BlockSmem sm;
-    __shared__ uint32_t s_used, s_cnt;
-    extern __shared__ __align__(16) unsigned char s_dyn[];
+// The whole threshold compress of one worker by the G CTAs of one group (this CTA is number b of
+// them); the group's barriers count on the worker's own workspace header.
+static __device__ __forceinline__ void threshold_multi_body(const ThrMultiArgs& a, const uint32_t G, const uint32_t b,
+                                                            BlockSmem& sm, uint32_t& s_used, uint32_t& s_cnt,
+                                                            unsigned char* s_dyn) {
     uint32_t* const rec = reinterpret_cast<uint32_t*>(s_dyn);                  // [per*kWarps] off<<10 | cnt
     uint32_t* const rec2 = rec + (size_t)a.per * kWarps;                       // [per*kWarps] first slot of the chunk
     uint32_t* const seg = rec2 + (size_t)a.per * kWarps;                       // [per][kSegWords]
     uint32_t* const tab_tile0 = seg + (size_t)a.per * kSegWords;               // [ntab] first tile of every tensor
     uint32_t* const tab_stile0 = tab_tile0 + a.ntab;                           // [ntab] first sample tile
-    uint2* const pool = a.cand + (size_t)blockIdx.x * a.pool_cap;
+    uint2* const pool = a.cand + (size_t)b * a.pool_cap;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t G = gridDim.x, b = blockIdx.x;
     WsHeader* hdr = a.ws.hdr;
     uint32_t passed = 0, n_stamp = 0;
     const uint32_t first = min(a.ntiles, b * a.per), last = min(a.ntiles, first + a.per);
@@ -158,7 +156,7 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
         tab_tile0[t] = a.desc[t].tile0;
         tab_stile0[t] = a.desc[t].stile0;
     }
-    phase_stamp(hdr, n_stamp);
+    phase_stamp(hdr, n_stamp, b);
     __syncthreads();
     auto owner = [&](const uint32_t* tab, uint32_t tile) -> uint32_t {    // last t with tab[t] <= tile
         uint32_t lo = 0, hi = a.ntab;
@@ -217,8 +215,8 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
     }
     __syncthreads();
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
-    if (!grid_wait(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_wait(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     // ---------------------------------------------------------------- exact tau, one CTA per tensor
     for (uint32_t q = b; q < a.n_reg; q += G) {
@@ -258,8 +256,8 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
         if (ok) tau = prefix;
         if (tid == 0) a.tsel[t].T = tau;                  // ~0: nothing is a hit (cannot happen for a valid plan)
     }
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     // ---------------------------------------------------------------- fold + hits, segment by segment
     uint32_t nseg = 0;
@@ -394,8 +392,8 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
         for (int w = 0; w < kWarps; ++w) tot += rec[i * kWarps + w] & 1023u;
         a.tile_cnt[first + i] = tot;
     }
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
 
     if (ld_cg(&hdr->overflow) == 0u) {
         // ------------------------------------------------------------ slots and emission
@@ -468,7 +466,7 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
             }
         }
         __syncthreads();
-        phase_stamp(hdr, n_stamp);
+        phase_stamp(hdr, n_stamp, b);
         exit_stamp(hdr);
         return;
     }
@@ -481,10 +479,43 @@ k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
             a.r[pr.x] = __uint_as_float(pr.y);
         }
     }
-    if (!grid_barrier(hdr, passed, &sm.ok)) return;
-    phase_stamp(hdr, n_stamp);
+    if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
+    phase_stamp(hdr, n_stamp, b);
     threshold_emit_body<false, true>(a.desc, a.T, a.ntiles, nullptr, a.r, a.out_idx, a.out_val, a.out_count, a.ws,
                                      a.tsel, 0u, 0);
+}
+
+// (three CTAs per SM: 80 registers and no spills beat four at 64 registers, see k_topk_single)
+static __global__ void __launch_bounds__(kBlock, 3)
+k_threshold_multi(const __grid_constant__ ThrMultiArgs a) {
+    __shared__ BlockSmem sm;
+    __shared__ uint32_t s_used, s_cnt;
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    threshold_multi_body(a, gridDim.x, blockIdx.x, sm, s_used, s_cnt, s_dyn);
+}
+
+// Several workers' threshold compress calls in one cooperative launch, one group of CTAs per
+// worker (see k_topk_workers).
+struct ThrWorkersArgs {
+    uint32_t W, G;                               // workers in this launch, CTAs per worker
+    ThrMultiArgs per[kWorkersPerLaunch];
+};
+static_assert(sizeof(ThrWorkersArgs) <= 4000, "kernel parameters stay below 4 KB");
+
+static __global__ void __launch_bounds__(kBlock, 3)
+k_threshold_workers(const __grid_constant__ ThrWorkersArgs wa) {
+    __shared__ BlockSmem sm;
+    __shared__ uint32_t s_used, s_cnt;
+    __shared__ ThrMultiArgs s_args;               // this CTA's worker
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    const uint32_t w = blockIdx.x % wa.W, b = blockIdx.x / wa.W;
+    {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(&wa.per[w]);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&s_args);
+        for (uint32_t i = threadIdx.x; i < sizeof(ThrMultiArgs) / 4; i += kBlock) dst[i] = src[i];
+    }
+    __syncthreads();
+    threshold_multi_body(s_args, wa.G, b, sm, s_used, s_cnt, s_dyn);
 }
 
 }  // namespace gc

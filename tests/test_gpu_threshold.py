@@ -116,6 +116,55 @@ def test_threshold_config4_resnet_workers_and_decode():
     assert np.array_equal(to_np_u32(out), bits(want))
 
 
+def check_threshold_workers(sizes, density, W, grads_fn, steps=2, cap_factor=0.0):
+    """`steps` gc_compress_workers calls of a threshold plan for W workers; every worker's pairs,
+    counts, residual and status against the oracle after every step."""
+    plan = api.Plan(sizes, density, mode=api.GC_THRESHOLD, device=0, cap_factor=cap_factor)
+    T, n = len(sizes), plan.total_n
+    caps, offs = plan.tensor_cap(), plan.tensor_out_offset()
+    strides = [plan.query(api.GC_Q_TENSOR_STRIDE, t) for t in range(T)]
+    workers = [GpuWorker(plan) for _ in range(W)]
+    r_cpu = [np.zeros(n, np.float32) for _ in range(W)]
+    for step in range(steps):
+        grads = [grads_fn(w, step) for w in range(W)]
+        for wk in workers:
+            wk.idx.fill_(-1); wk.val.fill_(float("nan")); wk.count.fill_(-1)
+        plan.compress_workers([g.cuda() for g in grads], [wk.residual for wk in workers], [wk.idx for wk in workers],
+                              [wk.val for wk in workers], [wk.count for wk in workers], [wk.ws for wk in workers])
+        for w, wk in enumerate(workers):
+            st, det = plan.last_status(wk.ws)
+            g_cpu = grads[w].cpu().numpy()
+            cnt, gi, gv = wk.count.cpu().numpy(), to_np_u32(wk.idx), to_np_u32(wk.val)
+            off, truncated = 0, False
+            for t, sz in enumerate(sizes):
+                oi, ov, hits, _ = oracle.threshold_compress(g_cpu[off:off + sz], r_cpu[w][off:off + sz], density,
+                                                            strides[t], caps[t], index_base=off)
+                assert cnt[t] == oi.size and cnt[T + t] == hits, (step, w, t)
+                assert np.array_equal(gi[offs[t]:offs[t] + oi.size], oi), (step, w, t)
+                assert same_f32_bits(gv[offs[t]:offs[t] + oi.size], bits(ov)), (step, w, t)
+                truncated |= hits > caps[t]
+                off += sz
+            assert same_f32_bits(to_np_u32(wk.residual[:n]), bits(r_cpu[w])), (step, w)
+            assert st == (api.GC_W_TRUNCATED if truncated else api.GC_OK), (st, det)
+    return plan, workers
+
+
+@pytest.mark.parametrize("W", [2, 5, 8, 13])
+def test_threshold_workers_call_matches_the_oracle(W):
+    """gc_compress_workers in threshold mode on a plan of several tensors: the workers share
+    cooperative launches (groups of CTAs), each exactly as a call of its own; a tight capacity
+    factor makes some workers truncate."""
+    sizes = [300_000, 5, 1_500_001, 131_072, 64, 0, 131_071, 700_003, 4097, 1000]
+    n = sum(sizes)
+    check_threshold_workers(sizes, 0.004, W, lambda w, s: randn(n, 9000 + 50 * w + s, 10.0 ** (w % 3 - 1)),
+                            steps=2, cap_factor=1.0)
+
+
+def test_threshold_workers_call_on_the_resnet_workload():
+    w = synth.workload(3)
+    check_threshold_workers(w.sizes, w.density, w.workers, lambda wk, s: synth.gradient(w, wk, s, device="cuda"), steps=2)
+
+
 @pytest.mark.parametrize("config_id", [2, 4], ids=["bert_110m", "gpt2_medium_355m"])
 def test_threshold_full_size_one_tensor_workloads(config_id):
     """One full-size step of the threshold variant on the 110M- and the 355M-element workload (the
