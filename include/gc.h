@@ -76,6 +76,21 @@ typedef struct gc_plan_s gc_plan_t;
 #define GC_Q_MODE              10
 #define GC_Q_KERNEL_LAUNCHES   11   /* kernels + memsets enqueued by the library so far (host count) */
 #define GC_Q_CANDIDATE_CAPACITY 12  /* slots of the internal candidate list (top-k mode)            */
+#define GC_Q_COMPRESS_ROUTE     13  /* which kernels gc_compress takes for this plan: GC_ROUTE_*    */
+
+/* values of GC_Q_COMPRESS_ROUTE (a diagnostic: the result never depends on the route) */
+#define GC_ROUTE_NONE             0 /* nothing to launch (host-only plan, or no elements)                      */
+#define GC_ROUTE_TOPK_ONE         1 /* one cooperative launch, one-tensor kernel                               */
+#define GC_ROUTE_TOPK_MANY        2 /* one cooperative launch, many-tensor kernel                              */
+#define GC_ROUTE_TOPK_GENERAL     3 /* one cooperative launch, general candidate kernel (global histograms per
+                                       level): plans the two kernels above do not take -- candidate sets too
+                                       large for a CTA's region (densities of several per cent on large
+                                       tensors), tensors beyond their tile limits, unsampled tensors          */
+#define GC_ROUTE_TOPK_STAGED      4 /* the general candidate path as separate launches                         */
+#define GC_ROUTE_EXACT            5 /* exact multi-pass kernels only                                           */
+#define GC_ROUTE_THRESHOLD_ONE    6 /* threshold mode, one cooperative launch, one-tensor kernel               */
+#define GC_ROUTE_THRESHOLD_MANY   7 /* threshold mode, one cooperative launch, many-tensor kernel              */
+#define GC_ROUTE_THRESHOLD_STAGED 8 /* threshold mode, sample levels and the emission as separate launches     */
 
 /*
  * gc_plan -- describe the flat gradient once; computes k per tensor, output offsets and the

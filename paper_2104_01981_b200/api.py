@@ -23,7 +23,9 @@ GC_MAX_WORKERS = 64
 GC_K_COUNT = 16
 (GC_Q_N_TENSORS, GC_Q_TOTAL_N, GC_Q_TOTAL_CAP, GC_Q_WORKSPACE_BYTES, GC_Q_TENSOR_N, GC_Q_TENSOR_K,
  GC_Q_TENSOR_CAP, GC_Q_TENSOR_OFFSET, GC_Q_TENSOR_OUT_OFFSET, GC_Q_TENSOR_STRIDE, GC_Q_MODE,
- GC_Q_KERNEL_LAUNCHES, GC_Q_CANDIDATE_CAPACITY) = range(13)
+ GC_Q_KERNEL_LAUNCHES, GC_Q_CANDIDATE_CAPACITY, GC_Q_COMPRESS_ROUTE) = range(14)
+(GC_ROUTE_NONE, GC_ROUTE_TOPK_ONE, GC_ROUTE_TOPK_MANY, GC_ROUTE_TOPK_GENERAL, GC_ROUTE_TOPK_STAGED, GC_ROUTE_EXACT,
+ GC_ROUTE_THRESHOLD_ONE, GC_ROUTE_THRESHOLD_MANY, GC_ROUTE_THRESHOLD_STAGED) = range(9)
 GC_OPT_PATH, GC_OPT_SAMPLE_RANK_PERMILLE, GC_OPT_CANDIDATE_CAPACITY, GC_OPT_DECODE_ROUTE = 0, 1, 2, 3
 GC_DECODE_AUTO, GC_DECODE_NARROW, GC_DECODE_WIDE = 0, 1, 2
 GC_OPT_DECODE_ORDER = 4

@@ -48,6 +48,7 @@ struct gc_plan_s {
            control_bytes = 0, off_tinfo = 0, off_cidx = 0, ws_bytes = 0;
     int sm_count = 0;
     int grid_thr = 0, grid_decode[2] = {0, 0};
+    int grid_decode8 = 0, grid_decode8_apply = 0;      // k_decode_tiles with eight pre-loaded entries per thread (one tile buffer)
     int grid_decode_seg[2] = {0, 0}, grid_decode_seg_apply = 0;    // k_decode_segments: one / two tile buffers; with optimizer
     bool wide_ok = false;                         // k_decode_wide may use up to 64 KB of dynamic shared memory
     std::vector<std::pair<size_t, int>> wide_occ[2];      // (shared-memory bytes -> CTAs per SM), plain / with optimizer
@@ -494,20 +495,30 @@ struct DecodeRoute {
     uint32_t win = 0;
     size_t smem = 0;
     int grid = 0;
+    int rounds = kDecRounds;    // (narrow) entries a thread pre-loads per tile: kDecRounds or twice that
 };
 template <bool APPLY>
-static DecodeRoute decode_route(gc_plan_t* p, uint32_t W) {
+static DecodeRoute decode_route(gc_plan_t* p, uint32_t W, bool zero_first) {
     DecodeRoute r;
-    if (!p->wide_ok || W == 0 || p->total_n == 0) return r;
+    if (W == 0 || p->total_n == 0) return r;
     const uint64_t avg = (p->total_cap * (uint64_t)kDecTile + p->total_n - 1) / p->total_n;     // per worker and tile
     const uint64_t need = avg + avg / 2 + 16;
     uint32_t Wp = 1;
     while (Wp < W && Wp < 64) Wp <<= 1;
-    const uint64_t narrow_window = (uint64_t)kDecRounds * (kDecBlock / Wp);
-    // measured: the narrow kernel wins as long as most tiles fit its window
+    uint64_t narrow_window = (uint64_t)kDecRounds * (kDecBlock / Wp);
     r.any = p->decode_order == GC_ORDER_ANY;
+    // Tiles that start at +0 take the narrow kernel's counted route from a few workers on; there a
+    // window of twice the size (eight pre-loaded entries per thread) still beats the rings, so
+    // lists up to that density stay with the narrow kernel (16 workers at 1 %: measured below).
+    if (!r.any && zero_first && W >= kDecCountedFrom && avg + avg / 4 > narrow_window &&
+        avg + avg / 4 <= 2 * narrow_window && p->grid_decode8 > 0) {
+        r.rounds = 2 * kDecRounds;
+        narrow_window *= 2;
+    }
+    // measured: the narrow kernel wins as long as most tiles fit its window
     r.wide = r.any || (p->decode_route == GC_DECODE_AUTO ? avg + avg / 4 > narrow_window
                                                           : p->decode_route == GC_DECODE_WIDE);
+    if (!p->wide_ok) r.wide = false;
     if (!r.wide) return r;
     uint32_t win = 32;
     while (win < need && win < 1024) win <<= 1;
@@ -533,6 +544,8 @@ static DecodeRoute decode_route(gc_plan_t* p, uint32_t W) {
 }
 
 extern "C" {
+
+static int compress_route(const gc_plan_s* p);
 
 uint32_t gc_version(void) { return 1u; }
 
@@ -680,16 +693,23 @@ int gc_plan(gc_plan_t** out, int device, uint32_t n_tensors, const uint64_t* siz
     }
     p->grid_thr = p->sm_count * blocks_per_sm(k_threshold_emit, kBlock);
     {
-        cudaError_t ed = cudaFuncSetAttribute(k_decode_tiles<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t ed = cudaFuncSetAttribute(k_decode_tiles<false, kDecRounds>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)(2 * kDecTileBytes));
         for (int nbuf = 1; nbuf <= 2; ++nbuf) {
             int nb = 0;
             if (ed == cudaSuccess)
-                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_tiles<false>, kDecBlock,
+                ed = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_decode_tiles<false, kDecRounds>, kDecBlock,
                                                                    nbuf * kDecTileBytes);
             if (ed != cudaSuccess || nb < 1) { (void)cudaGetLastError(); nb = 0; }
             p->grid_decode[nbuf - 1] = p->sm_count * nb;     // 0: fall back to one launch per worker
         }
+        int nb8 = 0, nb8a = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb8, k_decode_tiles<false, 2 * kDecRounds>, kDecBlock,
+                                                          kDecTileBytes) != cudaSuccess || nb8 < 1) { (void)cudaGetLastError(); nb8 = 0; }
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb8a, k_decode_tiles<true, 2 * kDecRounds>, kDecBlock,
+                                                          kDecTileBytes) != cudaSuccess || nb8a < 1) { (void)cudaGetLastError(); nb8a = 0; }
+        p->grid_decode8 = p->sm_count * nb8;
+        p->grid_decode8_apply = p->sm_count * nb8a;
     }
     {
         // lists with per-tensor counts (plans of several tensors): the segment-walking tile kernel
@@ -768,6 +788,7 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
         case GC_Q_MODE: *value = (uint64_t)p->mode; return GC_OK;
         case GC_Q_KERNEL_LAUNCHES: *value = p->launches; return GC_OK;
         case GC_Q_CANDIDATE_CAPACITY: *value = p->cand_cap; return GC_OK;
+        case GC_Q_COMPRESS_ROUTE: *value = (uint64_t)compress_route(p); return GC_OK;
         default: break;
     }
     if (tensor >= p->T) return GC_E_INVALID;
@@ -781,6 +802,22 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
         case GC_Q_TENSOR_STRIDE: *value = d.stride; return GC_OK;
         default: return GC_E_INVALID;
     }
+}
+
+// Which kernels a gc_compress call on this plan takes (GC_ROUTE_*); the dispatch below and
+// GC_Q_COMPRESS_ROUTE both ask here.
+static int compress_route(const gc_plan_s* p) {
+    if (p->device < 0 || p->total_n == 0) return GC_ROUTE_NONE;
+    if (p->mode == GC_THRESHOLD) {
+        if (p->path == GC_PATH_AUTO && p->thr_grid > 0) return GC_ROUTE_THRESHOLD_ONE;
+        if (p->path == GC_PATH_AUTO && p->thrm_grid > 0) return GC_ROUTE_THRESHOLD_MANY;
+        return GC_ROUTE_THRESHOLD_STAGED;
+    }
+    if (p->path == GC_PATH_EXACT) return GC_ROUTE_EXACT;
+    if (p->path == GC_PATH_AUTO && p->single_grid > 0) return GC_ROUTE_TOPK_ONE;
+    if (p->path == GC_PATH_AUTO && p->multi_grid > 0) return GC_ROUTE_TOPK_MANY;
+    if (p->path == GC_PATH_AUTO && p->grid_fused > 0) return GC_ROUTE_TOPK_GENERAL;
+    return GC_ROUTE_TOPK_STAGED;
 }
 
 // Argument block of the many-tensor kernel for one worker's buffers and a given geometry.
@@ -863,7 +900,8 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
     const int gcp = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
     char* wb = static_cast<char*>(workspace);
-    if (p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thr_grid > 0) {
+    const int route = compress_route(p);
+    if (route == GC_ROUTE_THRESHOLD_ONE) {
         // one large tensor: sample, exact threshold, fold + hits and emission in one cooperative launch
         ThrSingleArgs ta;
         ta.d = p->desc[0]; ta.desc = p->d_desc; ta.ntiles = nt; ta.maxt = p->thr_maxt; ta.pool_cap = p->thr_pool;
@@ -884,7 +922,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
                                                args, p->thr_smem, s));
         return GC_OK;
     }
-    if (p->mode == GC_THRESHOLD && p->path == GC_PATH_AUTO && p->thrm_grid > 0) {
+    if (route == GC_ROUTE_THRESHOLD_MANY) {
         // several tensors: sample, exact thresholds, fold + hits and emission in one cooperative launch
         MultiGeom mg;
         mg.G = p->thrm_grid; mg.per = p->thrm_per; mg.pool = p->thrm_pool; mg.ntab = p->thrm_ntab; mg.smem = p->thrm_smem;
@@ -895,7 +933,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
                                                args, p->thrm_smem, s));
         return GC_OK;
     }
-    if (p->mode == GC_THRESHOLD) {
+    if (route == GC_ROUTE_THRESHOLD_STAGED) {
         // exact order statistic of the sample (three radix levels), then one fused pass
         WsView sws = ws;
         sws.sel = reinterpret_cast<TensorSel*>(wb + p->off_ssel);
@@ -913,7 +951,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
-    if (p->path == GC_PATH_EXACT) {
+    if (route == GC_ROUTE_EXACT) {
         // exact multi-pass path on its own: fold + three histogram levels + ordered compaction
         { Timed tm(p, s, GC_K_FOLD_HIST);
           k_hist<0, SRC_FOLD><<<gh, kBlock, 0, s>>>(p->d_desc, p->T, nt, grad, residual, ws); }
@@ -939,7 +977,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     cv.group_cnt = reinterpret_cast<unsigned long long*>(wb + p->off_gstate);
     cv.cap = p->cand_cap;
     cv.ssel = sws.sel;
-    if (p->path == GC_PATH_AUTO && p->single_grid > 0) {
+    if (route == GC_ROUTE_TOPK_ONE) {
         // one large tensor: candidates stay in shared memory
         SingleArgs sa;
         sa.d = p->desc[0]; sa.desc = p->d_desc; sa.ntiles = nt; sa.maxt = p->single_maxt; sa.rows = p->single_rows;
@@ -960,7 +998,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         GC_CUDA(p, cudaLaunchCooperativeKernel(kfn, dim3(p->single_grid), dim3(kBlock), args, p->single_smem, s));
         return GC_OK;
     }
-    if (p->path == GC_PATH_AUTO && p->multi_grid > 0) {
+    if (route == GC_ROUTE_TOPK_MANY) {
         // many tensors: one cooperative launch, four grid barriers
         MultiGeom mg;
         mg.G = p->multi_grid; mg.per = p->multi_per; mg.pool = p->multi_pool; mg.full = p->multi_full;
@@ -972,7 +1010,7 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         GC_CUDA(p, cudaLaunchCooperativeKernel(kfn, dim3(p->multi_grid), dim3(kBlock), args, p->multi_smem, s));
         return GC_OK;
     }
-    if (p->path == GC_PATH_AUTO && p->grid_fused > 0) {
+    if (route == GC_ROUTE_TOPK_GENERAL) {
         // everything in one cooperative launch
         FusedArgs fa;
         fa.desc = p->d_desc; fa.T = p->T; fa.ntiles = nt; fa.nstiles = p->nstiles; fa.ngroups = p->ngroups;
@@ -1171,7 +1209,7 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
         const int grid = (int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode[nbuf - 1]);
         const int use_bulk = (reinterpret_cast<uintptr_t>(dense_out) & 15u) == 0 ? 1 : 0;
         Timed tm(p, s, GC_K_DECODE_TILES);
-        const DecodeRoute rt = decode_route<false>(p, W);
+        const DecodeRoute rt = decode_route<false>(p, W, zero_first != 0);
         if (rt.wide) {
             auto kw = rt.any ? k_decode_any<false> : k_decode_wide<false>;
             kw<<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
@@ -1180,10 +1218,15 @@ int gc_decompress_accumulate(gc_plan_t* p, uint32_t W, const uint32_t* const* id
             GC_CUDA(p, cudaGetLastError());
             return GC_OK;
         }
-        k_decode_tiles<false><<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap,
-                                                                            (uint32_t)p->total_n, dense_out,
-                                                                            zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr,
-                                                                            ApplyArgs{});
+        if (rt.rounds != kDecRounds)
+            k_decode_tiles<false, 2 * kDecRounds><<<(int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode8), kDecBlock,
+                                                    kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n,
+                                                                        dense_out, zero_first ? 1 : 0, use_bulk, 1, ws.hdr,
+                                                                        ApplyArgs{});
+        else
+            k_decode_tiles<false, kDecRounds><<<grid, kDecBlock, nbuf * kDecTileBytes, s>>>(
+                ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, dense_out, zero_first ? 1 : 0, use_bulk, nbuf, ws.hdr,
+                ApplyArgs{});
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
@@ -1260,7 +1303,7 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
-    const DecodeRoute rt = decode_route<true>(p, W);
+    const DecodeRoute rt = decode_route<true>(p, W, true);
     if (rt.wide) {
         auto kw = rt.any ? k_decode_any<true> : k_decode_wide<true>;
         kw<<<(int)std::min<uint32_t>(ntl, (uint32_t)rt.grid), kDecBlock, rt.smem, s>>>(
@@ -1268,8 +1311,13 @@ int gc_decompress_apply_momentum(gc_plan_t* p, uint32_t W, const uint32_t* const
         GC_CUDA(p, cudaGetLastError());
         return GC_OK;
     }
-    k_decode_tiles<true><<<grid, kDecBlock, kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n,
-                                                                nullptr, 1, 0, 1, ws.hdr, ap);
+    if (rt.rounds != kDecRounds && p->grid_decode8_apply > 0)
+        k_decode_tiles<true, 2 * kDecRounds><<<(int)std::min<uint32_t>(ntl, (uint32_t)p->grid_decode8_apply), kDecBlock,
+                                               kDecTileBytes, s>>>(ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n,
+                                                                   nullptr, 1, 0, 1, ws.hdr, ap);
+    else
+        k_decode_tiles<true, kDecRounds><<<grid, kDecBlock, kDecTileBytes, s>>>(
+            ls, W, (uint32_t)p->total_cap, (uint32_t)p->total_n, nullptr, 1, 0, 1, ws.hdr, ap);
     GC_CUDA(p, cudaGetLastError());
     return GC_OK;
 }

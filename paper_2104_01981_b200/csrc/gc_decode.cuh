@@ -120,19 +120,121 @@ __device__ __forceinline__ void stage_tile(float* s_tile, const float* out, uint
     }
 }
 
-template <bool APPLY>
-static __global__ void __launch_bounds__(kDecBlock)
+// Counted route of the narrow kernels, for tiles that start at +0 and enough workers that their
+// W block-wide steps would cost more than this.  Every pre-loaded entry inside [seg_lo, seg_hi)
+// first counts itself into its element -- the tile doubles as the counter array -- which tells
+// how many workers hit the element and gives each hitter a distinct arrival number.  One hit:
+// the entry is stored.  Two hits: the first arrival stores, the second adds; fp32 addition is
+// commutative, so (+0 + a) + b is the worker-order result whichever came first.  Three or more:
+// there the order matters; those entries go to a short list and one thread per element sums
+// them by worker number.  Returns false when the list overflowed: the touched elements are
+// back at +0 and the caller applies the entries on the ordered route.  Called by the whole CTA.
+constexpr uint32_t kDecCountedFrom = 4;      // workers from which the counted route is taken
+constexpr int kDecConfCap = 128;             // colliding entries (three and more hits) a tile may hold
+template <int R>
+__device__ __forceinline__ bool counted_apply(float* s_tile, uint32_t lo, uint32_t seg_lo, uint32_t seg_hi,
+                                              uint32_t (&ix)[R], const float (&v)[R], uint32_t my_w,
+                                              uint32_t c0, WsHeader* hdr, uint4* s_conf, uint32_t* s_nconf, int tid) {
+    int* const t_cnt = reinterpret_cast<int*>(s_tile);
+    // per entry one byte: arrival number (6 bits) | min(hits, 3) << 6.  Four entries: a register
+    // each (packing them cost registers and 5 % of the time); eight entries: packed into 64 bits,
+    // which keeps that form at 64 registers and four CTAs per SM.
+    constexpr bool kPacked = R > 4;
+    uint32_t oh_a[kPacked ? 1 : R] = {};
+    unsigned long long oh_p = 0ull;
+    auto put = [&](int rd, uint32_t bits) { if constexpr (kPacked) oh_p |= (unsigned long long)bits << (8 * rd); else oh_a[rd] |= bits; };
+    auto get = [&](int rd) -> uint32_t { if constexpr (kPacked) return (uint32_t)(oh_p >> (8 * rd)) & 255u; else return oh_a[rd]; };
+#pragma unroll
+    for (int rd = 0; rd < R; ++rd) {
+        if (ix[rd] < seg_hi) {
+            if (ix[rd] >= seg_lo) put(rd, (uint32_t)atomicAdd(&t_cnt[ix[rd] - lo], 1) & 63u);
+            else { record_status(hdr, -1 /*GC_E_INVALID*/, c0); ix[rd] = 0xFFFFFFFFu; }     // list not ascending: skipped
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rd = 0; rd < R; ++rd)
+        if (ix[rd] < seg_hi) put(rd, min((uint32_t)t_cnt[ix[rd] - lo], 3u) << 6);
+    __syncthreads();                                       // every count has been read
+    bool conflict = false;
+#pragma unroll
+    for (int rd = 0; rd < R; ++rd) {
+        if (ix[rd] >= seg_hi) continue;
+        const uint32_t b8 = get(rd);
+        if ((b8 >> 6) <= 2u) {
+            if ((b8 & 63u) == 0u) s_tile[ix[rd] - lo] = __fadd_rn(0.0f, v[rd]);
+        } else {
+            const uint32_t slot = atomicAdd(s_nconf, 1u);
+            if (slot < (uint32_t)kDecConfCap) s_conf[slot] = make_uint4(ix[rd] - lo, my_w, __float_as_uint(v[rd]), 0u);
+            conflict = true;
+        }
+    }
+    bool done = true;
+    if (__syncthreads_or(conflict ? 1 : 0)) {
+        const uint32_t nc = *s_nconf;
+        if (nc > (uint32_t)kDecConfCap) {
+            // more colliding entries than the list holds: every touched element goes back to +0
+            __syncthreads();
+#pragma unroll
+            for (int rd = 0; rd < R; ++rd) if (ix[rd] < seg_hi) s_tile[ix[rd] - lo] = 0.0f;
+            done = false;
+        } else if ((uint32_t)tid < nc) {
+            // one thread per element with three or more hits: the entry of the lowest worker sums them all
+            const uint4 me = s_conf[tid];
+            bool lowest = true;
+            for (uint32_t j = 0; j < nc; ++j) lowest = lowest && !(s_conf[j].x == me.x && s_conf[j].y < me.y);
+            if (lowest) {
+                float sum = 0.0f;
+                uint32_t next_from = 0u;                   // workers below this one have been added
+                while (true) {
+                    uint32_t best = 0xFFFFFFFFu, bj = 0;
+                    for (uint32_t j = 0; j < nc; ++j) {
+                        const uint4 e = s_conf[j];
+                        if (e.x == me.x && e.y >= next_from && e.y < best) { best = e.y; bj = j; }
+                    }
+                    if (best == 0xFFFFFFFFu) break;
+                    sum = __fadd_rn(sum, __uint_as_float(s_conf[bj].z));
+                    next_from = best + 1u;
+                }
+                s_tile[me.x] = sum;
+            }
+        }
+    }
+    if (done) {
+#pragma unroll
+        for (int rd = 0; rd < R; ++rd)
+            if (ix[rd] < seg_hi && get(rd) == ((2u << 6) | 1u))
+                s_tile[ix[rd] - lo] = __fadd_rn(s_tile[ix[rd] - lo], v[rd]);
+    }
+    __syncthreads();
+    return done;
+}
+
+// R = entries a thread pre-loads per tile (R, or twice that for lists that are denser
+// than four per thread and worker but still fit eight).
+template <bool APPLY, int R>
+// (the eight-entry form is held to 64 registers: four CTAs per SM measured better than three;
+// holding the four-entry form to 40 registers for six CTAs per SM measured worse than five)
+static __global__ void __launch_bounds__(kDecBlock, R == kDecRounds ? 0 : 4)
 k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float* __restrict__ out,
                int zero_first, int use_bulk, int nbuf, WsHeader* hdr, ApplyArgs ap) {
     // nbuf tile buffers: with two, one fills while the other drains (pays off when there are few
     // workers per tile; with many workers more resident CTAs are worth more than the overlap)
     extern __shared__ __align__(128) float s_tiles[];
-    __shared__ uint32_t s_cur[64], s_len[64];
+    __shared__ uint32_t s_cur[64], s_len[64], s_nconf;
+    __shared__ uint4 s_conf[kDecConfCap];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
     const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
     const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
     if (t0 >= t1) return;
+#ifdef GC_PROBE_DECODE_SPREAD
+    if (tid == 0) {
+        unsigned long long ts;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
+        atomicMin(reinterpret_cast<unsigned long long*>(hdr) + 40, ts);
+    }
+#endif
 
     // length of each worker's list, and where it enters this CTA's run of tiles
     for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
@@ -160,27 +262,30 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
         const uint32_t hi = min(total_n, lo + (uint32_t)kDecTile);
         const bool full = hi - lo == (uint32_t)kDecTile;
         stage_tile(s_tile, out, lo, hi, full, zero_first, use_bulk, tid);
-        // pre-load the next kDecRounds * E entries of every worker
+        // pre-load the next R * E entries of every worker
         const uint32_t c0 = live ? s_cur[my_w] : 0u;
-        uint32_t ix[kDecRounds];
-        float v[kDecRounds];
+        uint32_t ix[R];
+        float v[R];
         uint32_t nin = 0;
 #pragma unroll
-        for (int rd = 0; rd < kDecRounds; ++rd) {
+        for (int rd = 0; rd < R; ++rd) {
             const uint32_t p = c0 + (uint32_t)(rd * E + sub);
             ix[rd] = 0xFFFFFFFFu; v[rd] = 0.f;
             if (live && p < my_len) { ix[rd] = __ldg(ls.idx[my_w] + p); v[rd] = __ldg(ls.val[my_w] + p); }
         }
 #pragma unroll
-        for (int rd = 0; rd < kDecRounds; ++rd) nin += ix[rd] < hi;       // sorted lists: the ins are a prefix
+        for (int rd = 0; rd < R; ++rd) nin += ix[rd] < hi;       // sorted lists: the ins are a prefix
         // a worker whose pre-loaded entries all fall inside may have more: then the tile takes
         // the strictly sequential path so that worker order is kept for every element
-        const bool maybe_more = (ix[kDecRounds - 1] < hi) && sub == E - 1;
+        const bool maybe_more = (ix[R - 1] < hi) && sub == E - 1;
+        if (tid == 0) s_nconf = 0u;
         if (!__syncthreads_or(maybe_more ? 1 : 0)) {                      // (also: tile staged, cursors read)
-            for (uint32_t q = 0; q < W; ++q) {                             // apply in worker order
+            const bool counted = zero_first && W >= kDecCountedFrom &&
+                                 counted_apply<R>(s_tile, lo, lo, hi, ix, v, my_w, c0, hdr, s_conf, &s_nconf, tid);
+            for (uint32_t q = 0; q < W && !counted; ++q) {                 // apply in worker order
                 if (my_w == q) {
 #pragma unroll
-                    for (int rd = 0; rd < kDecRounds; ++rd) {
+                    for (int rd = 0; rd < R; ++rd) {
                         if (ix[rd] < hi) {
                             if (ix[rd] >= lo) s_tile[ix[rd] - lo] = __fadd_rn(s_tile[ix[rd] - lo], v[rd]);
                             else record_status(hdr, -1 /*GC_E_INVALID*/, c0);      // list not ascending
@@ -229,6 +334,15 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
         record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
     if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+#ifdef GC_PROBE_DECODE_SPREAD
+    if (tid == 0) {          // probe build only: when every CTA ended, and on which SM
+        unsigned long long ts; uint32_t smid;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        unsigned long long* dbg = reinterpret_cast<unsigned long long*>(hdr) + 64;
+        dbg[2 * blockIdx.x] = ts; dbg[2 * blockIdx.x + 1] = ((unsigned long long)(t1 - t0) << 16) | smid;
+    }
+#endif
 }
 
 // Tiled decode of lists that carry per-tensor counts (threshold mode, plans of several tensors):
@@ -244,7 +358,8 @@ static __global__ void __launch_bounds__(kDecBlock)
 k_decode_segments(DecodeLists ls, uint32_t W, const TensorDesc* __restrict__ desc, uint32_t T,
                   const uint32_t* __restrict__ tile_tensor, uint32_t total_n, float* __restrict__ out, int zero_first, int use_bulk, int nbuf, WsHeader* hdr, ApplyArgs ap) {
     extern __shared__ __align__(128) float s_tiles[];
-    __shared__ uint32_t s_cur[64], s_len[64];
+    __shared__ uint32_t s_cur[64], s_len[64], s_nconf;
+    __shared__ uint4 s_conf[kDecConfCap];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t ntl = (total_n + kDecTile - 1) / kDecTile;
     const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
@@ -305,8 +420,11 @@ k_decode_segments(DecodeLists ls, uint32_t W, const TensorDesc* __restrict__ des
 #pragma unroll
             for (int rd = 0; rd < kDecRounds; ++rd) nin += ix[rd] < seg_hi;
             const bool maybe_more = (ix[kDecRounds - 1] < seg_hi) && sub == E - 1;
+            if (tid == 0) s_nconf = 0u;
             if (!__syncthreads_or(maybe_more ? 1 : 0)) {                  // (also: tile staged, cursors read)
-                for (uint32_t q = 0; q < W; ++q) {                         // apply in worker order
+                const bool counted = zero_first && W >= kDecCountedFrom &&
+                                     counted_apply<kDecRounds>(s_tile, lo, seg_lo, seg_hi, ix, v, my_w, c0, hdr, s_conf, &s_nconf, tid);
+                for (uint32_t q = 0; q < W && !counted; ++q) {             // apply in worker order
                     if (my_w == q) {
 #pragma unroll
                         for (int rd = 0; rd < kDecRounds; ++rd) {

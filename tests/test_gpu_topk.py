@@ -295,6 +295,32 @@ def test_config4_eight_resnet_workers_in_one_call_then_decode():
     assert np.array_equal(to_np_u32(out), bits(want))
 
 
+def test_which_plans_take_which_route():
+    """The five workloads take the one-tensor or the many-tensor kernel; a candidate set too large
+    for the per-CTA regions (20 % of 20M elements) takes the general candidate kernel, and that
+    route is exact too; the path option and the mode pick the others."""
+    for cfg, want in ((0, api.GC_ROUTE_TOPK_ONE), (1, api.GC_ROUTE_TOPK_MANY), (2, api.GC_ROUTE_TOPK_ONE),
+                      (3, api.GC_ROUTE_TOPK_MANY), (4, api.GC_ROUTE_TOPK_ONE)):
+        w = synth.workload(cfg)
+        assert api.Plan(w.sizes, w.density, device=0).query(api.GC_Q_COMPRESS_ROUTE) == want, cfg
+        thr = api.Plan(w.sizes, w.density, mode=api.GC_THRESHOLD, device=0).query(api.GC_Q_COMPRESS_ROUTE)
+        assert thr == (api.GC_ROUTE_THRESHOLD_ONE if len(w.sizes) == 1 else api.GC_ROUTE_THRESHOLD_MANY), cfg
+    n = 20_000_000
+    plan = api.Plan([n], 0.2, device=0)
+    assert plan.query(api.GC_Q_COMPRESS_ROUTE) == api.GC_ROUTE_TOPK_GENERAL
+    gen = torch.Generator(device="cuda").manual_seed(12)
+    grads = [torch.randn(n, device="cuda", generator=gen) for _ in range(2)]
+    seen = []
+    check_topk_against_oracle([n], 0.2, grads, expect_counters=seen.append)
+    assert all(c[1] == 0 and c[2] == 0 for c in seen), seen
+    many = api.Plan([3_000_000] * 4, 0.3, device=0)
+    assert many.query(api.GC_Q_COMPRESS_ROUTE) in (api.GC_ROUTE_TOPK_MANY, api.GC_ROUTE_TOPK_GENERAL)
+    for opt, want in ((api.GC_PATH_EXACT, api.GC_ROUTE_EXACT), (api.GC_PATH_STAGED, api.GC_ROUTE_TOPK_STAGED)):
+        plan.set_option(api.GC_OPT_PATH, opt)
+        assert plan.query(api.GC_Q_COMPRESS_ROUTE) == want
+    assert api.Plan([100], 0.1, device=-1).query(api.GC_Q_COMPRESS_ROUTE) == api.GC_ROUTE_NONE
+
+
 def test_candidate_path_needs_no_redo_in_error_feedback_steady_state():
     """Re-using a few gradients makes unsent entries pile up just below the threshold (a cliff in
     the magnitude distribution).  The sampled threshold is an exact order statistic, so the
