@@ -268,6 +268,8 @@ class Rig:
         self.plan = api.Plan(w.sizes, w.density, mode=self.mode, device=device_index)
         if path != "auto":
             self.plan.set_option(api.GC_OPT_PATH, {"exact": api.GC_PATH_EXACT, "staged": api.GC_PATH_STAGED}[path])
+        # the bench owns its workspaces and nothing else writes to them between calls
+        self.plan.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
         self.n, self.k, self.W = self.plan.total_n, self.plan.total_cap, w.workers
         n, W = self.n, self.W
         self.stream = torch.cuda.current_stream()

@@ -145,6 +145,20 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                equals it where one worker hits.  Applies to the tiled decode of
  *                                both decode calls; lists with counts of many-tensor plans keep
  *                                their fixed-order kernel.
+ *   GC_OPT_WORKSPACE_PRIVATE     0 (default): every gc_compress starts with a launch that clears the
+ *                                control block of the workspace, so a workspace may be shared by
+ *                                plans or refilled by the caller between calls.  1: the caller
+ *                                promises that between two gc_compress calls of THIS plan on a
+ *                                workspace nothing else writes to it (the decode calls of this plan
+ *                                are fine, and so is a zero-filled or a fresh workspace for the first
+ *                                call).  The one-tensor top-k kernel cleans the control block as it
+ *                                goes (each section right after the grid barrier that follows its
+ *                                last reader, the rest at the start of the next launch), so its
+ *                                calls then do without the clearing launch.  A broken promise is
+ *                                caught by a mark in the workspace header: the kernel leaves at once
+ *                                and GC_E_INVALID is recorded in the device status; after any error
+ *                                status read through gc_last_status the next call clears again.
+ *                                Other plans' routes ignore the option.
  * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
  */
 #define GC_OPT_PATH                  0
@@ -155,6 +169,7 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
 #define GC_DECODE_NARROW 1
 #define GC_DECODE_WIDE   2
 #define GC_OPT_DECODE_ORDER          4
+#define GC_OPT_WORKSPACE_PRIVATE     5
 #define GC_ORDER_FIXED   0
 #define GC_ORDER_ANY     1
 #define GC_PATH_AUTO   0

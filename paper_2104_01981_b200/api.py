@@ -29,6 +29,7 @@ GC_K_COUNT = 16
 GC_OPT_PATH, GC_OPT_SAMPLE_RANK_PERMILLE, GC_OPT_CANDIDATE_CAPACITY, GC_OPT_DECODE_ROUTE = 0, 1, 2, 3
 GC_DECODE_AUTO, GC_DECODE_NARROW, GC_DECODE_WIDE = 0, 1, 2
 GC_OPT_DECODE_ORDER = 4
+GC_OPT_WORKSPACE_PRIVATE = 5
 GC_ORDER_FIXED, GC_ORDER_ANY = 0, 1
 GC_PATH_AUTO, GC_PATH_EXACT, GC_PATH_STAGED = 0, 1, 2
 

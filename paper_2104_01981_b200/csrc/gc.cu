@@ -69,6 +69,8 @@ struct gc_plan_s {
     size_t thrm_smem = 0;
     int grid_multi_max = 0;                 // resident CTAs of k_topk_multi (0 = not available)
     size_t multi_smem_max = 0, thrm_smem_max = 0;   // dynamic shared memory those occupancy figures were taken with
+    bool ws_private = false;                // GC_OPT_WORKSPACE_PRIVATE
+    std::vector<const void*> clean_ws;      // workspaces the one-tensor top-k kernel ran on last (and left clean), if private
     uint32_t wk_W = 0, wk_batch = 0;        // gc_compress_workers: workers per launch chosen for the last W seen
     MultiGeom wk_geom;
     uint32_t multi_ntab = 0;
@@ -750,6 +752,7 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
         case GC_OPT_PATH:
             if (value != GC_PATH_AUTO && value != GC_PATH_EXACT && value != GC_PATH_STAGED) return GC_E_INVALID;
             p->path = (int)value;
+            p->clean_ws.clear();
             return GC_OK;
         case GC_OPT_SAMPLE_RANK_PERMILLE:
             if (value < 1 || value > 100000) return GC_E_INVALID;
@@ -764,6 +767,11 @@ int gc_plan_set_option(gc_plan_t* p, int option, uint64_t value) {
             if (value > p->cand_cap_alloc) return GC_E_INVALID;
             p->cand_cap = (uint32_t)value;
             p->wk_W = 0;
+            return GC_OK;
+        case GC_OPT_WORKSPACE_PRIVATE:
+            if (value > 1) return GC_E_INVALID;
+            p->ws_private = value != 0;
+            p->clean_ws.clear();
             return GC_OK;
         case GC_OPT_DECODE_ORDER:
             if (value != GC_ORDER_FIXED && value != GC_ORDER_ANY) return GC_E_INVALID;
@@ -886,7 +894,15 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         return GC_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsView ws = view(p, workspace);
-    {
+    const int route = compress_route(p);
+    // The one-tensor top-k kernel leaves the control block as the next launch needs it; when the
+    // caller has promised that nobody else touches the workspace, the clearing launch is skipped
+    // for a workspace that kernel ran on last (the kernel checks a mark in the header and leaves
+    // with GC_E_INVALID if the promise was broken).
+    const auto known = std::find(p->clean_ws.begin(), p->clean_ws.end(), (const void*)workspace);
+    const bool kept_clean = p->ws_private && route == GC_ROUTE_TOPK_ONE && known != p->clean_ws.end();
+    if (known != p->clean_ws.end()) p->clean_ws.erase(known);
+    if (!kept_clean) {
         Timed tm(p, s, GC_K_CLEAR_CTRL);
         const size_t n16 = p->control_bytes / 16;             // control_bytes is a multiple of 256
         const int gc = (int)std::min<size_t>((n16 + kBlock - 1) / kBlock, (size_t)p->sm_count * 8);
@@ -900,7 +916,6 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     const int gh = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_hist);
     const int gcp = (int)std::min<uint32_t>(nt, (uint32_t)p->grid_compact);
     char* wb = static_cast<char*>(workspace);
-    const int route = compress_route(p);
     if (route == GC_ROUTE_THRESHOLD_ONE) {
         // one large tensor: sample, exact threshold, fold + hits and emission in one cooperative launch
         ThrSingleArgs ta;
@@ -992,6 +1007,17 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         sa.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
         sa.seg_tot = reinterpret_cast<uint32_t*>(wb + p->off_rowseg);
         sa.ws = ws; sa.gws = gws;
+        sa.ctrl = reinterpret_cast<uint4*>(workspace); sa.ctrl_units = (uint32_t)(p->control_bytes / 16);
+        sa.early[0][0] = (uint32_t)(p->off_hist5 / 16); sa.early[0][1] = (uint32_t)((p->off_hist5 + sizeof(uint32_t) * kHistBins) / 16);
+        sa.early[1][0] = (uint32_t)(p->off_fine / 16); sa.early[1][1] = (uint32_t)((p->off_fine + sizeof(uint32_t) * (size_t)kFineBins) / 16);
+        sa.early[2][0] = (uint32_t)(p->off_age / 16); sa.early[2][1] = (uint32_t)((p->off_age + sizeof(uint32_t) * 1024) / 16);
+        sa.clean_sig = 0xC1EA9B10C5ull ^ ((unsigned long long)p->control_bytes << 24) ^ ((unsigned long long)p->single_grid << 52) ^
+                       (unsigned long long)p->total_n;
+        sa.expect_clean = kept_clean ? 1u : 0u;
+        if (p->ws_private) {
+            if (p->clean_ws.size() >= 2 * GC_MAX_WORKERS) p->clean_ws.erase(p->clean_ws.begin());     // (oldest forgotten)
+            p->clean_ws.push_back(workspace);
+        }
         void* args[] = {&sa};
         Timed tm(p, s, GC_K_FUSED);
         const void* kfn = bf16 ? (const void*)k_topk_single<GradBF16> : (const void*)k_topk_single<GradF32>;
@@ -1332,6 +1358,10 @@ int gc_last_status(gc_plan_t* p, const void* workspace, void* stream, int32_t* s
     GC_CUDA(p, cudaStreamSynchronize(s));
     *status = h.status;
     if (detail) *detail = h.detail;
+    if (h.status < 0) {                                   // a failed launch leaves no clean block behind
+        const auto known = std::find(p->clean_ws.begin(), p->clean_ws.end(), workspace);
+        if (known != p->clean_ws.end()) p->clean_ws.erase(known);
+    }
     return GC_OK;
 }
 

@@ -73,11 +73,14 @@ struct WsHeader {            // head of the workspace, 256 bytes
     uint32_t n_failed;       // tensors whose candidate set turned out too small
     uint32_t barrier;        // arrivals at the grid barriers of the fused kernel (monotonic)
     uint32_t n_stamps;       // phase time stamps recorded by CTA 0 of the fused kernel
-    uint32_t pad0[3];
+    uint32_t exit_count;     // CTAs of the one-tensor top-k kernel that have left (back to 0 when the last one leaves)
+    uint32_t pad0[2];
     unsigned long long stamp[20];   // %globaltimer (ns) at the start and after each phase
     unsigned long long t_last_exit; // latest exit of any CTA of the fused kernel (ns)
-    uint32_t reserved[2];
+    unsigned long long clean_mark;  // set by a launch of the one-tensor top-k kernel that left the control block clean
 };
+// (as 32-bit words of the header: what that kernel does not reset at its start)
+constexpr uint32_t kHdrBarrierWord = 15, kHdrExitWord = 17, kHdrSigWord = 62;
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
 struct WsView {              // host-computed pointers into the workspace

@@ -321,6 +321,71 @@ def test_which_plans_take_which_route():
     assert api.Plan([100], 0.1, device=-1).query(api.GC_Q_COMPRESS_ROUTE) == api.GC_ROUTE_NONE
 
 
+@pytest.mark.parametrize("options", [{}, {api.GC_OPT_SAMPLE_RANK_PERMILLE: 30}, {api.GC_OPT_CANDIDATE_CAPACITY: 4}],
+                         ids=["plain", "starved", "overflow"])
+def test_private_workspace_skips_the_clearing_launch_and_stays_exact(options):
+    """GC_OPT_WORKSPACE_PRIVATE: from the second call on a workspace, the one-tensor kernel runs
+    without the clearing launch in front of it (one launch per call) because it leaves the control
+    block clean itself -- also when the safety net ran.  Five error-feedback steps, alternating two
+    workspaces, every step against the oracle."""
+    n = 3_000_001
+    plan = api.Plan([n], 0.01, device=0)
+    plan.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
+    for opt, value in options.items():
+        plan.set_option(opt, value)
+    k = plan.total_cap
+    wss = [plan.alloc_workspace(), plan.alloc_workspace()]
+    idx, val, cnt = plan.alloc_outputs()
+    r = torch.zeros(n, device="cuda")
+    r_cpu = np.zeros(n, np.float32)
+    for step in range(6):
+        ws = wss[step % 2]
+        g = randn(n, 5000 + step)
+        idx.fill_(-1); val.fill_(float("nan"))
+        before = plan.launches()
+        plan.compress(g.cuda(), r, idx, val, cnt, ws)
+        assert plan.launches() - before == (2 if step < 2 else 1), step        # first use of a workspace: cleared once
+        st, det = plan.last_status(ws)
+        assert st == api.GC_OK, (step, st, det)
+        oi, ov = oracle.topk_compress_tensors([n], [k], g.numpy(), r_cpu)
+        assert np.array_equal(to_np_u32(idx[:k]), oi), step
+        assert np.array_equal(to_np_u32(val[:k]), bits(ov)), step
+        assert np.array_equal(to_np_u32(r), bits(r_cpu)), step
+        if step == 3:                                  # a decode of this plan in between is fine (status word only)
+            dense = torch.empty(n, device="cuda")
+            plan.decompress_accumulate([idx], [val], None, dense, True, ws)
+
+
+def test_private_workspace_broken_promise_is_caught():
+    """The caller overwrites a workspace it promised to leave alone: the next call must end at once
+    with GC_E_INVALID in the device status (no barrier is entered on counters that cannot be
+    trusted), and the call after that -- cleared again -- is exact."""
+    n = 1_000_003
+    plan = api.Plan([n], 0.01, device=0)
+    plan.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
+    k = plan.total_cap
+    ws = plan.alloc_workspace()
+    idx, val, cnt = plan.alloc_outputs()
+    r = torch.zeros(n, device="cuda")
+    r_cpu = np.zeros(n, np.float32)
+    g = randn(n, 1)
+    plan.compress(g.cuda(), r, idx, val, None, ws)
+    assert plan.last_status(ws)[0] == api.GC_OK
+    oracle.topk_compress_tensors([n], [k], g.numpy(), r_cpu)
+    for fill in (0x5A, 0):                             # junk, and a zero fill (the mark is gone either way)
+        ws.fill_(fill)
+        r_keep = r.clone()
+        plan.compress(g.cuda(), r, idx, val, None, ws)
+        st, det = plan.last_status(ws)
+        assert st == api.GC_E_INVALID, (fill, st, det)
+        assert torch.equal(r, r_keep)                  # the kernel left before touching anything
+        g2 = randn(n, 2 + fill)
+        plan.compress(g2.cuda(), r, idx, val, None, ws)
+        assert plan.last_status(ws)[0] == api.GC_OK
+        oi, ov = oracle.topk_compress_tensors([n], [k], g2.numpy(), r_cpu)
+        assert np.array_equal(to_np_u32(idx[:k]), oi) and np.array_equal(to_np_u32(r), bits(r_cpu))
+
+
 def test_candidate_path_needs_no_redo_in_error_feedback_steady_state():
     """Re-using a few gradients makes unsent entries pile up just below the threshold (a cliff in
     the magnitude distribution).  The sampled threshold is an exact order statistic, so the
