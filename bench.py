@@ -518,6 +518,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others):
     prof = {("c3_bert_base_110m_student_t", "topk", "compress_fused"): "k_topk_single_c3_bert110m.md",
             ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): "k_threshold_single_c3_bert110m.md",
             ("c2_resnet50_layerwise", "topk", "compress_fused"): "k_topk_multi_c2_resnet50.md",
+            ("c4_resnet50_8workers", "topk", "compress_fused"): "k_topk_workers_c4_resnet50_8workers.md",
             }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None)
     ncu_traffic, ncu_src = profile_traffic(prof) if prof else (None, None)
 
@@ -630,8 +631,13 @@ def run_ecrm(args, rank: int, world: int, local_rank: int):
     def only_add(i):
         ecrm.parity_add(sets[i % len(sets)][2], de, ds, p_entry, p_state, None, stream)
 
+    def fused_step(i):
+        rows, g, prow = sets[i % len(sets)]
+        ecrm.rows_step_parity(ecrm.ECRM_MOMENTUM, rows, prow, g, entry, state, p_entry, p_state, 0.01, 0.9, None, stream)
+
     clocks = ClockSampler(local_rank, os.path.join(tempfile.gettempdir(), f"gc_clocks_ecrm_{rank}.csv"))
     ms = timed(step, args.steps)
+    ms_fused = timed(fused_step, args.steps)
     ms_step = timed(only_step, args.steps)
     ms_add = timed(only_add, args.steps)
     # encoder / decoder over whole shards (k = 4 shards of 1 GiB), degraded reads of m rows
@@ -647,8 +653,8 @@ def run_ecrm(args, rank: int, world: int, local_rank: int):
     sh2 = [x.view(-1, dim) for x in shards]
     ms_rd = timed(lambda i: ecrm.degraded_read(rd_rows, None, sh2[1:], parity.view(-1, dim), rd_out, None, stream), n_cd)
     clk = clocks.stop()
-    ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd = reduce_max_over_ranks([ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd],
-                                                                        world, dev)
+    ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd, ms_fused = reduce_max_over_ranks(
+        [ms, ms_step, ms_add, ms_enc, ms_dec, ms_rd, ms_fused], world, dev)
     if rank != 0:
         return
     row_b = dim * 4
@@ -678,6 +684,12 @@ def run_ecrm(args, rank: int, world: int, local_rank: int):
         "rows_per_s": m_eff * world * args.steps / (ms * 1e-3),
         "kernels": {
             "rows_step": {"ms_per_launch": ms_step / args.steps, "GB_per_s": step_gbs},
+            "rows_step_parity_fused": {"ms_per_launch": ms_fused / args.steps,
+                                       "bytes": m_eff * (9 * row_b + 8),     # g, e, s, pe, ps read; e, s, pe, ps written
+                                       "GB_per_s": m_eff * (9 * row_b + 8) / (ms_fused / args.steps * 1e-3) / 1e9,
+                                       "rows_per_s": m_eff * world * args.steps / (ms_fused * 1e-3),
+                                       "what": "ecrm_rows_step_parity: the same update when data and parity shard share the "
+                                               "GPU (the differences stay in registers)"},
             "parity_add": {"ms_per_launch": ms_add / args.steps,
                            "GB_per_s": bytes_add / (ms_add / args.steps * 1e-3) / 1e9},
             "encode_k4": {"ms_per_launch": ms_enc / n_cd, "GB_per_s": (k + 1) * 4 * shard_n / (ms_enc / n_cd * 1e-3) / 1e9},

@@ -96,6 +96,22 @@ int ecrm_parity_add(uint32_t m, const uint32_t *prow, const float *d_entry, cons
                     uint32_t *bad_rows, void *stream);
 
 /*
+ * ecrm_rows_step_parity -- ecrm_rows_step and ecrm_parity_add of the same rows in one pass, for a
+ * data shard whose parity shard lives on the same GPU (Section 3.3.2: the differences that
+ * server-side propagation would send never leave the chip, so they are not written out).
+ * For every j < m: the optimizer step on row rows[j] of entry / state exactly as in
+ * ecrm_rows_step, then p_entry[prow[j]] += fl(entry' - entry) and p_state[prow[j]] +=
+ * fl(state' - state), one rounding per operation -- bit for bit what the two calls give.
+ *   rows, prow   device, uint32[m]; every data row and every parity row at most once per call
+ *   the parity arrays must not be the data arrays; a row number out of range (either table)
+ *   skips the row and is counted in *bad_rows
+ * Moves 9 rows of dim floats per updated row instead of 13.
+ */
+int ecrm_rows_step_parity(int optimizer, uint32_t m, const uint32_t *rows, const uint32_t *prow, const float *grad,
+                          float *entry, float *state, uint64_t n_rows, float *p_entry, float *p_state,
+                          uint64_t n_prows, uint32_t dim, float lr, float hyper, uint32_t *bad_rows, void *stream);
+
+/*
  * ecrm_degraded_read -- out[j] = ((parity[prow[j]] - shards[0][srow[0][j]]) - shards[1][srow[1][j]]) ...
  * for j < m: rows of the failed server rebuilt on the fly.
  *   prow      device, uint32[m]: parity row of request j

@@ -106,6 +106,57 @@ __global__ void __launch_bounds__(kThreads) k_ecrm_rows_step(uint32_t m, const u
     }
 }
 
+// The optimizer step and the parity update of the same rows in one pass, for a data shard whose
+// parity lives on the same GPU: the two differences stay in registers.  One warp per row.
+template <int OPT>
+__global__ void __launch_bounds__(kThreads) k_ecrm_rows_step_parity(uint32_t m, const uint32_t* __restrict__ rows,
+                                                                     const uint32_t* __restrict__ prow,
+                                                                     const float* __restrict__ grad, float* __restrict__ entry,
+                                                                     float* __restrict__ state, uint64_t n_rows,
+                                                                     float* __restrict__ p_entry, float* __restrict__ p_state,
+                                                                     uint64_t n_prows, uint32_t dim4, float lr, float hyper,
+                                                                     uint32_t* bad_rows) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = (uint64_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const uint64_t nwarps = (uint64_t)gridDim.x * kWarpsPerCta;
+    for (uint64_t j = warp; j < m; j += nwarps) {
+        const uint32_t row = __ldg(rows + j), pr = __ldg(prow + j);
+        if (row >= n_rows || pr >= n_prows) {
+            if (lane == 0 && bad_rows != nullptr) atomicAdd(bad_rows, 1u);
+            continue;
+        }
+        const float4* g4 = reinterpret_cast<const float4*>(grad) + j * dim4;
+        float4* e4 = reinterpret_cast<float4*>(entry) + (uint64_t)row * dim4;
+        float4* s4 = reinterpret_cast<float4*>(state) + (uint64_t)row * dim4;
+        float4* pe4 = reinterpret_cast<float4*>(p_entry) + (uint64_t)pr * dim4;
+        float4* ps4 = reinterpret_cast<float4*>(p_state) + (uint64_t)pr * dim4;
+        for (uint32_t c = lane; c < dim4; c += 32) {
+            const float4 g = __ldcs(g4 + c);
+            const float4 e = e4[c], s = s4[c], pe = pe4[c], ps = ps4[c];
+            const float gv[4] = {g.x, g.y, g.z, g.w}, ev[4] = {e.x, e.y, e.z, e.w}, sv[4] = {s.x, s.y, s.z, s.w};
+            const float pev[4] = {pe.x, pe.y, pe.z, pe.w}, psv[4] = {ps.x, ps.y, ps.z, ps.w};
+            float en[4], sn[4], pen[4], psn[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (OPT == ECRM_ADAGRAD) {
+                    sn[q] = __fadd_rn(sv[q], __fmul_rn(gv[q], gv[q]));
+                    const float step = __fdiv_rn(lr, __fsqrt_rn(__fadd_rn(sn[q], hyper)));
+                    en[q] = __fsub_rn(ev[q], __fmul_rn(step, gv[q]));
+                } else {
+                    sn[q] = __fadd_rn(__fmul_rn(hyper, sv[q]), gv[q]);
+                    en[q] = __fsub_rn(ev[q], __fmul_rn(lr, sn[q]));
+                }
+                pen[q] = __fadd_rn(pev[q], __fsub_rn(en[q], ev[q]));      // parity += fl(new - old), as the two calls do
+                psn[q] = __fadd_rn(psv[q], __fsub_rn(sn[q], sv[q]));
+            }
+            e4[c] = make_float4(en[0], en[1], en[2], en[3]);
+            s4[c] = make_float4(sn[0], sn[1], sn[2], sn[3]);
+            pe4[c] = make_float4(pen[0], pen[1], pen[2], pen[3]);
+            ps4[c] = make_float4(psn[0], psn[1], psn[2], psn[3]);
+        }
+    }
+}
+
 // One warp per parity row: p += d (entry and, if given, state).
 __global__ void __launch_bounds__(kThreads) k_ecrm_parity_add(uint32_t m, const uint32_t* __restrict__ prow,
                                                                const float* __restrict__ d_entry,
@@ -241,6 +292,30 @@ int ecrm_rows_step(int optimizer, uint32_t m, const uint32_t* rows, const float*
     else
         k_ecrm_rows_step<ECRM_MOMENTUM><<<grid, kThreads, 0, s>>>(m, rows, grad, entry, state, n_rows, dim / 4, lr,
                                                                    hyper, d_entry, d_state, bad_rows);
+    return launched();
+}
+
+int ecrm_rows_step_parity(int optimizer, uint32_t m, const uint32_t* rows, const uint32_t* prow, const float* grad,
+                          float* entry, float* state, uint64_t n_rows, float* p_entry, float* p_state, uint64_t n_prows,
+                          uint32_t dim, float lr, float hyper, uint32_t* bad_rows, void* stream) {
+    if (optimizer != ECRM_ADAGRAD && optimizer != ECRM_MOMENTUM) return ECRM_E_INVALID;
+    if (dim == 0 || (dim & 3u) != 0 || n_rows == 0 || n_rows > 0xFFFFFFFFull || n_prows == 0 || n_prows > 0xFFFFFFFFull)
+        return ECRM_E_INVALID;
+    if (m == 0) return ECRM_OK;
+    if (rows == nullptr || prow == nullptr || grad == nullptr || entry == nullptr || state == nullptr ||
+        p_entry == nullptr || p_state == nullptr)
+        return ECRM_E_INVALID;
+    if (!aligned16(grad) || !aligned16(entry) || !aligned16(state) || !aligned16(p_entry) || !aligned16(p_state))
+        return ECRM_E_INVALID;
+    if (p_entry == entry || p_state == state || p_entry == state || p_state == entry) return ECRM_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int grid = grid_for_rows(m);
+    if (optimizer == ECRM_ADAGRAD)
+        k_ecrm_rows_step_parity<ECRM_ADAGRAD><<<grid, kThreads, 0, s>>>(m, rows, prow, grad, entry, state, n_rows, p_entry,
+                                                                         p_state, n_prows, dim / 4, lr, hyper, bad_rows);
+    else
+        k_ecrm_rows_step_parity<ECRM_MOMENTUM><<<grid, kThreads, 0, s>>>(m, rows, prow, grad, entry, state, n_rows, p_entry,
+                                                                          p_state, n_prows, dim / 4, lr, hyper, bad_rows);
     return launched();
 }
 

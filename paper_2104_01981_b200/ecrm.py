@@ -33,10 +33,11 @@ def lib() -> ctypes.CDLL:
         l.ecrm_decode.argtypes = [u32, pp, vp, vp, u64, vp]
         l.ecrm_rows_step.argtypes = [ctypes.c_int, u32, vp, vp, vp, vp, u64, u32, f32, f32, vp, vp, vp, vp]
         l.ecrm_parity_add.argtypes = [u32, vp, vp, vp, vp, vp, u64, u32, vp, vp]
+        l.ecrm_rows_step_parity.argtypes = [ctypes.c_int, u32, vp, vp, vp, vp, vp, u64, vp, vp, u64, u32, f32, f32, vp, vp]
         l.ecrm_degraded_read.argtypes = [u32, u32, vp, pp, pp, vp, u64, u32, vp, vp, vp]
         l.ecrm_placement.argtypes = [u32, u64, ctypes.POINTER(u32), ctypes.POINTER(u32)]
         for f in (l.ecrm_encode, l.ecrm_decode, l.ecrm_rows_step, l.ecrm_parity_add, l.ecrm_degraded_read,
-                  l.ecrm_placement):
+                  l.ecrm_placement, l.ecrm_rows_step_parity):
             f.restype = ctypes.c_int
         _configured = True
     return l
@@ -87,6 +88,16 @@ def parity_add(prow: torch.Tensor, d_entry: torch.Tensor, d_state: Optional[torc
     return _check("ecrm_parity_add", lib().ecrm_parity_add(prow.numel(), _ptr(prow), _ptr(d_entry), _ptr(d_state),
                                                            _ptr(p_entry), _ptr(p_state), n_prows, dim,
                                                            _ptr(bad_rows), _stream(stream)))
+
+
+def rows_step_parity(optimizer: int, rows: torch.Tensor, prow: torch.Tensor, grad: torch.Tensor, entry: torch.Tensor,
+                     state: torch.Tensor, p_entry: torch.Tensor, p_state: torch.Tensor, lr: float, hyper: float,
+                     bad_rows: Optional[torch.Tensor] = None, stream=None) -> int:
+    n_rows, dim = entry.shape
+    return _check("ecrm_rows_step_parity",
+                  lib().ecrm_rows_step_parity(optimizer, rows.numel(), _ptr(rows), _ptr(prow), _ptr(grad), _ptr(entry),
+                                              _ptr(state), n_rows, _ptr(p_entry), _ptr(p_state), p_entry.shape[0], dim,
+                                              lr, hyper, _ptr(bad_rows), _stream(stream)))
 
 
 def degraded_read(prow: torch.Tensor, srows: Optional[Sequence[Optional[torch.Tensor]]],

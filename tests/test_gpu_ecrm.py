@@ -44,6 +44,43 @@ def test_encode_decode_match_oracle_bitwise(k, n):
     assert same(work, eo.decode(want, [s.numpy() for s in shards[1:]]))
 
 
+@pytest.mark.parametrize("optimizer,lr,hyper", [(ecrm.ECRM_ADAGRAD, 0.05, 1e-8), (ecrm.ECRM_MOMENTUM, 0.01, 0.9)])
+@pytest.mark.parametrize("n_rows,p_rows,m,dim", [(1, 1, 1, 4), (100, 40, 30, 128), (5000, 1300, 1237, 128),
+                                                 (999, 333, 333, 132), (200_000, 50_000, 20_000, 128)])
+def test_fused_rows_step_and_parity_match_oracle_bitwise(optimizer, lr, hyper, n_rows, p_rows, m, dim):
+    """The optimizer step with the parity update fused behind it (data shard and parity shard on
+    one GPU): entry, state, parity entry and parity state after three steps equal the oracle's
+    step followed by its parity update, bit for bit; rows out of range are skipped and counted."""
+    entry = synth.ecrm_tables(n_rows, dim, 1, seed=n_rows + dim)[0]
+    state = torch.zeros(n_rows, dim)
+    p_entry, p_state = synth.ecrm_tables(p_rows, dim, 1, seed=7)[0] * 3.0, torch.zeros(p_rows, dim)
+    d = [t.cuda() for t in (entry, state, p_entry, p_state)]
+    h = [t.numpy().copy() for t in (entry, state, p_entry, p_state)]
+    bad = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(m)
+    for step in range(3):
+        rows, g = synth.ecrm_batch(n_rows, m, dim, seed=100 * step + m)
+        prow = torch.from_numpy(rng.permutation(p_rows)[:m].astype(np.uint32).view(np.int32))   # distinct parity rows
+        ecrm.rows_step_parity(optimizer, rows.cuda(), prow.cuda(), g.cuda(), d[0], d[1], d[2], d[3], lr, hyper, bad)
+        rows_np, prow_np = rows.numpy().view(np.uint32), prow.numpy().view(np.uint32)
+        wde, wds = eo.rows_step(optimizer, rows_np, g.numpy(), h[0], h[1], lr, hyper)
+        eo.parity_add(prow_np, wde, wds, h[2], h[3])
+        assert same(d[0], h[0]) and same(d[1], h[1]) and same(d[2], h[2]) and same(d[3], h[3]), step
+    assert bad.item() == 0
+    if m >= 3:                                     # a data row and a parity row out of range: both skipped
+        rows, g = synth.ecrm_batch(n_rows, m, dim, seed=999)
+        prow = torch.from_numpy(rng.permutation(p_rows)[:m].astype(np.uint32).view(np.int32))
+        rows_bad, prow_bad = rows.clone(), prow.clone()
+        rows_bad[1] = n_rows
+        prow_bad[2] = p_rows + 5
+        ecrm.rows_step_parity(optimizer, rows_bad.cuda(), prow_bad.cuda(), g.cuda(), d[0], d[1], d[2], d[3], lr, hyper, bad)
+        keep = np.ones(m, bool); keep[[1, 2]] = False
+        wde, wds = eo.rows_step(optimizer, rows.numpy().view(np.uint32)[keep], g.numpy()[keep], h[0], h[1], lr, hyper)
+        eo.parity_add(prow.numpy().view(np.uint32)[keep], wde, wds, h[2], h[3])
+        assert same(d[0], h[0]) and same(d[1], h[1]) and same(d[2], h[2]) and same(d[3], h[3])
+        assert bad.item() == 2
+
+
 def test_integer_valued_shards_are_recovered_exactly():
     shards = synth.ecrm_tables(5000, 128, 4, seed=3, device="cuda", integer_valued=True)
     parity = torch.empty_like(shards[0])
