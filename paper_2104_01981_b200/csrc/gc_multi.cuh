@@ -372,7 +372,7 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
                     if (!interior) c = c && ((valid >> (4 * j + e)) & 1u);
                     cnt[j] += c;
                     cm |= (uint32_t)c << (4 * j + e);
-                    hm |= (uint32_t)(key >= tau_z) << (4 * j + e);
+                    if (!interior) hm |= (uint32_t)(key >= tau_z) << (4 * j + e);
                 }
             }
             uint32_t rk[kVpt], wtot;
@@ -386,13 +386,16 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
             const uint32_t em = fits ? cm : 0u;             // goes to the candidate list
             const uint32_t zm = fits ? (hm & cm) : 0u;      // ... and leaves +0 in the residual (probably sent)
             if (interior) {
+                // +0 where the key reaches tau_z (implies a candidate: tau_z >= tau), a elsewhere; a chunk
+                // that did not fit keeps all its values (no key reaches 2^31)
+                const uint32_t tz = fits ? tau_z : 0x80000000u;
 #pragma unroll
                 for (int j = 0; j < kVpt; ++j) {
                     float4 o;
-                    o.x = ((zm >> (4 * j + 0)) & 1u) ? 0.0f : av[j][0];
-                    o.y = ((zm >> (4 * j + 1)) & 1u) ? 0.0f : av[j][1];
-                    o.z = ((zm >> (4 * j + 2)) & 1u) ? 0.0f : av[j][2];
-                    o.w = ((zm >> (4 * j + 3)) & 1u) ? 0.0f : av[j][3];
+                    o.x = key_of(av[j][0]) >= tz ? 0.0f : av[j][0];
+                    o.y = key_of(av[j][1]) >= tz ? 0.0f : av[j][1];
+                    o.z = key_of(av[j][2]) >= tz ? 0.0f : av[j][2];
+                    o.w = key_of(av[j][3]) >= tz ? 0.0f : av[j][3];
                     __stcs(reinterpret_cast<float4*>(a.r + tg.base + my_off + j * 128), o);    // streaming: evict first
                 }
             } else {
@@ -407,20 +410,22 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
             }
             const bool staged = wtot <= (uint32_t)kEmitStage;
             if (fits && wtot != 0u) {
-                if (em != 0u) {
+                // one round per candidate of the lane that has the most, instead of sixteen predicated
+                // blocks that every warp walks through (see the one-tensor kernel)
+                for (uint32_t m = em; m != 0u; m &= m - 1u) {
+                    const uint32_t bq = (uint32_t)__ffs((int)m) - 1u, j = bq >> 2;      // element 4 j + e of this thread
+                    float s8[8], s4[4];                                                 // its value by a select tree
 #pragma unroll
-                    for (int j = 0; j < kVpt; ++j) {
-                        uint32_t pos = rk[j];
+                    for (int q = 0; q < 8; ++q) s8[q] = (bq & 8u) ? av[2 + q / 4][q % 4] : av[q / 4][q % 4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if ((em >> (4 * j + e)) & 1u) {
-                                const uint2 pr = make_uint2(tg.base + my_off + j * 128 + e, __float_as_uint(av[j][e]));
-                                if (staged) sm.emit[warp][pos] = pr; else pool[off + pos] = pr;
-                                atomicAdd(&sm.hist[min((key_of(av[j][e]) - tau) >> shift, 2047u)], 1u);
-                                ++pos;
-                            }
-                        }
-                    }
+                    for (int q = 0; q < 4; ++q) s4[q] = (bq & 4u) ? s8[4 + q] : s8[q];
+                    const float s20 = (bq & 2u) ? s4[2] : s4[0], s21 = (bq & 2u) ? s4[3] : s4[1];
+                    const float v = (bq & 1u) ? s21 : s20;
+                    const uint32_t rkj = (bq & 8u) ? ((bq & 4u) ? rk[3] : rk[2]) : ((bq & 4u) ? rk[1] : rk[0]);
+                    const uint32_t pos = rkj + (uint32_t)__popc(em & ((1u << bq) - 1u) & (0xFu << (4u * j)));
+                    const uint2 pr = make_uint2(tg.base + my_off + j * 128u + (bq & 3u), __float_as_uint(v));
+                    if (staged) sm.emit[warp][pos] = pr; else pool[off + pos] = pr;
+                    atomicAdd(&sm.hist[min((key_of(v) - tau) >> shift, 2047u)], 1u);
                 }
                 if (staged) {
                     __syncwarp();
