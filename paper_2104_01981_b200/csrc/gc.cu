@@ -812,6 +812,38 @@ int gc_plan_query(const gc_plan_t* p, int what, uint32_t tensor, uint64_t* value
     }
 }
 
+// The control block as the self-cleaning kernels see it (see CleanArgs): up to three early sections.
+static CleanArgs clean_args(const gc_plan_s* p, void* workspace, int route, bool expect_clean) {
+    CleanArgs c{};
+    c.ctrl = reinterpret_cast<uint4*>(workspace);
+    c.ctrl_units = (uint32_t)(p->control_bytes / 16);
+    auto range = [&](int q, size_t off, size_t bytes) { c.early[q][0] = (uint32_t)(off / 16); c.early[q][1] = (uint32_t)((off + bytes) / 16); };
+    if (route == GC_ROUTE_TOPK_ONE) {
+        range(0, p->off_hist5, sizeof(uint32_t) * kHistBins);                 // coarse sample histogram
+        range(1, p->off_fine, sizeof(uint32_t) * (size_t)kFineBins);          // fine sample histogram
+        range(2, p->off_age, sizeof(uint32_t) * 1024);                        // arrivals per SM
+    } else {
+        range(0, p->off_shist, sizeof(uint32_t) * (size_t)kHistBins * p->T);  // coarse sample histogram per tensor
+    }
+    c.mark = 0xC1EA9B10C5ull ^ ((unsigned long long)p->control_bytes << 24) ^ ((unsigned long long)route << 56) ^
+             (unsigned long long)p->total_n;
+    c.expect_clean = expect_clean ? 1u : 0u;
+    return c;
+}
+
+// Workspaces this plan's self-cleaning kernels ran on last (GC_OPT_WORKSPACE_PRIVATE).
+static bool take_clean(gc_plan_s* p, const void* workspace) {       // forgets it: the coming launch dirties it
+    const auto known = std::find(p->clean_ws.begin(), p->clean_ws.end(), workspace);
+    if (known == p->clean_ws.end()) return false;
+    p->clean_ws.erase(known);
+    return true;
+}
+static void note_clean(gc_plan_s* p, const void* workspace) {
+    if (!p->ws_private) return;
+    if (p->clean_ws.size() >= 2 * GC_MAX_WORKERS) p->clean_ws.erase(p->clean_ws.begin());     // (oldest forgotten)
+    p->clean_ws.push_back(workspace);
+}
+
 // Which kernels a gc_compress call on this plan takes (GC_ROUTE_*); the dispatch below and
 // GC_Q_COMPRESS_ROUTE both ask here.
 static int compress_route(const gc_plan_s* p) {
@@ -830,7 +862,7 @@ static int compress_route(const gc_plan_s* p) {
 
 // Argument block of the many-tensor kernel for one worker's buffers and a given geometry.
 static MultiArgs multi_args(const gc_plan_s* p, const MultiGeom& mg, const void* grad, float* residual,
-                            uint32_t* out_idx, float* out_val, uint32_t* out_count, void* workspace) {
+                            uint32_t* out_idx, float* out_val, uint32_t* out_count, void* workspace, bool expect_clean) {
     char* wb = static_cast<char*>(workspace);
     WsView ws = view(p, workspace);
     WsView gws = ws;                 // redo of failed tensors: own records, gated by the main ones
@@ -853,6 +885,7 @@ static MultiArgs multi_args(const gc_plan_s* p, const MultiGeom& mg, const void*
     ma.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
     ma.skeys = reinterpret_cast<uint4*>(wb + p->off_skeys);
     ma.ws = ws; ma.gws = gws;
+    ma.cl = clean_args(p, workspace, GC_ROUTE_TOPK_MANY, expect_clean);
     return ma;
 }
 
@@ -899,9 +932,8 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
     // caller has promised that nobody else touches the workspace, the clearing launch is skipped
     // for a workspace that kernel ran on last (the kernel checks a mark in the header and leaves
     // with GC_E_INVALID if the promise was broken).
-    const auto known = std::find(p->clean_ws.begin(), p->clean_ws.end(), (const void*)workspace);
-    const bool kept_clean = p->ws_private && route == GC_ROUTE_TOPK_ONE && known != p->clean_ws.end();
-    if (known != p->clean_ws.end()) p->clean_ws.erase(known);
+    const bool self_cleaning = route == GC_ROUTE_TOPK_ONE || route == GC_ROUTE_TOPK_MANY;
+    const bool kept_clean = take_clean(p, workspace) && p->ws_private && self_cleaning;
     if (!kept_clean) {
         Timed tm(p, s, GC_K_CLEAR_CTRL);
         const size_t n16 = p->control_bytes / 16;             // control_bytes is a multiple of 256
@@ -1007,17 +1039,8 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         sa.tile_cnt = reinterpret_cast<uint32_t*>(wb + p->off_tinfo);
         sa.seg_tot = reinterpret_cast<uint32_t*>(wb + p->off_rowseg);
         sa.ws = ws; sa.gws = gws;
-        sa.ctrl = reinterpret_cast<uint4*>(workspace); sa.ctrl_units = (uint32_t)(p->control_bytes / 16);
-        sa.early[0][0] = (uint32_t)(p->off_hist5 / 16); sa.early[0][1] = (uint32_t)((p->off_hist5 + sizeof(uint32_t) * kHistBins) / 16);
-        sa.early[1][0] = (uint32_t)(p->off_fine / 16); sa.early[1][1] = (uint32_t)((p->off_fine + sizeof(uint32_t) * (size_t)kFineBins) / 16);
-        sa.early[2][0] = (uint32_t)(p->off_age / 16); sa.early[2][1] = (uint32_t)((p->off_age + sizeof(uint32_t) * 1024) / 16);
-        sa.clean_sig = 0xC1EA9B10C5ull ^ ((unsigned long long)p->control_bytes << 24) ^ ((unsigned long long)p->single_grid << 52) ^
-                       (unsigned long long)p->total_n;
-        sa.expect_clean = kept_clean ? 1u : 0u;
-        if (p->ws_private) {
-            if (p->clean_ws.size() >= 2 * GC_MAX_WORKERS) p->clean_ws.erase(p->clean_ws.begin());     // (oldest forgotten)
-            p->clean_ws.push_back(workspace);
-        }
+        sa.cl = clean_args(p, workspace, GC_ROUTE_TOPK_ONE, kept_clean);
+        note_clean(p, workspace);
         void* args[] = {&sa};
         Timed tm(p, s, GC_K_FUSED);
         const void* kfn = bf16 ? (const void*)k_topk_single<GradBF16> : (const void*)k_topk_single<GradF32>;
@@ -1029,7 +1052,8 @@ static int compress_impl(gc_plan_t* p, const void* grad_any, bool bf16, float* r
         MultiGeom mg;
         mg.G = p->multi_grid; mg.per = p->multi_per; mg.pool = p->multi_pool; mg.full = p->multi_full;
         mg.ntab = p->multi_ntab; mg.smem = p->multi_smem;
-        MultiArgs ma = multi_args(p, mg, grad_any, residual, out_idx, out_val, out_count, workspace);
+        MultiArgs ma = multi_args(p, mg, grad_any, residual, out_idx, out_val, out_count, workspace, kept_clean);
+        note_clean(p, workspace);
         void* args[] = {&ma};
         Timed tm(p, s, GC_K_FUSED);
         const void* kfn = bf16 ? (const void*)k_topk_multi<GradBF16> : (const void*)k_topk_multi<GradF32>;
@@ -1174,12 +1198,18 @@ int gc_compress_workers(gc_plan_t* p, uint32_t W, const float* const* grads, flo
         WorkersArgs wa;
         ThrWorkersArgs ta;
         wa.W = ta.W = wn; wa.G = ta.G = mg.G;
+        // the clearing launch is skipped only if every workspace of this launch was left clean
+        bool kept_clean = p->ws_private && topk_multi;
+        for (uint32_t i = 0; i < wn; ++i) kept_clean = take_clean(p, workspaces[w0 + i]) && kept_clean;
         for (uint32_t i = 0; i < wn; ++i) {
             const uint32_t w = w0 + i;
             cm.p[i] = reinterpret_cast<uint4*>(workspaces[w]);
             uint32_t* const oc = out_count ? out_count[w] : nullptr;
-            if (topk_multi) wa.per[i] = multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w]);
-            else ta.per[i] = thr_multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w]);
+            if (topk_multi) {
+                wa.per[i] = multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w], kept_clean);
+                note_clean(p, workspaces[w]);
+            }
+            if (!topk_multi) ta.per[i] = thr_multi_args(p, mg, grads[w], residuals[w], out_idx[w], out_val[w], oc, workspaces[w]);
             if (oc != nullptr && p->n_empty > 0) {
                 Timed tm(p, s, GC_K_CLEAR_CTRL);
                 GC_CUDA(p, cudaMemsetAsync(oc, 0, sizeof(uint32_t) * 2 * (size_t)p->T, s));
@@ -1189,7 +1219,7 @@ int gc_compress_workers(gc_plan_t* p, uint32_t W, const float* const* grads, flo
             cm.p[i] = nullptr;
             if (topk_multi) wa.per[i] = wa.per[0]; else ta.per[i] = ta.per[0];
         }
-        {
+        if (!kept_clean) {
             Timed tm(p, s, GC_K_CLEAR_CTRL);
             const size_t n16 = p->control_bytes / 16;
             const unsigned gx = (unsigned)std::min<size_t>((n16 + kBlock - 1) / kBlock, (size_t)p->sm_count * 8 / wn + 1);
@@ -1358,10 +1388,7 @@ int gc_last_status(gc_plan_t* p, const void* workspace, void* stream, int32_t* s
     GC_CUDA(p, cudaStreamSynchronize(s));
     *status = h.status;
     if (detail) *detail = h.detail;
-    if (h.status < 0) {                                   // a failed launch leaves no clean block behind
-        const auto known = std::find(p->clean_ws.begin(), p->clean_ws.end(), workspace);
-        if (known != p->clean_ws.end()) p->clean_ws.erase(known);
-    }
+    if (h.status < 0) (void)take_clean(p, workspace);    // a failed launch leaves no clean block behind
     return GC_OK;
 }
 

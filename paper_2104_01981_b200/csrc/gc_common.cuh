@@ -73,13 +73,13 @@ struct WsHeader {            // head of the workspace, 256 bytes
     uint32_t n_failed;       // tensors whose candidate set turned out too small
     uint32_t barrier;        // arrivals at the grid barriers of the fused kernel (monotonic)
     uint32_t n_stamps;       // phase time stamps recorded by CTA 0 of the fused kernel
-    uint32_t exit_count;     // CTAs of the one-tensor top-k kernel that have left (back to 0 when the last one leaves)
+    uint32_t exit_count;     // CTAs of a fused top-k launch that have left (back to 0 when the last one leaves)
     uint32_t pad0[2];
     unsigned long long stamp[20];   // %globaltimer (ns) at the start and after each phase
     unsigned long long t_last_exit; // latest exit of any CTA of the fused kernel (ns)
-    unsigned long long clean_mark;  // set by a launch of the one-tensor top-k kernel that left the control block clean
+    unsigned long long clean_mark;  // set by a fused top-k launch that left the control block clean (see CleanArgs)
 };
-// (as 32-bit words of the header: what that kernel does not reset at its start)
+// (as 32-bit words of the header: what those kernels do not reset at their start)
 constexpr uint32_t kHdrBarrierWord = 15, kHdrExitWord = 17, kHdrSigWord = 62;
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -388,6 +388,76 @@ __device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, in
 }
 __device__ __forceinline__ bool grid_barrier(WsHeader* hdr, uint32_t& passed, int* s_ok) {
     return grid_barrier(hdr, passed, s_ok, gridDim.x);
+}
+
+// ----------------------------------------------------------------------------- a control block that stays clean
+// The fused top-k kernels leave the control block of the workspace as their next launch needs to
+// find it, so that launch can do without the clearing launch in front of it.  Everything that is
+// first written after the first grid barrier is zeroed at the START of a launch, a slice per CTA
+// (the writers come after the barrier, so there is no ordering problem); the sections written
+// before the first barrier ("early": at most three ranges) are zeroed right after the barrier that
+// follows their last reader; the barrier counter is reset by the CTA that leaves last (an exit
+// counter in the header), which then sets a 64-bit mark.  When the host has skipped the clearing
+// launch (on the caller's promise that nobody else writes to the workspace), the kernel first
+// checks the mark and leaves at once if it is missing: no barrier is entered on a counter that
+// cannot be trusted.  G CTAs share the block, this is CTA b of them.
+struct CleanArgs {
+    uint4* ctrl;                     // the control block (= the workspace), in 16-byte units
+    uint32_t ctrl_units;             // its length
+    uint32_t early[3][2];            // [begin, end) in units of the sections written before the first barrier
+    unsigned long long mark;         // what the header's mark reads after a launch that left the block clean
+    uint32_t expect_clean;           // the host skipped the clearing launch
+};
+__device__ __forceinline__ unsigned long long* clean_mark_ptr(WsHeader* hdr) {
+    return reinterpret_cast<unsigned long long*>(reinterpret_cast<uint32_t*>(hdr) + kHdrSigWord);
+}
+// First thing in the kernel (after anything that must see the CTAs in their order of arrival).
+// Returns false if the launch must end here.  Contains a block-wide barrier for CTA 0.
+__device__ __forceinline__ bool clean_begin(const CleanArgs& c, WsHeader* hdr, uint32_t G, uint32_t b, int tid) {
+    if (c.expect_clean != 0u && ld_cg(clean_mark_ptr(hdr)) != c.mark) {
+        if (b == 0 && tid == 0) record_status(hdr, -1 /*GC_E_INVALID*/, 0xC1EA0000ull);
+        return false;                // every CTA sees the same word
+    }
+    const uint32_t per = (c.ctrl_units + G - 1) / G;
+    const uint32_t u0 = max(b * per, 16u), u1 = min(c.ctrl_units, (b + 1u) * per);     // (the header is 16 units)
+    for (uint32_t u = u0 + (uint32_t)tid; u < u1; u += kBlock) {
+        const bool is_early = (u >= c.early[0][0] && u < c.early[0][1]) || (u >= c.early[1][0] && u < c.early[1][1]) ||
+                              (u >= c.early[2][0] && u < c.early[2][1]);
+        if (!is_early) c.ctrl[u] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (b == 0) {                    // the header: all but the barrier's, the exit counter's and the mark's words
+        if (tid < 64 && tid != (int)kHdrBarrierWord && tid != (int)kHdrExitWord && tid != (int)kHdrSigWord &&
+            tid != (int)kHdrSigWord + 1)
+            reinterpret_cast<uint32_t*>(hdr)[tid] = 0u;
+        __syncthreads();
+    }
+    return true;
+}
+// After the first barrier: every CTA has read the mark, the block is in use.
+__device__ __forceinline__ void clean_in_use(WsHeader* hdr, uint32_t b, int tid) {
+    if (b == 0 && tid == 0) *clean_mark_ptr(hdr) = 0ull;
+}
+// After the barrier that follows the last reader of the early sections.
+__device__ __forceinline__ void clean_early(const CleanArgs& c, uint32_t G, uint32_t b, int tid) {
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+        const uint32_t len = c.early[q][1] - c.early[q][0], per = (len + G - 1) / G;
+        for (uint32_t u = c.early[q][0] + b * per + (uint32_t)tid; u < min(c.early[q][1], c.early[q][0] + (b + 1u) * per); u += kBlock)
+            c.ctrl[u] = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+// Last step of a launch that ends normally (whole CTA calls; its writes come after every CTA's own
+// cleaning: fence, then the counter).
+__device__ __forceinline__ void leave_clean(const CleanArgs& c, WsHeader* hdr, uint32_t G, int tid) {
+    if (tid == 0) {
+        uint32_t* const w = reinterpret_cast<uint32_t*>(hdr);
+        __threadfence();
+        if (atomicAdd(w + kHdrExitWord, 1u) == G - 1u) {
+            w[kHdrBarrierWord] = 0u; w[kHdrExitWord] = 0u;
+            __threadfence();
+            *clean_mark_ptr(hdr) = c.mark;
+        }
+    }
 }
 
 }  // namespace gc

@@ -56,6 +56,7 @@ struct MultiArgs {
     uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
     uint4* skeys;                    // [nstiles * kBlock] the sampled keys, one group of four per entry
     WsView ws, gws;
+    CleanArgs cl;                    // the control block is left clean for the next launch (early section: shist)
 };
 
 // segment record (one per tensor a CTA's tile run touches), kSegWords words in shared memory
@@ -112,6 +113,7 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WsHeader* hdr = a.ws.hdr;
     uint32_t passed = 0, n_stamp = 0;
+    if (!clean_begin(a.cl, hdr, G, b, tid)) return;
     // The CTAs launched last are the youngest on their SMs and advance the slowest (see RowMap in
     // the one-tensor kernel), so whatever the full runs leave over is spread evenly over them.
     uint32_t first, last;
@@ -229,6 +231,7 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     if (!grid_wait(hdr, passed, &sm.ok, G)) return;
     phase_stamp(hdr, n_stamp, b);
+    clean_in_use(hdr, b, tid);
 
     // ---------------------------------------------------------------- bracket per tensor, one CTA each
     // tau = the srank-th largest sampled key (22 bits when the kept keys allow the second radix
@@ -295,6 +298,7 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     }
     if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
     phase_stamp(hdr, n_stamp, b);
+    clean_early(a.cl, G, b, tid);      // the sample histograms have had their last reader (the brackets)
 
     // ---------------------------------------------------------------- fold + candidates, segment by segment
     uint32_t nseg = 0;
@@ -640,7 +644,7 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
         __syncthreads();
         phase_stamp(hdr, n_stamp, b);
         exit_stamp(hdr);
-        if (ld_cg(&hdr->n_failed) == 0u) return;
+        if (ld_cg(&hdr->n_failed) == 0u) { leave_clean(a.cl, hdr, G, tid); return; }
     } else {
         // a candidate region overflowed: every recorded candidate gets its value back
         for (uint32_t c = tid; c < ntl * kWarps; c += kBlock) {
@@ -663,6 +667,8 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     hist_body<2, SRC_RESID>(sm, a.desc, a.T, a.ntiles, nullptr, a.r, a.gws, G, b);
     if (!grid_barrier(hdr, passed, &sm.ok, G)) return;
     compact_body(sm, a.desc, a.T, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
+    __syncthreads();
+    leave_clean(a.cl, hdr, G, tid);
 }
 
 template <typename GL>

@@ -90,22 +90,6 @@ __device__ __forceinline__ uint32_t aged_column(const RowMap& rm, const uint32_t
     return aged ? min(age, 2u) * rm.gA + smid : b;
 }
 
-// Last step of a launch that ends normally: the CTA that leaves last (an exit counter in the
-// header) resets the barrier counter and that counter and sets the mark of a clean exit; its
-// writes come after every CTA's own cleaning (fence, then the counter).
-__device__ __forceinline__ void leave_clean(WsHeader* hdr, unsigned long long* sig, unsigned long long value,
-                                            uint32_t G, int tid) {
-    if (tid == 0) {
-        uint32_t* const w = reinterpret_cast<uint32_t*>(hdr);
-        __threadfence();
-        if (atomicAdd(w + kHdrExitWord, 1u) == G - 1u) {
-            w[kHdrBarrierWord] = 0u; w[kHdrExitWord] = 0u;
-            __threadfence();
-            *sig = value;
-        }
-    }
-}
-
 struct SingleArgs {
     TensorDesc d;                    // the tensor (by value)
     const TensorDesc* desc;          // device table (for the redo phases)
@@ -128,14 +112,7 @@ struct SingleArgs {
     uint32_t* tile_cnt;              // [ntiles] candidates above the band bin, per tile
     uint32_t* seg_tot;               // [maxt][ceil(G/32)] the same summed over each run of 32 CTAs of a row (zeroed)
     WsView ws, gws;
-    // The kernel leaves the control block of the workspace as it needs to find it, so that the
-    // next call on the same workspace can do without the clearing launch in front of it:
-    uint4* ctrl;                     // the control block (= the workspace), in 16-byte units
-    uint32_t ctrl_units;             // its length
-    uint32_t early[3][2];            // [begin, end) in units of the three sections that are written before the first
-                                     // barrier (coarse sample histogram, fine sample histogram, arrivals per SM)
-    unsigned long long clean_sig;    // what the header's mark reads when the previous launch left the block clean
-    uint32_t expect_clean;           // the host skipped the clearing launch: leave at once unless the mark is there
+    CleanArgs cl;                    // the control block is left clean for the next launch
 };
 
 
@@ -262,38 +239,12 @@ k_topk_single(const __grid_constant__ SingleArgs a) {
     uint32_t passed = 0, n_stamp = 0;
     const RowMap& rm = a.rows;
     __shared__ uint32_t s_age[2];
-    unsigned long long* const sig = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint32_t*>(hdr) + kHdrSigWord);
     // This CTA's age among the CTAs of its SM = its arrival number at the SM's counter, taken
     // first thing: the number has to reflect the order in which the CTAs really started (a load
     // in front of it was measured to cost the fold pass 10 us: the shares no longer matched).
     uint32_t my_age = 0, my_sm = 0;
     if (tid == 0) my_age = note_age(a.age, my_sm);
-    if (a.expect_clean != 0u && ld_cg(sig) != a.clean_sig) {
-        // the clearing launch was skipped on the caller's promise that nobody else touches this
-        // workspace, and the mark of a clean exit is not there: nothing can be trusted, not even
-        // the barrier counter.  Every CTA sees the same word and leaves.
-        if (b == 0 && tid == 0) record_status(hdr, -1 /*GC_E_INVALID*/, 0xC1EA0000ull);
-        return;
-    }
-    // Everything in the control block that is first written after the first grid barrier is
-    // zeroed here, a slice per CTA (the three early sections were zeroed by the previous launch
-    // after their last reader, or by the clearing launch); CTA 0 also resets the header words
-    // that are not the barrier's, the exit counter's or the mark's.
-    {
-        const uint32_t per = (a.ctrl_units + G - 1) / G;
-        const uint32_t u0 = max(b * per, 16u), u1 = min(a.ctrl_units, (b + 1u) * per);     // (the header is 16 units)
-        for (uint32_t u = u0 + (uint32_t)tid; u < u1; u += kBlock) {
-            const bool is_early = (u >= a.early[0][0] && u < a.early[0][1]) || (u >= a.early[1][0] && u < a.early[1][1]) ||
-                                  (u >= a.early[2][0] && u < a.early[2][1]);
-            if (!is_early) a.ctrl[u] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        if (b == 0) {
-            if (tid < 64 && tid != (int)kHdrBarrierWord && tid != (int)kHdrExitWord && tid != (int)kHdrSigWord &&
-                tid != (int)kHdrSigWord + 1)
-                reinterpret_cast<uint32_t*>(hdr)[tid] = 0u;
-            __syncthreads();
-        }
-    }
+    if (!clean_begin(a.cl, hdr, G, b, tid)) return;
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
     for (uint32_t i = tid; i < a.maxt * kWarps; i += kBlock) rec2[i] = 0u;
     for (uint32_t i = tid; i < a.maxt; i += kBlock) row_mid[i] = 0u;
@@ -355,7 +306,7 @@ k_topk_single(const __grid_constant__ SingleArgs a) {
         flush_hist(sm, a.hist5 + 0 * kHistBins, 1 << level_bits(0));
         if (!grid_barrier(hdr, passed, &sm.ok)) return;
         phase_stamp(hdr, n_stamp);
-        if (b == 0 && tid == 0) *sig = 0ull;             // (every CTA has read it) the block is in use
+        clean_in_use(hdr, b, tid);
         {
             col = aged_column(rm, a.age, s_age[0], s_age[1], G, b, tid);
             n_own = rm.rows_of(col);
@@ -528,13 +479,8 @@ k_topk_single(const __grid_constant__ SingleArgs a) {
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     phase_stamp(hdr, n_stamp);
     // the three early sections have had their last reader (the bracket, right after the first
-    // barrier): they are zeroed for the next launch, a slice per CTA
-#pragma unroll
-    for (int q = 0; q < 3; ++q) {
-        const uint32_t len = a.early[q][1] - a.early[q][0], per = (len + G - 1) / G;
-        for (uint32_t u = a.early[q][0] + b * per + (uint32_t)tid; u < min(a.early[q][1], a.early[q][0] + (b + 1u) * per); u += kBlock)
-            a.ctrl[u] = make_uint4(0u, 0u, 0u, 0u);
-    }
+    // barrier): they are zeroed for the next launch
+    clean_early(a.cl, G, b, tid);
 
     // ---------------------------------------------------------------- band bin of the threshold
     // `good` is the same in every CTA: it only depends on global data read after a barrier
@@ -760,7 +706,7 @@ k_topk_single(const __grid_constant__ SingleArgs a) {
             __syncthreads();
             phase_stamp(hdr, n_stamp);
             exit_stamp(hdr);
-            leave_clean(hdr, sig, a.clean_sig, G, tid);
+            leave_clean(a.cl, hdr, G, tid);
             return;
         }
     }
@@ -786,7 +732,7 @@ k_topk_single(const __grid_constant__ SingleArgs a) {
     if (!grid_barrier(hdr, passed, &sm.ok)) return;
     compact_body(sm, a.desc, 1u, a.ntiles, a.r, a.out_idx, a.out_val, a.out_count, a.gws, 0);
     __syncthreads();
-    leave_clean(hdr, sig, a.clean_sig, G, tid);
+    leave_clean(a.cl, hdr, G, tid);
 }
 
 }  // namespace gc

@@ -356,6 +356,60 @@ def test_private_workspace_skips_the_clearing_launch_and_stays_exact(options):
             plan.decompress_accumulate([idx], [val], None, dense, True, ws)
 
 
+@pytest.mark.parametrize("options", [{}, {api.GC_OPT_SAMPLE_RANK_PERMILLE: 30}, {api.GC_OPT_CANDIDATE_CAPACITY: 100}],
+                         ids=["plain", "starved", "overflow"])
+def test_private_workspace_many_tensors_and_workers_call(options):
+    """The same promise for plans of several tensors: gc_compress runs one launch per call from the
+    second call on a workspace, gc_compress_workers one launch for all its workers; every step of
+    every worker against the oracle, with the safety-net routes forced as well."""
+    sizes = [300_000, 5, 1_500_001, 131_072, 64, 0, 131_071, 700_003, 4097, 1000]
+    plan = api.Plan(sizes, 0.005, device=0)
+    plan.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
+    for opt, value in options.items():
+        plan.set_option(opt, value)
+    ks, n, W = plan.tensor_k(), plan.total_n, 3
+    tot = sum(ks)
+    workers = [GpuWorker(plan) for _ in range(W)]
+    r_cpu = [np.zeros(n, np.float32) for _ in range(W)]
+
+    def check(w, g):
+        workers[w].check_status()
+        oi, ov = oracle.topk_compress_tensors(sizes, ks, g.numpy(), r_cpu[w])
+        assert np.array_equal(to_np_u32(workers[w].idx[:tot]), oi)
+        assert np.array_equal(to_np_u32(workers[w].val[:tot]), bits(ov))
+        assert np.array_equal(to_np_u32(workers[w].residual[:n]), bits(r_cpu[w]))
+
+    for step in range(4):                              # one worker, plain calls
+        g = randn(n, 7000 + step)
+        before = plan.launches()
+        workers[0].step(g.cuda())
+        # (the plan has an empty tensor, so the counts are pre-zeroed by a memset per call)
+        assert plan.launches() - before == (3 if step == 0 else 2), step
+        check(0, g)
+    for step in range(3):                              # all workers in one call
+        gs = [randn(n, 7100 + 10 * step + w) for w in range(W)]
+        before = plan.launches()
+        plan.compress_workers([g.cuda() for g in gs], [wk.residual for wk in workers], [wk.idx for wk in workers],
+                              [wk.val for wk in workers], [wk.count for wk in workers], [wk.ws for wk in workers])
+        assert plan.launches() - before == W + (2 if step == 0 else 1), step  # workers 1 and 2 are new to the plan at first
+        for w in range(W):
+            check(w, gs[w])
+    # a foreign write to one worker's workspace: that call reports it, the next one is exact again
+    workers[1].ws.fill_(0x33)
+    gs = [randn(n, 7200 + w) for w in range(W)]
+    r_keep = workers[1].residual.clone()
+    plan.compress_workers([g.cuda() for g in gs], [wk.residual for wk in workers], [wk.idx for wk in workers],
+                          [wk.val for wk in workers], None, [wk.ws for wk in workers])
+    assert plan.last_status(workers[1].ws)[0] == api.GC_E_INVALID
+    assert torch.equal(workers[1].residual, r_keep)
+    check(0, gs[0]); check(2, gs[2])
+    gs2 = [randn(n, 7300 + w) for w in range(W)]
+    plan.compress_workers([g.cuda() for g in gs2], [wk.residual for wk in workers], [wk.idx for wk in workers],
+                          [wk.val for wk in workers], None, [wk.ws for wk in workers])
+    for w in range(W):
+        check(w, gs2[w])
+
+
 def test_private_workspace_broken_promise_is_caught():
     """The caller overwrites a workspace it promised to leave alone: the next call must end at once
     with GC_E_INVALID in the device status (no barrier is entered on counters that cannot be
