@@ -234,6 +234,57 @@ static __device__ __noinline__ void tiny_tensor_warp(const uint32_t off, const u
     if (out_count != nullptr && lane == 0) { out_count[t] = k; out_count[T + t] = k; }
 }
 
+// Exact top-k of one small tensor (it fits one tile) with a FEW entries to keep (k <= kFewK), by
+// one CTA: the tile is read once and stays in registers; round q finds the largest entry that
+// comes strictly after winner q - 1 in the order (key descending, index ascending) -- a scan of
+// the thread's 16 values, a warp-wide and a block-wide maximum, ONE barrier per round instead of
+// the twenty-odd of the three histogram levels.  The winners are then ranked by index.
+constexpr uint32_t kFewK = 8;
+template <typename GL = GradF32>
+static __device__ __noinline__ void small_tensor_fewk(BlockSmem& sm, const TensorDesc& d, uint32_t t, uint32_t T,
+                                                      const void* __restrict__ g, float* __restrict__ r,
+                                                      uint32_t* __restrict__ out_idx, float* __restrict__ out_val,
+                                                      uint32_t* __restrict__ out_count) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const TileGeom tg = tile_geom(d, 0u);
+    Tile tl;
+    load_tile<true, GL>(g, r, tg, warp, lane, tl);           // r = a = g + r; the winners get +0 below
+    unsigned long long* const slot = reinterpret_cast<unsigned long long*>(sm.hist);     // [2][kWarps], by round parity
+    uint32_t* const widx = sm.hist + 4 * kWarps;                                         // [kFewK] winners' flat indices
+    __syncthreads();                                         // (whoever used sm.hist before is done)
+    unsigned long long win = ~0ull;
+    for (uint32_t q = 0; q < d.k; ++q) {
+        unsigned long long best = 0ull;                      // order word: key << 32 | ~flat index (never 0)
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t f = vec_index(tg.base, warp, lane, j) + e;
+                const unsigned long long o = ((unsigned long long)key_of(tl.a[j][e]) << 32) | (unsigned long long)(~f);
+                if (((tl.valid >> (4 * j + e)) & 1u) && o < win && o > best) best = o;
+            }
+        }
+        best = warp_max64(best);
+        if (lane == 0) slot[(q & 1u) * kWarps + warp] = best;
+        __syncthreads();
+        win = 0ull;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { const unsigned long long o = slot[(q & 1u) * kWarps + w]; win = o > win ? o : win; }
+        if (tid == 0) widx[q] = ~(uint32_t)win;
+    }
+    __syncthreads();                                         // the winners' list is complete; r = a is visible block-wide
+    if ((uint32_t)tid < d.k) {
+        const uint32_t f = widx[tid];
+        uint32_t rank = 0;
+        for (uint32_t q = 0; q < d.k; ++q) rank += widx[q] < f ? 1u : 0u;
+        out_idx[d.out_off + rank] = f;
+        out_val[d.out_off + rank] = ld_cg(r + f);            // bit copy of a (written by the owning thread of this CTA)
+        r[f] = 0.0f;
+    }
+    if (out_count != nullptr && tid == 0) { out_count[t] = d.k; out_count[T + t] = d.k; }
+    __syncthreads();
+}
+
 // All small tensors of the plan, dealt out to the CTAs round-robin.
 static __device__ void small_tensors_body(BlockSmem& sm, const TensorDesc* __restrict__ desc, uint32_t T,
                                           const uint32_t* __restrict__ small_ids, uint32_t n_small,

@@ -225,7 +225,8 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     for (uint32_t q = a.n_tiny + (2u * G - 1u - b - ((a.n_tiny + kWarps - 1u) / kWarps) % G) % G; q < a.n_small; q += G) {
         const uint32_t t = a.small_ids[q];
         const TensorDesc d = a.desc[t];
-        small_tensor_body<GL>(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
+        if (d.k <= kFewK) small_tensor_fewk<GL>(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
+        else small_tensor_body<GL>(sm, d, t, a.T, a.g, a.r, a.out_idx, a.out_val, a.out_count);
     }
     __syncthreads();
     for (int i = tid; i < 2048; i += kBlock) sm.hist[i] = 0u;
