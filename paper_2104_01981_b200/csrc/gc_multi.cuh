@@ -463,15 +463,13 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     const bool overflowed = ld_cg(&hdr->overflow) != 0u;
     if (!overflowed && nseg != 0u) {
         // ------------------------------------------------------------ band bin per segment, counts above it
-        for (uint32_t sidx = 0; sidx < nseg; ++sidx) {
+        for (uint32_t sidx = (uint32_t)warp; sidx < nseg; sidx += kWarps) {      // a warp per segment, all at once
             uint32_t* s = seg + (size_t)sidx * kSegWords;
             const uint32_t t = s[SG_T];
-            const uint32_t want_k[1] = {s[SG_K]};
-            Picked pa[1];
-            block_select_multi<2048, 1>(sm, a.bhist + (size_t)t * kHistBins, want_k, pa);
-            const bool ok = pa[0].ok && pa[0].count <= kMultiMidCap;
-            if (tid == 0) {
-                s[SG_A] = pa[0].bin; s[SG_ABOVE] = pa[0].above; s[SG_M] = pa[0].count; s[SG_OK] = ok ? 1u : 0u;
+            const Picked pa = warp_select_2048(a.bhist + (size_t)t * kHistBins, s[SG_K], lane);
+            const bool ok = pa.ok && pa.count <= kMultiMidCap;
+            if (lane == 0) {
+                s[SG_A] = pa.bin; s[SG_ABOVE] = pa.above; s[SG_M] = pa.count; s[SG_OK] = ok ? 1u : 0u;
                 if (!ok) {          // every CTA that sees this tensor decides the same; count it once
                     const uint32_t old = atomicOr(&a.ws.sel[t].flags, kSelFailed);
                     if ((old & kSelFailed) == 0u) atomicAdd(&hdr->n_failed, 1u);

@@ -173,6 +173,53 @@ __device__ void block_select_multi(BlockSmem& sm, const uint32_t* hist, const ui
     __syncthreads();
 }
 
+// The same for ONE rank by ONE warp (all 32 lanes call): the 2048 bins are read once with sixteen
+// coalesced 16-byte loads per lane, so the eight warps of a CTA can each settle a different
+// histogram at the same time, without a block-wide barrier.  Lane l holds, in round i, the four
+// bins 4 (32 i + l) .. + 3; a "row" is the 128 bins of one round.
+__device__ __forceinline__ Picked warp_select_2048(const uint32_t* hist, uint32_t k, int lane) {
+    uint32_t rows[16], total = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {                        // eight loads in flight at a time (registers)
+        uint4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = ld_cg(reinterpret_cast<const uint4*>(hist) + 32 * (8 * h + i) + lane);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            rows[8 * h + i] = __reduce_add_sync(0xFFFFFFFFu, v[i].x + v[i].y + v[i].z + v[i].w);
+            total += rows[8 * h + i];
+        }
+    }
+    Picked p; p.bin = 0xFFFFFFFFu; p.above = 0u; p.count = 0u; p.ok = false;
+    if (k == 0u || total < k) return p;
+    // the row that holds the rank, from the top, and the count above that row
+    uint32_t above = 0; int R = -1;
+#pragma unroll
+    for (int i = 15; i >= 0; --i)
+        if (R < 0) { if (above + rows[i] >= k) R = i; else above += rows[i]; }
+    const uint4 vr = ld_cg(reinterpret_cast<const uint4*>(hist) + 32 * R + lane);      // (that row once more)
+    // inside the row, lanes from the top: position q stands for lane 31 - q
+    const uint32_t mine = vr.x + vr.y + vr.z + vr.w;
+    const uint32_t t = __shfl_sync(0xFFFFFFFFu, mine, 31 - lane);
+    const uint32_t inc = warp_incl_scan(t, lane);
+    const unsigned hit = __ballot_sync(0xFFFFFFFFu, above + inc >= k);
+    const int q = __ffs(hit) - 1;                                          // (hit != 0: the row holds the rank)
+    const uint32_t above_l = above + __shfl_sync(0xFFFFFFFFu, inc - t, q);
+    const int L = 31 - q;
+    const uint32_t c3 = __shfl_sync(0xFFFFFFFFu, vr.w, L), c2 = __shfl_sync(0xFFFFFFFFu, vr.z, L);
+    const uint32_t c1 = __shfl_sync(0xFFFFFFFFu, vr.y, L), c0 = __shfl_sync(0xFFFFFFFFu, vr.x, L);
+    const uint32_t base = 4u * (32u * (uint32_t)R + (uint32_t)L);
+    uint32_t ab = above_l;
+    if (ab + c3 >= k) { p.bin = base + 3u; p.count = c3; }
+    else { ab += c3;
+        if (ab + c2 >= k) { p.bin = base + 2u; p.count = c2; }
+        else { ab += c2;
+            if (ab + c1 >= k) { p.bin = base + 1u; p.count = c1; }
+            else { ab += c1; p.bin = base; p.count = c0; } } }
+    p.above = ab; p.ok = true;
+    return p;
+}
+
 // Rank `rank` (1 = largest) among the values f(entry) of the short-list entries that f accepts,
 // by radix select over `nbits` bits, 11 at a time from the top, with the histogram in shared
 // memory.  Every CTA runs this on the same list and gets the same answer.  Entries come from
