@@ -29,6 +29,7 @@ namespace gc {
 constexpr uint32_t kMultiMidCap = kMidFast;      // short list per tensor (entries stay in registers)
 constexpr uint32_t kSegWords = 16;               // shared-memory words per segment record
 constexpr uint32_t kRefineTiles = 32;            // samples of up to this many sample tiles are ranked a second time
+constexpr uint32_t kWarpMid = 128;               // short lists up to this length are settled by one warp
 
 struct MultiArgs {
     const TensorDesc* desc;
@@ -513,9 +514,81 @@ __device__ __forceinline__ void topk_multi_body(const MultiArgs& a, const uint32
     if (!overflowed) {
         if (nseg != 0u) {
             // -------------------------------------------------------- threshold, tie cut and slots per segment
+            // Short lists of up to kWarpMid entries (nearly all: a band bin holds a handful of
+            // candidates) are settled by a warp each, all segments of the CTA at once and without a
+            // block-wide barrier: every entry's place in the order (key descending, index ascending)
+            // is counted directly against all others, which settles threshold and tie cut in one go.
+            for (uint32_t sidx = (uint32_t)warp; sidx < nseg; sidx += kWarps) {
+                uint32_t* s = seg + (size_t)sidx * kSegWords;
+                const uint32_t m = s[SG_M];
+                if (s[SG_OK] == 0u || m > kWarpMid) continue;
+                const uint32_t t = s[SG_T];
+                const TensorDesc d = a.desc[t];
+                const uint2* mid = a.mid + (size_t)t * kMultiMidCap;
+                uint2 e[kWarpMid / 32];
+#pragma unroll
+                for (uint32_t u = 0; u < kWarpMid / 32; ++u)
+                    e[u] = u * 32u + lane < m ? ld_cg(mid + u * 32u + lane) : make_uint2(0xFFFFFFFFu, 0u);
+                // candidates above the band bin in the tensor's tiles before this segment
+                const uint32_t nbefore = first + s[SG_TILE0] - d.tile0;
+                uint32_t part = 0;
+                for (uint32_t q = lane; q < nbefore; q += 32u) part += ld_cg(a.tile_cnt + d.tile0 + q);
+                part = __reduce_add_sync(0xFFFFFFFFu, part);
+                const uint32_t krem = s[SG_K] - s[SG_ABOVE];             // entries of the short list that are sent (1 .. m)
+                // place of every own entry: entries that come before it in the order
+                uint32_t place[kWarpMid / 32];
+#pragma unroll
+                for (uint32_t u = 0; u < kWarpMid / 32; ++u) place[u] = 0u;
+#pragma unroll
+                for (uint32_t uo = 0; uo < kWarpMid / 32; ++uo) {
+                    if (uo * 32u >= m) break;                            // (uniform)
+                    const uint32_t lim = min(32u, m - uo * 32u);
+                    for (uint32_t l = 0; l < lim; ++l) {
+                        const uint32_t ox = __shfl_sync(0xFFFFFFFFu, e[uo].x, (int)l);
+                        const uint32_t ok = __shfl_sync(0xFFFFFFFFu, e[uo].y, (int)l) & kKeyMask;
+#pragma unroll
+                        for (uint32_t u = 0; u < kWarpMid / 32; ++u) {
+                            const uint32_t key = e[u].y & kKeyMask;
+                            place[u] += (ok > key || (ok == key && ox < e[u].x)) ? 1u : 0u;
+                        }
+                    }
+                }
+                // the last entry that is sent gives the threshold key and the tie cut; sent entries before
+                // the segment shift its first slot, inside it they join the count of their chunk
+                const uint32_t seg_end = s[SG_BASE0] + s[SG_NTILE] * (uint32_t)kTile;
+                uint32_t before = 0, tk = 0, cut = 0;
+                bool have = false;
+#pragma unroll
+                for (uint32_t u = 0; u < kWarpMid / 32; ++u) {
+                    if (u * 32u + lane >= m) continue;
+                    if (place[u] == krem - 1u) { have = true; tk = e[u].y & kKeyMask; cut = e[u].x; }
+                    if (place[u] < krem) {
+                        if (e[u].x < s[SG_BEGIN]) ++before;
+                        else if (e[u].x < seg_end) atomicAdd(&rec2[chunk_of(s, e[u].x)], 1u);
+                    }
+                }
+                before = __reduce_add_sync(0xFFFFFFFFu, before);
+                const unsigned who = __ballot_sync(0xFFFFFFFFu, have);
+                const bool good = who != 0u;                             // (the list holds at least krem entries)
+                const int src = good ? __ffs(who) - 1 : 0;
+                tk = __shfl_sync(0xFFFFFFFFu, tk, src); cut = __shfl_sync(0xFFFFFFFFu, cut, src);
+                __syncwarp();
+                if (lane == 0) {
+                    s[SG_TKEY] = tk; s[SG_CUT] = cut;
+                    s[SG_OUT] = d.out_off + part + before;             // slot of the segment's first sent entry
+                    if (!good) {        // cannot happen unless the list changed under us: report, send nothing
+                        s[SG_OK] = 0u;
+                        record_status(hdr, -1 /*GC_E_INVALID*/, 0xE0000000ull + t);
+                    } else if (a.out_count != nullptr && first + s[SG_TILE0] == d.tile0) {
+                        a.out_count[t] = d.k; a.out_count[a.T + t] = d.k;
+                    }
+                }
+            }
+            __syncthreads();
+            // longer short lists: the whole CTA, one segment after the other (radix select in shared memory)
             for (uint32_t sidx = 0; sidx < nseg; ++sidx) {
                 uint32_t* s = seg + (size_t)sidx * kSegWords;
-                if (s[SG_OK] == 0u) continue;
+                if (s[SG_OK] == 0u || s[SG_M] <= kWarpMid) continue;
                 const uint32_t t = s[SG_T], m = s[SG_M];
                 const TensorDesc d = a.desc[t];
                 const uint2* mid = a.mid + (size_t)t * kMultiMidCap;
