@@ -228,13 +228,6 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     const uint32_t per = (ntl + gridDim.x - 1) / gridDim.x;
     const uint32_t t0 = blockIdx.x * per, t1 = min(ntl, t0 + per);
     if (t0 >= t1) return;
-#ifdef GC_PROBE_DECODE_SPREAD
-    if (tid == 0) {
-        unsigned long long ts;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
-        atomicMin(reinterpret_cast<unsigned long long*>(hdr) + 40, ts);
-    }
-#endif
 
     // length of each worker's list, and where it enters this CTA's run of tiles
     for (uint32_t w = warp; w < W; w += kDecBlock / 32) {
@@ -334,15 +327,6 @@ k_decode_tiles(DecodeLists ls, uint32_t W, uint32_t cnt, uint32_t total_n, float
     if (t1 == ntl && tid < (int)W && s_cur[tid] < s_len[tid])
         record_status(hdr, -1 /*GC_E_INVALID*/, s_cur[tid]);   // leftovers point at or beyond total_n
     if (use_bulk && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-#ifdef GC_PROBE_DECODE_SPREAD
-    if (tid == 0) {          // probe build only: when every CTA ended, and on which SM
-        unsigned long long ts; uint32_t smid;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts));
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        unsigned long long* dbg = reinterpret_cast<unsigned long long*>(hdr) + 64;
-        dbg[2 * blockIdx.x] = ts; dbg[2 * blockIdx.x + 1] = ((unsigned long long)(t1 - t0) << 16) | smid;
-    }
-#endif
 }
 
 // Tiled decode of lists that carry per-tensor counts (threshold mode, plans of several tensors):
