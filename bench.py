@@ -519,6 +519,7 @@ def _report(args, w, rank, world, dev, plan, n, k, W, sets, res, others):
             ("c3_bert_base_110m_student_t", "threshold", "compress_fused"): "k_threshold_single_c3_bert110m.md",
             ("c2_resnet50_layerwise", "topk", "compress_fused"): "k_topk_multi_c2_resnet50.md",
             ("c4_resnet50_8workers", "topk", "compress_fused"): "k_topk_workers_c4_resnet50_8workers.md",
+            ("c4_resnet50_8workers", "threshold", "compress_fused"): "k_threshold_workers_c4_resnet50_8workers.md",
             }.get((w.name, args.mode, dom) if args.grad_dtype == "f32" else None)
     ncu_traffic, ncu_src = profile_traffic(prof) if prof else (None, None)
 
