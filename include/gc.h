@@ -151,14 +151,15 @@ int gc_plan(gc_plan_t **out, int device, uint32_t n_tensors, const uint64_t *siz
  *                                promises that between two gc_compress calls of THIS plan on a
  *                                workspace nothing else writes to it (the decode calls of this plan
  *                                are fine, and so is a zero-filled or a fresh workspace for the first
- *                                call).  The one-tensor top-k kernel cleans the control block as it
- *                                goes (each section right after the grid barrier that follows its
- *                                last reader, the rest at the start of the next launch), so its
+ *                                call).  The fused top-k kernels (one tensor, many tensors, and the
+ *                                shared launch of gc_compress_workers) clean the control block as
+ *                                they go (each section right after the grid barrier that follows its
+ *                                last reader, the rest at the start of the next launch), so their
  *                                calls then do without the clearing launch.  A broken promise is
  *                                caught by a mark in the workspace header: the kernel leaves at once
  *                                and GC_E_INVALID is recorded in the device status; after any error
  *                                status read through gc_last_status the next call clears again.
- *                                Other plans' routes ignore the option.
+ *                                The threshold, staged and exact routes ignore the option.
  * Errors: GC_E_INVALID (unknown option or value), GC_E_CUDA.
  */
 #define GC_OPT_PATH                  0
