@@ -618,3 +618,50 @@ def test_host_buffer_entry_point_with_alternating_staging_buffers(sizes):
         st, det = plan.last_status(ws)
         assert st == api.GC_OK, (st, det)
     plan.profile_enable(0)
+
+
+@pytest.mark.parametrize("mode", [api.GC_TOPK, api.GC_THRESHOLD], ids=["topk", "threshold"])
+def test_private_workspaces_under_changing_call_patterns(mode):
+    """Sixty steps on private workspaces that are served in turn by one gc_compress_workers call,
+    by one gc_compress call per worker, and by a two-worker call plus single calls, with a decode on
+    one of the workspaces in between, quantised (tie-heavy) gradients every fifth step and thirty
+    times larger ones every seventh: every step bit-equal to a second plan that clears its one
+    shared workspace before every call (that plan's route is what the tests above hold against
+    the oracle)."""
+    rng = np.random.default_rng(11)
+    sizes = [int(rng.integers(1, 200_000)) for _ in range(30)] + [5, 0, 4096, 4097]
+    W, n = 5, None
+    pa = api.Plan(sizes, 0.004, mode=mode, device=0)
+    pa.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
+    pb = api.Plan(sizes, 0.004, mode=mode, device=0)
+    n = pa.total_n
+    wa, wsb = [GpuWorker(pa) for _ in range(W)], pb.alloc_workspace()
+    wb = [GpuWorker(pb) for _ in range(W)]
+    da, db = torch.empty(n, device="cuda"), torch.empty(n, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    scale = torch.rand(n, device="cuda", generator=gen) * 2 + 0.01
+    for s in range(60):
+        g = [torch.randn(n, device="cuda", generator=gen) * scale * (1.0 if s % 7 else 30.0) for _ in range(W)]
+        if s % 5 == 3:
+            g = [torch.round(x * 4) / 4 for x in g]
+        for wk in wa + wb:
+            wk.idx.fill_(-1); wk.val.fill_(float("nan"))
+        first = 0 if s % 3 == 0 else (W if s % 3 == 1 else 2)      # workers served by the shared call
+        if first:
+            pa.compress_workers(g[:first] if first < W else g, [wk.residual for wk in wa[:first]],
+                                [wk.idx for wk in wa[:first]], [wk.val for wk in wa[:first]],
+                                [wk.count for wk in wa[:first]], [wk.ws for wk in wa[:first]])
+        for w in range(first, W):
+            pa.compress(g[w], wa[w].residual, wa[w].idx, wa[w].val, wa[w].count, wa[w].ws)
+        for w in range(W):
+            pb.compress(g[w], wb[w].residual, wb[w].idx, wb[w].val, wb[w].count, wsb)
+        pa.decompress_accumulate([wk.idx for wk in wa], [wk.val for wk in wa], [wk.count for wk in wa], da, True,
+                                 wa[s % W].ws)
+        pb.decompress_accumulate([wk.idx for wk in wb], [wk.val for wk in wb], [wk.count for wk in wb], db, True, wsb)
+        for w in range(W):
+            assert pa.last_status(wa[w].ws)[0] >= 0, (s, w)
+            assert torch.equal(wa[w].count, wb[w].count), (s, w)
+            assert torch.equal(wa[w].idx, wb[w].idx), (s, w)
+            assert torch.equal(wa[w].val.view(torch.int32), wb[w].val.view(torch.int32)), (s, w)
+            assert torch.equal(wa[w].residual.view(torch.int32), wb[w].residual.view(torch.int32)), (s, w)
+        assert torch.equal(da.view(torch.int32), db.view(torch.int32)), s
