@@ -317,7 +317,12 @@ void plan_single(gc_plan_s* p) {
     if (p->mode != GC_TOPK || p->T != 1 || p->grid_single_max <= 0) return;
     const TensorDesc& d = p->desc[0];
     if (d.sstride == 0 || d.ntiles == 0 || d.off != 0) return;
-    const uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
+    uint32_t G = std::min<uint32_t>((uint32_t)p->grid_single_max, d.ntiles);
+    // Small tensors are all latency (a CTA has a handful of tiles and five phases to walk through):
+    // there two CTAs per SM get through the phases sooner than three (2M-10M elements: 31-49 us
+    // against 37-51 us).  From about 12M elements on the third CTA pays for itself; below 300
+    // tiles there is a CTA per tile anyway (fewer were no faster).
+    if (d.ntiles <= 3000u) G = std::min<uint32_t>(G, 2u * (uint32_t)p->sm_count);
     uint32_t maxt = (d.ntiles + G - 1) / G;
     const RowMap rm = make_row_map(p, d.ntiles, G, maxt, p->density >= 0.005 ? kSingleSkew : kSingleSkewSparse);
     if (maxt > kSingleMaxT || G > 640) return;                       // chunk records and totals must stay small
