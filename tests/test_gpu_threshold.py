@@ -237,3 +237,11 @@ def test_threshold_random_plans_match_the_oracle(seed):
     scales = torch.cat([torch.full((s,), float(10.0 ** rng.integers(-2, 2))) for s in sizes])
     grads = [randn(n, 6000 + 10 * seed + s) * scales for s in range(2)]
     check_threshold(sizes, density, grads, stride=stride, cap_factor=cap_factor)
+
+
+@pytest.mark.parametrize("tiles", [296, 297, 2500, 2501])
+def test_threshold_one_tensor_plans_around_the_grid_rule(tiles):
+    """The one-tensor threshold kernel runs on two CTAs per SM up to 2500 tiles and on three beyond:
+    both sides of the rule and of the 296-CTA grid, ragged last tile, two steps against the oracle."""
+    n = tiles * 4096 - 7
+    check_threshold([n], 0.004, [randn(n, 9300 + tiles), randn(n, 9400 + tiles)])

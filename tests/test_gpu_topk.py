@@ -665,3 +665,12 @@ def test_private_workspaces_under_changing_call_patterns(mode):
             assert torch.equal(wa[w].val.view(torch.int32), wb[w].val.view(torch.int32)), (s, w)
             assert torch.equal(wa[w].residual.view(torch.int32), wb[w].residual.view(torch.int32)), (s, w)
         assert torch.equal(da.view(torch.int32), db.view(torch.int32)), s
+
+
+@pytest.mark.parametrize("tiles", [296, 297, 593, 2999, 3000, 3001])
+def test_one_tensor_plans_around_the_grid_rule(tiles):
+    """One-tensor plans of up to 3000 tiles run on two CTAs per SM, larger ones on three: sizes on
+    both sides of that rule and where a CTA's share of tiles changes (296 CTAs), with a ragged
+    last tile, two steps each against the oracle."""
+    n = tiles * 4096 - 5
+    check_topk_against_oracle([n], 0.004, [randn(n, 9100 + tiles), randn(n, 9200 + tiles)])
