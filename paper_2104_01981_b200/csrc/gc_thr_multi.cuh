@@ -230,14 +230,15 @@ static __device__ __forceinline__ void threshold_multi_body(const ThrMultiArgs& 
         int have = level_bits(0);                          // key bits fixed so far
         while (ok && have < 31) {
             const int w = min(11, 31 - have), sh = 31 - have - w;       // this level: bits [sh, sh + w)
-            for (uint32_t q0 = tid; q0 < nk; q0 += 4 * kBlock) {
-                uint4 kv[4];
+            constexpr int kKeyBatch = 8;                   // loads in flight per thread: one CTA walks a whole tensor's keys
+            for (uint32_t q0 = tid; q0 < nk; q0 += kKeyBatch * kBlock) {
+                uint4 kv[kKeyBatch];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
+                for (int u = 0; u < kKeyBatch; ++u)
                     kv[u] = q0 + u * kBlock < nk ? ld_cg(sk + q0 + u * kBlock)
                                                  : make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kKeyBatch; ++u) {
                     const uint32_t kk[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
