@@ -674,3 +674,45 @@ def test_one_tensor_plans_around_the_grid_rule(tiles):
     last tile, two steps each against the oracle."""
     n = tiles * 4096 - 5
     check_topk_against_oracle([n], 0.004, [randn(n, 9100 + tiles), randn(n, 9200 + tiles)])
+
+
+def test_calls_on_a_side_stream():
+    """Every call enqueues on the stream it is given and on no other: compress, the workers call,
+    decode and the fused optimizer step on a non-blocking side stream that is held back by a
+    long-running kernel, while the default stream stays idle; the results are read after the
+    side stream alone has been waited for, and compared with the oracle."""
+    sizes = [250_000, 0, 7, 1_200_003, 4096, 66_000]
+    plan = api.Plan(sizes, 0.004, device=0)
+    ks, n, W = plan.tensor_k(), plan.total_n, 3
+    tot = sum(ks)
+    workers = [GpuWorker(plan) for _ in range(W)]
+    gs = [randn(n, 9500 + w) for w in range(W)]
+    gd = [g.cuda() for g in gs]
+    dense = torch.empty(n, device="cuda")
+    param, vel = torch.ones(n, device="cuda"), torch.zeros(n, device="cuda")
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        torch.cuda._sleep(20_000_000)                       # about 10 ms: everything below queues up behind it
+        plan.compress(gd[0], workers[0].residual, workers[0].idx, workers[0].val, workers[0].count, workers[0].ws, side)
+        plan.compress_workers(gd[1:], [wk.residual for wk in workers[1:]], [wk.idx for wk in workers[1:]],
+                              [wk.val for wk in workers[1:]], [wk.count for wk in workers[1:]],
+                              [wk.ws for wk in workers[1:]], side)
+        plan.decompress_accumulate([wk.idx for wk in workers], [wk.val for wk in workers], None, dense, True,
+                                   workers[0].ws, side)
+        plan.decompress_apply_momentum([wk.idx for wk in workers], [wk.val for wk in workers], None, param, vel,
+                                       0.1, 0.9, 0.5, workers[0].ws, side)
+    side.synchronize()
+    lists = []
+    for w in range(W):
+        r_cpu = np.zeros(n, np.float32)
+        oi, ov = oracle.topk_compress_tensors(sizes, ks, gs[w].numpy(), r_cpu)
+        assert np.array_equal(to_np_u32(workers[w].idx[:tot]), oi), w
+        assert np.array_equal(to_np_u32(workers[w].val[:tot]), bits(ov)), w
+        assert np.array_equal(to_np_u32(workers[w].residual[:n]), bits(r_cpu)), w
+        lists.append((oi, ov))
+    want = oracle.decode_accumulate(lists, np.empty(n, np.float32), True)
+    assert np.array_equal(to_np_u32(dense), bits(want))
+    p_cpu, v_cpu = np.ones(n, np.float32), np.zeros(n, np.float32)
+    oracle.decode_apply_momentum(lists, p_cpu, v_cpu, 0.1, 0.9, 0.5)
+    assert np.array_equal(to_np_u32(param), bits(p_cpu)) and np.array_equal(to_np_u32(vel), bits(v_cpu))
