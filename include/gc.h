@@ -24,7 +24,8 @@
  *     ordinary process memory.  The caller owns every buffer it passes in, including the
  *     workspace; the plan owns only its own small host and device tables.
  *   - gc_compress and gc_decompress_accumulate enqueue work on the given stream and return
- *     without synchronising.  No call allocates device memory except gc_plan.
+ *     without synchronising (they may be captured in a CUDA graph; a plan option must not be
+ *     changed between capture and replay).  No call allocates device memory except gc_plan.
  *   - A plan is bound to one device.  Every call that touches the device (compress, decode,
  *     gc_last_*, gc_compress_host) must be made while that device is the current one and
  *     returns GC_E_INVALID otherwise; gc_plan leaves the caller's current device as it was.

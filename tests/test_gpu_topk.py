@@ -716,3 +716,51 @@ def test_calls_on_a_side_stream():
     p_cpu, v_cpu = np.ones(n, np.float32), np.zeros(n, np.float32)
     oracle.decode_apply_momentum(lists, p_cpu, v_cpu, 0.1, 0.9, 0.5)
     assert np.array_equal(to_np_u32(param), bits(p_cpu)) and np.array_equal(to_np_u32(vel), bits(v_cpu))
+
+
+@pytest.mark.parametrize("sizes", [[1_300_001], [200_000, 3, 0, 900_001, 4096]], ids=["one", "many"])
+def test_step_captured_in_a_cuda_graph(sizes):
+    """A compress + decode step captured once in a CUDA graph (cooperative launch included) and
+    replayed on fresh gradients copied into the captured buffer: every replay against the oracle.
+    The workspace is private and warmed, so the captured step holds no clearing launch."""
+    plan = api.Plan(sizes, 0.005, device=0)
+    plan.set_option(api.GC_OPT_WORKSPACE_PRIVATE, 1)
+    ks, n = plan.tensor_k(), plan.total_n
+    tot = sum(ks)
+    wk = GpuWorker(plan)
+    g_dev = torch.zeros(n, device="cuda")
+    dense = torch.empty(n, device="cuda")
+    side = torch.cuda.Stream()
+    r_cpu = np.zeros(n, np.float32)
+
+    def step():
+        plan.compress(g_dev, wk.residual, wk.idx, wk.val, wk.count, wk.ws, side)
+        plan.decompress_accumulate([wk.idx], [wk.val], None, dense, True, wk.ws, side)
+
+    def check(g):
+        oi, ov = oracle.topk_compress_tensors(sizes, ks, g.numpy(), r_cpu)
+        assert np.array_equal(to_np_u32(wk.idx[:tot]), oi)
+        assert np.array_equal(to_np_u32(wk.val[:tot]), bits(ov))
+        assert np.array_equal(to_np_u32(wk.residual[:n]), bits(r_cpu))
+        assert np.array_equal(to_np_u32(dense), bits(oracle.decode_accumulate([(oi, ov)], np.empty(n, np.float32), True)))
+
+    g0 = randn(n, 9600)
+    g_dev.copy_(g0.cuda())
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        step()                                              # warm: clears once, leaves the workspace clean
+    side.synchronize()
+    check(g0)
+    graph = torch.cuda.CUDAGraph()
+    before = plan.launches()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+    assert plan.launches() - before == (2 if len(sizes) == 1 else 3)    # (many: the plan has an empty tensor, counts pre-zeroed)
+    for i in range(3):
+        g = randn(n, 9601 + i)
+        g_dev.copy_(g.cuda())
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert plan.last_status(wk.ws)[0] == api.GC_OK
+        check(g)
