@@ -109,7 +109,12 @@ typedef struct gc_plan_s gc_plan_t;
  *   density        in (0, 1]
  *   mode           GC_TOPK or GC_THRESHOLD
  *   sample_stride  threshold mode: sample one 4-element group out of this many (0 = 64);
- *                  tensors of <= 65,536 elements are always sampled in full
+ *                  tensors of <= 65,536 elements are always sampled in full.  Every sampled
+ *                  group is a scattered 32-byte DRAM access in g and in r, and on tensors of
+ *                  100M elements and more that is a tenth of the call at stride 64 (110M
+ *                  elements: 262 us against 238 us at stride 512, whose sample still holds
+ *                  214,000 elements); the stride is part of the result's definition, so the
+ *                  library does not choose it
  *   cap_factor     threshold mode: per-tensor output capacity = min(n, ceil(cap_factor*k))
  *                  (0 = 2.0; must be >= 1)
  * Allocates a few KB of device memory for the tensor table (freed by gc_destroy).
